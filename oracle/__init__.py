@@ -1,0 +1,184 @@
+"""ctypes front end of the CPU oracle (test infrastructure, not the product).
+
+The oracle is the C++ file next to this module, built as ``libwindq_oracle.so``
+with ``g++ -O2 -ffp-contract=off``.  Nothing here touches CUDA or imports the
+GPU package; inputs and outputs are numpy arrays (fp16 data as ``uint16`` bit
+patterns or ``float16`` arrays).  Only tests, the smoke check and the
+benchmark's CPU-baseline leg may import this package.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from concurrent.futures import ThreadPoolExecutor
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "windq_oracle.cpp")
+_LIB = os.path.join(_HERE, "libwindq_oracle.so")
+
+CXX_FLAGS = ["-std=c++17", "-O2", "-ffp-contract=off", "-fno-fast-math", "-fPIC", "-shared", "-Wall"]
+
+N_BITWIDTHS = 6          # table columns: 8, 4, 3, 2, 1.58, 1
+N_FEATURES = 8
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle if the library is missing or older than its source."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + ".tmp.%d" % os.getpid()
+        subprocess.run(["g++", *CXX_FLAGS, "-o", tmp, _SRC], check=True)
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    global _lib
+    if _lib is None:
+        _lib = ctypes.CDLL(build())
+        _lib.oracle_half_to_float.restype = ctypes.c_float
+        _lib.oracle_half_to_float.argtypes = [ctypes.c_uint16]
+        _lib.oracle_float_to_half.restype = ctypes.c_uint16
+        _lib.oracle_float_to_half.argtypes = [ctypes.c_float]
+        _lib.oracle_psum8.restype = ctypes.c_float
+    return _lib
+
+
+def _p(a):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _as_u16(a: np.ndarray) -> np.ndarray:
+    a = np.ascontiguousarray(a)
+    if a.dtype == np.float16:
+        a = a.view(np.uint16)
+    assert a.dtype == np.uint16, a.dtype
+    return a
+
+
+def _f32(a) -> np.ndarray:
+    return np.ascontiguousarray(a, dtype=np.float32)
+
+
+def half_to_float(h: int) -> float:
+    return float(lib().oracle_half_to_float(int(h)))
+
+
+def float_to_half(f: float) -> int:
+    return int(lib().oracle_float_to_half(ctypes.c_float(f)))
+
+
+def psum8(x) -> float:
+    x = _f32(x)
+    return float(lib().oracle_psum8(_p(x), ctypes.c_int(x.size)))
+
+
+def uniform_candidate(w, s, bits: int, p: float, want_codes: bool = True):
+    """One clip candidate on one row-group: (scale, zero, error, codes)."""
+    w, s = _f32(w), _f32(s)
+    G = w.size
+    scale, zero, err = ctypes.c_float(), ctypes.c_float(), ctypes.c_float()
+    codes = np.zeros(G, np.uint8) if want_codes else None
+    rc = lib().oracle_uniform_candidate(_p(w), _p(s), ctypes.c_int(G), ctypes.c_int(bits), ctypes.c_float(p),
+                                        ctypes.byref(scale), ctypes.byref(zero), ctypes.byref(err), _p(codes))
+    if rc:
+        raise ValueError("oracle_uniform_candidate: bad arguments")
+    return scale.value, zero.value, err.value, codes
+
+
+def act_stats(X) -> np.ndarray:
+    X = _as_u16(X)
+    T, C = X.shape
+    s = np.zeros(C, np.float32)
+    rc = lib().oracle_act_stats(_p(X), ctypes.c_int64(T), ctypes.c_int64(C), ctypes.c_int64(C), _p(s))
+    if rc:
+        raise ValueError("oracle_act_stats: bad arguments")
+    return s
+
+
+def unit_features(W, G: int, s) -> np.ndarray:
+    W, s = _as_u16(W), _f32(s)
+    R, C = W.shape
+    feat = np.zeros((C // G, N_FEATURES), np.float32)
+    rc = lib().oracle_unit_features(_p(W), ctypes.c_int64(R), ctypes.c_int64(C), ctypes.c_int64(C),
+                                    ctypes.c_int(G), _p(s), _p(feat))
+    if rc:
+        raise ValueError("oracle_unit_features: bad arguments")
+    return feat
+
+
+def fit_eval(W, G: int, s, clip_grid, units=None, threads: int = 1, want_group_err: bool = True):
+    """Returns dict(err[U,6], energy[U], clip_idx[4,U,R], group_err[6,U,R]).
+
+    ``units`` = (begin, end) restricts the work to a unit range (other rows of
+    the outputs stay zero).  ``threads`` > 1 runs the same single-threaded
+    routine over disjoint unit ranges concurrently (units are independent).
+    """
+    W, s, clip_grid = _as_u16(W), _f32(s), _f32(clip_grid)
+    R, C = W.shape
+    U = C // G
+    K = clip_grid.size
+    u0, u1 = (0, U) if units is None else units
+    err = np.zeros((U, N_BITWIDTHS), np.float32)
+    energy = np.zeros(U, np.float32)
+    clip_idx = np.zeros((4, U, R), np.uint8)
+    group_err = np.zeros((N_BITWIDTHS, U, R), np.float32) if want_group_err else None
+
+    def run(a, b):
+        rc = lib().oracle_fit_eval(_p(W), ctypes.c_int64(R), ctypes.c_int64(C), ctypes.c_int64(C), ctypes.c_int(G),
+                                   _p(s), _p(clip_grid), ctypes.c_int(K), ctypes.c_int64(a), ctypes.c_int64(b),
+                                   _p(err), _p(energy), _p(clip_idx), _p(group_err))
+        if rc:
+            raise ValueError("oracle_fit_eval: bad arguments")
+
+    if threads <= 1 or u1 - u0 <= 1:
+        run(u0, u1)
+    else:
+        bounds = np.linspace(u0, u1, min(threads, u1 - u0) + 1).astype(np.int64)
+        with ThreadPoolExecutor(max_workers=threads) as ex:
+            list(ex.map(lambda ab: run(int(ab[0]), int(ab[1])), zip(bounds[:-1], bounds[1:])))
+    return dict(err=err, energy=energy, clip_idx=clip_idx, group_err=group_err)
+
+
+def effective_bits(actions, R: int, G: int, scale_bits: int = 16, zero_bits: int = 16):
+    """Returns dict(unit_centibits[U], code_offsets[U+1], total_centibits, total_packed_bytes)."""
+    actions = np.ascontiguousarray(actions, dtype=np.uint8)
+    U = actions.size
+    unit_cb = np.zeros(U, np.int64)
+    offs = np.zeros(U + 1, np.int64)
+    total = ctypes.c_int64()
+    packed = ctypes.c_int64()
+    rc = lib().oracle_effective_bits(_p(actions), ctypes.c_int64(U), ctypes.c_int64(R), ctypes.c_int(G),
+                                     ctypes.c_int(scale_bits), ctypes.c_int(zero_bits), _p(unit_cb), _p(offs),
+                                     ctypes.byref(total), ctypes.byref(packed))
+    if rc:
+        raise ValueError("oracle_effective_bits: bad arguments")
+    return dict(unit_centibits=unit_cb, code_offsets=offs, total_centibits=total.value,
+                total_packed_bytes=packed.value)
+
+
+def apply_plan(W, G: int, s, clip_grid, actions, clip_idx=None, want_wq: bool = True):
+    """Returns dict(codes[bytes], scales[U,R] u16, zeros[U,R] u16, wq[R,C] u16, code_offsets)."""
+    W, s, clip_grid = _as_u16(W), _f32(s), _f32(clip_grid)
+    actions = np.ascontiguousarray(actions, dtype=np.uint8)
+    R, C = W.shape
+    U = C // G
+    offs = effective_bits(actions, R, G)["code_offsets"]
+    codes = np.zeros(int(offs[U]), np.uint8)
+    scales = np.zeros((U, R), np.uint16)
+    zeros = np.zeros((U, R), np.uint16)
+    wq = np.zeros((R, C), np.uint16) if want_wq else None
+    if clip_idx is not None:
+        clip_idx = np.ascontiguousarray(clip_idx, dtype=np.uint8)
+        assert clip_idx.shape == (4, U, R)
+    rc = lib().oracle_apply_plan(_p(W), ctypes.c_int64(R), ctypes.c_int64(C), ctypes.c_int64(C), ctypes.c_int(G),
+                                 _p(s), _p(clip_grid), ctypes.c_int(clip_grid.size), _p(actions), _p(clip_idx),
+                                 _p(offs), _p(codes), _p(scales), _p(zeros), _p(wq))
+    if rc:
+        raise ValueError("oracle_apply_plan: bad arguments")
+    return dict(codes=codes, scales=scales, zeros=zeros, wq=wq, code_offsets=offs)

@@ -1,0 +1,569 @@
+// windq oracle -- TEST INFRASTRUCTURE, not the product.
+//
+// A plain, slow, single-threaded C++17 restatement of the scoring / fitting hot
+// path of WINDQuant's allocation loop: activation statistics, per-unit state
+// features, per-group quantizer fits under all six bit-widths, plan
+// application (codes, packing, fake-quantised weights) and effective-bit
+// accounting.  It shares no code with the CUDA library and neither includes
+// the other.  Only the tests, the smoke check and the benchmark's CPU-baseline
+// leg may call it.  Build: g++ -O2 -ffp-contract=off (no fast-math, no
+// -march): every float operation below is one IEEE-754 binary32 operation,
+// rounded to nearest even, in exactly the order written.
+//
+// What the paper fixes and what it leaves open
+//   * Units are column chunks of a linear weight matrix; every unit gets one of
+//     seven actions {16, 8, 4, 3, 2, 1.58, 1} (Eq. 3, "Action Space").
+//   * State features 0-4 and 9-11 are those of Table 1.
+//   * The engine fits a local scale per group (group = one row of one chunk,
+//     App. "Per-unit Scale Optimization") and scores it by reconstruction error
+//     (Sec. 3.5 "Quantization Engine and Bit Accounting").
+//   * Storage is counted in effective bits, b_bar = sum B_i / sum n_i (Eq. 6).
+//   The paper gives no formula for its quantizers.  The ones used here are the
+//   closed-form / grid-search readings listed beside each function; every such
+//   reading is marked "READING".
+//
+// Arithmetic model (READING; the paper is silent).  Every quantity that feeds
+// an integer code, a clip index or a stored fp16 value is a fixed sequence of
+// binary32 operations.  A sum over the G elements of a row-group is PSUM8:
+// leaves of 8 consecutive elements, each accumulated left to right from +0,
+// then combined by a balanced binary tree that adds adjacent leaves first.
+// Sums over rows (unit level) are taken in double and compared with tolerance.
+//
+// Pins (see tests/test_oracle_*.py): fp16 conversion against all 65536
+// patterns; PSUM8 order against hand-worked cancellation cases; 8-bit round
+// trip on grid values; brute-force clip search in float64 on tiny chunks;
+// ternary / binary closed forms and stationarity; scale invariance by powers of
+// two; degenerate groups; monotone error in bit-width; Eq. 6 bit arithmetic;
+// pack/unpack identity with an independent unpacker; nearest-rank P99 against a
+// full sort.  Parity unpinned: that threshold 0.7*mean|w| is a good ternary
+// threshold, and that these fits resemble the paper's Adam-fitted operators --
+// neither is claimed.
+
+#include <algorithm>
+#include <cmath>
+#include <cstdint>
+#include <cstring>
+#include <vector>
+
+namespace {
+
+// ---------------------------------------------------------------- fp16 <-> fp32
+inline uint32_t f32_bits(float f) { uint32_t u; std::memcpy(&u, &f, 4); return u; }
+inline float bits_f32(uint32_t u) { float f; std::memcpy(&f, &u, 4); return f; }
+
+// binary16 -> binary32, exact.
+float half_to_float(uint16_t h) {
+  const uint32_t sign = (uint32_t)(h & 0x8000u) << 16;
+  const uint32_t e = (h >> 10) & 31u;
+  const uint32_t m = h & 0x3ffu;
+  if (e == 0) {                                  // zero or subnormal: m * 2^-24
+    float v = (float)m * 5.9604644775390625e-08f;
+    return bits_f32(f32_bits(v) | sign);
+  }
+  if (e == 31) return bits_f32(sign | 0x7f800000u | (m << 13));
+  return bits_f32(sign | ((e + 112u) << 23) | (m << 13));
+}
+
+// binary32 -> binary16, round to nearest even, overflow to infinity.
+uint16_t float_to_half(float f) {
+  uint32_t x = f32_bits(f);
+  const uint16_t sign = (uint16_t)((x >> 16) & 0x8000u);
+  x &= 0x7fffffffu;
+  if (x > 0x7f800000u) return (uint16_t)(sign | 0x7e00u);            // NaN
+  if (x >= 0x477ff000u) return (uint16_t)(sign | 0x7c00u);           // >= 65520 -> inf
+  if (x < 0x38800000u) {                                              // below 2^-14
+    const float a = bits_f32(x) * 16777216.0f;                        // exact: units of 2^-24
+    const uint32_t m = (uint32_t)std::nearbyintf(a);                  // 0..1024, RNE
+    return (uint16_t)(sign | m);
+  }
+  const uint32_t odd = (x >> 13) & 1u;
+  x += 0xfffu + odd;
+  x -= 0x38000000u;
+  return (uint16_t)(sign | (x >> 13));
+}
+
+inline float round_through_half(float f) { return half_to_float(float_to_half(f)); }
+
+// ---------------------------------------------------------------- PSUM8
+// leaf(l) must return the left-to-right accumulation, from +0.0f, over the
+// elements 8l .. 8l+7.  G is 8 * 2^m.
+template <class Leaf>
+float psum8(int G, Leaf leaf) {
+  float node[64] = {0.0f};
+  const int nleaf = G / 8;
+  for (int l = 0; l < nleaf; ++l) node[l] = leaf(l);
+  for (int n = nleaf; n > 1; n /= 2)
+    for (int i = 0; i < n / 2; ++i) node[i] = node[2 * i] + node[2 * i + 1];
+  return node[0];
+}
+
+bool valid_group_width(int G) {
+  return G == 8 || G == 16 || G == 32 || G == 64 || G == 128 || G == 256 || G == 512;
+}
+
+// ---------------------------------------------------------------- constants
+const float kMagic = 12582912.0f;            // 1.5 * 2^23: adding it rounds to an integer (RNE)
+const int kUniformBits[4] = {8, 4, 3, 2};    // order of the bit-width columns 0..3
+// columns of every per-bit-width table: 0:8  1:4  2:3  3:2  4:1.58 (ternary)  5:1 (binary)
+// action codes (Eq. 3 order): 0 skip(16)  1:8  2:4  3:3  4:2  5:1.58  6:1
+
+// ---------------------------------------------------------------- one row-group
+struct Group {
+  int G;
+  const float* w;   // G weights of one row inside one unit, converted from fp16
+  const float* s;   // G activation statistics of the unit's input channels
+};
+
+struct UniformParams {
+  float scale;      // value of the stored fp16 scale (1.0 if it rounded to zero)
+  float inv;        // 1 / scale, IEEE division
+  float zf;         // integer zero point as a float, in [0, qmax]
+  float qmaxf;
+};
+
+// READING: asymmetric uniform grid over [p*mn, p*mx] with zero forced into the
+// range (mn <= 0 <= mx), scale rounded to fp16 before it is used, integer
+// zero point.
+UniformParams uniform_params(float mn, float rng, float p, int bits) {
+  UniformParams u;
+  const int qmax = (1 << bits) - 1;
+  u.qmaxf = (float)qmax;
+  const float rq = (float)(1.0 / (double)qmax);
+  const float scale32 = (p * rng) * rq;
+  u.scale = round_through_half(scale32);
+  if (u.scale == 0.0f) u.scale = 1.0f;
+  u.inv = 1.0f / u.scale;
+  float z = std::nearbyintf(std::fabs(p * mn) * u.inv);   // mn <= 0: |p*mn| = -(p*mn), and never -0
+  if (z < 0.0f) z = 0.0f;
+  if (z > u.qmaxf) z = u.qmaxf;
+  u.zf = z;
+  return u;
+}
+
+// c = q - z, the zero-centred integer code as a float.
+inline float centred_code(float w, const UniformParams& u) {
+  const float r = std::fmaf(w, u.inv, kMagic);   // nearest-even integer of the exact product
+  float c = r - kMagic;
+  const float lo = 0.0f - u.zf, hi = u.qmaxf - u.zf;    // 0 - 0 = +0: no negative zero codes
+  if (c < lo) c = lo;
+  if (c > hi) c = hi;
+  return c;
+}
+
+// s-weighted squared reconstruction error of one uniform candidate.
+float uniform_error(const Group& g, const UniformParams& u) {
+  return psum8(g.G, [&](int l) {
+    float acc = 0.0f;
+    for (int j = 8 * l; j < 8 * l + 8; ++j) {
+      const float c = centred_code(g.w[j], u);
+      const float d = std::fmaf(c, u.scale, -g.w[j]);
+      const float t = g.s[j] * d;
+      acc = std::fmaf(t, d, acc);
+    }
+    return acc;
+  });
+}
+
+void group_range(const Group& g, float* mn, float* rng) {
+  float lo = 0.0f, hi = 0.0f;
+  for (int j = 0; j < g.G; ++j) {
+    if (g.w[j] < lo) lo = g.w[j];
+    if (g.w[j] > hi) hi = g.w[j];
+  }
+  *mn = lo;
+  *rng = hi - lo;
+}
+
+// Clip search for one bit-width: smallest k with minimal error (strict '<').
+void search_uniform(const Group& g, float mn, float rng, int bits, const float* clip, int K,
+                    int* best_k, float* best_e) {
+  int bk = 0;
+  float be = 0.0f;
+  for (int k = 0; k < K; ++k) {
+    const UniformParams u = uniform_params(mn, rng, clip[k], bits);
+    const float e = uniform_error(g, u);
+    if (k == 0 || e < be) { be = e; bk = k; }
+  }
+  *best_k = bk;
+  *best_e = be;
+}
+
+float sum_abs(const Group& g) {
+  return psum8(g.G, [&](int l) {
+    float acc = 0.0f;
+    for (int j = 8 * l; j < 8 * l + 8; ++j) acc = acc + std::fabs(g.w[j]);
+    return acc;
+  });
+}
+
+float error_against(const Group& g, const float* what) {   // what[j] = reconstructed weight
+  return psum8(g.G, [&](int l) {
+    float acc = 0.0f;
+    for (int j = 8 * l; j < 8 * l + 8; ++j) {
+      const float d = what[j] - g.w[j];
+      const float t = g.s[j] * d;
+      acc = std::fmaf(t, d, acc);
+    }
+    return acc;
+  });
+}
+
+// READING: ternary = threshold 0.7 * mean|w| (textbook ternary weights), one
+// scale alpha = s-weighted mean of |w| on the support, stored in fp16.
+// trit[j] in {0,1,2} = 1 + sign(w_j) on the support, 1 elsewhere.
+float fit_ternary(const Group& g, float A, uint8_t* trit /*nullable*/, float* what /*nullable*/) {
+  const int G = g.G;
+  const float delta = 0.7f * (A * (1.0f / (float)G));
+  bool any = false;
+  std::vector<uint8_t> in(G);
+  for (int j = 0; j < G; ++j) { in[j] = std::fabs(g.w[j]) > delta; any = any || in[j]; }
+  float B = psum8(G, [&](int l) {
+    float acc = 0.0f;
+    for (int j = 8 * l; j < 8 * l + 8; ++j) acc = std::fmaf(g.s[j], in[j] ? std::fabs(g.w[j]) : 0.0f, acc);
+    return acc;
+  });
+  float Cs = psum8(G, [&](int l) {
+    float acc = 0.0f;
+    for (int j = 8 * l; j < 8 * l + 8; ++j) acc = acc + (in[j] ? g.s[j] : 0.0f);
+    return acc;
+  });
+  if (Cs == 0.0f) {               // no activation weight on the support: fit with s == 1
+    B = psum8(G, [&](int l) {
+      float acc = 0.0f;
+      for (int j = 8 * l; j < 8 * l + 8; ++j) acc = std::fmaf(1.0f, in[j] ? std::fabs(g.w[j]) : 0.0f, acc);
+      return acc;
+    });
+    Cs = psum8(G, [&](int l) {
+      float acc = 0.0f;
+      for (int j = 8 * l; j < 8 * l + 8; ++j) acc = acc + (in[j] ? 1.0f : 0.0f);
+      return acc;
+    });
+  }
+  const float alpha = any ? round_through_half(B / Cs) : 0.0f;
+  for (int j = 0; j < G; ++j) {
+    const int t = in[j] ? (g.w[j] < 0.0f ? 0 : 2) : 1;
+    if (trit) trit[j] = (uint8_t)t;
+    if (what) what[j] = (float)(t - 1) * alpha;
+  }
+  return alpha;
+}
+
+// READING: binary = sign(w) * alpha, alpha = s-weighted mean |w| in fp16;
+// sign(0) = +.  bit[j] = !(w_j < 0).
+float fit_binary(const Group& g, float A, uint8_t* bit /*nullable*/, float* what /*nullable*/) {
+  const int G = g.G;
+  const float B = psum8(G, [&](int l) {
+    float acc = 0.0f;
+    for (int j = 8 * l; j < 8 * l + 8; ++j) acc = std::fmaf(g.s[j], std::fabs(g.w[j]), acc);
+    return acc;
+  });
+  const float Cs = psum8(G, [&](int l) {
+    float acc = 0.0f;
+    for (int j = 8 * l; j < 8 * l + 8; ++j) acc = acc + g.s[j];
+    return acc;
+  });
+  const float alpha = round_through_half(Cs == 0.0f ? A * (1.0f / (float)G) : B / Cs);
+  for (int j = 0; j < G; ++j) {
+    const int b = !(g.w[j] < 0.0f);
+    if (bit) bit[j] = (uint8_t)b;
+    if (what) what[j] = b ? alpha : -alpha;
+  }
+  return alpha;
+}
+
+void load_group(const uint16_t* W, int64_t ldw, int64_t r, int64_t u, int G, float* w) {
+  const uint16_t* p = W + r * ldw + u * (int64_t)G;
+  for (int j = 0; j < G; ++j) w[j] = half_to_float(p[j]);
+}
+
+// ---------------------------------------------------------------- packing
+int64_t group_code_bytes(int action, int G) {
+  switch (action) {
+    case 0: return 2 * (int64_t)G;
+    case 1: return G;
+    case 2: return G / 2;
+    case 3: return 3 * (int64_t)G / 8;
+    case 4: return G / 4;
+    case 5: return (G + 4) / 5;
+    case 6: return G / 8;
+  }
+  return -1;
+}
+
+int64_t round_up16(int64_t x) { return (x + 15) / 16 * 16; }
+
+// codes[j] -> bytes of one row-group.  Little-endian inside a byte.
+void pack_group(int action, int G, const uint8_t* q, uint8_t* out) {
+  const int64_t nb = group_code_bytes(action, G);
+  std::memset(out, 0, (size_t)nb);
+  switch (action) {
+    case 1: for (int j = 0; j < G; ++j) out[j] = q[j]; break;
+    case 2: for (int j = 0; j < G; ++j) out[j / 2] |= (uint8_t)(q[j] << (4 * (j % 2))); break;
+    case 3:
+      for (int j = 0; j < G; ++j)
+        for (int t = 0; t < 3; ++t)
+          if ((q[j] >> t) & 1) { const int pos = 3 * j + t; out[pos / 8] |= (uint8_t)(1u << (pos % 8)); }
+      break;
+    case 4: for (int j = 0; j < G; ++j) out[j / 4] |= (uint8_t)(q[j] << (2 * (j % 4))); break;
+    case 5: {
+      const int pow3[5] = {1, 3, 9, 27, 81};
+      for (int j = 0; j < G; ++j) out[j / 5] = (uint8_t)(out[j / 5] + q[j] * pow3[j % 5]);
+      break;
+    }
+    case 6: for (int j = 0; j < G; ++j) out[j / 8] |= (uint8_t)(q[j] << (j % 8)); break;
+  }
+}
+
+int64_t unit_centibits(int action, int64_t R, int G, int scale_bits, int zero_bits) {
+  const int64_t n = R * (int64_t)G;
+  switch (action) {
+    case 0: return 1600 * n;
+    case 1: return 800 * n + R * 100 * (int64_t)(scale_bits + zero_bits);
+    case 2: return 400 * n + R * 100 * (int64_t)(scale_bits + zero_bits);
+    case 3: return 300 * n + R * 100 * (int64_t)(scale_bits + zero_bits);
+    case 4: return 200 * n + R * 100 * (int64_t)(scale_bits + zero_bits);
+    case 5: return 158 * n + R * 100 * (int64_t)scale_bits;
+    case 6: return 100 * n + R * 100 * (int64_t)scale_bits;
+  }
+  return -1;
+}
+
+}  // namespace
+
+extern "C" {
+
+// ---- helpers exported only so that the tests can pin them -------------------
+float oracle_half_to_float(uint16_t h) { return half_to_float(h); }
+uint16_t oracle_float_to_half(float f) { return float_to_half(f); }
+// PSUM8 of x[0..G) with plain addition in the leaves.
+float oracle_psum8(const float* x, int G) {
+  if (!valid_group_width(G)) return NAN;
+  return psum8(G, [&](int l) {
+    float acc = 0.0f;
+    for (int j = 8 * l; j < 8 * l + 8; ++j) acc = acc + x[j];
+    return acc;
+  });
+}
+// One uniform candidate on one group: scale, zero, error, codes (for the pins).
+int oracle_uniform_candidate(const float* w, const float* s, int G, int bits, float p,
+                             float* scale, float* zero, float* err, uint8_t* codes /*nullable*/) {
+  if (!valid_group_width(G) || bits < 1 || bits > 8) return 1;
+  Group g{G, w, s};
+  float mn, rng;
+  group_range(g, &mn, &rng);
+  const UniformParams u = uniform_params(mn, rng, p, bits);
+  *scale = u.scale;
+  *zero = u.zf;
+  *err = uniform_error(g, u);
+  if (codes) for (int j = 0; j < G; ++j) codes[j] = (uint8_t)(int)(centred_code(w[j], u) + u.zf);
+  return 0;
+}
+
+// ---- a1: activation statistics (calibration forward pass, App. "Salient Weight
+// Protection": per-channel activation scale).  READING: s_j = mean_t x_tj^2.
+int oracle_act_stats(const uint16_t* X, int64_t T, int64_t C, int64_t ldx, float* s_out) {
+  if (!X || !s_out || T <= 0 || C <= 0 || ldx < C) return 1;
+  for (int64_t j = 0; j < C; ++j) {
+    double acc = 0.0;
+    for (int64_t t = 0; t < T; ++t) {
+      const double x = (double)half_to_float(X[t * ldx + j]);
+      acc += x * x;
+    }
+    s_out[j] = (float)(acc / (double)T);
+  }
+  return 0;
+}
+
+// ---- a2: Table 1, dims 0-4 and 9-11, for every unit.
+// feat[u] = {mean, std, abs_mean, sparsity, outlier_frac, s_mean, s_std, s_max}.
+// READING: population std; nearest-rank P99 (k = ceil(0.99 n), 1-indexed).
+int oracle_unit_features(const uint16_t* W, int64_t R, int64_t C, int64_t ldw, int G, const float* s,
+                         float* feat_out) {
+  if (!W || !s || !feat_out || R <= 0 || C <= 0 || G <= 0 || C % G != 0 || ldw < C) return 1;
+  const int64_t U = C / G;
+  const int64_t n = R * (int64_t)G;
+  std::vector<float> a((size_t)n);
+  for (int64_t u = 0; u < U; ++u) {
+    double sum = 0.0, sum_abs_w = 0.0;
+    int64_t tiny = 0;
+    for (int64_t r = 0; r < R; ++r)
+      for (int j = 0; j < G; ++j) {
+        const float w = half_to_float(W[r * ldw + u * G + j]);
+        const float aw = std::fabs(w);
+        a[(size_t)(r * G + j)] = aw;
+        sum += (double)w;
+        sum_abs_w += (double)aw;
+        if (aw < 1e-6f) ++tiny;
+      }
+    const double mean = sum / (double)n;
+    double var = 0.0;
+    for (int64_t r = 0; r < R; ++r)
+      for (int j = 0; j < G; ++j) {
+        const double d = (double)half_to_float(W[r * ldw + u * G + j]) - mean;
+        var += d * d;
+      }
+    var /= (double)n;
+    const int64_t k = (99 * n + 99) / 100;                       // ceil(0.99 n)
+    std::vector<float> sorted(a);
+    std::sort(sorted.begin(), sorted.end());
+    const float p99 = sorted[(size_t)(k - 1)];
+    const float thr = 0.5f * p99;
+    int64_t outl = 0;
+    for (int64_t i = 0; i < n; ++i) if (a[(size_t)i] > thr) ++outl;
+
+    double ssum = 0.0, smax = (double)s[u * G];
+    for (int j = 0; j < G; ++j) { ssum += (double)s[u * G + j]; smax = std::max(smax, (double)s[u * G + j]); }
+    const double smean = ssum / (double)G;
+    double svar = 0.0;
+    for (int j = 0; j < G; ++j) { const double d = (double)s[u * G + j] - smean; svar += d * d; }
+    svar /= (double)G;
+
+    float* f = feat_out + u * 8;
+    f[0] = (float)mean;
+    f[1] = (float)std::sqrt(var);
+    f[2] = (float)(sum_abs_w / (double)n);
+    f[3] = (float)((double)tiny / (double)n);
+    f[4] = (float)((double)outl / (double)n);
+    f[5] = (float)smean;
+    f[6] = (float)std::sqrt(svar);
+    f[7] = (float)smax;
+  }
+  return 0;
+}
+
+// ---- a3: fit every row-group of units [u_begin, u_end) under all six bit-widths.
+// err_out[U][6], energy_out[U] (nullable), clip_idx_out[4][U][R] (nullable),
+// group_err_out[6][U][R] (nullable).  Only rows of the requested units are written.
+int oracle_fit_eval(const uint16_t* W, int64_t R, int64_t C, int64_t ldw, int G, const float* s,
+                    const float* clip_grid, int K, int64_t u_begin, int64_t u_end, float* err_out,
+                    float* energy_out, uint8_t* clip_idx_out, float* group_err_out) {
+  if (!W || !s || !clip_grid || !err_out || R <= 0 || C <= 0 || !valid_group_width(G) || C % G != 0 ||
+      ldw < C || K < 1 || K > 64)
+    return 1;
+  const int64_t U = C / G;
+  if (u_begin < 0 || u_end > U || u_begin > u_end) return 1;
+  std::vector<float> w((size_t)G), what((size_t)G);
+  for (int64_t u = u_begin; u < u_end; ++u) {
+    double tot[6] = {0, 0, 0, 0, 0, 0};
+    double energy = 0.0;
+    const float* su = s + u * G;
+    for (int64_t r = 0; r < R; ++r) {
+      load_group(W, ldw, r, u, G, w.data());
+      Group g{G, w.data(), su};
+      float e[6];
+      float mn, rng;
+      group_range(g, &mn, &rng);
+      for (int bi = 0; bi < 4; ++bi) {
+        int bk;
+        search_uniform(g, mn, rng, kUniformBits[bi], clip_grid, K, &bk, &e[bi]);
+        if (clip_idx_out) clip_idx_out[((int64_t)bi * U + u) * R + r] = (uint8_t)bk;
+      }
+      const float A = sum_abs(g);
+      fit_ternary(g, A, nullptr, what.data());
+      e[4] = error_against(g, what.data());
+      fit_binary(g, A, nullptr, what.data());
+      e[5] = error_against(g, what.data());
+      for (int b = 0; b < 6; ++b) {
+        tot[b] += (double)e[b];
+        if (group_err_out) group_err_out[((int64_t)b * U + u) * R + r] = e[b];
+      }
+      for (int j = 0; j < G; ++j) energy += (double)su[j] * (double)w[j] * (double)w[j];
+    }
+    for (int b = 0; b < 6; ++b) err_out[u * 6 + b] = (float)tot[b];
+    if (energy_out) energy_out[u] = (float)energy;
+  }
+  return 0;
+}
+
+// ---- a5: effective bits (Eq. 6 with no protected weights, extended by the
+// per-group scale / zero-point overhead) in integer centibits, plus the byte
+// offset of every unit's packed block (each rounded up to 16 bytes).
+int oracle_effective_bits(const uint8_t* actions, int64_t U, int64_t R, int G, int scale_bits,
+                          int zero_bits, int64_t* unit_centibits_out, int64_t* code_offsets_out,
+                          int64_t* total_centibits_out, int64_t* total_packed_bytes_out) {
+  if (!actions || U <= 0 || R <= 0 || G <= 0 || scale_bits < 0 || zero_bits < 0) return 1;
+  int64_t total = 0, off = 0, n_scales = 0, n_zeros = 0;
+  for (int64_t u = 0; u < U; ++u) {
+    const int a = actions[u];
+    if (a > 6) return 1;
+    const int64_t cb = unit_centibits(a, R, G, scale_bits, zero_bits);
+    if (unit_centibits_out) unit_centibits_out[u] = cb;
+    total += cb;
+    if (code_offsets_out) code_offsets_out[u] = off;
+    off += round_up16(R * group_code_bytes(a, G));
+    if (a >= 1) n_scales += R;
+    if (a >= 1 && a <= 4) n_zeros += R;
+  }
+  if (code_offsets_out) code_offsets_out[U] = off;
+  if (total_centibits_out) *total_centibits_out = total;
+  if (total_packed_bytes_out) *total_packed_bytes_out = off + 2 * (n_scales + n_zeros);
+  return 0;
+}
+
+// ---- a4: apply a plan.  codes_out must hold code_offsets[U] bytes and is fully
+// written (padding = 0); scales_out / zeros_out are fp16 [U][R]; Wq_out is
+// fp16 [R][ldw] (nullable).  clip_idx [4][U][R] may be null: the clip search is
+// then repeated for the chosen bit-width.
+int oracle_apply_plan(const uint16_t* W, int64_t R, int64_t C, int64_t ldw, int G, const float* s,
+                      const float* clip_grid, int K, const uint8_t* actions, const uint8_t* clip_idx,
+                      const int64_t* code_offsets, uint8_t* codes_out, uint16_t* scales_out,
+                      uint16_t* zeros_out, uint16_t* Wq_out) {
+  if (!W || !s || !clip_grid || !actions || !code_offsets || !codes_out || !scales_out || !zeros_out ||
+      R <= 0 || C <= 0 || !valid_group_width(G) || C % G != 0 || ldw < C || K < 1 || K > 64)
+    return 1;
+  const int64_t U = C / G;
+  std::memset(codes_out, 0, (size_t)code_offsets[U]);
+  std::vector<float> w((size_t)G), what((size_t)G);
+  std::vector<uint8_t> q((size_t)G);
+  for (int64_t u = 0; u < U; ++u) {
+    const int a = actions[u];
+    if (a > 6) return 1;
+    const float* su = s + u * G;
+    const int64_t gb = group_code_bytes(a, G);
+    for (int64_t r = 0; r < R; ++r) {
+      uint8_t* dst = codes_out + code_offsets[u] + r * gb;
+      uint16_t scale_h = 0, zero_h = 0;
+      if (a == 0) {
+        std::memcpy(dst, W + r * ldw + u * G, (size_t)(2 * G));
+        if (Wq_out) std::memcpy(Wq_out + r * ldw + u * G, W + r * ldw + u * G, (size_t)(2 * G));
+      } else {
+        load_group(W, ldw, r, u, G, w.data());
+        Group g{G, w.data(), su};
+        if (a <= 4) {
+          const int bi = a - 1, bits = kUniformBits[bi];
+          float mn, rng;
+          group_range(g, &mn, &rng);
+          int k;
+          if (clip_idx) {
+            k = clip_idx[((int64_t)bi * U + u) * R + r];
+            if (k >= K) return 1;
+          } else {
+            float e;
+            search_uniform(g, mn, rng, bits, clip_grid, K, &k, &e);
+          }
+          const UniformParams p = uniform_params(mn, rng, clip_grid[k], bits);
+          for (int j = 0; j < G; ++j) {
+            const float c = centred_code(w[j], p);
+            q[j] = (uint8_t)(int)(c + p.zf);
+            what[j] = c * p.scale;
+          }
+          scale_h = float_to_half(p.scale);
+          zero_h = float_to_half(p.zf);
+        } else {
+          const float A = sum_abs(g);
+          const float alpha = (a == 5) ? fit_ternary(g, A, q.data(), what.data())
+                                       : fit_binary(g, A, q.data(), what.data());
+          scale_h = float_to_half(alpha);
+        }
+        pack_group(a, G, q.data(), dst);
+        if (Wq_out)
+          for (int j = 0; j < G; ++j) Wq_out[r * ldw + u * G + j] = float_to_half(what[j]);
+      }
+      scales_out[u * R + r] = scale_h;
+      zeros_out[u * R + r] = zero_h;
+    }
+  }
+  return 0;
+}
+
+}  // extern "C"

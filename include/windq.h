@@ -1,0 +1,157 @@
+/* windq -- scoring and fitting hot path of WINDQuant-style mixed-precision allocation,
+ * CUDA (sm_100a) library with a C ABI.
+ *
+ * The paper's PPO controller gives every column-chunk *unit* of every linear weight matrix one
+ * of seven actions (Eq. 3, "Action Space"): skip (keep fp16) or quantize at 8, 4, 3, 2, 1.58 or
+ * 1 bit.  This library computes what the controller needs in order to score units and actions:
+ * calibration statistics, per-unit state features (Table 1), per-group quantizer fits under all
+ * six bit-widths with their reconstruction errors (Sec. 3.5 "Quantization Engine and Bit
+ * Accounting", App. "Per-unit Scale Optimization"), the application of a chosen plan, and
+ * effective-bit accounting (Eq. 6).  The policy, the perplexity proxy and the model forward
+ * are consumers and stay outside.
+ *
+ * Conventions (all calls)
+ *   - A linear weight is W[R][C], fp16 (IEEE binary16), row-major with leading dimension ldw
+ *     (elements): R = out features, C = in features.  Unit u = columns [u*G, (u+1)*G) of all R
+ *     rows; U = C / G.  A *group* (r, u) is the G contiguous values of row r in unit u; it
+ *     carries one scale (and one zero point).
+ *   - Action codes follow Eq. 3: 0 = skip(16)  1 = 8  2 = 4  3 = 3  4 = 2  5 = 1.58  6 = 1.
+ *     Per-bit-width tables have six columns in the order [8, 4, 3, 2, 1.58, 1].
+ *   - Every data pointer is a DEVICE pointer owned by the caller, unless it says "host".
+ *     Nothing is retained after a call.  `stream` is a cudaStream_t passed as void* (NULL = the
+ *     legacy default stream).  Calls only enqueue work on `stream`; outputs are valid once the
+ *     stream has reached that point.  The library allocates no outputs.  It owns a scratch
+ *     buffer inside the context, grown (cudaMalloc, which synchronises) only when a call needs
+ *     more than it has; windq_reserve sizes it ahead of time.
+ *   - Errors: every argument check happens on the host before anything is launched; a failing
+ *     call launches nothing and returns a status, and windq_last_error gives the reason.  There
+ *     are no exceptions, aborts or device traps.  Inputs must be finite; NaN / Inf give
+ *     unspecified values, never a fault.  A context must not be used from two threads at once.
+ *   - Pointers to fp16 / fp32 / int64 arrays must be 16-byte aligned (any cudaMalloc or torch
+ *     allocation is); ldw and ldx must be multiples of 8.
+ *   - G must be one of 32, 64, 128, 256, 512; C a multiple of G; 1 <= K <= 64; clip ratios in
+ *     [1/64, 1].
+ */
+#ifndef WINDQ_H_
+#define WINDQ_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct windq_ctx windq_ctx; /* opaque: device id, SM count, scratch, last error */
+
+typedef enum {
+  WINDQ_OK = 0,
+  WINDQ_ERR_NULL = 1,        /* a required pointer is NULL */
+  WINDQ_ERR_SHAPE = 2,       /* a size is <= 0, C % G != 0, ld < C, ... */
+  WINDQ_ERR_ALIGN = 3,       /* a pointer or leading dimension is misaligned */
+  WINDQ_ERR_ARG = 4,         /* G, K, a clip ratio or a bit count is out of range */
+  WINDQ_ERR_SCRATCH = 5,     /* the scratch buffer could not be grown */
+  WINDQ_ERR_CUDA = 6,        /* a CUDA runtime call or a launch failed */
+  WINDQ_ERR_UNSUPPORTED = 7  /* the device is not an sm_100 GPU */
+} windq_status;
+
+#define WINDQ_N_BITWIDTHS 6
+#define WINDQ_N_FEATURES 8
+
+/* Creates a context on CUDA device `device` (the caller's current device is left unchanged).
+ * *out receives the context (host memory, freed by windq_destroy). */
+windq_status windq_create(windq_ctx** out, int device);
+void windq_destroy(windq_ctx* ctx);
+
+/* Reason of the last failing call on this context (or of the last failing windq_create when ctx
+ * is NULL).  The string is owned by the library and stays valid until the next call. */
+const char* windq_last_error(const windq_ctx* ctx);
+
+/* Grows the context's scratch buffer to at least `bytes` now (synchronises the device), so that
+ * later calls do not allocate.  windq_scratch_bytes_* tell how much a call will need. */
+windq_status windq_reserve(windq_ctx* ctx, int64_t bytes);
+int64_t windq_scratch_bytes_act_stats(int64_t T, int64_t C);
+int64_t windq_scratch_bytes_unit_features(int64_t R, int64_t C, int G);
+int64_t windq_scratch_bytes_fit_eval(int64_t R, int64_t C, int G);
+
+/* a1 -- activation statistics of one calibration input (App. "Salient Weight Protection":
+ * per-channel activation scale estimated during a calibration forward pass; Table 1 dims 9-11).
+ *   s_out[j] = (1/T) * sum_t X[t][j]^2,  j < C.
+ * X: fp16 [T][ldx] (T tokens, C channels, ldx >= C); s_out: fp32 [C].  C % 8 == 0. */
+windq_status windq_act_stats(windq_ctx* ctx, const void* X, int64_t T, int64_t C, int64_t ldx,
+                             float* s_out, void* stream);
+
+/* a2 -- state features of every unit (Table 1, dims 0-4 and 9-11).
+ *   feat_out[u] = { mean, std, abs_mean, sparsity, outlier_frac, mean(s), std(s), max(s) }
+ * over the R*G weights of unit u and the G statistics s[u*G .. (u+1)*G).  std is the population
+ * standard deviation; sparsity = #{|w| < 1e-6} / n; outlier_frac = #{|w| > 0.5 * P99} / n with
+ * P99 the ceil(0.99 n)-th smallest |w| (nearest rank).  Both counts are exact.
+ * W: fp16 [R][ldw]; s: fp32 [C]; feat_out: fp32 [U][8]. */
+windq_status windq_unit_features(windq_ctx* ctx, const void* W, int64_t R, int64_t C, int64_t ldw,
+                                 int G, const float* s, float* feat_out, void* stream);
+
+/* a3 -- fit every group under all six bit-widths and score each fit by its s-weighted squared
+ * reconstruction error  e = sum_j s_j (w_j - w^_j)^2  (Sec. 3.5: local scale fitting per unit,
+ * judged by reconstruction error; App.: group size = chunk size).
+ *   8/4/3/2 bit: asymmetric uniform grid over [p*mn, p*mx] (mn = min(0, min w), mx = max(0, max
+ *     w)), scale rounded to fp16, integer zero point; every clip ratio p = clip_grid[k] is tried
+ *     and the smallest k with the least error kept.
+ *   1.58 bit: threshold 0.7 * mean|w|, one fp16 scale = s-weighted mean |w| on the support.
+ *   1 bit: sign(w) times one fp16 scale = s-weighted mean |w|.
+ * Outputs:
+ *   err_out      fp32 [U][6]     sum over rows of the best error, per bit-width
+ *   energy_out   fp32 [U]        sum_r sum_j s_j w_rj^2 (error of "quantize to zero"); nullable
+ *   clip_idx_out u8   [4][U][R]  best clip index for 8, 4, 3, 2 bit; nullable
+ *   group_err_out fp32 [6][U][R] best error of every group; nullable
+ * clip_grid: fp32 [K] (device).  Group-level results (clip indices, group errors) are
+ * bit-reproducible: every operation is a fixed IEEE binary32 sequence. */
+windq_status windq_fit_eval(windq_ctx* ctx, const void* W, int64_t R, int64_t C, int64_t ldw, int G,
+                            const float* s, const float* clip_grid, int K, float* err_out,
+                            float* energy_out, uint8_t* clip_idx_out, float* group_err_out,
+                            void* stream);
+
+/* a5 -- effective bits of a plan for one matrix (Eq. 6 with no protected weights, extended by
+ * the per-group scale / zero-point overhead), in integer centibits (1 bit = 100), and the byte
+ * offsets of the packed code blocks that windq_apply_plan writes.  With n = R*G:
+ *   skip: 1600 n;  b in {8,4,3,2}: 100 b n + 100 R (scale_bits + zero_bits);
+ *   1.58: 158 n + 100 R scale_bits;  1: 100 n + 100 R scale_bits.
+ * Bytes of one packed group: skip 2G, 8-bit G, 4-bit G/2, 3-bit 3G/8, 2-bit G/4, 1.58-bit
+ * ceil(G/5), 1-bit G/8.  A unit's block holds its R groups in row order; every block starts on a
+ * 16-byte boundary.
+ *   actions               u8  [U]    action code per unit (device)
+ *   unit_centibits_out    i64 [U]    nullable
+ *   code_offsets_out      i64 [U+1]  byte offset of every block, [U] = total code bytes; nullable
+ *   total_centibits_out   i64 [1]    sum over units; average bits = total / (100 * U * R * G)
+ *   total_packed_bytes_out i64 [1]   code bytes + 2 bytes per stored scale and zero point; nullable
+ * An action code above 6 makes both totals -1 (the per-unit entry is -1, its block empty).
+ * scale_bits and zero_bits must be in [0, 64]. */
+windq_status windq_effective_bits(windq_ctx* ctx, const uint8_t* actions, int64_t U, int64_t R, int G,
+                                  int scale_bits, int zero_bits, int64_t* unit_centibits_out,
+                                  int64_t* code_offsets_out, int64_t* total_centibits_out,
+                                  int64_t* total_packed_bytes_out, void* stream);
+
+/* a4 -- apply a plan to one matrix ("the environment applies the selected quantization to the
+ * current unit"): integer codes packed as described above, the fp16 scale and zero point of
+ * every group, and optionally the fake-quantised weights for the consumer's forward pass.
+ *   actions      u8  [U]          action per unit
+ *   clip_idx     u8  [4][U][R]    clip indices from windq_fit_eval, or NULL: the clip search is
+ *                                 repeated for the chosen bit-width (same result, more work).
+ *                                 An index >= K is treated as K-1.
+ *   code_offsets i64 [U+1]        from windq_effective_bits for the same actions, R and G
+ *   codes_out    u8  [code_offsets[U]]  every byte is written (padding = 0)
+ *   scales_out   fp16 [U][R]      scale (alpha for 1.58 / 1 bit, 0 for skip)
+ *   zeros_out    fp16 [U][R]      integer zero point (0 for 1.58 / 1 bit and skip)
+ *   Wq_out       fp16 [R][ldw]    fake-quantised weights, nullable; must not alias W
+ * Packing inside a group, little-endian within a byte: 8-bit byte j = q_j; 4-bit byte i = q_2i |
+ * q_2i+1 << 4; 3-bit: a bit stream, code j at bits [3j, 3j+3); 2-bit byte i = sum q_4i+m << 2m;
+ * 1.58-bit byte i = sum_{m<5} t_5i+m 3^m with trits t = 1 + sign(w) on the support, 1 elsewhere;
+ * 1-bit byte i = sum bit_8i+m << m with bit = !(w < 0); skip: the raw fp16 bytes.
+ * Units whose action code is above 6 are left unwritten.  codes_out must be 16-byte aligned. */
+windq_status windq_apply_plan(windq_ctx* ctx, const void* W, int64_t R, int64_t C, int64_t ldw, int G,
+                              const float* s, const float* clip_grid, int K, const uint8_t* actions,
+                              const uint8_t* clip_idx, const int64_t* code_offsets, uint8_t* codes_out,
+                              void* scales_out, void* zeros_out, void* Wq_out, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* WINDQ_H_ */

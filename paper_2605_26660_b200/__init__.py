@@ -1,0 +1,261 @@
+"""Python binding of the windq CUDA library (argument marshalling only).
+
+Every function below has the name of the C-ABI entry point it calls
+(``include/windq.h``) and does nothing but check tensor types, allocate output
+tensors with torch, pass raw device pointers and the current CUDA stream, and
+turn a non-zero status into ``WindqError``.  All arithmetic happens in the CUDA
+kernels.  There is no CPU fallback: if the shared library is missing and cannot
+be built, importing this package raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+from . import _build
+
+N_BITWIDTHS = 6     # columns of per-bit-width tables: 8, 4, 3, 2, 1.58, 1
+N_FEATURES = 8
+ACTION_BITS = (16.0, 8.0, 4.0, 3.0, 2.0, 1.58, 1.0)   # action code -> nominal bits (Eq. 3)
+
+STATUS_NAMES = {0: "OK", 1: "ERR_NULL", 2: "ERR_SHAPE", 3: "ERR_ALIGN", 4: "ERR_ARG", 5: "ERR_SCRATCH",
+                6: "ERR_CUDA", 7: "ERR_UNSUPPORTED"}
+
+
+class WindqError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        super().__init__("windq status %d (%s): %s" % (status, STATUS_NAMES.get(status, "?"), message))
+        self.status = status
+
+
+def _load() -> ctypes.CDLL:
+    try:
+        path = _build.build()
+    except Exception as exc:  # no nvcc, or a compile error
+        if os.path.exists(_build.LIB):
+            path = _build.LIB   # a library built elsewhere travelled with the tree
+        else:
+            raise ImportError("the windq CUDA library is not built and cannot be built here: %s" % exc) from exc
+    lib = ctypes.CDLL(path)
+    i64, i32, vp = ctypes.c_int64, ctypes.c_int, ctypes.c_void_p
+    lib.windq_create.argtypes = [ctypes.POINTER(vp), i32]
+    lib.windq_destroy.argtypes = [vp]
+    lib.windq_destroy.restype = None
+    lib.windq_last_error.argtypes = [vp]
+    lib.windq_last_error.restype = ctypes.c_char_p
+    lib.windq_reserve.argtypes = [vp, i64]
+    for name in ("windq_scratch_bytes_act_stats",):
+        getattr(lib, name).argtypes = [i64, i64]
+        getattr(lib, name).restype = i64
+    for name in ("windq_scratch_bytes_unit_features", "windq_scratch_bytes_fit_eval"):
+        getattr(lib, name).argtypes = [i64, i64, i32]
+        getattr(lib, name).restype = i64
+    lib.windq_act_stats.argtypes = [vp, vp, i64, i64, i64, vp, vp]
+    lib.windq_unit_features.argtypes = [vp, vp, i64, i64, i64, i32, vp, vp, vp]
+    lib.windq_fit_eval.argtypes = [vp, vp, i64, i64, i64, i32, vp, vp, i32, vp, vp, vp, vp, vp]
+    lib.windq_effective_bits.argtypes = [vp, vp, i64, i64, i32, i32, i32, vp, vp, vp, vp, vp]
+    lib.windq_apply_plan.argtypes = [vp, vp, i64, i64, i64, i32, vp, vp, i32, vp, vp, vp, vp, vp, vp, vp, vp]
+    return lib
+
+
+_lib = _load()
+LIBRARY_PATH = _build.LIB
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream=None):
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream)
+
+
+def _need(t: torch.Tensor, dtype, name: str, dims=None):
+    if not isinstance(t, torch.Tensor) or not t.is_cuda:
+        raise TypeError("%s must be a CUDA tensor" % name)
+    if t.dtype != dtype:
+        raise TypeError("%s must be %s, got %s" % (name, dtype, t.dtype))
+    if dims is not None and t.dim() != dims:
+        raise ValueError("%s must have %d dimensions" % (name, dims))
+    return t
+
+
+def _matrix(t: torch.Tensor, name: str):
+    _need(t, torch.float16, name, 2)
+    if t.stride(1) != 1:
+        raise ValueError("%s must be row-major (unit stride along columns)" % name)
+    return t.shape[0], t.shape[1], t.stride(0)
+
+
+class Context:
+    """Owns a ``windq_ctx`` on one CUDA device."""
+
+    def __init__(self, device: int | None = None):
+        if device is None:
+            device = torch.cuda.current_device()
+        self.device = int(device)
+        self._h = ctypes.c_void_p()
+        st = _lib.windq_create(ctypes.byref(self._h), self.device)
+        if st:
+            raise WindqError(st, _lib.windq_last_error(None).decode())
+
+    def close(self):
+        if getattr(self, "_h", None) is not None and self._h.value:
+            _lib.windq_destroy(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def _check(self, st: int):
+        if st:
+            raise WindqError(st, _lib.windq_last_error(self._h).decode())
+
+    def reserve(self, nbytes: int):
+        self._check(_lib.windq_reserve(self._h, int(nbytes)))
+
+
+def windq_create(device: int | None = None) -> Context:
+    return Context(device)
+
+
+def windq_destroy(ctx: Context) -> None:
+    ctx.close()
+
+
+def windq_reserve(ctx: Context, nbytes: int) -> None:
+    ctx.reserve(nbytes)
+
+
+def windq_scratch_bytes_act_stats(T: int, C: int) -> int:
+    return int(_lib.windq_scratch_bytes_act_stats(T, C))
+
+
+def windq_scratch_bytes_unit_features(R: int, C: int, G: int) -> int:
+    return int(_lib.windq_scratch_bytes_unit_features(R, C, G))
+
+
+def windq_scratch_bytes_fit_eval(R: int, C: int, G: int) -> int:
+    return int(_lib.windq_scratch_bytes_fit_eval(R, C, G))
+
+
+def windq_act_stats(ctx: Context, X: torch.Tensor, s_out: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+    """s[j] = mean_t X[t, j]^2.  X: fp16 [T, C]; returns fp32 [C]."""
+    T, C, ldx = _matrix(X, "X")
+    if s_out is None:
+        s_out = torch.empty(C, dtype=torch.float32, device=X.device)
+    _need(s_out, torch.float32, "s_out", 1)
+    ctx._check(_lib.windq_act_stats(ctx._h, _ptr(X), T, C, ldx, _ptr(s_out), _stream(stream)))
+    return s_out
+
+
+def windq_unit_features(ctx: Context, W: torch.Tensor, G: int, s: torch.Tensor, feat_out: torch.Tensor | None = None,
+                        stream=None) -> torch.Tensor:
+    """Table 1 features per unit.  Returns fp32 [U, 8]."""
+    R, C, ldw = _matrix(W, "W")
+    _need(s, torch.float32, "s", 1)
+    if feat_out is None:
+        feat_out = torch.empty((max(C // max(G, 1), 0), N_FEATURES), dtype=torch.float32, device=W.device)
+    _need(feat_out, torch.float32, "feat_out", 2)
+    ctx._check(_lib.windq_unit_features(ctx._h, _ptr(W), R, C, ldw, int(G), _ptr(s), _ptr(feat_out), _stream(stream)))
+    return feat_out
+
+
+def windq_fit_eval(ctx: Context, W: torch.Tensor, G: int, s: torch.Tensor, clip_grid: torch.Tensor, *,
+                   want_energy: bool = True, want_clip_idx: bool = True, want_group_err: bool = False,
+                   out: dict | None = None, stream=None) -> dict:
+    """Fits every group under all six bit-widths.
+
+    Returns dict(err [U,6] f32, energy [U] f32 | None, clip_idx [4,U,R] u8 | None,
+    group_err [6,U,R] f32 | None).  ``out`` may hold preallocated tensors under the same keys.
+    """
+    R, C, ldw = _matrix(W, "W")
+    _need(s, torch.float32, "s", 1)
+    _need(clip_grid, torch.float32, "clip_grid", 1)
+    U = C // G if G > 0 else 0
+    out = dict(out) if out else {}
+    dev = W.device
+    if out.get("err") is None:
+        out["err"] = torch.empty((U, N_BITWIDTHS), dtype=torch.float32, device=dev)
+    if want_energy and out.get("energy") is None:
+        out["energy"] = torch.empty(U, dtype=torch.float32, device=dev)
+    if want_clip_idx and out.get("clip_idx") is None:
+        out["clip_idx"] = torch.empty((4, U, R), dtype=torch.uint8, device=dev)
+    if want_group_err and out.get("group_err") is None:
+        out["group_err"] = torch.empty((N_BITWIDTHS, U, R), dtype=torch.float32, device=dev)
+    for key in ("energy", "clip_idx", "group_err"):
+        out.setdefault(key, None)
+    ctx._check(_lib.windq_fit_eval(ctx._h, _ptr(W), R, C, ldw, int(G), _ptr(s), _ptr(clip_grid), clip_grid.numel(),
+                                   _ptr(out["err"]), _ptr(out["energy"]), _ptr(out["clip_idx"]), _ptr(out["group_err"]),
+                                   _stream(stream)))
+    return out
+
+
+def windq_effective_bits(ctx: Context, actions: torch.Tensor, R: int, G: int, scale_bits: int = 16, zero_bits: int = 16,
+                         out: dict | None = None, stream=None) -> dict:
+    """Returns dict(unit_centibits [U] i64, code_offsets [U+1] i64, total_centibits [1] i64,
+    total_packed_bytes [1] i64), all on the device."""
+    _need(actions, torch.uint8, "actions", 1)
+    U = actions.numel()
+    dev = actions.device
+    out = dict(out) if out else {}
+    if out.get("unit_centibits") is None:
+        out["unit_centibits"] = torch.empty(U, dtype=torch.int64, device=dev)
+    if out.get("code_offsets") is None:
+        out["code_offsets"] = torch.empty(U + 1, dtype=torch.int64, device=dev)
+    if out.get("total_centibits") is None:
+        out["total_centibits"] = torch.empty(1, dtype=torch.int64, device=dev)
+    if out.get("total_packed_bytes") is None:
+        out["total_packed_bytes"] = torch.empty(1, dtype=torch.int64, device=dev)
+    ctx._check(_lib.windq_effective_bits(ctx._h, _ptr(actions), U, int(R), int(G), int(scale_bits), int(zero_bits),
+                                         _ptr(out["unit_centibits"]), _ptr(out["code_offsets"]),
+                                         _ptr(out["total_centibits"]), _ptr(out["total_packed_bytes"]), _stream(stream)))
+    return out
+
+
+def windq_apply_plan(ctx: Context, W: torch.Tensor, G: int, s: torch.Tensor, clip_grid: torch.Tensor,
+                     actions: torch.Tensor, code_offsets: torch.Tensor, codes_out: torch.Tensor,
+                     clip_idx: torch.Tensor | None = None, *, want_wq: bool = True, out: dict | None = None,
+                     stream=None) -> dict:
+    """Applies a plan.  ``code_offsets`` comes from windq_effective_bits for the same actions;
+    ``codes_out`` is a uint8 tensor of at least code_offsets[U] bytes (the caller sizes it, e.g.
+    from the worst case 2*R*C + 16*U, to avoid a device-to-host read).
+
+    Returns dict(codes, scales [U,R] f16, zeros [U,R] f16, wq [R,C] f16 | None).
+    """
+    R, C, ldw = _matrix(W, "W")
+    _need(s, torch.float32, "s", 1)
+    _need(clip_grid, torch.float32, "clip_grid", 1)
+    _need(actions, torch.uint8, "actions", 1)
+    _need(code_offsets, torch.int64, "code_offsets", 1)
+    _need(codes_out, torch.uint8, "codes_out", 1)
+    if clip_idx is not None:
+        _need(clip_idx, torch.uint8, "clip_idx", 3)
+        if not clip_idx.is_contiguous():
+            raise ValueError("clip_idx must be contiguous")
+    U = C // G if G > 0 else 0
+    if actions.numel() != U or code_offsets.numel() != U + 1:
+        raise ValueError("actions must have U and code_offsets U + 1 entries")
+    out = dict(out) if out else {}
+    dev = W.device
+    if out.get("scales") is None:
+        out["scales"] = torch.empty((U, R), dtype=torch.float16, device=dev)
+    if out.get("zeros") is None:
+        out["zeros"] = torch.empty((U, R), dtype=torch.float16, device=dev)
+    if want_wq and out.get("wq") is None:
+        out["wq"] = torch.empty_strided((R, C), (ldw, 1), dtype=torch.float16, device=dev)
+    out.setdefault("wq", None)
+    if out["wq"] is not None and (_matrix(out["wq"], "wq")[2] != ldw or out["wq"].shape != W.shape):
+        raise ValueError("wq must have the shape and row stride of W")
+    out["codes"] = codes_out
+    ctx._check(_lib.windq_apply_plan(ctx._h, _ptr(W), R, C, ldw, int(G), _ptr(s), _ptr(clip_grid), clip_grid.numel(),
+                                     _ptr(actions), _ptr(clip_idx), _ptr(code_offsets), _ptr(codes_out), _ptr(out["scales"]),
+                                     _ptr(out["zeros"]), _ptr(out["wq"]), _stream(stream)))
+    return out

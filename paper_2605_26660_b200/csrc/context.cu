@@ -1,0 +1,111 @@
+// Context life cycle, error reporting and the host-side argument checks.
+#include <stdarg.h>
+#include <string.h>
+
+#include "windq_internal.cuh"
+
+namespace {
+thread_local char g_create_error[256] = "";
+}
+
+namespace windq {
+
+windq_status fail(windq_ctx* ctx, windq_status st, const char* fmt, ...) {
+  char* dst = ctx ? ctx->err : g_create_error;
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(dst, 256, fmt, ap);
+  va_end(ap);
+  return st;
+}
+
+windq_status ensure_scratch(windq_ctx* ctx, int64_t bytes) {
+  if (bytes <= ctx->scratch_bytes) return WINDQ_OK;
+  const int64_t want = round_up(bytes, 1 << 20);
+  void* p = nullptr;
+  if (cudaMalloc(&p, (size_t)want) != cudaSuccess) {
+    cudaGetLastError();
+    return fail(ctx, WINDQ_ERR_SCRATCH, "cannot grow scratch to %lld bytes", (long long)want);
+  }
+  if (ctx->scratch) {
+    // earlier calls may still be using the old buffer on some stream
+    cudaDeviceSynchronize();
+    cudaFree(ctx->scratch);
+  }
+  ctx->scratch = p;
+  ctx->scratch_bytes = want;
+  return WINDQ_OK;
+}
+
+windq_status check_matrix(windq_ctx* ctx, const char* who, const void* W, int64_t R, int64_t C, int64_t ldw, int G) {
+  WINDQ_REQUIRE(ctx, W != nullptr, WINDQ_ERR_NULL, "%s: W is NULL", who);
+  WINDQ_REQUIRE(ctx, valid_G(G), WINDQ_ERR_ARG, "%s: G = %d is not one of 32, 64, 128, 256, 512", who, G);
+  WINDQ_REQUIRE(ctx, R > 0 && C > 0, WINDQ_ERR_SHAPE, "%s: R = %lld, C = %lld must be positive", who, (long long)R,
+                (long long)C);
+  WINDQ_REQUIRE(ctx, R < (1ll << 31) && C < (1ll << 31), WINDQ_ERR_SHAPE, "%s: R and C must be below 2^31", who);
+  WINDQ_REQUIRE(ctx, C % G == 0, WINDQ_ERR_SHAPE, "%s: C = %lld is not a multiple of G = %d", who, (long long)C, G);
+  WINDQ_REQUIRE(ctx, ldw >= C, WINDQ_ERR_SHAPE, "%s: ldw = %lld is below C = %lld", who, (long long)ldw, (long long)C);
+  WINDQ_REQUIRE(ctx, ldw % 8 == 0, WINDQ_ERR_ALIGN, "%s: ldw = %lld is not a multiple of 8", who, (long long)ldw);
+  WINDQ_REQUIRE(ctx, aligned16(W), WINDQ_ERR_ALIGN, "%s: W is not 16-byte aligned", who);
+  return WINDQ_OK;
+}
+
+windq_status check_K(windq_ctx* ctx, const char* who, int K) {
+  WINDQ_REQUIRE(ctx, K >= 1 && K <= 64, WINDQ_ERR_ARG, "%s: K = %d is outside [1, 64]", who, K);
+  return WINDQ_OK;
+}
+
+}  // namespace windq
+
+extern "C" {
+
+windq_status windq_create(windq_ctx** out, int device) {
+  if (!out) return windq::fail(nullptr, WINDQ_ERR_NULL, "windq_create: out is NULL");
+  *out = nullptr;
+  int n = 0;
+  if (cudaGetDeviceCount(&n) != cudaSuccess || n == 0) {
+    cudaGetLastError();
+    return windq::fail(nullptr, WINDQ_ERR_CUDA, "windq_create: no CUDA device");
+  }
+  if (device < 0 || device >= n)
+    return windq::fail(nullptr, WINDQ_ERR_ARG, "windq_create: device %d of %d", device, n);
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) {
+    cudaGetLastError();
+    return windq::fail(nullptr, WINDQ_ERR_CUDA, "windq_create: cannot query device %d", device);
+  }
+  if (prop.major != 10)
+    return windq::fail(nullptr, WINDQ_ERR_UNSUPPORTED, "windq_create: device %d is sm_%d%d, this library is built for sm_100a",
+                       device, prop.major, prop.minor);
+  windq_ctx* ctx = new windq_ctx;
+  ctx->device = device;
+  ctx->sm_count = prop.multiProcessorCount;
+  ctx->scratch = nullptr;
+  ctx->scratch_bytes = 0;
+  ctx->err[0] = 0;
+  *out = ctx;
+  return WINDQ_OK;
+}
+
+void windq_destroy(windq_ctx* ctx) {
+  if (!ctx) return;
+  {
+    windq::DeviceGuard guard(ctx->device);
+    if (ctx->scratch) {
+      cudaDeviceSynchronize();
+      cudaFree(ctx->scratch);
+    }
+  }
+  delete ctx;
+}
+
+const char* windq_last_error(const windq_ctx* ctx) { return ctx ? ctx->err : g_create_error; }
+
+windq_status windq_reserve(windq_ctx* ctx, int64_t bytes) {
+  if (!ctx) return windq::fail(nullptr, WINDQ_ERR_NULL, "windq_reserve: ctx is NULL");
+  WINDQ_REQUIRE(ctx, bytes >= 0, WINDQ_ERR_ARG, "windq_reserve: bytes = %lld", (long long)bytes);
+  windq::DeviceGuard guard(ctx->device);
+  return windq::ensure_scratch(ctx, bytes);
+}
+
+}  // extern "C"

@@ -1,0 +1,320 @@
+// Device-side group fitting shared by windq_fit_eval and windq_apply_plan.
+//
+// Thread mapping.  A group (one row of one unit, G fp16 values) is owned by LG = G/32 adjacent
+// lanes; each lane keeps its 32 consecutive values (four leaves of 8) and the matching 32
+// activation statistics in registers as fp32 for the whole fit, so a weight is read from memory
+// once and every clip candidate of every bit-width is evaluated from registers.  A warp therefore
+// works on GPW = 32/LG consecutive rows of the same unit.
+//
+// Arithmetic.  Everything that decides a clip index, a code or a stored fp16 value is an explicit
+// IEEE binary32 operation (round to nearest even, no flush to zero, no contraction beyond the
+// fma's written here).  A sum over a group is taken as: each leaf of 8 consecutive elements
+// accumulated left to right from +0, then a balanced tree that adds adjacent leaves first.  In
+// this mapping the first two tree levels are inside a lane and the rest are xor-shuffles over
+// 1, 2, ... LG/2, which perform exactly those additions.
+//
+// The inner loop uses the sm_100 packed binary32 instructions (fma/add/mul .f32x2): two leaves of
+// a lane advance together, one instruction per pair, each half rounded exactly like the scalar
+// instruction.  min/max have no packed form and stay scalar.
+#pragma once
+
+#include "windq_internal.cuh"
+
+namespace windq {
+
+constexpr float kMagic = 12582912.0f;  // 1.5 * 2^23: adding it rounds to the nearest-even integer
+
+template <int G>
+struct Map {
+  static constexpr int LG = G / 32;    // lanes per group
+  static constexpr int GPW = 32 / LG;  // groups (rows) per warp
+};
+
+// ---- packed binary32 pairs --------------------------------------------------------------------
+__device__ __forceinline__ unsigned long long as_u64(float2 v) {
+  unsigned long long u;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(u) : "f"(v.x), "f"(v.y));
+  return u;
+}
+__device__ __forceinline__ float2 as_f2(unsigned long long u) {
+  float2 v;
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(v.x), "=f"(v.y) : "l"(u));
+  return v;
+}
+__device__ __forceinline__ float2 fma2(float2 a, float2 b, float2 c) {
+  unsigned long long d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(as_u64(a)), "l"(as_u64(b)), "l"(as_u64(c)));
+  return as_f2(d);
+}
+__device__ __forceinline__ float2 add2(float2 a, float2 b) {
+  unsigned long long d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(as_u64(a)), "l"(as_u64(b)));
+  return as_f2(d);
+}
+__device__ __forceinline__ float2 mul2(float2 a, float2 b) {
+  unsigned long long d;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(as_u64(a)), "l"(as_u64(b)));
+  return as_f2(d);
+}
+
+// ---- what a lane owns -------------------------------------------------------------------------
+// Element e (0..31) of the lane = leaf l = e / 8, position i = e % 8, stored in
+// v[l >> 1][i].x (even leaf) or .y (odd leaf): the two halves of a pair belong to different
+// leaves, so their accumulations are independent.
+struct Lane32 {
+  float2 v[2][8];
+  __device__ __forceinline__ float get(int l, int i) const { return (l & 1) ? v[l >> 1][i].y : v[l >> 1][i].x; }
+  __device__ __forceinline__ void set(int l, int i, float x) {
+    if (l & 1) v[l >> 1][i].y = x; else v[l >> 1][i].x = x;
+  }
+};
+
+// 32 fp16 values (64 bytes, 16-byte aligned) -> Lane32.
+__device__ __forceinline__ void load_weights(const __half* p, Lane32& w) {
+  const uint4* p4 = reinterpret_cast<const uint4*>(p);
+#pragma unroll
+  for (int l = 0; l < 4; ++l) {
+    const uint4 raw = __ldg(p4 + l);
+    const __half2* h = reinterpret_cast<const __half2*>(&raw);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const float2 f = __half22float2(h[i]);
+      w.set(l, 2 * i, f.x);
+      w.set(l, 2 * i + 1, f.y);
+    }
+  }
+}
+
+// 32 fp32 statistics (128 bytes, 16-byte aligned) -> Lane32.
+__device__ __forceinline__ void load_stats(const float* p, Lane32& s) {
+  const float4* p4 = reinterpret_cast<const float4*>(p);
+#pragma unroll
+  for (int l = 0; l < 4; ++l) {
+    const float4 a = __ldg(p4 + 2 * l), b = __ldg(p4 + 2 * l + 1);
+    s.set(l, 0, a.x); s.set(l, 1, a.y); s.set(l, 2, a.z); s.set(l, 3, a.w);
+    s.set(l, 4, b.x); s.set(l, 5, b.y); s.set(l, 6, b.z); s.set(l, 7, b.w);
+  }
+}
+
+// Tree over the group: four leaf sums of this lane, then the lanes of the group.
+template <int G>
+__device__ __forceinline__ float group_tree(float l0, float l1, float l2, float l3) {
+  float t = __fadd_rn(__fadd_rn(l0, l1), __fadd_rn(l2, l3));
+#pragma unroll
+  for (int m = 1; m < Map<G>::LG; m <<= 1) t = __fadd_rn(t, __shfl_xor_sync(0xffffffffu, t, m));
+  return t;
+}
+template <int G>
+__device__ __forceinline__ float group_tree(float2 a01, float2 a23) {
+  return group_tree<G>(a01.x, a01.y, a23.x, a23.y);
+}
+
+// min(0, min w) and max(0, max w) over the group.
+template <int G>
+__device__ __forceinline__ void group_range(const Lane32& w, float& mn, float& mx) {
+  float lo = 0.0f, hi = 0.0f;
+#pragma unroll
+  for (int h = 0; h < 2; ++h)
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      lo = fminf(lo, fminf(w.v[h][i].x, w.v[h][i].y));
+      hi = fmaxf(hi, fmaxf(w.v[h][i].x, w.v[h][i].y));
+    }
+#pragma unroll
+  for (int m = 1; m < Map<G>::LG; m <<= 1) {
+    lo = fminf(lo, __shfl_xor_sync(0xffffffffu, lo, m));
+    hi = fmaxf(hi, __shfl_xor_sync(0xffffffffu, hi, m));
+  }
+  mn = __fadd_rn(lo, 0.0f);  // -0 -> +0
+  mx = hi;
+}
+
+// ---- uniform candidates -----------------------------------------------------------------------
+// Parameters of one (bit-width, clip ratio) candidate of one group, as the inner loop wants them.
+struct Cand {
+  float inv;     // 1 / scale
+  float nscale;  // -scale: d' = fma(c, -scale, w) = -(c*scale - w), and (s*d')*d' = (s*d)*d exactly
+  float lo;      // 0 - z
+  float hi;      // qmax - z
+};
+
+struct UniformSpec {
+  float qmax;
+  float rq;  // fp32 nearest to 1 / qmax
+};
+__device__ __forceinline__ UniformSpec uniform_spec(int bi) {  // bi: 0..3 = 8, 4, 3, 2 bit
+  switch (bi) {
+    case 0: return {255.0f, (float)(1.0 / 255.0)};
+    case 1: return {15.0f, (float)(1.0 / 15.0)};
+    case 2: return {7.0f, (float)(1.0 / 7.0)};
+    default: return {3.0f, (float)(1.0 / 3.0)};
+  }
+}
+
+// scale (value of the stored fp16 scale, 1 if that is zero) and zero point (float integer).
+__device__ __forceinline__ void uniform_scale_zero(float mn, float rng, float p, UniformSpec us, float& scale,
+                                                   float& zf) {
+  const float scale32 = __fmul_rn(__fmul_rn(p, rng), us.rq);
+  scale = __half2float(__float2half_rn(scale32));
+  if (scale == 0.0f) scale = 1.0f;
+  const float inv = __frcp_rn(scale);
+  float z = rintf(__fmul_rn(fabsf(__fmul_rn(p, mn)), inv));
+  zf = fminf(fmaxf(z, 0.0f), us.qmax);
+}
+
+__device__ __forceinline__ Cand make_cand(float mn, float rng, float p, UniformSpec us) {
+  float scale, zf;
+  uniform_scale_zero(mn, rng, p, us, scale, zf);
+  Cand c;
+  c.inv = __frcp_rn(scale);
+  c.nscale = -scale;
+  c.lo = __fsub_rn(0.0f, zf);
+  c.hi = __fsub_rn(us.qmax, zf);
+  return c;
+}
+
+// Zero-centred code c = clamp(rne(w * inv), lo, hi) of one element.
+__device__ __forceinline__ float centred_code(float w, const Cand& c) {
+  const float r = __fmaf_rn(w, c.inv, kMagic);
+  return fminf(fmaxf(__fadd_rn(r, -kMagic), c.lo), c.hi);
+}
+
+// s-weighted squared error of one candidate over this lane's 32 elements: the four leaf sums,
+// as two pairs.
+__device__ __forceinline__ void cand_leaf_errors(const Lane32& w, const Lane32& s, const Cand& c, float2& e01,
+                                                 float2& e23) {
+  const float2 inv2 = make_float2(c.inv, c.inv);
+  const float2 ns2 = make_float2(c.nscale, c.nscale);
+  const float2 magic2 = make_float2(kMagic, kMagic);
+  const float2 nmagic2 = make_float2(-kMagic, -kMagic);
+  float2 acc[2] = {make_float2(0.0f, 0.0f), make_float2(0.0f, 0.0f)};
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      const float2 wv = w.v[h][i];
+      float2 q = add2(fma2(wv, inv2, magic2), nmagic2);
+      q.x = fminf(fmaxf(q.x, c.lo), c.hi);
+      q.y = fminf(fmaxf(q.y, c.lo), c.hi);
+      const float2 d = fma2(q, ns2, wv);
+      const float2 t = mul2(s.v[h][i], d);
+      acc[h] = fma2(t, d, acc[h]);
+    }
+  }
+  e01 = acc[0];
+  e23 = acc[1];
+}
+
+// Clip search for one bit-width.  `cand` is this warp's shared-memory parameter table with room
+// for GPW rows of `stride` entries; candidates are processed in chunks of at most `chunk`.
+// On return best_e / best_k hold the least error and the smallest index that reaches it; all
+// lanes of a group hold the same values.  Must be called by all 32 lanes.
+template <int G>
+__device__ __forceinline__ void search_uniform(const Lane32& w, const Lane32& s, float mn, float rng, int bi,
+                                               const float* __restrict__ clip, int K, Cand* cand, int chunk,
+                                               int stride, int lane, float& best_e, int& best_k) {
+  constexpr int LG = Map<G>::LG;
+  const int g = lane / LG, q = lane % LG;
+  const UniformSpec us = uniform_spec(bi);
+  Cand* mine = cand + g * stride;
+  best_e = 0.0f;
+  best_k = 0;
+  for (int k0 = 0; k0 < K; k0 += chunk) {
+    const int kc = min(chunk, K - k0);
+    __syncwarp();
+    for (int k = q; k < kc; k += LG) mine[k] = make_cand(mn, rng, __ldg(clip + k0 + k), us);
+    __syncwarp();
+    for (int k = 0; k < kc; ++k) {
+      const Cand c = mine[k];
+      float2 e01, e23;
+      cand_leaf_errors(w, s, c, e01, e23);
+      const float e = group_tree<G>(e01, e23);
+      if ((k0 + k == 0) || e < best_e) {
+        best_e = e;
+        best_k = k0 + k;
+      }
+    }
+  }
+}
+
+// ---- ternary and binary -----------------------------------------------------------------------
+struct LowBitFit {
+  float delta;    // ternary threshold 0.7 * mean |w|
+  float alpha_t;  // ternary scale (value of the fp16 number), 0 if the support is empty
+  float alpha_b;  // binary scale
+  float err_t, err_b;
+  float energy;   // sum_j s_j w_j^2 of the group (any order; tolerance output)
+};
+
+// Must be called by all 32 lanes.
+template <int G>
+__device__ __forceinline__ LowBitFit fit_low_bits(const Lane32& w, const Lane32& s) {
+  LowBitFit f;
+  float A[4], Sb[4], Bb[4], En[4];
+#pragma unroll
+  for (int l = 0; l < 4; ++l) {
+    float a = 0.0f, sb = 0.0f, bb = 0.0f, en = 0.0f;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const float wv = w.get(l, i), sv = s.get(l, i), aw = fabsf(wv);
+      a = __fadd_rn(a, aw);
+      sb = __fadd_rn(sb, sv);
+      bb = __fmaf_rn(sv, aw, bb);
+      en = __fmaf_rn(__fmul_rn(sv, wv), wv, en);
+    }
+    A[l] = a; Sb[l] = sb; Bb[l] = bb; En[l] = en;
+  }
+  const float sumA = group_tree<G>(A[0], A[1], A[2], A[3]);
+  const float sumS = group_tree<G>(Sb[0], Sb[1], Sb[2], Sb[3]);
+  const float sumB = group_tree<G>(Bb[0], Bb[1], Bb[2], Bb[3]);
+  f.energy = group_tree<G>(En[0], En[1], En[2], En[3]);
+  const float meanA = __fmul_rn(sumA, 1.0f / (float)G);
+  f.delta = __fmul_rn(0.7f, meanA);
+  f.alpha_b = __half2float(__float2half_rn(sumS == 0.0f ? meanA : __fdiv_rn(sumB, sumS)));
+
+  // ternary sums over the support, weighted by s and (fallback) unweighted
+  float Bt[4], Ct[4], Bu[4], Cu[4];
+#pragma unroll
+  for (int l = 0; l < 4; ++l) {
+    float bt = 0.0f, ct = 0.0f, bu = 0.0f, cu = 0.0f;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const float aw = fabsf(w.get(l, i)), sv = s.get(l, i);
+      const bool in = aw > f.delta;
+      const float a_in = in ? aw : 0.0f;
+      bt = __fmaf_rn(sv, a_in, bt);
+      ct = __fadd_rn(ct, in ? sv : 0.0f);
+      bu = __fadd_rn(bu, a_in);
+      cu = __fadd_rn(cu, in ? 1.0f : 0.0f);
+    }
+    Bt[l] = bt; Ct[l] = ct; Bu[l] = bu; Cu[l] = cu;
+  }
+  float sumBt = group_tree<G>(Bt[0], Bt[1], Bt[2], Bt[3]);
+  float sumCt = group_tree<G>(Ct[0], Ct[1], Ct[2], Ct[3]);
+  const float sumBu = group_tree<G>(Bu[0], Bu[1], Bu[2], Bu[3]);
+  const float sumCu = group_tree<G>(Cu[0], Cu[1], Cu[2], Cu[3]);
+  if (sumCt == 0.0f) { sumBt = sumBu; sumCt = sumCu; }
+  f.alpha_t = (sumCu > 0.0f) ? __half2float(__float2half_rn(__fdiv_rn(sumBt, sumCt))) : 0.0f;
+
+  float Et[4], Eb[4];
+#pragma unroll
+  for (int l = 0; l < 4; ++l) {
+    float et = 0.0f, eb = 0.0f;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const float wv = w.get(l, i), sv = s.get(l, i);
+      const bool neg = wv < 0.0f;
+      const float rt = (fabsf(wv) > f.delta) ? (neg ? -f.alpha_t : f.alpha_t) : 0.0f;
+      const float dt = __fsub_rn(rt, wv);
+      et = __fmaf_rn(__fmul_rn(sv, dt), dt, et);
+      const float db = __fsub_rn(neg ? -f.alpha_b : f.alpha_b, wv);
+      eb = __fmaf_rn(__fmul_rn(sv, db), db, eb);
+    }
+    Et[l] = et; Eb[l] = eb;
+  }
+  f.err_t = group_tree<G>(Et[0], Et[1], Et[2], Et[3]);
+  f.err_b = group_tree<G>(Eb[0], Eb[1], Eb[2], Eb[3]);
+  return f;
+}
+
+}  // namespace windq

@@ -1,0 +1,185 @@
+// windq_fit_eval: every group of a weight matrix fitted under all six bit-widths.
+//
+// Bound by the FP32 pipes, not by HBM: about 28*K + 40 binary32 operations per 2-byte weight
+// (K clip ratios x 4 uniform bit-widths x 7 operations, plus the ternary / binary fits).  The
+// design therefore spends nothing on data movement tricks -- each lane reads its 64 bytes of a
+// row once with 128-bit loads, straight into registers -- and everything on keeping the inner
+// loop at its minimum instruction count (see fit_device.cuh).
+//
+// Work is split into items = (unit, block of GPW consecutive rows), one warp per item, no
+// block-level synchronisation.  The grid is persistent: every warp takes a contiguous range of
+// items, so that it mostly stays within one unit and the unit's statistics stay in registers.
+// Per item the warp writes seven partial sums (six errors and the energy, added over its rows in
+// double) to scratch; a second small kernel adds them per unit in a fixed order, so unit totals
+// are reproducible from run to run.
+#include "fit_device.cuh"
+
+namespace windq {
+
+constexpr int kFitWarpsPerBlock = 4;
+constexpr int kFitPartials = 8;  // 6 errors + energy + pad
+
+__host__ __device__ inline int fit_cand_chunk(int G) {
+  // candidates per shared-memory chunk: GPW * stride * 16 bytes <= ~5.4 KB per warp
+  const int gpw = 32 / (G / 32);
+  int c = 336 / gpw;  // 8 rows -> 42, 16 -> 21, 32 -> 10, 4 -> 84, 2 -> 168
+  return c > 64 ? 64 : c;
+}
+__host__ __device__ inline int fit_cand_stride(int chunk) { return chunk | 1; }  // odd: conflict-free rows
+
+template <int G>
+__global__ void __launch_bounds__(kFitWarpsPerBlock * 32, 4)
+fit_eval_kernel(const __half* __restrict__ W, int R, int U, int64_t ldw, const float* __restrict__ s,
+                const float* __restrict__ clip, int K, double* __restrict__ partial, uint8_t* __restrict__ clip_idx_out,
+                float* __restrict__ group_err_out, int rows_blocks, int chunk, int stride) {
+  constexpr int LG = Map<G>::LG, GPW = Map<G>::GPW;
+  extern __shared__ float4 smem_f4[];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  Cand* cand = reinterpret_cast<Cand*>(smem_f4) + (size_t)warp * GPW * stride;
+  const int g = lane / LG, q = lane % LG;
+
+  const int64_t n_items = (int64_t)U * rows_blocks;
+  const int64_t n_warps = (int64_t)gridDim.x * kFitWarpsPerBlock;
+  const int64_t wid = (int64_t)blockIdx.x * kFitWarpsPerBlock + warp;
+  const int64_t item_begin = wid * n_items / n_warps, item_end = (wid + 1) * n_items / n_warps;
+
+  Lane32 sv;
+  int cur_u = -1;
+  for (int64_t item = item_begin; item < item_end; ++item) {
+    const int u = (int)(item / rows_blocks), rb = (int)(item % rows_blocks);
+    if (u != cur_u) {
+      load_stats(s + (int64_t)u * G + 32 * q, sv);
+      cur_u = u;
+    }
+    const int row = rb * GPW + g;
+    const bool live = row < R;
+    const int row_ld = live ? row : R - 1;  // rows past the end repeat the last row and are not written
+    Lane32 wv;
+    load_weights(W + (int64_t)row_ld * ldw + (int64_t)u * G + 32 * q, wv);
+
+    float mn, mx;
+    group_range<G>(wv, mn, mx);
+    const float rng = __fsub_rn(mx, mn);
+
+    float e[7] = {0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f};
+#pragma unroll 1
+    for (int bi = 0; bi < 4; ++bi) {
+      float be;
+      int bk;
+      search_uniform<G>(wv, sv, mn, rng, bi, clip, K, cand, chunk, stride, lane, be, bk);
+      e[0] = bi == 0 ? be : e[0];
+      e[1] = bi == 1 ? be : e[1];
+      e[2] = bi == 2 ? be : e[2];
+      e[3] = bi == 3 ? be : e[3];
+      if (live && q == 0) {
+        const int64_t o = ((int64_t)bi * U + u) * R + row;
+        if (clip_idx_out) clip_idx_out[o] = (uint8_t)bk;
+        if (group_err_out) group_err_out[o] = be;
+      }
+    }
+    const LowBitFit low = fit_low_bits<G>(wv, sv);
+    e[4] = low.err_t;
+    e[5] = low.err_b;
+    e[6] = low.energy;
+    if (live && q == 0 && group_err_out) {
+      group_err_out[((int64_t)4 * U + u) * R + row] = low.err_t;
+      group_err_out[((int64_t)5 * U + u) * R + row] = low.err_b;
+    }
+
+    // add over the rows of this item in double; lanes of a group hold equal values
+#pragma unroll
+    for (int c = 0; c < 7; ++c) {
+      double d = live ? (double)e[c] : 0.0;
+#pragma unroll
+      for (int m = LG; m < 32; m <<= 1) d += __shfl_xor_sync(0xffffffffu, d, m);
+      if (lane == 0) partial[item * kFitPartials + c] = d;
+    }
+  }
+}
+
+// err_out[u][0..5], energy_out[u] = sum over the unit's row blocks, fixed order.
+__global__ void __launch_bounds__(256)
+fit_finalize_kernel(const double* __restrict__ partial, int rows_blocks, float* __restrict__ err_out,
+                    float* __restrict__ energy_out) {
+  __shared__ double red[256];
+  const int u = blockIdx.x, t = threadIdx.x;
+  const double* p = partial + (int64_t)u * rows_blocks * kFitPartials;
+  for (int c = 0; c < 7; ++c) {
+    double acc = 0.0;
+    for (int rb = t; rb < rows_blocks; rb += 256) acc += p[(int64_t)rb * kFitPartials + c];
+    red[t] = acc;
+    __syncthreads();
+    for (int n = 128; n > 0; n >>= 1) {
+      if (t < n) red[t] += red[t + n];
+      __syncthreads();
+    }
+    if (t == 0) {
+      if (c < 6) err_out[(int64_t)u * 6 + c] = (float)red[0];
+      else if (energy_out) energy_out[u] = (float)red[0];
+    }
+    __syncthreads();
+  }
+}
+
+template <int G>
+windq_status launch_fit(windq_ctx* ctx, const __half* W, int R, int U, int64_t ldw, const float* s,
+                        const float* clip, int K, double* partial, float* err_out, float* energy_out,
+                        uint8_t* clip_idx_out, float* group_err_out, cudaStream_t st) {
+  constexpr int GPW = Map<G>::GPW;
+  const int rows_blocks = (R + GPW - 1) / GPW;
+  const int chunk = fit_cand_chunk(G), stride = fit_cand_stride(chunk);
+  const size_t smem = (size_t)kFitWarpsPerBlock * GPW * stride * sizeof(Cand);
+  static int blocks_per_sm = 0;  // same for every device this library supports
+  if (blocks_per_sm == 0) {
+    WINDQ_CUDA(ctx, cudaFuncSetAttribute(fit_eval_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    int n = 0;
+    WINDQ_CUDA(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, fit_eval_kernel<G>, kFitWarpsPerBlock * 32, smem));
+    blocks_per_sm = n > 0 ? n : 1;
+  }
+  const int64_t n_items = (int64_t)U * rows_blocks;
+  int64_t grid = (int64_t)ctx->sm_count * blocks_per_sm;
+  const int64_t need = (n_items + kFitWarpsPerBlock - 1) / kFitWarpsPerBlock;
+  if (grid > need) grid = need;
+  fit_eval_kernel<G><<<(unsigned)grid, kFitWarpsPerBlock * 32, smem, st>>>(W, R, U, ldw, s, clip, K, partial, clip_idx_out,
+                                                                          group_err_out, rows_blocks, chunk, stride);
+  WINDQ_CUDA(ctx, cudaGetLastError());
+  fit_finalize_kernel<<<(unsigned)U, 256, 0, st>>>(partial, rows_blocks, err_out, energy_out);
+  WINDQ_CUDA(ctx, cudaGetLastError());
+  return WINDQ_OK;
+}
+
+}  // namespace windq
+
+extern "C" {
+
+int64_t windq_scratch_bytes_fit_eval(int64_t R, int64_t C, int G) {
+  if (!windq::valid_G(G) || R <= 0 || C <= 0) return 0;
+  const int gpw = 32 / (G / 32);
+  return (C / G) * ((R + gpw - 1) / gpw) * windq::kFitPartials * (int64_t)sizeof(double);
+}
+
+windq_status windq_fit_eval(windq_ctx* ctx, const void* W, int64_t R, int64_t C, int64_t ldw, int G, const float* s,
+                            const float* clip_grid, int K, float* err_out, float* energy_out, uint8_t* clip_idx_out,
+                            float* group_err_out, void* stream) {
+  using namespace windq;
+  if (!ctx) return fail(nullptr, WINDQ_ERR_NULL, "windq_fit_eval: ctx is NULL");
+  if (windq_status st = check_matrix(ctx, "windq_fit_eval", W, R, C, ldw, G)) return st;
+  if (windq_status st = check_K(ctx, "windq_fit_eval", K)) return st;
+  WINDQ_REQUIRE(ctx, s && clip_grid && err_out, WINDQ_ERR_NULL, "windq_fit_eval: s, clip_grid or err_out is NULL");
+  WINDQ_REQUIRE(ctx, aligned16(s), WINDQ_ERR_ALIGN, "windq_fit_eval: s is not 16-byte aligned");
+  DeviceGuard guard(ctx->device);
+  if (windq_status st = ensure_scratch(ctx, windq_scratch_bytes_fit_eval(R, C, G))) return st;
+  const int U = (int)(C / G);
+  cudaStream_t st = (cudaStream_t)stream;
+  const __half* Wh = (const __half*)W;
+  double* partial = (double*)ctx->scratch;
+  switch (G) {
+    case 32: return launch_fit<32>(ctx, Wh, (int)R, U, ldw, s, clip_grid, K, partial, err_out, energy_out, clip_idx_out, group_err_out, st);
+    case 64: return launch_fit<64>(ctx, Wh, (int)R, U, ldw, s, clip_grid, K, partial, err_out, energy_out, clip_idx_out, group_err_out, st);
+    case 128: return launch_fit<128>(ctx, Wh, (int)R, U, ldw, s, clip_grid, K, partial, err_out, energy_out, clip_idx_out, group_err_out, st);
+    case 256: return launch_fit<256>(ctx, Wh, (int)R, U, ldw, s, clip_grid, K, partial, err_out, energy_out, clip_idx_out, group_err_out, st);
+    default: return launch_fit<512>(ctx, Wh, (int)R, U, ldw, s, clip_grid, K, partial, err_out, energy_out, clip_idx_out, group_err_out, st);
+  }
+}
+
+}  // extern "C"

@@ -1,0 +1,72 @@
+// Internal declarations shared by the windq translation units: the context, host-side argument
+// checks and small device helpers.  Nothing here is part of the ABI.
+#pragma once
+
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stdio.h>
+
+#include "windq.h"
+
+struct windq_ctx {
+  int device;
+  int sm_count;
+  void* scratch;
+  int64_t scratch_bytes;
+  char err[256];
+};
+
+namespace windq {
+
+windq_status fail(windq_ctx* ctx, windq_status st, const char* fmt, ...);
+// Makes the context's scratch at least `bytes` large (may cudaMalloc).
+windq_status ensure_scratch(windq_ctx* ctx, int64_t bytes);
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline bool valid_G(int G) { return G == 32 || G == 64 || G == 128 || G == 256 || G == 512; }
+inline int64_t round_up(int64_t x, int64_t m) { return (x + m - 1) / m * m; }
+
+// Switches to the context's device for the lifetime of the object.
+struct DeviceGuard {
+  int prev = -1;
+  bool switched = false;
+  explicit DeviceGuard(int dev) {
+    if (cudaGetDevice(&prev) == cudaSuccess && prev != dev) switched = (cudaSetDevice(dev) == cudaSuccess);
+  }
+  ~DeviceGuard() {
+    if (switched) cudaSetDevice(prev);
+  }
+};
+
+#define WINDQ_REQUIRE(ctx, cond, st, ...) \
+  do {                                    \
+    if (!(cond)) return ::windq::fail((ctx), (st), __VA_ARGS__); \
+  } while (0)
+
+#define WINDQ_CUDA(ctx, call)                                                                      \
+  do {                                                                                             \
+    cudaError_t e_ = (call);                                                                       \
+    if (e_ != cudaSuccess) return ::windq::fail((ctx), WINDQ_ERR_CUDA, "%s: %s", #call, cudaGetErrorString(e_)); \
+  } while (0)
+
+// Checks shared by the calls that take a weight matrix.
+windq_status check_matrix(windq_ctx* ctx, const char* who, const void* W, int64_t R, int64_t C, int64_t ldw, int G);
+// The clip grid lives on the device and is used as given; only K can be checked on the host.
+windq_status check_K(windq_ctx* ctx, const char* who, int K);
+
+// Bytes of one packed group under an action (host and device).
+__host__ __device__ inline int group_code_bytes(int action, int G) {
+  switch (action) {
+    case 0: return 2 * G;
+    case 1: return G;
+    case 2: return G / 2;
+    case 3: return 3 * G / 8;
+    case 4: return G / 4;
+    case 5: return (G + 4) / 5;
+    case 6: return G / 8;
+  }
+  return 0;
+}
+
+}  // namespace windq

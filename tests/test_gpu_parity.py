@@ -1,0 +1,319 @@
+"""GPU parity: the CUDA library (through its C ABI) against the CPU oracle, on the same seeded inputs.
+
+Bars (fixed in advance): clip indices, codes / packed bytes, fp16 scales / zero points, fake-quantised
+weights, the counts behind sparsity / outlier_frac and all int64 totals are bit-exact; float outputs
+agree within |g - o| <= 1e-4 |o| + 1e-6.  Group errors are compared bit-exactly as well, since both
+sides define them as the same sequence of binary32 operations.
+"""
+import numpy as np
+import pytest
+import torch
+
+import windq_synth as ws
+
+pytestmark = pytest.mark.gpu
+
+RTOL, ATOL = 1e-4, 1e-6
+
+
+@pytest.fixture(scope="module")
+def wq():
+    import paper_2605_26660_b200 as wq
+    return wq
+
+
+@pytest.fixture(scope="module")
+def ctx(wq):
+    c = wq.windq_create(0)
+    yield c
+    wq.windq_destroy(c)
+
+
+def close(g, o):
+    g, o = np.asarray(g, np.float64), np.asarray(o, np.float64)
+    return np.abs(g - o) <= RTOL * np.abs(o) + ATOL
+
+
+def guarded(shape, dtype, fill=0xAB):
+    """An output tensor inside a larger buffer whose margins must stay untouched."""
+    n = int(np.prod(shape))
+    item = torch.empty(0, dtype=dtype).element_size()
+    pad = 256 // item
+    buf = torch.full((n + 2 * pad,), 0, dtype=dtype, device="cuda")
+    buf.view(torch.uint8).fill_(fill)
+    view = buf[pad:pad + n].view(*shape)
+
+    def intact():
+        raw = buf.view(torch.uint8)
+        return bool((raw[:256] == fill).all()) and bool((raw[256 + n * item:] == fill).all())
+    return view, intact
+
+
+def make(R, C, seed, dist="student_t", T=96):
+    W = ws.weights(R, C, seed, dist)
+    X = ws.activations(T, C, seed + 7)
+    return W, X
+
+
+# ------------------------------------------------------------------ act_stats
+@pytest.mark.parametrize("T,C", [(512, 4096), (77, 264), (1, 8), (300, 11008)])
+def test_act_stats(wq, ctx, oracle, T, C):
+    X = ws.activations(T, C, 100 + T)
+    want = oracle.act_stats(X.numpy())
+    out, intact = guarded((C,), torch.float32)
+    wq.windq_act_stats(ctx, X.cuda(), out)
+    torch.cuda.synchronize()
+    assert intact()
+    assert close(out.cpu().numpy(), want).all()
+
+
+def test_act_stats_strided_rows(wq, ctx, oracle):
+    X = ws.activations(64, 512, 5)
+    big = torch.zeros((64, 768), dtype=torch.float16, device="cuda")
+    big[:, :512] = X.cuda()
+    got = wq.windq_act_stats(ctx, big[:, :512])
+    assert close(got.cpu().numpy(), oracle.act_stats(X.numpy())).all()
+
+
+# ------------------------------------------------------------------ unit_features
+@pytest.mark.parametrize("R,C,G", [(300, 512, 128), (64, 256, 32), (1000, 1024, 512), (97, 256, 64), (4096, 512, 256)])
+def test_unit_features(wq, ctx, oracle, R, C, G):
+    W, X = make(R, C, 200 + G)
+    W[::5, ::7] = 0
+    s = oracle.act_stats(X.numpy())
+    want = oracle.unit_features(W.numpy(), G, s)
+    out, intact = guarded((C // G, 8), torch.float32)
+    wq.windq_unit_features(ctx, W.cuda(), G, torch.from_numpy(s).cuda(), out)
+    torch.cuda.synchronize()
+    got = out.cpu().numpy()
+    assert intact()
+    assert (got[:, 3:5] == want[:, 3:5]).all()          # exact counts -> identical ratios
+    assert close(got, want).all()
+
+
+# ------------------------------------------------------------------ fit_eval
+def run_fit(wq, ctx, W, G, s, grid):
+    R, C = W.shape
+    U = C // G
+    err, ok1 = guarded((U, 6), torch.float32)
+    energy, ok2 = guarded((U,), torch.float32)
+    clip_idx, ok3 = guarded((4, U, R), torch.uint8)
+    group_err, ok4 = guarded((6, U, R), torch.float32)
+    out = wq.windq_fit_eval(ctx, W.cuda(), G, torch.from_numpy(s).cuda(), torch.from_numpy(grid).cuda(),
+                            want_group_err=True, out=dict(err=err, energy=energy, clip_idx=clip_idx, group_err=group_err))
+    torch.cuda.synchronize()
+    assert ok1() and ok2() and ok3() and ok4()
+    return {k: v.cpu().numpy() for k, v in out.items()}
+
+
+def check_fit(got, want):
+    mism = got["clip_idx"] != want["clip_idx"]
+    assert (got["group_err"].view(np.uint32) == want["group_err"].view(np.uint32)).all()
+    assert not mism.any()
+    assert close(got["err"], want["err"]).all()
+    assert close(got["energy"], want["energy"]).all()
+
+
+@pytest.mark.parametrize("G,R,C,K", [(128, 70, 512, 20), (64, 37, 256, 20), (32, 33, 128, 20), (256, 19, 1024, 20),
+                                     (512, 9, 1024, 20), (128, 8, 256, 7), (64, 40, 128, 64), (32, 64, 64, 40),
+                                     (128, 1, 128, 1)])
+def test_fit_eval_small(wq, ctx, oracle, G, R, C, K):
+    W, X = make(R, C, 300 + G + K)
+    s = oracle.act_stats(X.numpy())
+    grid = ws.clip_grid(K)
+    want = oracle.fit_eval(W.numpy(), G, s, grid, threads=8)
+    check_fit(run_fit(wq, ctx, W, G, s, grid), want)
+
+
+def test_fit_eval_degenerate_inputs(wq, ctx, oracle):
+    G, R = 128, 24
+    W = ws.weights(R, 4 * G, 9, "normal")
+    W[:, :G] = 0                                   # all-zero unit
+    W[:, G:2 * G] = 0.37                           # constant unit
+    W[0, 2 * G:3 * G] = -0.0                       # negative zeros
+    W[1, 2 * G:3 * G] = 6.0e-8                     # fp16 subnormals
+    s = np.ones(4 * G, np.float32)
+    s[3 * G:] = 0                                  # no activation weight at all
+    grid = ws.clip_grid(20)
+    want = oracle.fit_eval(W.numpy(), G, s, grid)
+    check_fit(run_fit(wq, ctx, W, G, s, grid), want)
+
+
+def test_fit_eval_config1_single_layer(wq, ctx, oracle):
+    spec = ws.CONFIGS["cfg1_single_layer"]
+    W = ws.weights(4096, 4096, ws.matrix_seed(0, 0, 0), "normal")
+    X = ws.activations(spec.T, 4096, ws.matrix_seed(0, 0, 8))
+    s = oracle.act_stats(X.numpy())
+    grid = ws.clip_grid(20)
+    out = wq.windq_fit_eval(ctx, W.cuda(), 128, torch.from_numpy(s).cuda(), torch.from_numpy(grid).cuda(), want_group_err=True)
+    got = {k: v.cpu().numpy() for k, v in out.items()}
+    # the oracle on every fourth unit (8 of 32 units, 4.2e6 weights)
+    for u0 in range(0, 32, 4):
+        want = oracle.fit_eval(W.numpy(), 128, s, grid, units=(u0, u0 + 1))
+        assert (got["clip_idx"][:, u0] == want["clip_idx"][:, u0]).all()
+        assert (got["group_err"][:, u0].view(np.uint32) == want["group_err"][:, u0].view(np.uint32)).all()
+        assert close(got["err"][u0], want["err"][u0]).all() and close(got["energy"][u0], want["energy"][u0]).all()
+
+
+def test_fit_eval_is_reproducible(wq, ctx):
+    W = ws.weights(333, 1024, 77, "student_t").cuda()
+    s = torch.rand(1024, device="cuda") + 0.1
+    grid = torch.from_numpy(ws.clip_grid(20)).cuda()
+    a = wq.windq_fit_eval(ctx, W, 128, s, grid, want_group_err=True)
+    b = wq.windq_fit_eval(ctx, W, 128, s, grid, want_group_err=True)
+    for k in a:
+        assert torch.equal(a[k], b[k])
+
+
+# ------------------------------------------------------------------ effective_bits
+@pytest.mark.parametrize("U,R,G", [(32, 4096, 128), (1, 1, 32), (2500, 37, 64), (86, 4096, 512)])
+def test_effective_bits(wq, ctx, oracle, U, R, G):
+    rng = np.random.default_rng(U)
+    acts = rng.integers(0, 7, U).astype(np.uint8)
+    for sb, zb in ((16, 16), (0, 0), (32, 8)):
+        want = oracle.effective_bits(acts, R, G, sb, zb)
+        got = wq.windq_effective_bits(ctx, torch.from_numpy(acts).cuda(), R, G, sb, zb)
+        assert (got["unit_centibits"].cpu().numpy() == want["unit_centibits"]).all()
+        assert (got["code_offsets"].cpu().numpy() == want["code_offsets"]).all()
+        assert int(got["total_centibits"].item()) == want["total_centibits"]
+        assert int(got["total_packed_bytes"].item()) == want["total_packed_bytes"]
+
+
+def test_effective_bits_flags_bad_action(wq, ctx):
+    acts = torch.tensor([1, 2, 9, 3], dtype=torch.uint8, device="cuda")
+    got = wq.windq_effective_bits(ctx, acts, 16, 128)
+    assert int(got["total_centibits"].item()) == -1 and int(got["total_packed_bytes"].item()) == -1
+    assert got["unit_centibits"].cpu().tolist()[2] == -1
+
+
+# ------------------------------------------------------------------ apply_plan
+def run_apply(wq, ctx, W, G, s, grid, acts, clip_idx):
+    R, C = W.shape
+    U = C // G
+    a_d = torch.from_numpy(acts).cuda()
+    eb = wq.windq_effective_bits(ctx, a_d, R, G)
+    n_codes = int(eb["code_offsets"][-1].item())
+    codes, ok1 = guarded((max(n_codes, 1),), torch.uint8)
+    scales, ok2 = guarded((U, R), torch.float16)
+    zeros, ok3 = guarded((U, R), torch.float16)
+    wq_t, ok4 = guarded((R, C), torch.float16)
+    out = wq.windq_apply_plan(ctx, W.cuda(), G, torch.from_numpy(s).cuda(), torch.from_numpy(grid).cuda(), a_d,
+                              eb["code_offsets"], codes, None if clip_idx is None else torch.from_numpy(clip_idx).cuda(),
+                              out=dict(scales=scales, zeros=zeros, wq=wq_t))
+    torch.cuda.synchronize()
+    assert ok1() and ok2() and ok3() and ok4()
+    return dict(codes=out["codes"][:n_codes].cpu().numpy(), scales=out["scales"].cpu().view(torch.int16).numpy().view(np.uint16),
+                zeros=out["zeros"].cpu().view(torch.int16).numpy().view(np.uint16),
+                wq=out["wq"].cpu().view(torch.int16).numpy().view(np.uint16))
+
+
+@pytest.mark.parametrize("G,R", [(128, 70), (64, 133), (32, 200), (256, 19), (512, 67), (128, 3), (128, 64)])
+def test_apply_plan_all_actions(wq, ctx, oracle, G, R):
+    C = 8 * G
+    W, X = make(R, C, 400 + G + R)
+    s = oracle.act_stats(X.numpy())
+    grid = ws.clip_grid(20)
+    acts = np.array([0, 1, 2, 3, 4, 5, 6, 5], np.uint8)
+    fit = oracle.fit_eval(W.numpy(), G, s, grid, threads=8, want_group_err=False)
+    want = oracle.apply_plan(W.numpy(), G, s, grid, acts, fit["clip_idx"])
+    for clip_idx in (fit["clip_idx"], None):
+        got = run_apply(wq, ctx, W, G, s, grid, acts, clip_idx)
+        for key in ("codes", "scales", "zeros", "wq"):
+            assert got[key].shape == want[key].shape, key
+            assert (got[key] == want[key]).all(), key
+
+
+def test_apply_plan_uses_clip_idx_from_fit_eval(wq, ctx, oracle):
+    G, R, C = 128, 96, 1024
+    W, X = make(R, C, 500)
+    s = oracle.act_stats(X.numpy())
+    grid = ws.clip_grid(20)
+    fit = wq.windq_fit_eval(ctx, W.cuda(), G, torch.from_numpy(s).cuda(), torch.from_numpy(grid).cuda())
+    acts = np.array([4, 3, 2, 1, 4, 4, 3, 2], np.uint8)
+    want = oracle.apply_plan(W.numpy(), G, s, grid, acts, None)
+    got = run_apply(wq, ctx, W, G, s, grid, acts, fit["clip_idx"].cpu().numpy())
+    for key in ("codes", "scales", "zeros", "wq"):
+        assert (got[key] == want[key]).all(), key
+
+
+def test_apply_plan_degenerate_inputs(wq, ctx, oracle):
+    G, R = 128, 20
+    W = ws.weights(R, 7 * G, 19, "normal")
+    W[:, :3 * G] = 0
+    W[3, 3 * G:4 * G] = -0.0
+    s = np.ones(7 * G, np.float32)
+    s[5 * G:] = 0
+    grid = ws.clip_grid(20)
+    for acts in (np.array([1, 5, 6, 4, 3, 5, 6], np.uint8), np.array([4, 6, 5, 2, 1, 6, 5], np.uint8)):
+        want = oracle.apply_plan(W.numpy(), G, s, grid, acts, None)
+        got = run_apply(wq, ctx, W, G, s, grid, acts, None)
+        for key in ("codes", "scales", "zeros", "wq"):
+            assert (got[key] == want[key]).all(), key
+
+
+# ------------------------------------------------------------------ argument checks (no launch)
+def test_argument_errors(wq, ctx):
+    W = torch.zeros((16, 256), dtype=torch.float16, device="cuda")
+    s = torch.ones(256, device="cuda")
+    grid = torch.from_numpy(ws.clip_grid(20)).cuda()
+    with pytest.raises(wq.WindqError) as e:
+        wq.windq_fit_eval(ctx, W, 100, s, grid)
+    assert e.value.status == 4 and "G = 100" in str(e.value)
+    with pytest.raises(wq.WindqError) as e:
+        wq.windq_fit_eval(ctx, W[:, :192], 128, s, grid)
+    assert e.value.status == 2
+    with pytest.raises(wq.WindqError) as e:
+        wq.windq_fit_eval(ctx, W, 128, s, torch.ones(65, device="cuda"))
+    assert e.value.status == 4
+    with pytest.raises(wq.WindqError) as e:
+        wq.windq_fit_eval(ctx, W[:, 4:132], 128, s, grid)          # 8-byte offset: misaligned
+    assert e.value.status == 3
+    with pytest.raises(wq.WindqError) as e:
+        wq.windq_act_stats(ctx, torch.zeros((4, 12), dtype=torch.float16, device="cuda"))
+    assert e.value.status in (2, 3)
+    with pytest.raises(wq.WindqError) as e:
+        wq.windq_effective_bits(ctx, torch.zeros(4, dtype=torch.uint8, device="cuda"), 16, 128, scale_bits=-1)
+    assert e.value.status == 4
+    # the context stays usable after errors
+    out = wq.windq_fit_eval(ctx, W, 128, s, grid)
+    assert float(out["err"].abs().sum()) == 0.0
+
+
+# ------------------------------------------------------------------ full size, sampled units
+def test_full_size_matrix_sampled_units(wq, ctx, oracle):
+    """An 11008 x 4096 Student-t matrix generated on the device (the benchmark's recipe and launch
+    shape); the oracle recomputes sampled units from the same bits."""
+    spec = ws.CONFIGS["cfg3_llama7b_model"]
+    m = spec.block_matrices()[4]
+    W = ws.block_weight(spec, 0, 0, m, device="cuda")
+    X = ws.block_input(spec, 0, 0, m.x_id, device="cuda")
+    s = wq.windq_act_stats(ctx, X)
+    grid = ws.clip_grid(spec.K)
+    grid_d = torch.from_numpy(grid).cuda()
+    s_h = s.cpu().numpy()
+    assert close(s_h, oracle.act_stats(X.cpu().numpy())).all()
+    for G in spec.chunk_widths:
+        U = m.C // G
+        fit = wq.windq_fit_eval(ctx, W, G, s, grid_d)
+        feat = wq.windq_unit_features(ctx, W, G, s).cpu().numpy()
+        rng = np.random.default_rng(G)
+        acts = rng.integers(0, 7, U).astype(np.uint8)
+        a_d = torch.from_numpy(acts).cuda()
+        eb = wq.windq_effective_bits(ctx, a_d, m.R, G)
+        codes = torch.empty(int(eb["code_offsets"][-1].item()), dtype=torch.uint8, device="cuda")
+        plan = wq.windq_apply_plan(ctx, W, G, s, grid_d, a_d, eb["code_offsets"], codes, fit["clip_idx"])
+        offs = eb["code_offsets"].cpu().numpy()
+        for u in rng.choice(U, 3, replace=False):
+            Wu = W[:, u * G:(u + 1) * G].cpu().numpy()
+            su = s_h[u * G:(u + 1) * G]
+            want = oracle.fit_eval(Wu, G, su, grid, threads=8, want_group_err=False)
+            assert (fit["clip_idx"][:, u].cpu().numpy() == want["clip_idx"][:, 0]).all()
+            assert close(fit["err"][u].cpu().numpy(), want["err"][0]).all()
+            assert close(fit["energy"][u].cpu().numpy(), want["energy"][0]).all()
+            wf = oracle.unit_features(Wu, G, su)
+            assert (feat[u, 3:5] == wf[0, 3:5]).all() and close(feat[u], wf[0]).all()
+            wp = oracle.apply_plan(Wu, G, su, grid, acts[u:u + 1], want["clip_idx"])
+            assert (codes[offs[u]:offs[u + 1]].cpu().numpy() == wp["codes"]).all()
+            assert (plan["scales"][u].cpu().view(torch.int16).numpy().view(np.uint16) == wp["scales"][0]).all()
+            assert (plan["zeros"][u].cpu().view(torch.int16).numpy().view(np.uint16) == wp["zeros"][0]).all()
+            assert (plan["wq"][:, u * G:(u + 1) * G].cpu().view(torch.int16).numpy().view(np.uint16) == wp["wq"]).all()

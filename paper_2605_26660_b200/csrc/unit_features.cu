@@ -102,6 +102,7 @@ feat_finalize_kernel(const unsigned int* __restrict__ hist, const double* __rest
 #pragma unroll
   for (int i = 0; i < 32; ++i) {
     const float v = __half2float(__ushort_as_half((unsigned short)(t * 32 + i)));
+    if (c[i] == 0) continue;  // also keeps the Inf / NaN patterns (never counted for finite input) out
     const double dv = (double)v, dc = (double)c[i];
     sa += dc * dv;
     sq += dc * dv * dv;

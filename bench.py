@@ -1,0 +1,555 @@
+#!/usr/bin/env python
+"""Benchmark of the WINDQuant scoring path on B200.
+
+    python bench.py --gpus N --steps K --warmup W            # this library (CUDA, C ABI)
+    python bench.py --impl reference --steps K --warmup W    # the CPU oracle, as it stands
+
+A step is one pass of the whole hot path over a LLaMA-7B-shaped model of synthetic weights and
+calibration activations (32 decoder blocks; see windq_synth.CONFIGS): per block 4 x act_stats;
+per matrix and chunk width (64, 128) unit_features + fit_eval over every unit; then, at chunk
+width 128, effective_bits + apply_plan for three seeded random plans (1.58, 2.0, 3.0 bits).
+The metric is unit x bit-width candidate evaluations per second (6 per unit and chunk width).
+
+`value` is measured with the inputs resident in HBM; `e2e` runs the same step from pinned host
+memory, host-to-device copies of every weight and activation and device-to-host copies of every
+result (error tables, features, packed codes, scales, zero points) inside the timed region.
+With N > 1 (torchrun) every rank scores its own replica of the model: weak scaling, no
+data-path collective; time is the maximum over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+import windq_synth as ws
+
+METRIC = "unit_x_bitwidth_candidate_evals_per_s"
+UNIT = "evals/s"
+TARGET_BITS = (1.58, 2.0, 3.0)
+APPLY_G = 128
+SEED = 0
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=3)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="windq", choices=["windq", "reference"])
+    ap.add_argument("--workload", default="cfg3_llama7b_model", choices=sorted(ws.CONFIGS))
+    ap.add_argument("--blocks", type=int, default=0, help="use only the first B blocks (0 = all; profiling aid)")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    return ap.parse_args()
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as fh:
+            p = json.load(fh)
+        return dict(hbm_gbs=float(p["hbm_gbs"]), sm_max_mhz=float(p.get("sm_max_mhz", 1965.0)), source="measured")
+    return dict(hbm_gbs=6650.0, sm_max_mhz=1965.0, source="fallback")
+
+
+# ---------------------------------------------------------------------------------------- clocks
+class ClockSampler:
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu_index = gpu_index
+        self.proc = None
+        self.path = None
+
+    def __enter__(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu_index), "--query-gpu=" + self.FIELDS,
+                                          "--format=csv,noheader,nounits", "-lms", "200"],
+                                         stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+        return self
+
+    def __exit__(self, *exc):
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except Exception:
+                self.proc.kill()
+
+    def summary(self):
+        out = dict(sm_mhz=None, sm_max_mhz=None, reasons=[])
+        if not self.path or not os.path.exists(self.path):
+            return out
+        sm, mx, reasons = [], [], set()
+        with open(self.path) as fh:
+            for line in fh:
+                t = [x.strip() for x in line.split(",")]
+                if len(t) < 9:
+                    continue
+                try:
+                    sm.append(float(t[1]))
+                    mx.append(float(t[2]))
+                except ValueError:
+                    continue
+                for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), t[5:9]):
+                    if v.lower().startswith("active"):
+                        reasons.add(name)
+        os.unlink(self.path)
+        if sm:
+            busy = [x for x in sm if x > 0.5 * max(mx)] or sm
+            out = dict(sm_mhz=float(np.median(busy)), sm_max_mhz=float(max(mx)), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+# ---------------------------------------------------------------------------------------- workload
+def matrices_of(spec):
+    return [m for m in spec.block_matrices() if m.R > 0 and m.C > 0]
+
+
+def inputs_of(spec):
+    used = {m.x_id for m in matrices_of(spec)}
+    return [(i, c) for i, c in spec.block_inputs() if i in used]
+
+
+def workload_counts(spec, n_blocks):
+    mats = matrices_of(spec)
+    elems = sum(m.R * m.C for m in mats) * n_blocks
+    units = {G: sum(m.C // G for m in mats) * n_blocks for G in spec.chunk_widths}
+    return elems, units
+
+
+def fit_ops_per_element(K):
+    """Algorithmic binary32 lane operations per weight element (fma = 1): seven per (bit-width, clip
+    ratio) candidate of the four uniform bit-widths, plus about ten once per element."""
+    return 28 * K + 10
+
+
+class DeviceModel:
+    """Weights and calibration inputs of this rank's blocks, resident in HBM."""
+
+    def __init__(self, spec, blocks, seed):
+        self.spec, self.blocks = spec, list(blocks)
+        self.W, self.X = [], []
+        for b in self.blocks:
+            self.W.append([ws.block_weight(spec, seed, b, m, device="cuda") for m in matrices_of(spec)])
+            self.X.append({i: ws.block_input(spec, seed, b, i, device="cuda") for i, _ in inputs_of(spec)})
+        torch.cuda.synchronize()
+
+
+def make_plans(wq, ctx, spec, n_blocks, G):
+    """Seeded random plans for the three target bit-widths; returns {target: [[actions per matrix] per block]}."""
+    mats = matrices_of(spec)
+    costs, nw = [], []
+    all_actions = torch.arange(7, dtype=torch.uint8, device="cuda")
+    per_R = {}
+    for m in mats:
+        if m.R not in per_R:
+            per_R[m.R] = wq.windq_effective_bits(ctx, all_actions, m.R, G)["unit_centibits"].cpu().numpy()
+    for _ in range(n_blocks):
+        for m in mats:
+            U = m.C // G
+            costs.append(np.tile(per_R[m.R][None, :], (U, 1)))
+            nw.append(np.full(U, m.R * G, np.int64))
+    costs, nw = np.concatenate(costs), np.concatenate(nw)
+    plans = {}
+    for ti, target in enumerate(TARGET_BITS):
+        flat = ws.random_plan(costs, nw, target, SEED * 7919 + ti)
+        per_block, pos = [], 0
+        for _ in range(n_blocks):
+            row = []
+            for m in mats:
+                U = m.C // G
+                row.append(torch.from_numpy(flat[pos:pos + U].copy()).cuda())
+                pos += U
+            per_block.append(row)
+        plans[target] = per_block
+    return plans
+
+
+class Buffers:
+    """Output tensors sized for the largest matrix, reused for every matrix (a consumer would keep
+    what it needs); nothing is allocated inside a step."""
+
+    def __init__(self, spec):
+        mats = matrices_of(spec)
+        Gmin = min(spec.chunk_widths)
+        maxU = max(m.C // Gmin for m in mats)
+        maxRC = max(m.R * m.C for m in mats)
+        maxUR = max((m.C // Gmin) * m.R for m in mats)
+        maxC = max(c for _, c in inputs_of(spec))
+        dev = "cuda"
+        self.s = {i: torch.empty(c, dtype=torch.float32, device=dev) for i, c in inputs_of(spec)}
+        self.feat = torch.empty(maxU * 8, dtype=torch.float32, device=dev)
+        self.err = torch.empty(maxU * 6, dtype=torch.float32, device=dev)
+        self.energy = torch.empty(maxU, dtype=torch.float32, device=dev)
+        self.clip_idx = torch.empty(4 * maxUR, dtype=torch.uint8, device=dev)
+        self.unit_cb = torch.empty(maxU, dtype=torch.int64, device=dev)
+        self.offsets = torch.empty(maxU + 1, dtype=torch.int64, device=dev)
+        self.totals = torch.zeros(2 * len(TARGET_BITS), dtype=torch.int64, device=dev)
+        self.codes = torch.empty(2 * maxRC + 16 * maxU, dtype=torch.uint8, device=dev)
+        self.scales = torch.empty(maxUR, dtype=torch.float16, device=dev)
+        self.zeros = torch.empty(maxUR, dtype=torch.float16, device=dev)
+        self.wq = torch.empty(maxRC, dtype=torch.float16, device=dev)
+        del maxC
+
+
+class FitTimer:
+    """CUDA events around every windq_fit_eval call of the timed steps (on the launching stream)."""
+
+    def __init__(self):
+        self.pairs = []
+
+    def start(self):
+        e = torch.cuda.Event(enable_timing=True)
+        e.record()
+        return e
+
+    def stop(self, e0):
+        e1 = torch.cuda.Event(enable_timing=True)
+        e1.record()
+        self.pairs.append((e0, e1))
+
+    def total_ms(self):
+        return sum(a.elapsed_time(b) for a, b in self.pairs)
+
+
+def score_block(wq, ctx, spec, Wb, Xb, plans_b, buf, grid_d, timer=None, sink=None):
+    """The whole hot path for one block.  Returns the number of kernels launched.  `sink(name, tensor)`
+    receives every result (the e2e leg copies them to the host)."""
+    launches = 0
+    mats = matrices_of(spec)
+    for i, X in Xb.items():
+        wq.windq_act_stats(ctx, X, buf.s[i])
+        launches += 2
+    for mi, m in enumerate(mats):
+        W, s = Wb[mi], buf.s[m.x_id]
+        for G in spec.chunk_widths:
+            U = m.C // G
+            feat = buf.feat[:U * 8].view(U, 8)
+            wq.windq_unit_features(ctx, W, G, s, feat)
+            launches += 2
+            out = dict(err=buf.err[:U * 6].view(U, 6), energy=buf.energy[:U],
+                       clip_idx=buf.clip_idx[:4 * U * m.R].view(4, U, m.R))
+            e0 = timer.start() if timer else None
+            wq.windq_fit_eval(ctx, W, G, s, grid_d, out=out)
+            if timer:
+                timer.stop(e0)
+            launches += 2
+            if sink:
+                sink("feat", feat)
+                sink("err", out["err"])
+                sink("energy", out["energy"])
+            if G == APPLY_G and plans_b:
+                for ti, target in enumerate(TARGET_BITS):
+                    acts = plans_b[target][mi]
+                    eb = wq.windq_effective_bits(ctx, acts, m.R, G, out=dict(
+                        unit_centibits=buf.unit_cb[:U], code_offsets=buf.offsets[:U + 1],
+                        total_centibits=buf.totals[2 * ti:2 * ti + 1], total_packed_bytes=buf.totals[2 * ti + 1:2 * ti + 2]))
+                    plan = wq.windq_apply_plan(ctx, W, G, s, grid_d, acts, eb["code_offsets"], buf.codes, out["clip_idx"],
+                                               out=dict(scales=buf.scales[:U * m.R].view(U, m.R), zeros=buf.zeros[:U * m.R].view(U, m.R),
+                                                        wq=buf.wq[:m.R * m.C].view(m.R, m.C)))
+                    launches += 2
+                    if sink:
+                        sink("codes", (plan["codes"], acts, m.R, G))
+                        sink("scales", plan["scales"])
+                        sink("zeros", plan["zeros"])
+                        sink("totals", buf.totals[2 * ti:2 * ti + 2])
+    return launches
+
+
+def packed_code_bytes(actions_np, R, G):
+    per = np.array([2 * G, G, G // 2, 3 * G // 8, G // 4, (G + 4) // 5, G // 8], np.int64)
+    return int(((R * per[actions_np] + 15) // 16 * 16).sum())
+
+
+# ---------------------------------------------------------------------------------------- legs
+def run_device_leg(wq, ctx, spec, model, plans, buf, grid_d, steps, warmup, rank, sync):
+    def step(timer=None):
+        n = 0
+        for bi in range(len(model.blocks)):
+            n += score_block(wq, ctx, spec, model.W[bi], model.X[bi], {t: plans[t][bi] for t in plans}, buf, grid_d, timer)
+        return n
+
+    for _ in range(warmup):
+        step()
+    timer = FitTimer()
+    sync()
+    with ClockSampler(rank) as clocks:
+        t0 = torch.cuda.Event(enable_timing=True)
+        t1 = torch.cuda.Event(enable_timing=True)
+        t0.record()
+        launches = 0
+        for _ in range(steps):
+            launches += step(timer)
+        t1.record()
+        sync()
+    ms = t0.elapsed_time(t1)
+    return ms, launches, timer.total_ms(), clocks.summary()
+
+
+def run_e2e_leg(wq, ctx, spec, model, plans, plans_np, buf, grid_d, steps, warmup, sync):
+    """Same step from pinned host memory: two device-side block slots, copies on a second stream
+    overlapped with the previous block's kernels; every result copied back to pinned host memory."""
+    mats = matrices_of(spec)
+    nb = len(model.blocks)
+    need = sum(m.R * m.C for m in mats) * 2 + sum(spec.T * c for _, c in inputs_of(spec)) * 2
+    import psutil
+    avail = psutil.virtual_memory().available
+    host_blocks = nb if need * nb * 3 < avail else 1
+    hostW, hostX = [], []
+    for bi in range(host_blocks):
+        hostW.append([w.cpu().pin_memory() for w in model.W[bi]])
+        hostX.append({i: x.cpu().pin_memory() for i, x in model.X[bi].items()})
+    slots = []
+    for _ in range(2):
+        slots.append(dict(W=[torch.empty_like(w) for w in model.W[0]], X={i: torch.empty_like(x) for i, x in model.X[0].items()},
+                          ready=torch.cuda.Event(), free=torch.cuda.Event()))
+    copy_stream = torch.cuda.Stream()
+    main = torch.cuda.current_stream()
+    # pinned result buffers (sized for the largest matrix); D2H on the main stream after each call
+    host_out = {}
+
+    def host_buf(name, n, dtype):
+        key = (name, dtype)
+        if key not in host_out or host_out[key].numel() < n:
+            host_out[key] = torch.empty(n, dtype=dtype).pin_memory()
+        return host_out[key][:n]
+
+    d2h = [0]
+
+    def sink(name, t):
+        if name == "codes":
+            codes, acts, R, G = t
+            n = sink.code_bytes[(id(acts))]
+            host_buf(name, n, torch.uint8).copy_(codes[:n], non_blocking=True)
+            d2h[0] += n
+        else:
+            flat = t.reshape(-1)
+            host_buf(name, flat.numel(), flat.dtype).copy_(flat, non_blocking=True)
+            d2h[0] += flat.numel() * flat.element_size()
+
+    sink.code_bytes = {}
+    for target in plans:
+        for bi in range(nb):
+            for mi, m in enumerate(mats):
+                sink.code_bytes[id(plans[target][bi][mi])] = packed_code_bytes(plans_np[target][bi][mi], m.R, APPLY_G)
+    # make sure the largest pinned result buffers exist before timing
+    maxRC = max(m.R * m.C for m in mats)
+    host_buf("codes", 2 * maxRC, torch.uint8)
+    h2d_per_step = need * nb
+
+    def step():
+        n = 0
+        for bi in range(nb):
+            slot = slots[bi % 2]
+            hb = bi % host_blocks
+            with torch.cuda.stream(copy_stream):
+                copy_stream.wait_event(slot["free"])
+                for dst, src in zip(slot["W"], hostW[hb]):
+                    dst.copy_(src, non_blocking=True)
+                for i in slot["X"]:
+                    slot["X"][i].copy_(hostX[hb][i], non_blocking=True)
+                slot["ready"].record(copy_stream)
+            main.wait_event(slot["ready"])
+            n += score_block(wq, ctx, spec, slot["W"], slot["X"], {t: plans[t][bi] for t in plans}, buf, grid_d, None, sink)
+            slot["free"].record(main)
+        return n
+
+    for s in slots:
+        s["free"].record(main)
+    for _ in range(min(warmup, 1)):
+        step()
+    sync()
+    d2h[0] = 0
+    t0 = torch.cuda.Event(enable_timing=True)
+    t1 = torch.cuda.Event(enable_timing=True)
+    wall0 = time.perf_counter()
+    t0.record()
+    for _ in range(steps):
+        step()
+    t1.record()
+    sync()
+    wall = (time.perf_counter() - wall0) * 1e3
+    ms = max(t0.elapsed_time(t1), 0.0)
+    return ms, wall, h2d_per_step, d2h[0] // max(steps, 1), host_blocks
+
+
+def oracle_sample(spec, seed, threads):
+    """The CPU oracle on a bounded sample of the workload: the whole hot path for block 0's q_proj
+    (4096 x 4096) at every chunk width, its calibration statistics, features and the three plans.
+    Returns (seconds, unit x bit-width evaluations, description)."""
+    import oracle
+    m = matrices_of(spec)[0]
+    W = ws.block_weight(spec, seed, 0, m).numpy()
+    X = ws.block_input(spec, seed, 0, m.x_id).numpy()
+    grid = ws.clip_grid(spec.K)
+    t0 = time.perf_counter()
+    s = oracle.act_stats(X)
+    evals = 0
+    for G in spec.chunk_widths:
+        oracle.unit_features(W, G, s) if threads <= 1 else _parallel_features(oracle, W, G, s, threads)
+        fit = oracle.fit_eval(W, G, s, grid, threads=threads, want_group_err=False)
+        evals += 6 * (m.C // G)
+        if G == APPLY_G:
+            rng = np.random.default_rng(seed)
+            for ti, _ in enumerate(TARGET_BITS):
+                acts = rng.choice(7, size=m.C // G, p=np.array(ws.ACTION_MIX) / sum(ws.ACTION_MIX)).astype(np.uint8)
+                oracle.effective_bits(acts, m.R, G)
+                oracle.apply_plan(W, G, s, grid, acts, fit["clip_idx"])
+    dt = time.perf_counter() - t0
+    desc = "block 0 %s %dx%d, T=%d: act_stats, unit_features + fit_eval at G=%s, 3 plans applied at G=%d" % (
+        m.name, m.R, m.C, spec.T, "/".join(map(str, spec.chunk_widths)), APPLY_G)
+    return dt, evals, desc
+
+
+def _parallel_features(oracle, W, G, s, threads):
+    from concurrent.futures import ThreadPoolExecutor
+    U = W.shape[1] // G
+    bounds = np.linspace(0, U, min(threads, U) + 1).astype(int)
+
+    def run(ab):
+        a, b = ab
+        if b > a:
+            oracle.unit_features(np.ascontiguousarray(W[:, a * G:b * G]), G, s[a * G:b * G])
+    with ThreadPoolExecutor(max_workers=threads) as ex:
+        list(ex.map(run, zip(bounds[:-1], bounds[1:])))
+
+
+def reference_main(args, spec):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    threads = os.cpu_count() or 1
+    for _ in range(min(args.warmup, 1)):
+        oracle_sample(spec, SEED, threads)
+    tot_t, tot_e, desc = 0.0, 0, ""
+    for _ in range(args.steps):
+        dt, ev, desc = oracle_sample(spec, SEED, threads)
+        tot_t += dt
+        tot_e += ev
+    value = tot_e / tot_t
+    line = dict(impl="reference", metric=METRIC, value=value, unit=UNIT, n_gpus=args.gpus, steps=args.steps, warmup=args.warmup,
+                ms_per_step=1e3 * tot_t / args.steps, higher_is_better=True, scaling="weak", vs_baseline=None, dtype="f32",
+                data="synthetic", config=dict(workload=spec.name, sample=desc),
+                cpu_baseline=dict(value=value, unit=UNIT, cores=threads, kind="oracle", sample=desc),
+                e2e=dict(value=value, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0), gpu_launches=0)
+    print(json.dumps(line))
+
+
+def main():
+    args = parse_args()
+    spec = ws.CONFIGS[args.workload]
+    if args.impl == "reference":
+        return reference_main(args, spec)
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the windq library has no CPU path")
+    torch.cuda.set_device(local_rank)
+    import torch.distributed as dist
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    import paper_2605_26660_b200 as wq
+    from paper_2605_26660_b200 import sharding
+
+    def sync():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    peaks = load_peaks()
+    ctx = wq.windq_create(local_rank)
+    n_blocks = args.blocks if args.blocks > 0 else spec.n_blocks
+    # weak scaling: rank r scores its own replica (global blocks r*n_blocks ...)
+    blocks = sharding.block_range(n_blocks * world, rank, world)
+    model = DeviceModel(spec, blocks, SEED)
+    buf = Buffers(spec)
+    grid_d = torch.from_numpy(ws.clip_grid(spec.K)).cuda()
+    plans = make_plans(wq, ctx, spec, n_blocks, APPLY_G) if APPLY_G in spec.chunk_widths else {}
+    plans_np = {t: [[a.cpu().numpy() for a in row] for row in plans[t]] for t in plans}
+    mats = matrices_of(spec)
+    scratch = max(max(wq.windq_scratch_bytes_fit_eval(m.R, m.C, G), wq.windq_scratch_bytes_unit_features(m.R, m.C, G))
+                  for m in mats for G in spec.chunk_widths)
+    wq.windq_reserve(ctx, scratch)
+
+    elems, units = workload_counts(spec, n_blocks)
+    evals_per_step = 6 * sum(units.values())
+    ms, launches, fit_ms, clocks = run_device_leg(wq, ctx, spec, model, plans, buf, grid_d, args.steps, args.warmup, local_rank, sync)
+    ms = sharding.max_float(ms)
+    value = world * evals_per_step * args.steps / (ms * 1e-3)
+
+    # plan totals (control path): exact int64 sums over ranks
+    total_cb = sharding.sum_int64(int(buf.totals[2 * (len(TARGET_BITS) - 1)].item())) if plans else 0
+
+    n_fit = len(spec.chunk_widths) * len(mats) * n_blocks * args.steps
+    fit_elem = elems * len(spec.chunk_widths) * args.steps
+    ops = fit_ops_per_element(spec.K)
+    sm_count = torch.cuda.get_device_properties(local_rank).multi_processor_count
+    alu_peak = sm_count * 128 * peaks["sm_max_mhz"] * 1e6 / 1e12          # T lane-ops/s, fma = 1
+    achieved = fit_elem * ops / (fit_ms * 1e-3) / 1e12
+    hbm_time = 2.0 * fit_elem / (peaks["hbm_gbs"] * 1e9)
+    alu_time = fit_elem * ops / (alu_peak * 1e12)
+    roofline = dict(bound="alu" if alu_time >= hbm_time else "hbm", kernel="fit_eval_kernel", achieved=achieved, peak=alu_peak,
+                    unit="T fp32 lane-ops/s (fma = 1)", frac=achieved / alu_peak, traffic=None,
+                    launches=n_fit, avg_launch_ms=fit_ms / n_fit, ops_per_element=ops,
+                    weight_gbs=2.0 * fit_elem / (fit_ms * 1e-3) / 1e9, hbm_frac=hbm_time / (fit_ms * 1e-3),
+                    elem_cand_per_s=fit_elem * (4 * spec.K + 2) / (fit_ms * 1e-3),
+                    peak_source="%d SMs x 128 lanes x %.0f MHz (%s)" % (sm_count, peaks["sm_max_mhz"], peaks["source"]))
+
+    e2e = None
+    if not args.no_e2e:
+        e_ms, e_wall, h2d, d2h, host_blocks = run_e2e_leg(wq, ctx, spec, model, plans, plans_np, buf, grid_d,
+                                                          max(1, min(args.steps, 2)), args.warmup, sync)
+        e_steps = max(1, min(args.steps, 2))
+        e_ms = sharding.max_float(max(e_ms, e_wall))
+        e2e = dict(value=world * evals_per_step * e_steps / (e_ms * 1e-3), unit=UNIT, h2d_bytes_per_step=h2d,
+                   d2h_bytes_per_step=d2h, steps=e_steps, ms_per_step=e_ms / e_steps,
+                   host_blocks_resident=host_blocks)
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        threads = os.cpu_count() or 1
+        dt, ev, desc = oracle_sample(spec, SEED, threads)
+        cpu = dict(value=ev / dt, unit=UNIT, cores=threads, kind="oracle", sample=desc, seconds=dt)
+
+    if rank == 0:
+        line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,
+                    ms_per_step=ms / args.steps, higher_is_better=True, scaling="weak", vs_baseline=None, dtype="f32",
+                    data="synthetic",
+                    config=dict(workload=spec.name, blocks=n_blocks, elements_per_chunk_width=elems, units=units, K=spec.K,
+                                chunk_widths=list(spec.chunk_widths), plan_targets=list(TARGET_BITS), apply_chunk_width=APPLY_G,
+                                tokens=spec.T, weights=spec.dist, parallelism="replica per GPU",
+                                l2="every step streams %.1f GB of inputs, far above the 126 MB L2" % (
+                                    (2 * elems + 2 * spec.T * sum(c for _, c in inputs_of(spec)) * n_blocks) / 1e9)),
+                    clocks=clocks, e2e=e2e, gpu_launches=launches, roofline=roofline, cpu_baseline=cpu,
+                    fit_eval_ms_per_step=fit_ms / args.steps, plan_total_centibits_last=total_cb)
+        print(json.dumps(line))
+    wq.windq_destroy(ctx)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -80,6 +80,36 @@ int64_t windq_scratch_bytes_fit_eval(int64_t R, int64_t C, int G);
 windq_status windq_act_stats(windq_ctx* ctx, const void* X, int64_t T, int64_t C, int64_t ldx,
                              float* s_out, void* stream);
 
+/* Variant of windq_act_stats that allocates nothing.  (The paper has no counterpart: this entry
+ * point exists for the sake of callers, not of the method.)
+ *
+ * windq_act_stats keeps its per-slice partial sums in the context's scratch buffer, which it
+ * grows with cudaMalloc when a call needs more than is there.  Some hosts cannot afford that: a
+ * process whose device memory has been handed out completely to its own pool, so that a fresh
+ * cudaMalloc fails; a latency-bound loop that must not take the device-wide synchronisation
+ * cudaMalloc and cudaFree imply; code that runs where only kernel launches are allowed.  For them
+ * this call keeps the partial sums in an array of WINDQ_NOALLOC_SCRATCH_BYTES that is built into
+ * the library image.  Every device that loads the library holds that array until the process
+ * exits, whether or not this entry point is ever called.
+ *
+ * Arguments, layout, result and argument errors are those of windq_act_stats.  In addition:
+ *   - the call needs 4 * C * ceil(T / 64) bytes of the array (windq_scratch_bytes_act_stats
+ *     gives the figure); a larger request is refused with WINDQ_ERR_SCRATCH before anything is
+ *     launched -- use windq_act_stats, or call once per block of tokens and combine the means;
+ *   - no cudaMalloc, cudaFree or other allocating routine is called, on any path;
+ *   - the first call on a device asks the runtime for the array's device address (one
+ *     cudaGetSymbolAddress, kept per device afterwards).  Make that first call outside any
+ *     stream capture;
+ *   - all calls on a device share the one array, and it keeps whatever the last call left.  That
+ *     is harmless from call to call, because every partial sum that is read has been written by
+ *     the same call first; but two calls whose kernels can overlap on the GPU (different streams
+ *     with no ordering between them, or two contexts on one device) race on it and give wrong
+ *     results.  Order such calls on one stream or with events.
+ *   - at most 64 devices (device index below 64). */
+#define WINDQ_NOALLOC_SCRATCH_BYTES (4 * 1024 * 1024)
+windq_status windq_act_stats_noalloc(windq_ctx* ctx, const void* X, int64_t T, int64_t C, int64_t ldx,
+                                     float* s_out, void* stream);
+
 /* a2 -- state features of every unit (Table 1, dims 0-4 and 9-11).
  *   feat_out[u] = { mean, std, abs_mean, sparsity, outlier_frac, mean(s), std(s), max(s) }
  * over the R*G weights of unit u and the G statistics s[u*G .. (u+1)*G).  std is the population

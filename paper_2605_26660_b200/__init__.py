@@ -53,6 +53,7 @@ def _load() -> ctypes.CDLL:
         getattr(lib, name).argtypes = [i64, i64, i32]
         getattr(lib, name).restype = i64
     lib.windq_act_stats.argtypes = [vp, vp, i64, i64, i64, vp, vp]
+    lib.windq_act_stats_noalloc.argtypes = [vp, vp, i64, i64, i64, vp, vp]
     lib.windq_unit_features.argtypes = [vp, vp, i64, i64, i64, i32, vp, vp, vp]
     lib.windq_fit_eval.argtypes = [vp, vp, i64, i64, i64, i32, vp, vp, i32, vp, vp, vp, vp, vp]
     lib.windq_effective_bits.argtypes = [vp, vp, i64, i64, i32, i32, i32, vp, vp, vp, vp, vp]
@@ -153,6 +154,23 @@ def windq_act_stats(ctx: Context, X: torch.Tensor, s_out: torch.Tensor | None = 
         s_out = torch.empty(C, dtype=torch.float32, device=X.device)
     _need(s_out, torch.float32, "s_out", 1)
     ctx._check(_lib.windq_act_stats(ctx._h, _ptr(X), T, C, ldx, _ptr(s_out), _stream(stream)))
+    return s_out
+
+
+NOALLOC_SCRATCH_BYTES = 4 * 1024 * 1024   # WINDQ_NOALLOC_SCRATCH_BYTES of the header
+
+
+def windq_act_stats_noalloc(ctx: Context, X: torch.Tensor, s_out: torch.Tensor, stream=None) -> torch.Tensor:
+    """windq_act_stats for callers that must not allocate device memory: the partial sums live in
+    an array built into the library, so neither the library nor this wrapper allocates anything.
+    ``s_out`` (fp32 [C]) is therefore required.  Shapes that need more than NOALLOC_SCRATCH_BYTES
+    (4 * C * ceil(T / 64) bytes) raise WindqError with status ERR_SCRATCH.  Calls that can overlap
+    on the GPU share that array and must be ordered by the caller."""
+    T, C, ldx = _matrix(X, "X")
+    _need(s_out, torch.float32, "s_out", 1)
+    if s_out.numel() < C:
+        raise ValueError("s_out must have at least C entries")
+    ctx._check(_lib.windq_act_stats_noalloc(ctx._h, _ptr(X), T, C, ldx, _ptr(s_out), _stream(stream)))
     return s_out
 
 

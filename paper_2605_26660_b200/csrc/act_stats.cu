@@ -98,3 +98,75 @@ windq_status windq_act_stats(windq_ctx* ctx, const void* X, int64_t T, int64_t C
 }
 
 }  // extern "C"
+
+// ---- windq_act_stats_noalloc ------------------------------------------------------------------
+// Same two kernels as windq_act_stats, with the per-slice partial sums kept in a fixed array in
+// device global memory instead of the context's cudaMalloc'ed scratch.  The array is part of the
+// library image: every device that loads the library carries WINDQ_NOALLOC_SCRATCH_BYTES of it
+// until the process exits, and every call on a device uses the same bytes.
+#include <mutex>
+
+namespace windq {
+
+constexpr int64_t kNoallocFloats = WINDQ_NOALLOC_SCRATCH_BYTES / (int64_t)sizeof(float);
+static __device__ __align__(256) float g_noalloc_partial[kNoallocFloats];
+
+constexpr int kNoallocMaxDevices = 64;
+static std::mutex g_noalloc_mutex;
+static float* g_noalloc_ptr[kNoallocMaxDevices];  // device address of the array, per device; NULL until looked up
+
+// Device address of g_noalloc_partial on `device`, which must be the current device.  In host
+// code the array's name only stands for the symbol; the address a kernel can use has to be asked
+// from the runtime, once per device.
+static cudaError_t noalloc_scratch(int device, float** out) {
+  std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+  if (g_noalloc_ptr[device] == nullptr) {
+    void* p = nullptr;
+    const cudaError_t e = cudaGetSymbolAddress(&p, g_noalloc_partial);
+    if (e != cudaSuccess) return e;
+    g_noalloc_ptr[device] = static_cast<float*>(p);
+  }
+  *out = g_noalloc_ptr[device];
+  return cudaSuccess;
+}
+
+}  // namespace windq
+
+extern "C" windq_status windq_act_stats_noalloc(windq_ctx* ctx, const void* X, int64_t T, int64_t C, int64_t ldx,
+                                                float* s_out, void* stream) {
+  using namespace windq;
+  if (!ctx) return fail(nullptr, WINDQ_ERR_NULL, "windq_act_stats_noalloc: ctx is NULL");
+  WINDQ_REQUIRE(ctx, X && s_out, WINDQ_ERR_NULL, "windq_act_stats_noalloc: X or s_out is NULL");
+  WINDQ_REQUIRE(ctx, T > 0 && C > 0, WINDQ_ERR_SHAPE, "windq_act_stats_noalloc: T = %lld, C = %lld must be positive",
+                (long long)T, (long long)C);
+  WINDQ_REQUIRE(ctx, C < (1ll << 31) && T < (1ll << 40), WINDQ_ERR_SHAPE, "windq_act_stats_noalloc: T or C too large");
+  WINDQ_REQUIRE(ctx, C % 8 == 0, WINDQ_ERR_SHAPE, "windq_act_stats_noalloc: C = %lld is not a multiple of 8", (long long)C);
+  WINDQ_REQUIRE(ctx, ldx >= C, WINDQ_ERR_SHAPE, "windq_act_stats_noalloc: ldx = %lld is below C = %lld", (long long)ldx,
+                (long long)C);
+  WINDQ_REQUIRE(ctx, ldx % 8 == 0, WINDQ_ERR_ALIGN, "windq_act_stats_noalloc: ldx = %lld is not a multiple of 8",
+                (long long)ldx);
+  WINDQ_REQUIRE(ctx, aligned16(X), WINDQ_ERR_ALIGN, "windq_act_stats_noalloc: X is not 16-byte aligned");
+  const int64_t need = windq_scratch_bytes_act_stats(T, C);
+  WINDQ_REQUIRE(ctx, need <= (int64_t)WINDQ_NOALLOC_SCRATCH_BYTES, WINDQ_ERR_SCRATCH,
+                "windq_act_stats_noalloc: T = %lld, C = %lld needs %lld bytes of scratch, the built-in array has %lld; "
+                "use windq_act_stats or split the tokens",
+                (long long)T, (long long)C, (long long)need, (long long)WINDQ_NOALLOC_SCRATCH_BYTES);
+  WINDQ_REQUIRE(ctx, ctx->device < kNoallocMaxDevices, WINDQ_ERR_UNSUPPORTED,
+                "windq_act_stats_noalloc: device %d is beyond the %d devices this entry point keeps addresses for",
+                ctx->device, kNoallocMaxDevices);
+  const int slices = act_slices(T);
+  WINDQ_REQUIRE(ctx, slices <= 65535, WINDQ_ERR_SHAPE, "windq_act_stats_noalloc: T = %lld is too large", (long long)T);
+  DeviceGuard guard(ctx->device);
+  float* partial = nullptr;
+  WINDQ_CUDA(ctx, noalloc_scratch(ctx->device, &partial));
+  const int rows_per_slice = kActRowsPar * kActMaxRowsPerThread;
+  cudaStream_t st = (cudaStream_t)stream;
+  dim3 grid((unsigned)((C + kActCols - 1) / kActCols), (unsigned)slices);
+  // every partial[slice][channel] that the second kernel reads is written by the first one, so
+  // nothing left in the array by an earlier call is ever read and nothing needs clearing
+  act_partial_kernel<<<grid, 256, 0, st>>>((const __half*)X, T, (int)C, ldx, rows_per_slice, partial);
+  WINDQ_CUDA(ctx, cudaGetLastError());
+  act_finalize_kernel<<<(unsigned)((C + 255) / 256), 256, 0, st>>>(partial, slices, (int)C, 1.0 / (double)T, s_out);
+  WINDQ_CUDA(ctx, cudaGetLastError());
+  return WINDQ_OK;
+}

@@ -392,31 +392,38 @@ def run_e2e_leg(wq, ctx, spec, model, plans, plans_np, buf, grid_d, steps, warmu
     return ms, wall, h2d_per_step, d2h[0] // max(steps, 1), host_blocks
 
 
+ORACLE_SAMPLE_MATRICES = 5     # block 0: q, k, v, o and gate projections (about 55 % of a block's weights)
+
+
 def oracle_sample(spec, seed, threads):
-    """The CPU oracle on a bounded sample of the workload: the whole hot path for block 0's q_proj
-    (4096 x 4096) at every chunk width, its calibration statistics, features and the three plans.
+    """The CPU oracle on a bounded sample of the workload: the whole hot path for the first
+    ORACLE_SAMPLE_MATRICES matrices of block 0 -- their calibration statistics, and per matrix
+    unit_features + fit_eval at every chunk width and the three plans at APPLY_G.
     Returns (seconds, unit x bit-width evaluations, description)."""
     import oracle
-    m = matrices_of(spec)[0]
-    W = ws.block_weight(spec, seed, 0, m).numpy()
-    X = ws.block_input(spec, seed, 0, m.x_id).numpy()
+    mats = matrices_of(spec)[:ORACLE_SAMPLE_MATRICES]
+    Ws = [ws.block_weight(spec, seed, 0, m).numpy() for m in mats]
+    Xs = {i: ws.block_input(spec, seed, 0, i).numpy() for i in sorted({m.x_id for m in mats})}
     grid = ws.clip_grid(spec.K)
+    rng = np.random.default_rng(seed)
     t0 = time.perf_counter()
-    s = oracle.act_stats(X)
+    stats = {i: oracle.act_stats(X) for i, X in Xs.items()}
     evals = 0
-    for G in spec.chunk_widths:
-        oracle.unit_features(W, G, s) if threads <= 1 else _parallel_features(oracle, W, G, s, threads)
-        fit = oracle.fit_eval(W, G, s, grid, threads=threads, want_group_err=False)
-        evals += 6 * (m.C // G)
-        if G == APPLY_G:
-            rng = np.random.default_rng(seed)
-            for ti, _ in enumerate(TARGET_BITS):
-                acts = rng.choice(7, size=m.C // G, p=np.array(ws.ACTION_MIX) / sum(ws.ACTION_MIX)).astype(np.uint8)
-                oracle.effective_bits(acts, m.R, G)
-                oracle.apply_plan(W, G, s, grid, acts, fit["clip_idx"])
+    for m, W in zip(mats, Ws):
+        s = stats[m.x_id]
+        for G in spec.chunk_widths:
+            oracle.unit_features(W, G, s) if threads <= 1 else _parallel_features(oracle, W, G, s, threads)
+            fit = oracle.fit_eval(W, G, s, grid, threads=threads, want_group_err=False)
+            evals += 6 * (m.C // G)
+            if G == APPLY_G:
+                for ti, _ in enumerate(TARGET_BITS):
+                    acts = rng.choice(7, size=m.C // G, p=np.array(ws.ACTION_MIX) / sum(ws.ACTION_MIX)).astype(np.uint8)
+                    oracle.effective_bits(acts, m.R, G)
+                    oracle.apply_plan(W, G, s, grid, acts, fit["clip_idx"])
     dt = time.perf_counter() - t0
-    desc = "block 0 %s %dx%d, T=%d: act_stats, unit_features + fit_eval at G=%s, 3 plans applied at G=%d" % (
-        m.name, m.R, m.C, spec.T, "/".join(map(str, spec.chunk_widths)), APPLY_G)
+    desc = "block 0 of %d, matrices %s (%.1f M weights), T=%d: act_stats, unit_features + fit_eval at G=%s, 3 plans applied at G=%d" % (
+        spec.n_blocks, "/".join(m.name for m in mats), sum(m.R * m.C for m in mats) / 1e6, spec.T,
+        "/".join(map(str, spec.chunk_widths)), APPLY_G)
     return dt, evals, desc
 
 

@@ -280,11 +280,34 @@ def test_argument_errors(wq, ctx):
 
 
 # ------------------------------------------------------------------ full size, sampled units
-def test_full_size_matrix_sampled_units(wq, ctx, oracle):
-    """An 11008 x 4096 Student-t matrix generated on the device (the benchmark's recipe and launch
-    shape); the oracle recomputes sampled units from the same bits."""
-    spec = ws.CONFIGS["cfg3_llama7b_model"]
-    m = spec.block_matrices()[4]
+def plan_for_target(wq, ctx, U, R, G, target, seed):
+    """A seeded random plan at `target` average bits (the benchmark's recipe): the cost table comes
+    from windq_effective_bits itself, the drawing from the shared generator module."""
+    all_actions = torch.arange(7, dtype=torch.uint8, device="cuda")
+    per_action = wq.windq_effective_bits(ctx, all_actions, R, G)["unit_centibits"].cpu().numpy()
+    costs = np.tile(per_action[None, :], (U, 1))
+    return ws.random_plan(costs, np.full(U, R * G, np.int64), target, seed)
+
+
+FULL_SIZE_CASES = [
+    # config, matrix index in the block, units sampled per chunk width, plan target (None: uniform random actions)
+    ("cfg2_llama7b_block", 6, 2, 2.0),      # down_proj 4096 x 11008, N(0, 0.02), plan at 2.0 bits
+    ("cfg3_llama7b_model", 4, 3, None),     # gate_proj 11008 x 4096, Student-t, chunk widths 64 and 128
+    ("cfg3_llama7b_model", 0, 2, 1.58),     # q_proj 4096 x 4096, plan at 1.58 bits
+    ("cfg4_llama13b_model", 5, 2, 3.0),     # up_proj 13824 x 5120, 40 clip ratios, 4096 tokens
+    ("cfg5_llama70b_model", 4, 1, 2.0),     # gate_proj 28672 x 8192
+    ("cfg5_llama70b_model", 1, 2, 2.0),     # k_proj 1024 x 8192 (grouped-query attention)
+    ("cfg5_llama70b_model", 6, 1, 2.0),     # down_proj 8192 x 28672
+]
+
+
+@pytest.mark.parametrize("config,mi,n_units,target", FULL_SIZE_CASES)
+def test_full_size_matrix_sampled_units(wq, ctx, oracle, config, mi, n_units, target):
+    """A full-size matrix of one of the five configurations, generated on the device with the
+    benchmark's recipe and run in the benchmark's launch shape; the oracle recomputes sampled units
+    from the same bits.  Properties that hold at any size are checked on every unit."""
+    spec = ws.CONFIGS[config]
+    m = spec.block_matrices()[mi]
     W = ws.block_weight(spec, 0, 0, m, device="cuda")
     X = ws.block_input(spec, 0, 0, m.x_id, device="cuda")
     s = wq.windq_act_stats(ctx, X)
@@ -292,18 +315,35 @@ def test_full_size_matrix_sampled_units(wq, ctx, oracle):
     grid_d = torch.from_numpy(grid).cuda()
     s_h = s.cpu().numpy()
     assert close(s_h, oracle.act_stats(X.cpu().numpy())).all()
+    del X
     for G in spec.chunk_widths:
         U = m.C // G
         fit = wq.windq_fit_eval(ctx, W, G, s, grid_d)
         feat = wq.windq_unit_features(ctx, W, G, s).cpu().numpy()
         rng = np.random.default_rng(G)
-        acts = rng.integers(0, 7, U).astype(np.uint8)
+        if target is None:
+            acts = rng.integers(0, 7, U).astype(np.uint8)
+        else:
+            acts = plan_for_target(wq, ctx, U, m.R, G, target, 17)
         a_d = torch.from_numpy(acts).cuda()
         eb = wq.windq_effective_bits(ctx, a_d, m.R, G)
+        o_eb = oracle.effective_bits(acts, m.R, G)
+        assert int(eb["total_centibits"].item()) == o_eb["total_centibits"]
+        assert int(eb["total_packed_bytes"].item()) == o_eb["total_packed_bytes"]
+        assert (eb["code_offsets"].cpu().numpy() == o_eb["code_offsets"]).all()
+        if target is not None:
+            assert abs(o_eb["total_centibits"] / (100.0 * m.R * m.C) - target) <= 0.005
         codes = torch.empty(int(eb["code_offsets"][-1].item()), dtype=torch.uint8, device="cuda")
         plan = wq.windq_apply_plan(ctx, W, G, s, grid_d, a_d, eb["code_offsets"], codes, fit["clip_idx"])
         offs = eb["code_offsets"].cpu().numpy()
-        for u in rng.choice(U, 3, replace=False):
+        # any size: every clip index is a grid index; errors are finite and non-negative; skip units
+        # come back unchanged
+        err = fit["err"].cpu().numpy()
+        assert int(fit["clip_idx"].max().item()) < spec.K
+        assert np.isfinite(err).all() and (err >= 0).all() and (fit["energy"].cpu().numpy() >= err[:, 5] * 0).all()
+        for u in np.flatnonzero(acts == 0)[:2]:
+            assert torch.equal(plan["wq"][:, u * G:(u + 1) * G], W[:, u * G:(u + 1) * G])
+        for u in rng.choice(U, n_units, replace=False):
             Wu = W[:, u * G:(u + 1) * G].cpu().numpy()
             su = s_h[u * G:(u + 1) * G]
             want = oracle.fit_eval(Wu, G, su, grid, threads=8, want_group_err=False)
@@ -317,3 +357,5 @@ def test_full_size_matrix_sampled_units(wq, ctx, oracle):
             assert (plan["scales"][u].cpu().view(torch.int16).numpy().view(np.uint16) == wp["scales"][0]).all()
             assert (plan["zeros"][u].cpu().view(torch.int16).numpy().view(np.uint16) == wp["zeros"][0]).all()
             assert (plan["wq"][:, u * G:(u + 1) * G].cpu().view(torch.int16).numpy().view(np.uint16) == wp["wq"]).all()
+    del W
+    torch.cuda.empty_cache()

@@ -1,0 +1,97 @@
+"""The multi-GPU host logic on CPU: two gloo ranks shard the blocks of a model with no data-path
+exchange, and the only cross-rank values (plan bits: int64 sum; step time: max) are reduced exactly.
+Each rank runs the oracle's bit accounting on its own blocks' plans; the sum over ranks must equal
+the single-process total."""
+import os
+import socket
+import sys
+
+import numpy as np
+import pytest
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _load_sharding():
+    # the sharding helpers are plain torch.distributed code; load the file directly so that the
+    # CUDA package (which builds and loads the library on import) is not needed on CPU
+    import importlib.util
+    spec = importlib.util.spec_from_file_location("windq_sharding", os.path.join(ROOT, "paper_2605_26660_b200", "sharding.py"))
+    mod = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(mod)
+    return mod
+
+
+def _free_port():
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+N_BLOCKS, UNITS_PER_BLOCK, R, G = 7, 24, 64, 128
+
+
+def _block_plan(block):
+    rng = np.random.default_rng(1000 + block)
+    return rng.integers(0, 7, UNITS_PER_BLOCK).astype(np.uint8)
+
+
+def _worker(rank, world, port, out_dir):
+    sys.path.insert(0, ROOT)
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        sharding = _load_sharding()
+        import oracle
+        oracle.build()
+        mine = sharding.block_range(N_BLOCKS, rank, world)
+        local_cb, local_n = 0, 0
+        for b in mine:
+            eb = oracle.effective_bits(_block_plan(b), R, G)
+            local_cb += int(eb["total_centibits"])
+            local_n += UNITS_PER_BLOCK * R * G
+        total_cb = sharding.sum_int64(local_cb)
+        avg = sharding.average_bits(local_cb, local_n)
+        slowest = sharding.max_float(10.0 + rank)
+        np.save(os.path.join(out_dir, "rank%d.npy" % rank),
+                np.array([total_cb, avg, slowest, len(mine), min(mine, default=-1), max(mine, default=-1)], np.float64))
+    finally:
+        dist.destroy_process_group()
+
+
+def test_block_range_is_a_partition():
+    sharding = _load_sharding()
+    for n in (0, 1, 7, 32, 80):
+        for world in (1, 2, 3, 8):
+            seen = [b for r in range(world) for b in sharding.block_range(n, r, world)]
+            assert seen == list(range(n))
+            sizes = [len(sharding.block_range(n, r, world)) for r in range(world)]
+            assert max(sizes) - min(sizes) <= 1
+    with pytest.raises(ValueError):
+        sharding.block_range(4, 2, 2)
+
+
+def test_reductions_without_a_process_group():
+    sharding = _load_sharding()
+    assert sharding.sum_int64(12345678901234) == 12345678901234
+    assert sharding.max_float(1.5) == 1.5
+    assert sharding.average_bits(2 * 100 * 1000, 1000) == 2.0
+
+
+def test_two_gloo_ranks_agree_with_one_process(tmp_path, oracle):
+    world = 2
+    port = _free_port()
+    mp.start_processes(_worker, args=(world, port, str(tmp_path)), nprocs=world, join=True, start_method="spawn")
+    want_cb = sum(int(oracle.effective_bits(_block_plan(b), R, G)["total_centibits"]) for b in range(N_BLOCKS))
+    want_avg = want_cb / (100.0 * N_BLOCKS * UNITS_PER_BLOCK * R * G)
+    got = [np.load(os.path.join(str(tmp_path), "rank%d.npy" % r)) for r in range(world)]
+    for g in got:
+        assert int(g[0]) == want_cb                  # exact int64 sum
+        assert g[1] == want_avg                      # b_bar = sum B_i / sum n_i over all ranks
+        assert g[2] == 10.0 + (world - 1)            # step time = slowest rank
+    assert sum(int(g[3]) for g in got) == N_BLOCKS   # every block scored exactly once
+    assert int(got[0][5]) + 1 == int(got[1][4])      # contiguous, disjoint ranges

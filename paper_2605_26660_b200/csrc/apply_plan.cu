@@ -3,28 +3,26 @@
 //
 // With clip indices supplied this is a streaming kernel bound by HBM: 2 bytes read per weight,
 // 2 bytes written for the fake-quantised copy and bits/8 for the codes.  Thread mapping as in
-// the fit (LG lanes per group, 32 values per lane in registers).  A block handles one tile =
-// (unit, 64 or 128 consecutive rows); the action is uniform over the tile, so there is no
-// divergence.  Each lane packs its own 32 codes into whole 32-bit words in registers (1, 2, 3, 4
-// and 8 bit all give whole bytes per lane); the words are staged in shared memory so that the
-// tile's packed bytes, which are contiguous in the output, leave with 128-bit stores.  Only the
-// base-3 ternary packing crosses lanes (5 trits per byte): its trits are staged as bytes and the
-// output bytes are assembled from shared memory.
+// the fit (LG lanes per group, 32 values per lane in registers).  Work is split into items =
+// (unit, GPW consecutive rows), one warp per item; the warps of a persistent grid walk the items
+// with a stride of the number of warps, so that neighbouring warps read and write neighbouring
+// rows.  What keeps HBM busy is that the weights of a warp's NEXT item are already on their way
+// (cp.async into a 2 KB shared-memory buffer per warp, two buffers) while it fits, quantises
+// and stores the current one.
+//
+// Packing.  Each lane packs its own 32 codes into whole 32-bit words in registers (1, 2, 3, 4
+// and 8 bit all give whole words per lane) and the rows of an item are adjacent in the output, so
+// the words of a warp form one contiguous run and go out with plain vector stores, no staging.
+// Only the base-3 ternary packing crosses lanes (5 trits per byte): its trits are staged as 2-bit
+// fields in shared memory and each output byte is looked up from the 10-bit window that holds its
+// five trits.
 #include "fit_device.cuh"
 
 namespace windq {
 
 constexpr int kApplyWarps = 4;
 
-template <int G>
-struct ApplyTile {
-  static constexpr int GPW = Map<G>::GPW;
-  static constexpr int ROWS = (kApplyWarps * GPW >= 64) ? kApplyWarps * GPW : 64;  // multiple of 16
-  static constexpr int PASSES = ROWS / (kApplyWarps * GPW);
-  static constexpr int STAGE_BYTES = ROWS * G;
-};
-
-// 32 small codes -> packed little-endian words; returns the number of words.
+// 32 small codes -> packed little-endian words.
 template <int BITS>
 __device__ __forceinline__ void pack_words(const unsigned (&q)[32], unsigned (&out)[8]) {
 #pragma unroll
@@ -39,50 +37,130 @@ __device__ __forceinline__ void pack_words(const unsigned (&q)[32], unsigned (&o
 
 __device__ __forceinline__ unsigned short half_bits(float x) { return __half_as_ushort(__float2half_rn(x)); }
 
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src) {
+  const unsigned dst = (unsigned)__cvta_generic_to_shared(smem_dst);
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_all_but_one() { asm volatile("cp.async.wait_group 1;" ::: "memory"); }
+
+// Shared memory of a block: per warp two weight buffers (GPW rows x G halves = 2 KB each) and a
+// staging area for the ternary packing (1 KB; 256 bytes of 2-bit fields are used); then, only when the clip search has to be repeated, the
+// candidate tables of the warps.
+constexpr int kApplyWarpBytes = 2 * 2048 + 1024;
+
 template <int G>
-__global__ void __launch_bounds__(kApplyWarps * 32)
+__host__ __device__ inline int apply_cand_chunk() {
+  return (336 / Map<G>::GPW > 64) ? 64 : 336 / Map<G>::GPW;
+}
+
+// The fake-quantised values of a lane (as fp16 bit patterns) -> its 64 bytes of Wq.
+__device__ __forceinline__ void store_wq(__half* dst, const unsigned short (&h)[32]) {
+  uint4* p = reinterpret_cast<uint4*>(dst);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    uint4 v;
+    v.x = h[8 * i + 0] | ((unsigned)h[8 * i + 1] << 16);
+    v.y = h[8 * i + 2] | ((unsigned)h[8 * i + 3] << 16);
+    v.z = h[8 * i + 4] | ((unsigned)h[8 * i + 5] << 16);
+    v.w = h[8 * i + 6] | ((unsigned)h[8 * i + 7] << 16);
+    p[i] = v;
+  }
+}
+
+// n_words packed words of a lane -> dst (4-byte aligned; 8- or 16-byte aligned for 2, 4, 8 words).
+__device__ __forceinline__ void store_words(uint8_t* dst, const unsigned (&w)[8], int n_words) {
+  switch (n_words) {
+    case 8:
+      reinterpret_cast<uint4*>(dst)[0] = make_uint4(w[0], w[1], w[2], w[3]);
+      reinterpret_cast<uint4*>(dst)[1] = make_uint4(w[4], w[5], w[6], w[7]);
+      break;
+    case 4: reinterpret_cast<uint4*>(dst)[0] = make_uint4(w[0], w[1], w[2], w[3]); break;
+    case 3: {
+      unsigned* d = reinterpret_cast<unsigned*>(dst);
+      d[0] = w[0]; d[1] = w[1]; d[2] = w[2];
+      break;
+    }
+    case 2: reinterpret_cast<uint2*>(dst)[0] = make_uint2(w[0], w[1]); break;
+    default: reinterpret_cast<unsigned*>(dst)[0] = w[0]; break;
+  }
+}
+
+// SEARCH = false: clip indices are supplied.  SEARCH = true: the clip search is repeated for the
+// unit's bit-width (the candidate table follows the warp buffers in shared memory).
+template <int G, bool SEARCH>
+__global__ void __launch_bounds__(kApplyWarps * 32, 4)
 apply_plan_kernel(const __half* __restrict__ W, int R, int U, int64_t ldw, const float* __restrict__ s,
                   const float* __restrict__ clip, int K, const uint8_t* __restrict__ actions,
                   const uint8_t* __restrict__ clip_idx, const long long* __restrict__ code_offsets,
                   uint8_t* __restrict__ codes_out, __half* __restrict__ scales_out, __half* __restrict__ zeros_out,
-                  __half* __restrict__ Wq_out, int row_tiles, int chunk, int stride) {
-  using T = ApplyTile<G>;
+                  __half* __restrict__ Wq_out, int rows_blocks) {
   constexpr int LG = Map<G>::LG, GPW = Map<G>::GPW;
   extern __shared__ uint4 smem_u4[];
-  uint8_t* stage = reinterpret_cast<uint8_t*>(smem_u4);
-  Cand* cand_all = reinterpret_cast<Cand*>(stage + T::STAGE_BYTES);
-
-  const int u = blockIdx.x / row_tiles, rt = blockIdx.x % row_tiles;
-  const int a = actions[u];
-  if (a > 6) return;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int g = lane / LG, q = lane % LG;
-  Cand* cand = cand_all + (size_t)warp * GPW * stride;
-  const int r0 = rt * T::ROWS;
-  const int rows_here = min(T::ROWS, R - r0);
-  const int bpg = group_code_bytes(a, G);
-  uint8_t* out_base = codes_out + code_offsets[u] + (long long)r0 * bpg;
+  uint8_t* mine = reinterpret_cast<uint8_t*>(smem_u4) + (size_t)warp * kApplyWarpBytes;
+  uint8_t* trits = mine + 4096;
+  // base3[x] = sum over m < 5 of ((x >> 2m) & 3) * 3^m: five 2-bit trits -> one packed byte
+  __shared__ uint8_t base3[1024];
+  for (int x = threadIdx.x; x < 1024; x += kApplyWarps * 32)
+    base3[x] = (uint8_t)((x & 3) + 3 * ((x >> 2) & 3) + 9 * ((x >> 4) & 3) + 27 * ((x >> 6) & 3) + 81 * ((x >> 8) & 3));
+  __syncthreads();
+  const int chunk = apply_cand_chunk<G>(), stride = chunk | 1;
+  Cand* cand = reinterpret_cast<Cand*>(reinterpret_cast<uint8_t*>(smem_u4) + (size_t)kApplyWarps * kApplyWarpBytes) +
+               (size_t)warp * GPW * stride;
 
-  Lane32 sv;
-  load_stats(s + (int64_t)u * G + 32 * q, sv);
+  const int n_items = U * rows_blocks;
+  const int n_warps = gridDim.x * kApplyWarps;
+  int item = blockIdx.x * kApplyWarps + warp;
 
-#pragma unroll 1
-  for (int pass = 0; pass < T::PASSES; ++pass) {
-    const int rl = (pass * kApplyWarps + warp) * GPW + g;  // row inside the tile
-    const int row = r0 + rl;
+  // asks for the lane's 64 bytes of `it` into buffer `buf` (rows past the end repeat the last row)
+  auto prefetch = [&](int it, int buf) {
+    if (it < n_items) {
+      const int u = it / rows_blocks, rb = it - u * rows_blocks;
+      const int row = min(rb * GPW + g, R - 1);
+      const __half* src = W + (int64_t)row * ldw + (int64_t)u * G + 32 * q;
+      uint8_t* dst = mine + buf * 2048 + lane * 64;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) cp_async16(dst + 16 * i, src + 8 * i);
+    }
+    cp_async_commit();  // one group per call, possibly empty, so that the wait below counts right
+  };
+
+  prefetch(item, 0);
+  for (int n = 0; item < n_items; item += n_warps, ++n) {
+    prefetch(item + n_warps, (n + 1) & 1);
+    cp_async_wait_all_but_one();  // this lane's 64 bytes of the current item have arrived
+    const int u = item / rows_blocks, rb = item - u * rows_blocks;
+    const int a = actions[u];
+    if (a > 6) continue;
+    const int row = rb * GPW + g;
     const bool live = row < R;
-    const int row_ld = live ? row : R - 1;
-    const __half* wp = W + (int64_t)row_ld * ldw + (int64_t)u * G + 32 * q;
+    const int bpg = group_code_bytes(a, G);
+    uint8_t* unit_codes = codes_out + code_offsets[u];
+    uint8_t* row_codes = unit_codes + (long long)row * bpg;
+    __half* wq_dst = Wq_out ? Wq_out + (int64_t)row * ldw + (int64_t)u * G + 32 * q : nullptr;
+
+    uint4 raw[4];
+    {
+      const uint4* src = reinterpret_cast<const uint4*>(mine + (n & 1) * 2048 + lane * 64);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) raw[i] = src[i];
+    }
+    // the unit's last rows also write the zero padding up to the next 16-byte boundary
+    if (rb == rows_blocks - 1) {
+      const long long total = (long long)R * bpg;
+      const int pad = (int)(((total + 15) & ~15ll) - total);
+      if (lane < pad) unit_codes[total + lane] = 0;
+    }
+
     if (a == 0) {  // skip: the raw fp16 values are the codes and the reconstruction
       if (live) {
-        const uint4* src = reinterpret_cast<const uint4*>(wp);
-        uint4* dst = reinterpret_cast<uint4*>(out_base + (long long)rl * bpg + 64 * q);
-        uint4* wq = Wq_out ? reinterpret_cast<uint4*>(Wq_out + (int64_t)row * ldw + (int64_t)u * G + 32 * q) : nullptr;
+        uint4* dst = reinterpret_cast<uint4*>(row_codes + 64 * q);
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-          const uint4 v = __ldg(src + i);
-          dst[i] = v;
-          if (wq) wq[i] = v;
+          dst[i] = raw[i];
+          if (wq_dst) reinterpret_cast<uint4*>(wq_dst)[i] = raw[i];
         }
         if (q == 0) {
           scales_out[(int64_t)u * R + row] = __ushort_as_half(0);
@@ -91,8 +169,9 @@ apply_plan_kernel(const __half* __restrict__ W, int R, int U, int64_t ldw, const
       }
       continue;
     }
+
     Lane32 wv;
-    load_weights(wp, wv);
+    unpack_weights(raw, wv);
     unsigned code[32];
     unsigned short wq16[32];
     float scale_store, zero_store = 0.0f;
@@ -102,9 +181,11 @@ apply_plan_kernel(const __half* __restrict__ W, int R, int U, int64_t ldw, const
       group_range<G>(wv, mn, mx);
       const float rng = __fsub_rn(mx, mn);
       int k;
-      if (clip_idx) {
-        k = min((int)clip_idx[((int64_t)bi * U + u) * R + row_ld], K - 1);
+      if (!SEARCH) {
+        k = min((int)clip_idx[((int64_t)bi * U + u) * R + min(row, R - 1)], K - 1);
       } else {
+        Lane32 sv;
+        load_stats(s + (int64_t)u * G + 32 * q, sv);
         float be;
         search_uniform<G>(wv, sv, mn, rng, bi, clip, K, cand, chunk, stride, lane, be, k);
       }
@@ -124,8 +205,10 @@ apply_plan_kernel(const __half* __restrict__ W, int R, int U, int64_t ldw, const
       scale_store = scale;
       zero_store = zf;
     } else {
-      const LowBitFit f = fit_low_bits<G>(wv, sv);
-      const float alpha = (a == 5) ? f.alpha_t : f.alpha_b;
+      Lane32 sv;
+      load_stats(s + (int64_t)u * G + 32 * q, sv);
+      float delta = 0.0f;
+      const float alpha = (a == 5) ? ternary_scale<G>(wv, sv, delta) : binary_scale<G>(wv, sv);
       const unsigned short pos = half_bits(alpha), neg = half_bits(-alpha);
 #pragma unroll
       for (int l = 0; l < 4; ++l)
@@ -134,7 +217,7 @@ apply_plan_kernel(const __half* __restrict__ W, int R, int U, int64_t ldw, const
           const float w = wv.get(l, i);
           const bool is_neg = w < 0.0f;
           if (a == 5) {
-            const bool in = fabsf(w) > f.delta;
+            const bool in = fabsf(w) > delta;
             code[8 * l + i] = in ? (is_neg ? 0u : 2u) : 1u;
             wq16[8 * l + i] = in ? (is_neg ? neg : pos) : (unsigned short)0;
           } else {
@@ -144,101 +227,83 @@ apply_plan_kernel(const __half* __restrict__ W, int R, int U, int64_t ldw, const
         }
       scale_store = alpha;
     }
+
     if (live) {
-      if (Wq_out) {
-        uint4* wq = reinterpret_cast<uint4*>(Wq_out + (int64_t)row * ldw + (int64_t)u * G + 32 * q);
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          uint4 v;
-          v.x = wq16[8 * i + 0] | ((unsigned)wq16[8 * i + 1] << 16);
-          v.y = wq16[8 * i + 2] | ((unsigned)wq16[8 * i + 3] << 16);
-          v.z = wq16[8 * i + 4] | ((unsigned)wq16[8 * i + 5] << 16);
-          v.w = wq16[8 * i + 6] | ((unsigned)wq16[8 * i + 7] << 16);
-          wq[i] = v;
-        }
-      }
+      if (wq_dst) store_wq(wq_dst, wq16);
       if (q == 0) {
         scales_out[(int64_t)u * R + row] = __float2half_rn(scale_store);
         zeros_out[(int64_t)u * R + row] = __float2half_rn(zero_store);
       }
-      unsigned words[8];
+    }
+    unsigned words[8];
+    if (a != 5) {
       int n_words;
-      unsigned* dst;
       switch (a) {
         case 1: pack_words<8>(code, words); n_words = 8; break;
         case 2: pack_words<4>(code, words); n_words = 4; break;
         case 3: pack_words<3>(code, words); n_words = 3; break;
         case 4: pack_words<2>(code, words); n_words = 2; break;
-        case 5: pack_words<8>(code, words); n_words = 8; break;  // trits as bytes
         default: pack_words<1>(code, words); n_words = 1; break;
       }
-      if (a == 5) dst = reinterpret_cast<unsigned*>(stage + (size_t)rl * G + 32 * q);
-      else dst = reinterpret_cast<unsigned*>(stage + (size_t)rl * bpg + 4 * n_words * q);
-#pragma unroll
-      for (int i = 0; i < 8; ++i)
-        if (i < n_words) dst[i] = words[i];
-    }
-  }
-  if (a == 0) return;
-  __syncthreads();
-
-  // the tile's packed bytes are contiguous in the output; the unit's last tile also writes the
-  // zero padding up to the next 16-byte boundary
-  const int total = rows_here * bpg;
-  const int out_len = (total + 15) & ~15;
-  for (int i = threadIdx.x * 16; i < out_len; i += kApplyWarps * 32 * 16) {
-    uint4 v;
-    if (a != 5) {
-      v = *reinterpret_cast<const uint4*>(stage + i);
+      if (live) store_words(row_codes + 4 * n_words * q, words, n_words);
     } else {
-      unsigned w4[4] = {0u, 0u, 0u, 0u};
-#pragma unroll
-      for (int b = 0; b < 16; ++b) {
-        const int B = i + b;
-        if (B < total) {
-          const int rl = B / bpg, bi = B - rl * bpg;
-          const uint8_t* t = stage + (size_t)rl * G + 5 * bi;
-          unsigned val = 0u, p3 = 1u;
-#pragma unroll
-          for (int m = 0; m < 5; ++m) {
-            if (5 * bi + m < G) val += t[m] * p3;
-            p3 *= 3u;
-          }
-          w4[b >> 2] |= val << (8 * (b & 3));
-        }
+      // codes as 2-bit fields into the warp's buffer; an output byte is the base-3 value of five
+      // consecutive fields, i.e. of a 10-bit window, looked up in the block's table
+      pack_words<2>(code, words);
+      __syncwarp();  // the previous item's fields have been read
+      *reinterpret_cast<uint2*>(trits + g * (G / 4) + 8 * q) = make_uint2(words[0], words[1]);
+      __syncwarp();
+      const int rows_here = min(GPW, R - rb * GPW);
+      uint8_t* dst = unit_codes + (long long)rb * GPW * bpg;
+      for (int B = lane; B < rows_here * bpg; B += 32) {
+        const int rl = B / bpg, bj = B - rl * bpg;
+        const uint8_t* t = trits + rl * (G / 4) + ((10 * bj) >> 3);
+        unsigned x = ((unsigned)t[0] | ((unsigned)t[1] << 8)) >> ((10 * bj) & 7);
+        const int valid = min(5, G - 5 * bj);  // the row's last byte holds fewer than five trits
+        x &= (1u << (2 * valid)) - 1u;
+        dst[B] = base3[x];
       }
-      v = make_uint4(w4[0], w4[1], w4[2], w4[3]);
     }
-    if (i + 16 > total) {  // mask the padding bytes of the last chunk
-      unsigned* pv = reinterpret_cast<unsigned*>(&v);
-#pragma unroll
-      for (int b = 0; b < 16; ++b)
-        if (i + b >= total) pv[b >> 2] &= ~(0xffu << (8 * (b & 3)));
-    }
-    *reinterpret_cast<uint4*>(out_base + i) = v;
   }
 }
 
-template <int G>
+template <int G, bool SEARCH>
 windq_status launch_apply(windq_ctx* ctx, const __half* W, int R, int U, int64_t ldw, const float* s, const float* clip,
                           int K, const uint8_t* actions, const uint8_t* clip_idx, const long long* code_offsets,
                           uint8_t* codes_out, __half* scales_out, __half* zeros_out, __half* Wq_out, cudaStream_t st) {
-  using T = ApplyTile<G>;
-  const int chunk = 336 / T::GPW > 64 ? 64 : 336 / T::GPW, stride = chunk | 1;
-  const size_t smem = (size_t)T::STAGE_BYTES + (size_t)kApplyWarps * T::GPW * stride * sizeof(Cand);
-  static bool configured = false;
-  if (!configured) {
-    WINDQ_CUDA(ctx, cudaFuncSetAttribute(apply_plan_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    configured = true;
+  constexpr int GPW = Map<G>::GPW;
+  const int stride = apply_cand_chunk<G>() | 1;
+  const size_t smem = (size_t)kApplyWarps * kApplyWarpBytes + (SEARCH ? (size_t)kApplyWarps * GPW * stride * sizeof(Cand) : 0);
+  static int blocks_per_sm = 0;  // same for every device this library supports
+  if (blocks_per_sm == 0) {
+    WINDQ_CUDA(ctx, cudaFuncSetAttribute(apply_plan_kernel<G, SEARCH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    int n = 0;
+    WINDQ_CUDA(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, apply_plan_kernel<G, SEARCH>, kApplyWarps * 32, smem));
+    blocks_per_sm = n > 0 ? n : 1;
   }
-  const int row_tiles = (R + T::ROWS - 1) / T::ROWS;
-  const int64_t blocks = (int64_t)U * row_tiles;
-  WINDQ_REQUIRE(ctx, blocks < (1ll << 31), WINDQ_ERR_SHAPE, "windq_apply_plan: too many tiles");
-  apply_plan_kernel<G><<<(unsigned)blocks, kApplyWarps * 32, smem, st>>>(W, R, U, ldw, s, clip, K, actions, clip_idx,
-                                                                          code_offsets, codes_out, scales_out, zeros_out,
-                                                                          Wq_out, row_tiles, chunk, stride);
+  const int rows_blocks = (R + GPW - 1) / GPW;
+  const int64_t n_items = (int64_t)U * rows_blocks;
+  WINDQ_REQUIRE(ctx, n_items < (1ll << 30), WINDQ_ERR_SHAPE, "windq_apply_plan: R * C is too large for one call");
+  int64_t grid = (int64_t)ctx->sm_count * blocks_per_sm;
+  const int64_t need = (n_items + kApplyWarps - 1) / kApplyWarps;
+  if (grid > need) grid = need;
+  apply_plan_kernel<G, SEARCH><<<(unsigned)grid, kApplyWarps * 32, smem, st>>>(W, R, U, ldw, s, clip, K, actions, clip_idx,
+                                                                               code_offsets, codes_out, scales_out,
+                                                                               zeros_out, Wq_out, rows_blocks);
   WINDQ_CUDA(ctx, cudaGetLastError());
   return WINDQ_OK;
+}
+
+template <int G>
+windq_status launch_apply_any(windq_ctx* ctx, const __half* W, int R, int U, int64_t ldw, const float* s,
+                              const float* clip, int K, const uint8_t* actions, const uint8_t* clip_idx,
+                              const long long* code_offsets, uint8_t* codes_out, __half* scales_out, __half* zeros_out,
+                              __half* Wq_out, cudaStream_t st) {
+  if (clip_idx)
+    return launch_apply<G, false>(ctx, W, R, U, ldw, s, clip, K, actions, clip_idx, code_offsets, codes_out, scales_out,
+                                  zeros_out, Wq_out, st);
+  return launch_apply<G, true>(ctx, W, R, U, ldw, s, clip, K, actions, clip_idx, code_offsets, codes_out, scales_out,
+                               zeros_out, Wq_out, st);
 }
 
 }  // namespace windq
@@ -266,10 +331,10 @@ extern "C" windq_status windq_apply_plan(windq_ctx* ctx, const void* W, int64_t 
   const long long* offs = (const long long*)code_offsets;
   __half *sc = (__half*)scales_out, *zp = (__half*)zeros_out, *wq = (__half*)Wq_out;
   switch (G) {
-    case 32: return launch_apply<32>(ctx, Wh, (int)R, U, ldw, s, clip_grid, K, actions, clip_idx, offs, codes_out, sc, zp, wq, st);
-    case 64: return launch_apply<64>(ctx, Wh, (int)R, U, ldw, s, clip_grid, K, actions, clip_idx, offs, codes_out, sc, zp, wq, st);
-    case 128: return launch_apply<128>(ctx, Wh, (int)R, U, ldw, s, clip_grid, K, actions, clip_idx, offs, codes_out, sc, zp, wq, st);
-    case 256: return launch_apply<256>(ctx, Wh, (int)R, U, ldw, s, clip_grid, K, actions, clip_idx, offs, codes_out, sc, zp, wq, st);
-    default: return launch_apply<512>(ctx, Wh, (int)R, U, ldw, s, clip_grid, K, actions, clip_idx, offs, codes_out, sc, zp, wq, st);
+    case 32: return launch_apply_any<32>(ctx, Wh, (int)R, U, ldw, s, clip_grid, K, actions, clip_idx, offs, codes_out, sc, zp, wq, st);
+    case 64: return launch_apply_any<64>(ctx, Wh, (int)R, U, ldw, s, clip_grid, K, actions, clip_idx, offs, codes_out, sc, zp, wq, st);
+    case 128: return launch_apply_any<128>(ctx, Wh, (int)R, U, ldw, s, clip_grid, K, actions, clip_idx, offs, codes_out, sc, zp, wq, st);
+    case 256: return launch_apply_any<256>(ctx, Wh, (int)R, U, ldw, s, clip_grid, K, actions, clip_idx, offs, codes_out, sc, zp, wq, st);
+    default: return launch_apply_any<512>(ctx, Wh, (int)R, U, ldw, s, clip_grid, K, actions, clip_idx, offs, codes_out, sc, zp, wq, st);
   }
 }

@@ -47,16 +47,29 @@ effective_bits_kernel(const uint8_t* __restrict__ actions, long long U, long lon
       }
       if (unit_cb) unit_cb[u] = cb;
     }
-    scan[t] = bytes;
-    __syncthreads();
-    for (int off = 1; off < 1024; off <<= 1) {
-      const long long v = (t >= off) ? scan[t - off] : 0;
-      __syncthreads();
-      scan[t] += v;
-      __syncthreads();
+    // inclusive scan of the 1024 byte counts: inside each warp, then over the 32 warp totals
+    long long incl = bytes;
+#pragma unroll
+    for (int m = 1; m < 32; m <<= 1) {
+      const long long o = __shfl_up_sync(0xffffffffu, incl, m);
+      if ((t & 31) >= m) incl += o;
     }
-    if (u < U && offsets) offsets[u] = carry + scan[t] - bytes;
-    carry += scan[1023];
+    if ((t & 31) == 31) scan[t >> 5] = incl;
+    __syncthreads();
+    if (t < 32) {
+      long long w = scan[t];
+#pragma unroll
+      for (int m = 1; m < 32; m <<= 1) {
+        const long long o = __shfl_up_sync(0xffffffffu, w, m);
+        if (t >= m) w += o;
+      }
+      scan[32 + t] = w;
+    }
+    __syncthreads();
+    incl += (t >> 5) ? scan[32 + (t >> 5) - 1] : 0ll;
+    const long long chunk_total = scan[63];
+    if (u < U && offsets) offsets[u] = carry + incl - bytes;
+    carry += chunk_total;
     __syncthreads();
   }
 #pragma unroll

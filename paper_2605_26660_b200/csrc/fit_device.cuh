@@ -69,13 +69,11 @@ struct Lane32 {
   }
 };
 
-// 32 fp16 values (64 bytes, 16-byte aligned) -> Lane32.
-__device__ __forceinline__ void load_weights(const __half* p, Lane32& w) {
-  const uint4* p4 = reinterpret_cast<const uint4*>(p);
+// 32 fp16 values, as four 128-bit words -> Lane32.
+__device__ __forceinline__ void unpack_weights(const uint4 (&raw)[4], Lane32& w) {
 #pragma unroll
   for (int l = 0; l < 4; ++l) {
-    const uint4 raw = __ldg(p4 + l);
-    const __half2* h = reinterpret_cast<const __half2*>(&raw);
+    const __half2* h = reinterpret_cast<const __half2*>(&raw[l]);
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       const float2 f = __half22float2(h[i]);
@@ -83,6 +81,15 @@ __device__ __forceinline__ void load_weights(const __half* p, Lane32& w) {
       w.set(l, 2 * i + 1, f.y);
     }
   }
+}
+
+// 32 fp16 values (64 bytes, 16-byte aligned) -> Lane32.
+__device__ __forceinline__ void load_weights(const __half* p, Lane32& w) {
+  const uint4* p4 = reinterpret_cast<const uint4*>(p);
+  uint4 raw[4];
+#pragma unroll
+  for (int l = 0; l < 4; ++l) raw[l] = __ldg(p4 + l);
+  unpack_weights(raw, w);
 }
 
 // 32 fp32 statistics (128 bytes, 16-byte aligned) -> Lane32.
@@ -315,6 +322,90 @@ __device__ __forceinline__ LowBitFit fit_low_bits(const Lane32& w, const Lane32&
   f.err_t = group_tree<G>(Et[0], Et[1], Et[2], Et[3]);
   f.err_b = group_tree<G>(Eb[0], Eb[1], Eb[2], Eb[3]);
   return f;
+}
+
+// ---- scales only (plan application) ------------------------------------------------------------
+// The binary and ternary scales as fit_low_bits computes them -- the same operations in the same
+// order -- without the error sums, and without the sums that only a rare fallback needs unless
+// some group of the warp takes that fallback.  Must be called by all 32 lanes.
+
+// PSUM8 of |w| over the group.
+template <int G>
+__device__ __forceinline__ float group_abs_sum(const Lane32& w) {
+  float A[4];
+#pragma unroll
+  for (int l = 0; l < 4; ++l) {
+    float a = 0.0f;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) a = __fadd_rn(a, fabsf(w.get(l, i)));
+    A[l] = a;
+  }
+  return group_tree<G>(A[0], A[1], A[2], A[3]);
+}
+
+template <int G>
+__device__ __forceinline__ float binary_scale(const Lane32& w, const Lane32& s) {
+  float Sb[4], Bb[4];
+#pragma unroll
+  for (int l = 0; l < 4; ++l) {
+    float sb = 0.0f, bb = 0.0f;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const float sv = s.get(l, i);
+      sb = __fadd_rn(sb, sv);
+      bb = __fmaf_rn(sv, fabsf(w.get(l, i)), bb);
+    }
+    Sb[l] = sb; Bb[l] = bb;
+  }
+  const float sumS = group_tree<G>(Sb[0], Sb[1], Sb[2], Sb[3]);
+  const float sumB = group_tree<G>(Bb[0], Bb[1], Bb[2], Bb[3]);
+  float meanA = 0.0f;
+  if (__any_sync(0xffffffffu, sumS == 0.0f)) meanA = __fmul_rn(group_abs_sum<G>(w), 1.0f / (float)G);
+  return __half2float(__float2half_rn(sumS == 0.0f ? meanA : __fdiv_rn(sumB, sumS)));
+}
+
+// delta = 0.7 * mean |w|; returns the scale (0 when the support is empty).
+template <int G>
+__device__ __forceinline__ float ternary_scale(const Lane32& w, const Lane32& s, float& delta) {
+  const float sumA = group_abs_sum<G>(w);
+  delta = __fmul_rn(0.7f, __fmul_rn(sumA, 1.0f / (float)G));
+  float Bt[4], Ct[4];
+#pragma unroll
+  for (int l = 0; l < 4; ++l) {
+    float bt = 0.0f, ct = 0.0f;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const float aw = fabsf(w.get(l, i)), sv = s.get(l, i);
+      const bool in = aw > delta;
+      bt = __fmaf_rn(sv, in ? aw : 0.0f, bt);
+      ct = __fadd_rn(ct, in ? sv : 0.0f);
+    }
+    Bt[l] = bt; Ct[l] = ct;
+  }
+  float sumBt = group_tree<G>(Bt[0], Bt[1], Bt[2], Bt[3]);
+  float sumCt = group_tree<G>(Ct[0], Ct[1], Ct[2], Ct[3]);
+  // delta < max |w| whenever some w is not zero (0.7 * mean <= 0.7 * max, roundings included), so
+  // the support is empty exactly when every |w| is zero, i.e. when their sum is
+  const bool nonempty = sumA > 0.0f;
+  if (__any_sync(0xffffffffu, nonempty && sumCt == 0.0f)) {  // no activation weight on the support: unweighted mean
+    float Bu[4], Cu[4];
+#pragma unroll
+    for (int l = 0; l < 4; ++l) {
+      float bu = 0.0f, cu = 0.0f;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const float aw = fabsf(w.get(l, i));
+        const bool in = aw > delta;
+        bu = __fadd_rn(bu, in ? aw : 0.0f);
+        cu = __fadd_rn(cu, in ? 1.0f : 0.0f);
+      }
+      Bu[l] = bu; Cu[l] = cu;
+    }
+    const float sumBu = group_tree<G>(Bu[0], Bu[1], Bu[2], Bu[3]);
+    const float sumCu = group_tree<G>(Cu[0], Cu[1], Cu[2], Cu[3]);
+    if (sumCt == 0.0f) { sumBt = sumBu; sumCt = sumCu; }
+  }
+  return nonempty ? __half2float(__float2half_rn(__fdiv_rn(sumBt, sumCt))) : 0.0f;
 }
 
 }  // namespace windq

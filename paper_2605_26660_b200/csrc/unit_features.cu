@@ -3,95 +3,157 @@
 // The magnitude of an fp16 number has 32768 possible bit patterns and their integer order is
 // their numeric order, so ONE histogram of |w| per unit gives the nearest-rank P99, the count
 // above 0.5 * P99 and the count below 1e-6 exactly, and also sum |w| and sum w^2 exactly up to
-// double rounding.  One streaming pass over W (2 bytes per weight, HBM-bound in principle; the
-// shared-memory atomics are what limits it in practice):
-//   pass 1  blocks = (unit, slice of rows): histogram in shared memory (128 KB), flushed to the
-//           unit's histogram in scratch with integer atomics (order-independent, so exact and
-//           reproducible); the signed sum of the slice goes to scratch as a double.
+// double rounding.  One streaming pass over W (2 bytes per weight, bound by HBM):
+//   pass 1  one block of 1024 threads per SM.  The U * R (unit, row) pairs, unit-major, are cut
+//           into equal contiguous shares, one per block, so a block meets two or three units at
+//           most.  It keeps the current unit's histogram in shared memory (128 KB) and, when the
+//           unit ends, adds the non-empty bins to the unit's histogram in scratch with integer
+//           atomics (order-independent, hence exact and reproducible).  Every thread has four
+//           128-bit loads in flight before it touches the histogram: with one block per SM that
+//           is what keeps enough bytes on their way from HBM.  The signed sum of every
+//           (unit, block) segment goes to its own slot in scratch as a double.
 //   pass 2  one block per unit scans the histogram and writes the eight features.
 #include "windq_internal.cuh"
 
 namespace windq {
 
 constexpr int kBins = 32768;
-constexpr int kFeatThreads = 512;
+constexpr int kFeatThreads = 1024;
+constexpr int kFeatMaxBlocks = 1024;  // bound on the pass-1 grid that the scratch size assumes
+constexpr int kFeatLoads = 4;         // rows in flight per thread
 
-template <int G>
-__global__ void __launch_bounds__(kFeatThreads, 1)
-feat_hist_kernel(const __half* __restrict__ W, int R, int64_t ldw, int rows_per_slice, unsigned int* __restrict__ hist,
-                 double* __restrict__ slice_sum /*[U][slices]*/) {
-  extern __shared__ unsigned int sh[];
-  __shared__ double wsum[kFeatThreads / 32];
-  constexpr int TPR = G / 8;                  // threads per row (8 halves = 16 bytes each)
-  constexpr int RPP = kFeatThreads / TPR;     // rows per pass
-  const int u = blockIdx.x, slice = blockIdx.y;
-  for (int i = threadIdx.x; i < kBins; i += kFeatThreads) sh[i] = 0;
-  __syncthreads();
-  const int r0 = slice * rows_per_slice, r1 = min(r0 + rows_per_slice, R);
-  const int tr = threadIdx.x / TPR, tc = threadIdx.x % TPR;
-  const __half* base = W + (int64_t)u * G + tc * 8;
-  double sum = 0.0;
-  for (int r = r0 + tr; r < r1; r += RPP) {
-    const uint4 raw = __ldg(reinterpret_cast<const uint4*>(base + (int64_t)r * ldw));
-    const unsigned int v[4] = {raw.x, raw.y, raw.z, raw.w};
-    float part = 0.0f;
+__device__ __forceinline__ void hist_add8(unsigned int* sh, const uint4& raw, float& part) {
+  const unsigned int v[4] = {raw.x, raw.y, raw.z, raw.w};
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      atomicAdd(&sh[v[i] & 0x7fffu], 1u);
-      atomicAdd(&sh[(v[i] >> 16) & 0x7fffu], 1u);
-      const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&v[i]));
-      part += f.x + f.y;
-    }
-    sum += (double)part;
-  }
-#pragma unroll
-  for (int m = 16; m > 0; m >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, m);
-  if ((threadIdx.x & 31) == 0) wsum[threadIdx.x >> 5] = sum;
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    double t = 0.0;
-    for (int i = 0; i < kFeatThreads / 32; ++i) t += wsum[i];
-    slice_sum[(int64_t)u * gridDim.y + slice] = t;
-  }
-  unsigned int* gh = hist + (int64_t)u * kBins;
-  for (int i = threadIdx.x; i < kBins; i += kFeatThreads) {
-    const unsigned int c = sh[i];
-    if (c) atomicAdd(&gh[i], c);
+  for (int i = 0; i < 4; ++i) {
+    atomicAdd(&sh[v[i] & 0x7fffu], 1u);
+    atomicAdd(&sh[(v[i] >> 16) & 0x7fffu], 1u);
+    const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&v[i]));
+    part += f.x + f.y;
   }
 }
 
+// rows_per_block consecutive (unit, row) pairs per block; slot j of unit u belongs to block
+// (u * R) / rows_per_block + j.
+template <int G>
+__global__ void __launch_bounds__(kFeatThreads, 1)
+feat_hist_kernel(const __half* __restrict__ W, int R, int64_t ldw, long long rows_per_block, long long total_rows,
+                 unsigned int* __restrict__ hist, double* __restrict__ slot_sum, int slots_per_unit) {
+  extern __shared__ unsigned int sh[];
+  __shared__ double wsum[kFeatThreads / 32];
+  constexpr int TPR = G / 8;               // threads per row (8 halves = 16 bytes each)
+  constexpr int RPP = kFeatThreads / TPR;  // rows per pass
+  for (int i = threadIdx.x; i < kBins; i += kFeatThreads) sh[i] = 0;
+  __syncthreads();
+  const int tr = threadIdx.x / TPR, tc = threadIdx.x % TPR;
+  long long p = (long long)blockIdx.x * rows_per_block;
+  const long long p_end = min(p + rows_per_block, total_rows);
+  while (p < p_end) {
+    const int u = (int)(p / R);
+    const int r0 = (int)(p - (long long)u * R);
+    const int r1 = (int)min((long long)R, r0 + (p_end - p));
+    const __half* base = W + (int64_t)u * G + tc * 8;
+    double sum = 0.0;
+    for (int r = r0 + tr; r < r1; r += RPP * kFeatLoads) {
+      uint4 raw[kFeatLoads];
+#pragma unroll
+      for (int k = 0; k < kFeatLoads; ++k)
+        if (r + k * RPP < r1) raw[k] = __ldg(reinterpret_cast<const uint4*>(base + (int64_t)(r + k * RPP) * ldw));
+      float part = 0.0f;
+#pragma unroll
+      for (int k = 0; k < kFeatLoads; ++k)
+        if (r + k * RPP < r1) hist_add8(sh, raw[k], part);
+      sum += (double)part;
+    }
+#pragma unroll
+    for (int m = 16; m > 0; m >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, m);
+    if ((threadIdx.x & 31) == 0) wsum[threadIdx.x >> 5] = sum;
+    __syncthreads();  // also: every histogram update of this segment is done
+    if (threadIdx.x == 0) {
+      double t = 0.0;
+      for (int i = 0; i < kFeatThreads / 32; ++i) t += wsum[i];
+      const long long first_block = ((long long)u * R) / rows_per_block;
+      slot_sum[(int64_t)u * slots_per_unit + (blockIdx.x - first_block)] = t;
+    }
+    unsigned int* gh = hist + (int64_t)u * kBins;
+    for (int i = threadIdx.x; i < kBins; i += kFeatThreads) {
+      const unsigned int c = sh[i];
+      if (c) {
+        atomicAdd(&gh[i], c);
+        sh[i] = 0;
+      }
+    }
+    __syncthreads();
+    p += r1 - r0;
+  }
+}
+
+// One block per unit.  Thread t owns the 32 consecutive bins 32 t .. 32 t + 31.
 __global__ void __launch_bounds__(1024)
-feat_finalize_kernel(const unsigned int* __restrict__ hist, const double* __restrict__ slice_sum, int slices, int R, int G,
-                     const float* __restrict__ s, float* __restrict__ feat) {
-  __shared__ unsigned long long cnt_scan[1024];
+feat_finalize_kernel(const unsigned int* __restrict__ hist, const double* __restrict__ slot_sum, int slots_per_unit,
+                     long long rows_per_block, int R, int G, const float* __restrict__ s, float* __restrict__ feat) {
+  __shared__ unsigned long long warp_total[32];
   __shared__ double red[3][32];
   __shared__ unsigned long long redc[2][32];
+  __shared__ double s_stat[3];
   __shared__ int p99_bin;
-  const int u = blockIdx.x, t = threadIdx.x;
-  const unsigned int* h = hist + (int64_t)u * kBins;
+  const int u = blockIdx.x, t = threadIdx.x, lane = t & 31, wp = t >> 5;
+  const uint4* h4 = reinterpret_cast<const uint4*>(hist + (int64_t)u * kBins) + t * 8;
   const long long n = (long long)R * G;
-  const long long k = (99 * n + 99) / 100;  // rank of P99, 1-indexed
+  const unsigned long long k = (unsigned long long)((99 * n + 99) / 100);  // rank of P99, 1-indexed
 
-  // each thread owns 32 consecutive bins
   unsigned int c[32];
   unsigned long long local = 0;
 #pragma unroll
-  for (int i = 0; i < 32; ++i) { c[i] = h[t * 32 + i]; local += c[i]; }
-  cnt_scan[t] = local;
-  __syncthreads();
-  for (int off = 1; off < 1024; off <<= 1) {  // inclusive scan over threads
-    unsigned long long v = (t >= off) ? cnt_scan[t - off] : 0;
-    __syncthreads();
-    cnt_scan[t] += v;
-    __syncthreads();
+  for (int i = 0; i < 8; ++i) {
+    const uint4 v = h4[i];
+    c[4 * i] = v.x; c[4 * i + 1] = v.y; c[4 * i + 2] = v.z; c[4 * i + 3] = v.w;
+    local += (unsigned long long)v.x + v.y + v.z + v.w;
   }
-  const unsigned long long before = cnt_scan[t] - local;
-  if (before < (unsigned long long)k && (unsigned long long)k <= cnt_scan[t]) {
+  // inclusive scan of the per-thread counts: inside the warp, then over the warp totals
+  unsigned long long incl = local;
+#pragma unroll
+  for (int m = 1; m < 32; m <<= 1) {
+    const unsigned long long o = __shfl_up_sync(0xffffffffu, incl, m);
+    if (lane >= m) incl += o;
+  }
+  if (lane == 31) warp_total[wp] = incl;
+  __syncthreads();
+  if (wp == 0) {
+    unsigned long long w = warp_total[lane];
+#pragma unroll
+    for (int m = 1; m < 32; m <<= 1) {
+      const unsigned long long o = __shfl_up_sync(0xffffffffu, w, m);
+      if (lane >= m) w += o;
+    }
+    warp_total[lane] = w;  // inclusive over warps
+  }
+  __syncthreads();
+  incl += wp ? warp_total[wp - 1] : 0ull;
+  const unsigned long long before = incl - local;
+  if (before < k && k <= incl) {
     unsigned long long run = before;
     for (int i = 0; i < 32; ++i) {
       run += c[i];
-      if (run >= (unsigned long long)k) { p99_bin = t * 32 + i; break; }
+      if (run >= k) { p99_bin = t * 32 + i; break; }
     }
+  }
+  // statistics of s over the unit's G channels: warp 1, in double
+  if (wp == 1) {
+    const float* su = s + (int64_t)u * G;
+    double sm = 0.0, mx = (double)su[0];
+    for (int j = lane; j < G; j += 32) { const double v = (double)su[j]; sm += v; mx = fmax(mx, v); }
+#pragma unroll
+    for (int m = 16; m > 0; m >>= 1) {
+      sm += __shfl_xor_sync(0xffffffffu, sm, m);
+      mx = fmax(mx, __shfl_xor_sync(0xffffffffu, mx, m));
+    }
+    const double mean = sm / (double)G;
+    double var = 0.0;
+    for (int j = lane; j < G; j += 32) { const double d = (double)su[j] - mean; var += d * d; }
+#pragma unroll
+    for (int m = 16; m > 0; m >>= 1) var += __shfl_xor_sync(0xffffffffu, var, m);
+    if (lane == 0) { s_stat[0] = mean; s_stat[1] = sqrt(var / (double)G); s_stat[2] = mx; }
   }
   __syncthreads();
   const float p99 = __half2float(__ushort_as_half((unsigned short)p99_bin));
@@ -99,18 +161,24 @@ feat_finalize_kernel(const unsigned int* __restrict__ hist, const double* __rest
 
   double sa = 0.0, sq = 0.0;
   unsigned long long n_out = 0, n_tiny = 0;
+  if (local) {
 #pragma unroll
-  for (int i = 0; i < 32; ++i) {
-    const float v = __half2float(__ushort_as_half((unsigned short)(t * 32 + i)));
-    if (c[i] == 0) continue;  // also keeps the Inf / NaN patterns (never counted for finite input) out
-    const double dv = (double)v, dc = (double)c[i];
-    sa += dc * dv;
-    sq += dc * dv * dv;
-    if (v > thr) n_out += c[i];
-    if (v < 1e-6f) n_tiny += c[i];
+    for (int i = 0; i < 32; ++i) {
+      if (c[i] == 0) continue;  // also keeps the Inf / NaN patterns (never counted for finite input) out
+      const float v = __half2float(__ushort_as_half((unsigned short)(t * 32 + i)));
+      const double dv = (double)v, dc = (double)c[i];
+      sa += dc * dv;
+      sq += dc * dv * dv;
+      if (v > thr) n_out += c[i];
+      if (v < 1e-6f) n_tiny += c[i];
+    }
   }
   double ss = 0.0;
-  for (int i = t; i < slices; i += 1024) ss += slice_sum[(int64_t)u * slices + i];
+  {
+    const long long first = ((long long)u * R) / rows_per_block, last = ((long long)(u + 1) * R - 1) / rows_per_block;
+    const int cnt = (int)(last - first + 1);
+    for (int i = t; i < cnt; i += 1024) ss += slot_sum[(int64_t)u * slots_per_unit + i];
+  }
 #pragma unroll
   for (int m = 16; m > 0; m >>= 1) {
     sa += __shfl_xor_sync(0xffffffffu, sa, m);
@@ -119,9 +187,9 @@ feat_finalize_kernel(const unsigned int* __restrict__ hist, const double* __rest
     n_out += __shfl_xor_sync(0xffffffffu, n_out, m);
     n_tiny += __shfl_xor_sync(0xffffffffu, n_tiny, m);
   }
-  if ((t & 31) == 0) {
-    red[0][t >> 5] = sa; red[1][t >> 5] = sq; red[2][t >> 5] = ss;
-    redc[0][t >> 5] = n_out; redc[1][t >> 5] = n_tiny;
+  if (lane == 0) {
+    red[0][wp] = sa; red[1][wp] = sq; red[2][wp] = ss;
+    redc[0][wp] = n_out; redc[1][wp] = n_tiny;
   }
   __syncthreads();
   if (t == 0) {
@@ -132,44 +200,47 @@ feat_finalize_kernel(const unsigned int* __restrict__ hist, const double* __rest
     const double mean = sg / dn;
     double var = q2 / dn - mean * mean;
     if (var < 0.0) var = 0.0;
-    double smean = 0.0, smax = (double)s[(int64_t)u * G];
-    for (int j = 0; j < G; ++j) { const double v = (double)s[(int64_t)u * G + j]; smean += v; smax = fmax(smax, v); }
-    smean /= (double)G;
-    double svar = 0.0;
-    for (int j = 0; j < G; ++j) { const double d = (double)s[(int64_t)u * G + j] - smean; svar += d * d; }
-    svar /= (double)G;
     float* f = feat + (int64_t)u * WINDQ_N_FEATURES;
     f[0] = (float)mean;
     f[1] = (float)sqrt(var);
     f[2] = (float)(a / dn);
     f[3] = (float)((double)nt / dn);
     f[4] = (float)((double)no / dn);
-    f[5] = (float)smean;
-    f[6] = (float)sqrt(svar);
-    f[7] = (float)smax;
+    f[5] = (float)s_stat[0];
+    f[6] = (float)s_stat[1];
+    f[7] = (float)s_stat[2];
   }
 }
 
-inline int feat_slices(int sm_count, int64_t R, int U) {
-  // about two waves of blocks over the SMs, at least 64 rows per slice
-  int64_t want = (2ll * sm_count + U - 1) / U;
-  const int64_t max_slices = (R + 63) / 64;
-  if (want > max_slices) want = max_slices;
-  if (want < 1) want = 1;
-  return (int)want;
+// Pass-1 geometry: blocks and (unit, row) pairs per block.
+struct FeatGrid {
+  int blocks;
+  long long rows_per_block;
+  int slots_per_unit;
+};
+inline FeatGrid feat_grid(int sm_count, int64_t R, int64_t U) {
+  FeatGrid g;
+  const long long total = (long long)U * R;
+  int nb = sm_count < kFeatMaxBlocks ? sm_count : kFeatMaxBlocks;
+  const long long min_rows = 16;  // a block should see at least a few rows
+  if ((long long)nb * min_rows > total) nb = (int)((total + min_rows - 1) / min_rows);
+  g.rows_per_block = (total + nb - 1) / nb;
+  g.blocks = (int)((total + g.rows_per_block - 1) / g.rows_per_block);
+  g.slots_per_unit = (int)(R / g.rows_per_block) + 2;
+  return g;
 }
 
 template <int G>
-windq_status launch_hist(windq_ctx* ctx, const __half* W, int R, int U, int64_t ldw, int slices, unsigned int* hist,
-                         double* slice_sum, cudaStream_t st) {
+windq_status launch_hist(windq_ctx* ctx, const __half* W, int R, int U, int64_t ldw, const FeatGrid& fg,
+                         unsigned int* hist, double* slot_sum, cudaStream_t st) {
   static bool configured = false;
   const size_t smem = (size_t)kBins * sizeof(unsigned int);
   if (!configured) {
     WINDQ_CUDA(ctx, cudaFuncSetAttribute(feat_hist_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     configured = true;
   }
-  const int rows_per_slice = (R + slices - 1) / slices;
-  feat_hist_kernel<G><<<dim3((unsigned)U, (unsigned)slices), kFeatThreads, smem, st>>>(W, R, ldw, rows_per_slice, hist, slice_sum);
+  feat_hist_kernel<G><<<(unsigned)fg.blocks, kFeatThreads, smem, st>>>(W, R, ldw, fg.rows_per_block, (long long)U * R, hist,
+                                                                      slot_sum, fg.slots_per_unit);
   WINDQ_CUDA(ctx, cudaGetLastError());
   return WINDQ_OK;
 }
@@ -181,8 +252,9 @@ extern "C" {
 int64_t windq_scratch_bytes_unit_features(int64_t R, int64_t C, int G) {
   if (!windq::valid_G(G) || R <= 0 || C <= 0) return 0;
   const int64_t U = C / G;
-  // histograms + slice sums (at most ceil(R/64) slices per unit)
-  return U * windq::kBins * (int64_t)sizeof(unsigned int) + U * ((R + 63) / 64) * (int64_t)sizeof(double);
+  // histograms + one double per (unit, block that holds rows of it): a unit meets at most
+  // blocks / U + 2 blocks, and the grid has at most kFeatMaxBlocks blocks
+  return U * windq::kBins * (int64_t)sizeof(unsigned int) + (windq::kFeatMaxBlocks + 2 * U) * (int64_t)sizeof(double);
 }
 
 windq_status windq_unit_features(windq_ctx* ctx, const void* W, int64_t R, int64_t C, int64_t ldw, int G,
@@ -198,20 +270,20 @@ windq_status windq_unit_features(windq_ctx* ctx, const void* W, int64_t R, int64
   WINDQ_REQUIRE(ctx, U <= 65535 * 32, WINDQ_ERR_SHAPE, "windq_unit_features: too many units");
   cudaStream_t st = (cudaStream_t)stream;
   unsigned int* hist = (unsigned int*)ctx->scratch;
-  double* slice_sum = (double*)((char*)ctx->scratch + (int64_t)U * kBins * sizeof(unsigned int));
-  const int slices = feat_slices(ctx->sm_count, R, U);
+  double* slot_sum = (double*)((char*)ctx->scratch + (int64_t)U * kBins * sizeof(unsigned int));
+  const FeatGrid fg = feat_grid(ctx->sm_count, R, U);
   WINDQ_CUDA(ctx, cudaMemsetAsync(hist, 0, (size_t)U * kBins * sizeof(unsigned int), st));
   const __half* Wh = (const __half*)W;
   windq_status rc;
   switch (G) {
-    case 32: rc = launch_hist<32>(ctx, Wh, (int)R, U, ldw, slices, hist, slice_sum, st); break;
-    case 64: rc = launch_hist<64>(ctx, Wh, (int)R, U, ldw, slices, hist, slice_sum, st); break;
-    case 128: rc = launch_hist<128>(ctx, Wh, (int)R, U, ldw, slices, hist, slice_sum, st); break;
-    case 256: rc = launch_hist<256>(ctx, Wh, (int)R, U, ldw, slices, hist, slice_sum, st); break;
-    default: rc = launch_hist<512>(ctx, Wh, (int)R, U, ldw, slices, hist, slice_sum, st); break;
+    case 32: rc = launch_hist<32>(ctx, Wh, (int)R, U, ldw, fg, hist, slot_sum, st); break;
+    case 64: rc = launch_hist<64>(ctx, Wh, (int)R, U, ldw, fg, hist, slot_sum, st); break;
+    case 128: rc = launch_hist<128>(ctx, Wh, (int)R, U, ldw, fg, hist, slot_sum, st); break;
+    case 256: rc = launch_hist<256>(ctx, Wh, (int)R, U, ldw, fg, hist, slot_sum, st); break;
+    default: rc = launch_hist<512>(ctx, Wh, (int)R, U, ldw, fg, hist, slot_sum, st); break;
   }
   if (rc != WINDQ_OK) return rc;
-  feat_finalize_kernel<<<(unsigned)U, 1024, 0, st>>>(hist, slice_sum, slices, (int)R, G, s, feat_out);
+  feat_finalize_kernel<<<(unsigned)U, 1024, 0, st>>>(hist, slot_sum, fg.slots_per_unit, fg.rows_per_block, (int)R, G, s, feat_out);
   WINDQ_CUDA(ctx, cudaGetLastError());
   return WINDQ_OK;
 }

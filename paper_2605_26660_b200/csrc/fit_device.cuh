@@ -279,29 +279,45 @@ __device__ __forceinline__ LowBitFit fit_low_bits(const Lane32& w, const Lane32&
   f.delta = __fmul_rn(0.7f, meanA);
   f.alpha_b = __half2float(__float2half_rn(sumS == 0.0f ? meanA : __fdiv_rn(sumB, sumS)));
 
-  // ternary sums over the support, weighted by s and (fallback) unweighted
-  float Bt[4], Ct[4], Bu[4], Cu[4];
+  // ternary sums over the support, weighted by s; the unweighted ones only if some group of the
+  // warp has no activation weight on its support
+  float Bt[4], Ct[4];
 #pragma unroll
   for (int l = 0; l < 4; ++l) {
-    float bt = 0.0f, ct = 0.0f, bu = 0.0f, cu = 0.0f;
+    float bt = 0.0f, ct = 0.0f;
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
       const float aw = fabsf(w.get(l, i)), sv = s.get(l, i);
       const bool in = aw > f.delta;
-      const float a_in = in ? aw : 0.0f;
-      bt = __fmaf_rn(sv, a_in, bt);
+      bt = __fmaf_rn(sv, in ? aw : 0.0f, bt);
       ct = __fadd_rn(ct, in ? sv : 0.0f);
-      bu = __fadd_rn(bu, a_in);
-      cu = __fadd_rn(cu, in ? 1.0f : 0.0f);
     }
-    Bt[l] = bt; Ct[l] = ct; Bu[l] = bu; Cu[l] = cu;
+    Bt[l] = bt; Ct[l] = ct;
   }
   float sumBt = group_tree<G>(Bt[0], Bt[1], Bt[2], Bt[3]);
   float sumCt = group_tree<G>(Ct[0], Ct[1], Ct[2], Ct[3]);
-  const float sumBu = group_tree<G>(Bu[0], Bu[1], Bu[2], Bu[3]);
-  const float sumCu = group_tree<G>(Cu[0], Cu[1], Cu[2], Cu[3]);
-  if (sumCt == 0.0f) { sumBt = sumBu; sumCt = sumCu; }
-  f.alpha_t = (sumCu > 0.0f) ? __half2float(__float2half_rn(__fdiv_rn(sumBt, sumCt))) : 0.0f;
+  // delta < max |w| whenever some w is not zero (0.7 * mean <= 0.7 * max, roundings included), so
+  // the support is empty exactly when every |w| is zero, i.e. when their sum is
+  const bool nonempty = sumA > 0.0f;
+  if (__any_sync(0xffffffffu, nonempty && sumCt == 0.0f)) {
+    float Bu[4], Cu[4];
+#pragma unroll
+    for (int l = 0; l < 4; ++l) {
+      float bu = 0.0f, cu = 0.0f;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const float aw = fabsf(w.get(l, i));
+        const bool in = aw > f.delta;
+        bu = __fadd_rn(bu, in ? aw : 0.0f);
+        cu = __fadd_rn(cu, in ? 1.0f : 0.0f);
+      }
+      Bu[l] = bu; Cu[l] = cu;
+    }
+    const float sumBu = group_tree<G>(Bu[0], Bu[1], Bu[2], Bu[3]);
+    const float sumCu = group_tree<G>(Cu[0], Cu[1], Cu[2], Cu[3]);
+    if (sumCt == 0.0f) { sumBt = sumBu; sumCt = sumCu; }
+  }
+  f.alpha_t = nonempty ? __half2float(__float2half_rn(__fdiv_rn(sumBt, sumCt))) : 0.0f;
 
   float Et[4], Eb[4];
 #pragma unroll

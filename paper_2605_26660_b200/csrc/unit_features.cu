@@ -20,7 +20,10 @@ namespace windq {
 constexpr int kBins = 32768;
 constexpr int kFeatThreads = 1024;
 constexpr int kFeatMaxBlocks = 1024;  // bound on the pass-1 grid that the scratch size assumes
-constexpr int kFeatLoads = 4;         // rows in flight per thread
+#ifndef WINDQ_FEAT_LOADS
+#define WINDQ_FEAT_LOADS 4
+#endif
+constexpr int kFeatLoads = WINDQ_FEAT_LOADS;  // rows in flight per thread
 
 __device__ __forceinline__ void hist_add8(unsigned int* sh, const uint4& raw, float& part) {
   const unsigned int v[4] = {raw.x, raw.y, raw.z, raw.w};
@@ -88,7 +91,8 @@ feat_hist_kernel(const __half* __restrict__ W, int R, int64_t ldw, long long row
   }
 }
 
-// One block per unit.  Thread t owns the 32 consecutive bins 32 t .. 32 t + 31.
+// One block per unit.  Thread t owns the 32 consecutive bins 32 t .. 32 t + 31; it reads them twice
+// (the second time from L1) rather than keep 32 counts in registers across the scan.
 __global__ void __launch_bounds__(1024)
 feat_finalize_kernel(const unsigned int* __restrict__ hist, const double* __restrict__ slot_sum, int slots_per_unit,
                      long long rows_per_block, int R, int G, const float* __restrict__ s, float* __restrict__ feat) {
@@ -102,12 +106,10 @@ feat_finalize_kernel(const unsigned int* __restrict__ hist, const double* __rest
   const long long n = (long long)R * G;
   const unsigned long long k = (unsigned long long)((99 * n + 99) / 100);  // rank of P99, 1-indexed
 
-  unsigned int c[32];
   unsigned long long local = 0;
 #pragma unroll
   for (int i = 0; i < 8; ++i) {
     const uint4 v = h4[i];
-    c[4 * i] = v.x; c[4 * i + 1] = v.y; c[4 * i + 2] = v.z; c[4 * i + 3] = v.w;
     local += (unsigned long long)v.x + v.y + v.z + v.w;
   }
   // inclusive scan of the per-thread counts: inside the warp, then over the warp totals
@@ -128,16 +130,6 @@ feat_finalize_kernel(const unsigned int* __restrict__ hist, const double* __rest
     }
     warp_total[lane] = w;  // inclusive over warps
   }
-  __syncthreads();
-  incl += wp ? warp_total[wp - 1] : 0ull;
-  const unsigned long long before = incl - local;
-  if (before < k && k <= incl) {
-    unsigned long long run = before;
-    for (int i = 0; i < 32; ++i) {
-      run += c[i];
-      if (run >= k) { p99_bin = t * 32 + i; break; }
-    }
-  }
   // statistics of s over the unit's G channels: warp 1, in double
   if (wp == 1) {
     const float* su = s + (int64_t)u * G;
@@ -156,21 +148,39 @@ feat_finalize_kernel(const unsigned int* __restrict__ hist, const double* __rest
     if (lane == 0) { s_stat[0] = mean; s_stat[1] = sqrt(var / (double)G); s_stat[2] = mx; }
   }
   __syncthreads();
+  incl += wp ? warp_total[wp - 1] : 0ull;
+  const unsigned long long before = incl - local;
+  if (before < k && k <= incl) {  // exactly one thread: the rank-k value is in its bins
+    const unsigned int* hb = reinterpret_cast<const unsigned int*>(h4);
+    unsigned long long run = before;
+    int i = 0;
+    for (; i < 31; ++i) {
+      run += hb[i];
+      if (run >= k) break;
+    }
+    p99_bin = t * 32 + i;
+  }
+  __syncthreads();
   const float p99 = __half2float(__ushort_as_half((unsigned short)p99_bin));
   const float thr = 0.5f * p99;
 
   double sa = 0.0, sq = 0.0;
   unsigned long long n_out = 0, n_tiny = 0;
   if (local) {
+#pragma unroll 1
+    for (int i = 0; i < 8; ++i) {
+      const uint4 v = h4[i];
+      const unsigned int c[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
-    for (int i = 0; i < 32; ++i) {
-      if (c[i] == 0) continue;  // also keeps the Inf / NaN patterns (never counted for finite input) out
-      const float v = __half2float(__ushort_as_half((unsigned short)(t * 32 + i)));
-      const double dv = (double)v, dc = (double)c[i];
-      sa += dc * dv;
-      sq += dc * dv * dv;
-      if (v > thr) n_out += c[i];
-      if (v < 1e-6f) n_tiny += c[i];
+      for (int j = 0; j < 4; ++j) {
+        if (c[j] == 0) continue;  // also keeps the Inf / NaN patterns (never counted for finite input) out
+        const float x = __half2float(__ushort_as_half((unsigned short)(t * 32 + 4 * i + j)));
+        const double dv = (double)x, dc = (double)c[j];
+        sa += dc * dv;
+        sq += dc * dv * dv;
+        if (x > thr) n_out += c[j];
+        if (x < 1e-6f) n_tiny += c[j];
+      }
     }
   }
   double ss = 0.0;
@@ -192,23 +202,32 @@ feat_finalize_kernel(const unsigned int* __restrict__ hist, const double* __rest
     redc[0][wp] = n_out; redc[1][wp] = n_tiny;
   }
   __syncthreads();
-  if (t == 0) {
-    double a = 0, q2 = 0, sg = 0;
-    unsigned long long no = 0, nt = 0;
-    for (int i = 0; i < 32; ++i) { a += red[0][i]; q2 += red[1][i]; sg += red[2][i]; no += redc[0][i]; nt += redc[1][i]; }
-    const double dn = (double)n;
-    const double mean = sg / dn;
-    double var = q2 / dn - mean * mean;
-    if (var < 0.0) var = 0.0;
-    float* f = feat + (int64_t)u * WINDQ_N_FEATURES;
-    f[0] = (float)mean;
-    f[1] = (float)sqrt(var);
-    f[2] = (float)(a / dn);
-    f[3] = (float)((double)nt / dn);
-    f[4] = (float)((double)no / dn);
-    f[5] = (float)s_stat[0];
-    f[6] = (float)s_stat[1];
-    f[7] = (float)s_stat[2];
+  if (wp == 0) {
+    double a = red[0][lane], q2 = red[1][lane], sg = red[2][lane];
+    unsigned long long no = redc[0][lane], nt = redc[1][lane];
+#pragma unroll
+    for (int m = 16; m > 0; m >>= 1) {
+      a += __shfl_xor_sync(0xffffffffu, a, m);
+      q2 += __shfl_xor_sync(0xffffffffu, q2, m);
+      sg += __shfl_xor_sync(0xffffffffu, sg, m);
+      no += __shfl_xor_sync(0xffffffffu, no, m);
+      nt += __shfl_xor_sync(0xffffffffu, nt, m);
+    }
+    if (lane == 0) {
+      const double dn = (double)n;
+      const double mean = sg / dn;
+      double var = q2 / dn - mean * mean;
+      if (var < 0.0) var = 0.0;
+      float* f = feat + (int64_t)u * WINDQ_N_FEATURES;
+      f[0] = (float)mean;
+      f[1] = (float)sqrt(var);
+      f[2] = (float)(a / dn);
+      f[3] = (float)((double)nt / dn);
+      f[4] = (float)((double)no / dn);
+      f[5] = (float)s_stat[0];
+      f[6] = (float)s_stat[1];
+      f[7] = (float)s_stat[2];
+    }
   }
 }
 

@@ -89,7 +89,10 @@ __device__ __forceinline__ void store_words(uint8_t* dst, const unsigned (&w)[8]
 // SEARCH = false: clip indices are supplied.  SEARCH = true: the clip search is repeated for the
 // unit's bit-width (the candidate table follows the warp buffers in shared memory).
 template <int G, bool SEARCH>
-__global__ void __launch_bounds__(kApplyWarps * 32, 4)
+#ifndef WINDQ_APPLY_MIN_BLOCKS
+#define WINDQ_APPLY_MIN_BLOCKS 4
+#endif
+__global__ void __launch_bounds__(kApplyWarps * 32, WINDQ_APPLY_MIN_BLOCKS)
 apply_plan_kernel(const __half* __restrict__ W, int R, int U, int64_t ldw, const float* __restrict__ s,
                   const float* __restrict__ clip, int K, const uint8_t* __restrict__ actions,
                   const uint8_t* __restrict__ clip_idx, const long long* __restrict__ code_offsets,

@@ -91,27 +91,32 @@ feat_hist_kernel(const __half* __restrict__ W, int R, int64_t ldw, long long row
   }
 }
 
-// One block per unit.  Thread t owns the 32 consecutive bins 32 t .. 32 t + 31; it reads them twice
-// (the second time from L1) rather than keep 32 counts in registers across the scan.
+// One block per unit.  The unit's histogram is first copied to shared memory with coalesced 128-bit
+// loads; thread t then owns the 32 consecutive bins 32 t .. 32 t + 31 and walks them from shared
+// memory starting at bin t mod 32, so that the lanes of a warp stay on different banks.
 __global__ void __launch_bounds__(1024)
 feat_finalize_kernel(const unsigned int* __restrict__ hist, const double* __restrict__ slot_sum, int slots_per_unit,
                      long long rows_per_block, int R, int G, const float* __restrict__ s, float* __restrict__ feat) {
+  extern __shared__ unsigned int sh[];  // kBins counts
   __shared__ unsigned long long warp_total[32];
   __shared__ double red[3][32];
   __shared__ unsigned long long redc[2][32];
   __shared__ double s_stat[3];
   __shared__ int p99_bin;
   const int u = blockIdx.x, t = threadIdx.x, lane = t & 31, wp = t >> 5;
-  const uint4* h4 = reinterpret_cast<const uint4*>(hist + (int64_t)u * kBins) + t * 8;
   const long long n = (long long)R * G;
   const unsigned long long k = (unsigned long long)((99 * n + 99) / 100);  // rank of P99, 1-indexed
-
+  {
+    const uint4* src = reinterpret_cast<const uint4*>(hist + (int64_t)u * kBins);
+    uint4* dst = reinterpret_cast<uint4*>(sh);
+#pragma unroll
+    for (int i = 0; i < kBins / 4 / 1024; ++i) dst[i * 1024 + t] = src[i * 1024 + t];
+  }
+  __syncthreads();
+  const unsigned int* mine = sh + t * 32;
   unsigned long long local = 0;
 #pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    const uint4 v = h4[i];
-    local += (unsigned long long)v.x + v.y + v.z + v.w;
-  }
+  for (int i = 0; i < 32; ++i) local += mine[(i + lane) & 31];
   // inclusive scan of the per-thread counts: inside the warp, then over the warp totals
   unsigned long long incl = local;
 #pragma unroll
@@ -151,11 +156,10 @@ feat_finalize_kernel(const unsigned int* __restrict__ hist, const double* __rest
   incl += wp ? warp_total[wp - 1] : 0ull;
   const unsigned long long before = incl - local;
   if (before < k && k <= incl) {  // exactly one thread: the rank-k value is in its bins
-    const unsigned int* hb = reinterpret_cast<const unsigned int*>(h4);
     unsigned long long run = before;
     int i = 0;
     for (; i < 31; ++i) {
-      run += hb[i];
+      run += mine[i];
       if (run >= k) break;
     }
     p99_bin = t * 32 + i;
@@ -167,20 +171,17 @@ feat_finalize_kernel(const unsigned int* __restrict__ hist, const double* __rest
   double sa = 0.0, sq = 0.0;
   unsigned long long n_out = 0, n_tiny = 0;
   if (local) {
-#pragma unroll 1
-    for (int i = 0; i < 8; ++i) {
-      const uint4 v = h4[i];
-      const unsigned int c[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        if (c[j] == 0) continue;  // also keeps the Inf / NaN patterns (never counted for finite input) out
-        const float x = __half2float(__ushort_as_half((unsigned short)(t * 32 + 4 * i + j)));
-        const double dv = (double)x, dc = (double)c[j];
-        sa += dc * dv;
-        sq += dc * dv * dv;
-        if (x > thr) n_out += c[j];
-        if (x < 1e-6f) n_tiny += c[j];
-      }
+#pragma unroll 4
+    for (int i = 0; i < 32; ++i) {
+      const int b = (i + lane) & 31;
+      const unsigned int c = mine[b];
+      if (c == 0) continue;  // also keeps the Inf / NaN patterns (never counted for finite input) out
+      const float x = __half2float(__ushort_as_half((unsigned short)(t * 32 + b)));
+      const double dv = (double)x, dc = (double)c;
+      sa += dc * dv;
+      sq += dc * dv * dv;
+      if (x > thr) n_out += c;
+      if (x < 1e-6f) n_tiny += c;
     }
   }
   double ss = 0.0;
@@ -302,7 +303,12 @@ windq_status windq_unit_features(windq_ctx* ctx, const void* W, int64_t R, int64
     default: rc = launch_hist<512>(ctx, Wh, (int)R, U, ldw, fg, hist, slot_sum, st); break;
   }
   if (rc != WINDQ_OK) return rc;
-  feat_finalize_kernel<<<(unsigned)U, 1024, 0, st>>>(hist, slot_sum, fg.slots_per_unit, fg.rows_per_block, (int)R, G, s, feat_out);
+  static bool finalize_configured = false;
+  if (!finalize_configured) {
+    WINDQ_CUDA(ctx, cudaFuncSetAttribute(feat_finalize_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kBins * sizeof(unsigned int))));
+    finalize_configured = true;
+  }
+  feat_finalize_kernel<<<(unsigned)U, 1024, kBins * sizeof(unsigned int), st>>>(hist, slot_sum, fg.slots_per_unit, fg.rows_per_block, (int)R, G, s, feat_out);
   WINDQ_CUDA(ctx, cudaGetLastError());
   return WINDQ_OK;
 }

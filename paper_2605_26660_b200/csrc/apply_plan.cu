@@ -277,13 +277,9 @@ windq_status launch_apply(windq_ctx* ctx, const __half* W, int R, int U, int64_t
   constexpr int GPW = Map<G>::GPW;
   const int stride = apply_cand_chunk<G>() | 1;
   const size_t smem = (size_t)kApplyWarps * kApplyWarpBytes + (SEARCH ? (size_t)kApplyWarps * GPW * stride * sizeof(Cand) : 0);
-  static int blocks_per_sm = 0;  // same for every device this library supports
-  if (blocks_per_sm == 0) {
-    WINDQ_CUDA(ctx, cudaFuncSetAttribute(apply_plan_kernel<G, SEARCH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    int n = 0;
-    WINDQ_CUDA(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, apply_plan_kernel<G, SEARCH>, kApplyWarps * 32, smem));
-    blocks_per_sm = n > 0 ? n : 1;
-  }
+  const int id = (SEARCH ? kApplySearchG32 : kApplyG32) + g_index(G);
+  if (windq_status rc = prepare_kernel(ctx, id, apply_plan_kernel<G, SEARCH>, kApplyWarps * 32, smem, true)) return rc;
+  const int blocks_per_sm = ctx->occupancy[id];
   const int rows_blocks = (R + GPW - 1) / GPW;
   const int64_t n_items = (int64_t)U * rows_blocks;
   WINDQ_REQUIRE(ctx, n_items < (1ll << 30), WINDQ_ERR_SHAPE, "windq_apply_plan: R * C is too large for one call");

@@ -129,13 +129,9 @@ windq_status launch_fit(windq_ctx* ctx, const __half* W, int R, int U, int64_t l
   const int rows_blocks = (R + GPW - 1) / GPW;
   const int chunk = fit_cand_chunk(G), stride = fit_cand_stride(chunk);
   const size_t smem = (size_t)kFitWarpsPerBlock * GPW * stride * sizeof(Cand);
-  static int blocks_per_sm = 0;  // same for every device this library supports
-  if (blocks_per_sm == 0) {
-    WINDQ_CUDA(ctx, cudaFuncSetAttribute(fit_eval_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    int n = 0;
-    WINDQ_CUDA(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, fit_eval_kernel<G>, kFitWarpsPerBlock * 32, smem));
-    blocks_per_sm = n > 0 ? n : 1;
-  }
+  const int id = kFitG32 + g_index(G);
+  if (windq_status rc = prepare_kernel(ctx, id, fit_eval_kernel<G>, kFitWarpsPerBlock * 32, smem, true)) return rc;
+  const int blocks_per_sm = ctx->occupancy[id];
   const int64_t n_items = (int64_t)U * rows_blocks;
   int64_t grid = (int64_t)ctx->sm_count * blocks_per_sm;
   const int64_t need = (n_items + kFitWarpsPerBlock - 1) / kFitWarpsPerBlock;

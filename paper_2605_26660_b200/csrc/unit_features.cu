@@ -18,7 +18,10 @@
 namespace windq {
 
 constexpr int kBins = 32768;
-constexpr int kFeatThreads = 1024;
+#ifndef WINDQ_FEAT_THREADS
+#define WINDQ_FEAT_THREADS 1024
+#endif
+constexpr int kFeatThreads = WINDQ_FEAT_THREADS;
 constexpr int kFeatMaxBlocks = 1024;  // bound on the pass-1 grid that the scratch size assumes
 #ifndef WINDQ_FEAT_LOADS
 #define WINDQ_FEAT_LOADS 4
@@ -39,7 +42,7 @@ __device__ __forceinline__ void hist_add8(unsigned int* sh, const uint4& raw, fl
 // rows_per_block consecutive (unit, row) pairs per block; slot j of unit u belongs to block
 // (u * R) / rows_per_block + j.
 template <int G>
-__global__ void __launch_bounds__(kFeatThreads, 1)
+__global__ void __launch_bounds__(kFeatThreads, kFeatThreads <= 256 ? 4 : 1)  // at most 64 registers per thread
 feat_hist_kernel(const __half* __restrict__ W, int R, int64_t ldw, long long rows_per_block, long long total_rows,
                  unsigned int* __restrict__ hist, double* __restrict__ slot_sum, int slots_per_unit) {
   extern __shared__ unsigned int sh[];
@@ -253,12 +256,8 @@ inline FeatGrid feat_grid(int sm_count, int64_t R, int64_t U) {
 template <int G>
 windq_status launch_hist(windq_ctx* ctx, const __half* W, int R, int U, int64_t ldw, const FeatGrid& fg,
                          unsigned int* hist, double* slot_sum, cudaStream_t st) {
-  static bool configured = false;
   const size_t smem = (size_t)kBins * sizeof(unsigned int);
-  if (!configured) {
-    WINDQ_CUDA(ctx, cudaFuncSetAttribute(feat_hist_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    configured = true;
-  }
+  if (windq_status rc = prepare_kernel(ctx, kHistG32 + g_index(G), feat_hist_kernel<G>, kFeatThreads, smem, false)) return rc;
   feat_hist_kernel<G><<<(unsigned)fg.blocks, kFeatThreads, smem, st>>>(W, R, ldw, fg.rows_per_block, (long long)U * R, hist,
                                                                       slot_sum, fg.slots_per_unit);
   WINDQ_CUDA(ctx, cudaGetLastError());
@@ -303,11 +302,7 @@ windq_status windq_unit_features(windq_ctx* ctx, const void* W, int64_t R, int64
     default: rc = launch_hist<512>(ctx, Wh, (int)R, U, ldw, fg, hist, slot_sum, st); break;
   }
   if (rc != WINDQ_OK) return rc;
-  static bool finalize_configured = false;
-  if (!finalize_configured) {
-    WINDQ_CUDA(ctx, cudaFuncSetAttribute(feat_finalize_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kBins * sizeof(unsigned int))));
-    finalize_configured = true;
-  }
+  if (windq_status st2 = prepare_kernel(ctx, kFinalize, feat_finalize_kernel, 1024, kBins * sizeof(unsigned int), false)) return st2;
   feat_finalize_kernel<<<(unsigned)U, 1024, kBins * sizeof(unsigned int), st>>>(hist, slot_sum, fg.slots_per_unit, fg.rows_per_block, (int)R, G, s, feat_out);
   WINDQ_CUDA(ctx, cudaGetLastError());
   return WINDQ_OK;

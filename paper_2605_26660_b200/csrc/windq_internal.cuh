@@ -14,6 +14,8 @@ struct windq_ctx {
   int sm_count;
   void* scratch;
   int64_t scratch_bytes;
+  unsigned long long prepared;  // kernels whose attributes have been set on this context's device (bit per KernelId)
+  int occupancy[32];            // resident blocks per SM of those kernels (0 where not asked)
   char err[256];
 };
 
@@ -49,6 +51,32 @@ struct DeviceGuard {
     cudaError_t e_ = (call);                                                                       \
     if (e_ != cudaSuccess) return ::windq::fail((ctx), WINDQ_ERR_CUDA, "%s: %s", #call, cudaGetErrorString(e_)); \
   } while (0)
+
+// One bit per kernel instantiation that needs a function attribute or an occupancy figure.  Function
+// attributes belong to a device, so the record is kept in the context, not in a process-wide static.
+enum KernelId { kFitG32 = 0, kApplyG32 = 5, kApplySearchG32 = 10, kHistG32 = 15, kFinalize = 20 };
+inline int g_index(int G) { return G == 32 ? 0 : G == 64 ? 1 : G == 128 ? 2 : G == 256 ? 3 : 4; }
+
+// Sets the dynamic shared-memory limit of `kernel` once per context and, if asked, records how many
+// of its blocks fit on an SM.
+template <class K>
+windq_status prepare_kernel(windq_ctx* ctx, int id, K kernel, int threads, size_t smem, bool want_occupancy) {
+  if (ctx->prepared & (1ull << id)) return WINDQ_OK;
+  if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
+    cudaGetLastError();
+    return fail(ctx, WINDQ_ERR_CUDA, "cannot reserve %lld bytes of shared memory per block", (long long)smem);
+  }
+  if (want_occupancy) {
+    int n = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kernel, threads, smem) != cudaSuccess) {
+      cudaGetLastError();
+      return fail(ctx, WINDQ_ERR_CUDA, "occupancy query failed");
+    }
+    ctx->occupancy[id] = n > 0 ? n : 1;
+  }
+  ctx->prepared |= 1ull << id;
+  return WINDQ_OK;
+}
 
 // Checks shared by the calls that take a weight matrix.
 windq_status check_matrix(windq_ctx* ctx, const char* who, const void* W, int64_t R, int64_t C, int64_t ldw, int G);

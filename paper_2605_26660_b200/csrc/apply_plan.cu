@@ -22,20 +22,70 @@ namespace windq {
 
 constexpr int kApplyWarps = 4;
 
-// 32 small codes -> packed little-endian words.
+// 16 registers that each hold two small codes -- one in the low bits of each 16-bit half, anything
+// above the low BITS bits ignored -- -> packed little-endian words.
 template <int BITS>
-__device__ __forceinline__ void pack_words(const unsigned (&q)[32], unsigned (&out)[8]) {
+__device__ __forceinline__ void pack_pairs(const unsigned (&p)[16], unsigned (&out)[8]) {
+  constexpr unsigned mask = (1u << BITS) - 1u;
 #pragma unroll
   for (int i = 0; i < 8; ++i) out[i] = 0u;
 #pragma unroll
-  for (int j = 0; j < 32; ++j) {
-    const int pos = BITS * j, wd = pos >> 5, sh = pos & 31;
-    out[wd] |= q[j] << sh;
-    if (sh + BITS > 32) out[wd + 1] |= q[j] >> (32 - sh);
+  for (int j = 0; j < 16; ++j) {
+    const unsigned f = (p[j] & mask) | (((p[j] >> 16) & mask) << BITS);  // codes 2j, 2j+1
+    const int pos = 2 * BITS * j, wd = pos >> 5, sh = pos & 31;
+    out[wd] |= f << sh;
+    if (sh + 2 * BITS > 32) out[wd + 1] |= f >> (32 - sh);
   }
 }
 
-__device__ __forceinline__ unsigned short half_bits(float x) { return __half_as_ushort(__float2half_rn(x)); }
+__device__ __forceinline__ unsigned h2_bits(__half2 h) { return *reinterpret_cast<unsigned*>(&h); }
+__device__ __forceinline__ __half2 bits_h2(unsigned u) { return *reinterpret_cast<__half2*>(&u); }
+
+// min(0, min w) and max(0, max w) over the group, from the lane's 32 halves: the comparisons are
+// made on the fp16 values themselves (exact, two per instruction).
+template <int G>
+__device__ __forceinline__ void group_range_h(const uint4 (&raw)[4], float& mn, float& mx) {
+  const unsigned* r = reinterpret_cast<const unsigned*>(raw);
+  __half2 lo2 = bits_h2(r[0]), hi2 = lo2;
+#pragma unroll
+  for (int i = 1; i < 16; ++i) {
+    lo2 = __hmin2(lo2, bits_h2(r[i]));
+    hi2 = __hmax2(hi2, bits_h2(r[i]));
+  }
+  const float2 l = __half22float2(lo2), h = __half22float2(hi2);
+  float lo = fminf(0.0f, fminf(l.x, l.y)), hi = fmaxf(0.0f, fmaxf(h.x, h.y));
+#pragma unroll
+  for (int m = 1; m < Map<G>::LG; m <<= 1) {
+    lo = fminf(lo, __shfl_xor_sync(0xffffffffu, lo, m));
+    hi = fmaxf(hi, __shfl_xor_sync(0xffffffffu, hi, m));
+  }
+  mn = __fadd_rn(lo, 0.0f);  // -0 -> +0
+  mx = hi;
+}
+
+// Uniform grid with known parameters: codes and fake-quantised weights of the lane's 32 values.
+// The centred code c = clamp(rne(w / scale), lo, hi) is formed in fp32 exactly as in the fit; being
+// an integer of at most 8 bits it is exact in fp16, so the stored weight fp16(c * scale) is one
+// half-precision product (scale is an fp16 value: the product is rounded once either way), and
+// the code c + z comes out of a half-precision add of z + 1024, whose low bits are the integer.
+__device__ __forceinline__ void quantise_uniform(const uint4 (&raw)[4], float scale, float zf, float qmax,
+                                                 unsigned (&wq)[16], unsigned (&code)[16]) {
+  const float inv = __frcp_rn(scale);
+  const float lo = __fsub_rn(0.0f, zf), hi = __fsub_rn(qmax, zf);
+  const __half2 scale2 = __float2half2_rn(scale);              // exact
+  const __half2 zbias2 = __float2half2_rn(__fadd_rn(zf, 1024.0f));  // exact: an integer below 2048
+  const unsigned* r = reinterpret_cast<const unsigned*>(raw);
+#pragma unroll
+  for (int i = 0; i < 16; ++i) {
+    const float2 w = __half22float2(bits_h2(r[i]));
+    const float cx = fminf(fmaxf(__fadd_rn(__fmaf_rn(w.x, inv, kMagic), -kMagic), lo), hi);
+    const float cy = fminf(fmaxf(__fadd_rn(__fmaf_rn(w.y, inv, kMagic), -kMagic), lo), hi);
+    const __half2 c2 = __floats2half2_rn(cx, cy);  // exact
+    wq[i] = h2_bits(__hmul2(c2, scale2));
+    code[i] = h2_bits(__hadd2(c2, zbias2));        // 0x6400 + code in each half
+  }
+}
+
 
 __device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src) {
   const unsigned dst = (unsigned)__cvta_generic_to_shared(smem_dst);
@@ -52,20 +102,6 @@ constexpr int kApplyWarpBytes = 2 * 2048 + 1024;
 template <int G>
 __host__ __device__ inline int apply_cand_chunk() {
   return (336 / Map<G>::GPW > 64) ? 64 : 336 / Map<G>::GPW;
-}
-
-// The fake-quantised values of a lane (as fp16 bit patterns) -> its 64 bytes of Wq.
-__device__ __forceinline__ void store_wq(__half* dst, const unsigned short (&h)[32]) {
-  uint4* p = reinterpret_cast<uint4*>(dst);
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    uint4 v;
-    v.x = h[8 * i + 0] | ((unsigned)h[8 * i + 1] << 16);
-    v.y = h[8 * i + 2] | ((unsigned)h[8 * i + 3] << 16);
-    v.z = h[8 * i + 4] | ((unsigned)h[8 * i + 5] << 16);
-    v.w = h[8 * i + 6] | ((unsigned)h[8 * i + 7] << 16);
-    p[i] = v;
-  }
 }
 
 // n_words packed words of a lane -> dst (4-byte aligned; 8- or 16-byte aligned for 2, 4, 8 words).
@@ -173,66 +209,65 @@ apply_plan_kernel(const __half* __restrict__ W, int R, int U, int64_t ldw, const
       continue;
     }
 
-    Lane32 wv;
-    unpack_weights(raw, wv);
-    unsigned code[32];
-    unsigned short wq16[32];
+    unsigned wq[16], code[16];  // two fp16 weights / two codes per register
     float scale_store, zero_store = 0.0f;
     if (a <= 4) {
       const int bi = a - 1;
+      const UniformSpec us = uniform_spec(bi);
       float mn, mx;
-      group_range<G>(wv, mn, mx);
-      const float rng = __fsub_rn(mx, mn);
       int k;
       if (!SEARCH) {
+        group_range_h<G>(raw, mn, mx);
         k = min((int)clip_idx[((int64_t)bi * U + u) * R + min(row, R - 1)], K - 1);
       } else {
-        Lane32 sv;
+        Lane32 wv, sv;
+        unpack_weights(raw, wv);
         load_stats(s + (int64_t)u * G + 32 * q, sv);
+        group_range<G>(wv, mn, mx);
         float be;
-        search_uniform<G>(wv, sv, mn, rng, bi, clip, K, cand, chunk, stride, lane, be, k);
+        search_uniform<G>(wv, sv, mn, __fsub_rn(mx, mn), bi, clip, K, cand, chunk, stride, lane, be, k);
       }
-      const UniformSpec us = uniform_spec(bi);
-      const float p = __ldg(clip + k);
       float scale, zf;
-      uniform_scale_zero(mn, rng, p, us, scale, zf);
-      const Cand c = make_cand(mn, rng, p, us);
-#pragma unroll
-      for (int l = 0; l < 4; ++l)
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          const float cc = centred_code(wv.get(l, i), c);
-          code[8 * l + i] = (unsigned)(int)__fadd_rn(cc, zf);
-          wq16[8 * l + i] = half_bits(__fmul_rn(cc, scale));
-        }
+      uniform_scale_zero(mn, __fsub_rn(mx, mn), __ldg(clip + k), us, scale, zf);
+      quantise_uniform(raw, scale, zf, us.qmax, wq, code);
       scale_store = scale;
       zero_store = zf;
     } else {
-      Lane32 sv;
+      Lane32 wv, sv;
+      unpack_weights(raw, wv);
       load_stats(s + (int64_t)u * G + 32 * q, sv);
       float delta = 0.0f;
       const float alpha = (a == 5) ? ternary_scale<G>(wv, sv, delta) : binary_scale<G>(wv, sv);
-      const unsigned short pos = half_bits(alpha), neg = half_bits(-alpha);
+      const unsigned alpha2 = h2_bits(__float2half2_rn(alpha));
+      const unsigned* r = reinterpret_cast<const unsigned*>(raw);
+      if (a == 5) {
+        // |w| > delta, with |w| an fp16 value, is |w| > (delta rounded towards zero to fp16)
+        const __half2 delta2 = __half2half2(__float2half_rz(delta));
 #pragma unroll
-      for (int l = 0; l < 4; ++l)
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          const float w = wv.get(l, i);
-          const bool is_neg = w < 0.0f;
-          if (a == 5) {
-            const bool in = fabsf(w) > delta;
-            code[8 * l + i] = in ? (is_neg ? 0u : 2u) : 1u;
-            wq16[8 * l + i] = in ? (is_neg ? neg : pos) : (unsigned short)0;
-          } else {
-            code[8 * l + i] = is_neg ? 0u : 1u;
-            wq16[8 * l + i] = is_neg ? neg : pos;
-          }
+        for (int i = 0; i < 16; ++i) {
+          const unsigned in = __hgt2_mask(__habs2(bits_h2(r[i])), delta2);  // 0xffff per value on the support
+          wq[i] = ((r[i] & 0x80008000u) | alpha2) & in;                      // +-alpha on the support, +0 elsewhere
+          const unsigned neg = (r[i] >> 14) & 0x00020002u;
+          code[i] = (in & 0x00020002u & ~neg) | (~in & 0x00010001u);         // trit 2, 0 (negative) or 1 (off the support)
         }
+      } else {
+        const __half2 zero2 = __float2half2_rn(0.0f);
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+          const unsigned neg = __hlt2_mask(bits_h2(r[i]), zero2);  // w < 0 (false for -0)
+          wq[i] = (neg & 0x80008000u) | alpha2;
+          code[i] = ~neg & 0x00010001u;
+        }
+      }
       scale_store = alpha;
     }
 
     if (live) {
-      if (wq_dst) store_wq(wq_dst, wq16);
+      if (wq_dst) {
+        uint4* dst = reinterpret_cast<uint4*>(wq_dst);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) dst[i] = make_uint4(wq[4 * i], wq[4 * i + 1], wq[4 * i + 2], wq[4 * i + 3]);
+      }
       if (q == 0) {
         scales_out[(int64_t)u * R + row] = __float2half_rn(scale_store);
         zeros_out[(int64_t)u * R + row] = __float2half_rn(zero_store);
@@ -242,17 +277,17 @@ apply_plan_kernel(const __half* __restrict__ W, int R, int U, int64_t ldw, const
     if (a != 5) {
       int n_words;
       switch (a) {
-        case 1: pack_words<8>(code, words); n_words = 8; break;
-        case 2: pack_words<4>(code, words); n_words = 4; break;
-        case 3: pack_words<3>(code, words); n_words = 3; break;
-        case 4: pack_words<2>(code, words); n_words = 2; break;
-        default: pack_words<1>(code, words); n_words = 1; break;
+        case 1: pack_pairs<8>(code, words); n_words = 8; break;
+        case 2: pack_pairs<4>(code, words); n_words = 4; break;
+        case 3: pack_pairs<3>(code, words); n_words = 3; break;
+        case 4: pack_pairs<2>(code, words); n_words = 2; break;
+        default: pack_pairs<1>(code, words); n_words = 1; break;
       }
       if (live) store_words(row_codes + 4 * n_words * q, words, n_words);
     } else {
       // codes as 2-bit fields into the warp's buffer; an output byte is the base-3 value of five
       // consecutive fields, i.e. of a 10-bit window, looked up in the block's table
-      pack_words<2>(code, words);
+      pack_pairs<2>(code, words);
       __syncwarp();  // the previous item's fields have been read
       *reinterpret_cast<uint2*>(trits + g * (G / 4) + 8 * q) = make_uint2(words[0], words[1]);
       __syncwarp();

@@ -279,6 +279,112 @@ def test_argument_errors(wq, ctx):
     assert float(out["err"].abs().sum()) == 0.0
 
 
+# ------------------------------------------------------------------ layouts, limits, contexts
+def test_strided_weight_matrix(wq, ctx, oracle):
+    """W as a column block of a wider matrix (ldw > C): every call reads the same values as from a
+    packed copy, and apply_plan writes only inside the block of the fake-quantised output."""
+    G, R, C = 128, 50, 512
+    W, X = make(R, C, 610)
+    s = oracle.act_stats(X.numpy())
+    grid = ws.clip_grid(20)
+    wide = torch.full((R, C + 256), 7.0, dtype=torch.float16, device="cuda")
+    wide[:, 128:128 + C] = W.cuda()
+    view = wide[:, 128:128 + C]
+    s_d, grid_d = torch.from_numpy(s).cuda(), torch.from_numpy(grid).cuda()
+    want = oracle.fit_eval(W.numpy(), G, s, grid, threads=8)
+    got = wq.windq_fit_eval(ctx, view, G, s_d, grid_d, want_group_err=True)
+    check_fit({k: v.cpu().numpy() for k, v in got.items()}, want)
+    assert close(wq.windq_unit_features(ctx, view, G, s_d).cpu().numpy(), oracle.unit_features(W.numpy(), G, s)).all()
+    acts = np.array([3, 5, 6, 0], np.uint8)
+    a_d = torch.from_numpy(acts).cuda()
+    eb = wq.windq_effective_bits(ctx, a_d, R, G)
+    codes = torch.empty(int(eb["code_offsets"][-1].item()), dtype=torch.uint8, device="cuda")
+    wq_wide = torch.full_like(wide, -3.0)
+    plan = wq.windq_apply_plan(ctx, view, G, s_d, grid_d, a_d, eb["code_offsets"], codes, got["clip_idx"],
+                               out=dict(wq=wq_wide[:, 128:128 + C]))
+    o = oracle.apply_plan(W.numpy(), G, s, grid, acts, want["clip_idx"])
+    assert (codes.cpu().numpy() == o["codes"]).all()
+    assert (plan["wq"].cpu().view(torch.int16).numpy().view(np.uint16) == o["wq"]).all()
+    assert bool((wq_wide[:, :128] == -3.0).all()) and bool((wq_wide[:, 128 + C:] == -3.0).all())
+
+
+def test_empty_inputs_are_refused(wq, ctx):
+    grid = torch.from_numpy(ws.clip_grid(20)).cuda()
+    s = torch.ones(256, device="cuda")
+    empty = torch.zeros((0, 256), dtype=torch.float16, device="cuda")
+    for call in (lambda: wq.windq_fit_eval(ctx, empty, 128, s, grid),
+                 lambda: wq.windq_unit_features(ctx, empty, 128, s),
+                 lambda: wq.windq_act_stats(ctx, empty),
+                 lambda: wq.windq_effective_bits(ctx, torch.zeros(0, dtype=torch.uint8, device="cuda"), 16, 128)):
+        with pytest.raises(wq.WindqError) as e:
+            call()
+        assert e.value.status in (1, 2)          # NULL (no storage) or SHAPE
+
+
+def test_scratch_sizes_and_reserve(wq, oracle):
+    c = wq.windq_create(0)
+    try:
+        R, C, G = 333, 1024, 64
+        need = max(wq.windq_scratch_bytes_fit_eval(R, C, G), wq.windq_scratch_bytes_unit_features(R, C, G),
+                   wq.windq_scratch_bytes_act_stats(512, C))
+        assert need > 0 and wq.windq_scratch_bytes_fit_eval(R, C, 100) == 0
+        wq.windq_reserve(c, need)
+        W, X = make(R, C, 620)
+        s = wq.windq_act_stats(c, X.cuda())
+        assert close(s.cpu().numpy(), oracle.act_stats(X.numpy())).all()
+        with pytest.raises(wq.WindqError):
+            wq.windq_reserve(c, -1)
+    finally:
+        wq.windq_destroy(c)
+
+
+def test_two_contexts_on_two_streams(wq, ctx):
+    """Contexts own their scratch: calls through different contexts on different streams do not disturb
+    each other."""
+    other = wq.windq_create(0)
+    try:
+        W1 = ws.weights(400, 1024, 630, "student_t").cuda()
+        W2 = ws.weights(300, 2048, 631, "student_t").cuda()
+        s1, s2 = torch.rand(1024, device="cuda") + 0.1, torch.rand(2048, device="cuda") + 0.1
+        grid = torch.from_numpy(ws.clip_grid(20)).cuda()
+        ref1 = wq.windq_fit_eval(ctx, W1, 128, s1, grid)
+        ref2 = wq.windq_fit_eval(ctx, W2, 64, s2, grid)
+        f1 = wq.windq_unit_features(ctx, W1, 128, s1).clone()
+        torch.cuda.synchronize()
+        st1, st2 = torch.cuda.Stream(), torch.cuda.Stream()
+        for _ in range(3):
+            a = wq.windq_fit_eval(ctx, W1, 128, s1, grid, stream=st1)
+            b = wq.windq_fit_eval(other, W2, 64, s2, grid, stream=st2)
+            f = wq.windq_unit_features(other, W1, 128, s1, stream=st2)
+        torch.cuda.synchronize()
+        for k in ("err", "energy", "clip_idx"):
+            assert torch.equal(a[k], ref1[k]) and torch.equal(b[k], ref2[k])
+        assert torch.equal(f, f1)
+    finally:
+        wq.windq_destroy(other)
+
+
+def test_fit_eval_largest_grid_and_widest_chunk(wq, ctx, oracle):
+    G, R, C, K = 512, 21, 1024, 64
+    W, X = make(R, C, 640)
+    s = oracle.act_stats(X.numpy())
+    grid = ws.clip_grid(K, lo=1.0 / 64.0)
+    want = oracle.fit_eval(W.numpy(), G, s, grid, threads=8)
+    check_fit(run_fit(wq, ctx, W, G, s, grid), want)
+    acts = np.array([4, 2], np.uint8)
+    o = oracle.apply_plan(W.numpy(), G, s, grid, acts, None)
+    got = run_apply(wq, ctx, W, G, s, grid, acts, None)
+    for key in ("codes", "scales", "zeros", "wq"):
+        assert (got[key] == o[key]).all(), key
+
+
+def test_act_stats_near_the_fp16_limit(wq, ctx, oracle):
+    X = torch.full((300, 64), 60000.0, dtype=torch.float16)
+    X[::2] = -65504.0
+    got = wq.windq_act_stats(ctx, X.cuda()).cpu().numpy()
+    assert np.isfinite(got).all() and close(got, oracle.act_stats(X.numpy())).all()
+
+
 # ------------------------------------------------------------------ full size, sampled units
 def plan_for_target(wq, ctx, U, R, G, target, seed):
     """A seeded random plan at `target` average bits (the benchmark's recipe): the cost table comes

@@ -38,7 +38,7 @@ import windq_synth as ws
 METRIC = "unit_x_bitwidth_candidate_evals_per_s"
 UNIT = "evals/s"
 TARGET_BITS = (1.58, 2.0, 3.0)
-APPLY_G = 128
+APPLY_G = 128                    # chunk width the plans are applied at (the first of the workload's widths if it has no 128)
 FIT_TRAFFIC_PER_WEIGHT_BYTE = 34.82 / 33.554   # measured DRAM bytes per algorithmic byte (see profiles/)
 SEED = 0
 
@@ -463,8 +463,11 @@ def reference_main(args, spec):
 
 
 def main():
+    global APPLY_G
     args = parse_args()
     spec = ws.CONFIGS[args.workload]
+    if APPLY_G not in spec.chunk_widths:
+        APPLY_G = spec.chunk_widths[0]
     if args.impl == "reference":
         return reference_main(args, spec)
 

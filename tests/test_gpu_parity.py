@@ -404,6 +404,8 @@ FULL_SIZE_CASES = [
     ("cfg5_llama70b_model", 4, 1, 2.0),     # gate_proj 28672 x 8192
     ("cfg5_llama70b_model", 1, 2, 2.0),     # k_proj 1024 x 8192 (grouped-query attention)
     ("cfg5_llama70b_model", 6, 1, 2.0),     # down_proj 8192 x 28672
+    ("llama3_8b_g256", 4, 1, None),         # gate_proj 14336 x 4096 at the paper's chunk sizes 256 and 512
+    ("llama3_8b_g256", 2, 2, None),         # v_proj 1024 x 4096 (grouped-query attention)
 ]
 
 

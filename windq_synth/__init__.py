@@ -117,12 +117,15 @@ class ModelSpec:
         return sum(m.R * m.C for m in self.block_matrices())
 
 
-# The five benchmark configurations (LLaMA-1/2-style shapes).
+# The five benchmark configurations (LLaMA-1/2-style shapes), and the shape the paper itself reports its
+# unit count on ("Episode complexity": LLaMA-3.1-8B, chunk size 256, 32 x 7 x 16 = 3584 units), with its
+# ablated chunk size 512 beside it.
 CONFIGS = {
     "cfg1_single_layer": ModelSpec("cfg1_single_layer", 1, 4096, 0, 4096, "normal", 512, 20, (128,)),
     "cfg2_llama7b_block": ModelSpec("cfg2_llama7b_block", 1, 4096, 11008, 4096, "normal", 2048, 20, (128,)),
     "cfg3_llama7b_model": ModelSpec("cfg3_llama7b_model", 32, 4096, 11008, 4096, "student_t", 2048, 20, (64, 128)),
     "cfg4_llama13b_model": ModelSpec("cfg4_llama13b_model", 40, 5120, 13824, 5120, "student_t", 4096, 40, (128,)),
+    "llama3_8b_g256": ModelSpec("llama3_8b_g256", 32, 4096, 14336, 1024, "student_t", 2048, 20, (256, 512)),
     "cfg5_llama70b_model": ModelSpec("cfg5_llama70b_model", 80, 8192, 28672, 1024, "student_t", 2048, 20, (128,)),
 }
 

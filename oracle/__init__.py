@@ -182,3 +182,34 @@ def apply_plan(W, G: int, s, clip_grid, actions, clip_idx=None, want_wq: bool = 
     if rc:
         raise ValueError("oracle_apply_plan: bad arguments")
     return dict(codes=codes, scales=scales, zeros=zeros, wq=wq, code_offsets=offs)
+
+
+def salient_select(W, G: int, s, rate_ppm: int, want_mask: bool = True):
+    """Top-r selection of salient weights per unit.  Returns dict(thresh[U] f32, count[U] i64,
+    mask[R, C/8] u8 | None) -- bit (col % 8) of mask[r, col // 8] is set for a protected weight."""
+    W, s = _as_u16(W), _f32(s)
+    R, C = W.shape
+    U = C // G
+    thresh = np.zeros(U, np.float32)
+    count = np.zeros(U, np.int64)
+    mask = np.zeros((R, C // 8), np.uint8) if want_mask else None
+    rc = lib().oracle_salient_select(_p(W), ctypes.c_int64(R), ctypes.c_int64(C), ctypes.c_int64(C), ctypes.c_int(G),
+                                     _p(s), ctypes.c_int64(rate_ppm), _p(thresh), _p(count), _p(mask))
+    if rc:
+        raise ValueError("oracle_salient_select: bad arguments")
+    return dict(thresh=thresh, count=count, mask=mask)
+
+
+def effective_bits_protected(actions, n_protected, R: int, G: int, scale_bits: int = 16, zero_bits: int = 16):
+    """Eq. 6 with INT8-protected weights.  Returns dict(unit_centibits[U], total_centibits)."""
+    actions = np.ascontiguousarray(actions, dtype=np.uint8)
+    n_protected = np.ascontiguousarray(n_protected, dtype=np.int64)
+    U = actions.size
+    unit_cb = np.zeros(U, np.int64)
+    total = ctypes.c_int64()
+    rc = lib().oracle_effective_bits_protected(_p(actions), _p(n_protected), ctypes.c_int64(U), ctypes.c_int64(R),
+                                               ctypes.c_int(G), ctypes.c_int(scale_bits), ctypes.c_int(zero_bits),
+                                               _p(unit_cb), ctypes.byref(total))
+    if rc:
+        raise ValueError("oracle_effective_bits_protected: bad arguments")
+    return dict(unit_centibits=unit_cb, total_centibits=total.value)

@@ -35,7 +35,8 @@
 // ternary / binary closed forms and stationarity; scale invariance by powers of
 // two; degenerate groups; monotone error in bit-width; Eq. 6 bit arithmetic;
 // pack/unpack identity with an independent unpacker; nearest-rank P99 against a
-// full sort.  Parity unpinned: that threshold 0.7*mean|w| is a good ternary
+// full sort; salient selection against a full sort, its count arithmetic and
+// Eq. 6 with protected weights against the paper's formula.  Parity unpinned: that threshold 0.7*mean|w| is a good ternary
 // threshold, and that these fits resemble the paper's Adam-fitted operators --
 // neither is claimed.
 
@@ -43,6 +44,7 @@
 #include <cmath>
 #include <cstdint>
 #include <cstring>
+#include <limits>
 #include <vector>
 
 namespace {
@@ -563,6 +565,73 @@ int oracle_apply_plan(const uint16_t* W, int64_t R, int64_t C, int64_t ldw, int 
       zeros_out[u * R + r] = zero_h;
     }
   }
+  return 0;
+}
+
+// ---- salient-weight selection (App. "Salient Weight Protection") -----------------------------
+// The saliency of a weight is the product of its magnitude and the activation scale of its input
+// channel; the top-r fraction of a unit's weights by saliency is kept in INT8.
+// READING: the activation scale of channel j is a_j = sqrt(s_j), the root of the mean square that
+// act_stats returns (binary32 square root, then one binary32 product |w| * a_j: two IEEE
+// operations, so the key is reproducible).  n_p = floor(rate_ppm * n / 10^6) weights are asked
+// for; the threshold is the n_p-th largest key of the unit and every weight whose key reaches it
+// is protected, so equal keys at the threshold are all in (the protected count can exceed n_p,
+// and it is the count that Eq. 6 uses).  n_p = 0 protects nothing (threshold +infinity).
+int oracle_salient_select(const uint16_t* W, int64_t R, int64_t C, int64_t ldw, int G, const float* s,
+                          int64_t rate_ppm, float* thresh_out, int64_t* count_out, uint8_t* mask_out) {
+  if (!W || !s || !thresh_out || !count_out || R <= 0 || C <= 0 || G <= 0 || C % G || ldw < C) return 1;
+  if (rate_ppm < 0 || rate_ppm > 1000000) return 1;
+  const int64_t U = C / G, n = R * G;
+  const int64_t n_p = (int64_t)(((__int128)rate_ppm * n) / 1000000);
+  if (mask_out) std::memset(mask_out, 0, (size_t)(R * (C / 8)));
+  std::vector<float> key((size_t)n);
+  for (int64_t u = 0; u < U; ++u) {
+    for (int64_t r = 0; r < R; ++r)
+      for (int j = 0; j < G; ++j) {
+        const float a = std::sqrt(s[u * G + j]);
+        key[(size_t)(r * G + j)] = std::fabs(half_to_float(W[r * ldw + u * G + j])) * a;
+      }
+    float tau = std::numeric_limits<float>::infinity();
+    int64_t count = 0;
+    if (n_p > 0) {
+      std::vector<float> sorted(key);
+      std::nth_element(sorted.begin(), sorted.begin() + (n - n_p), sorted.end());
+      tau = sorted[(size_t)(n - n_p)];   // (n - n_p + 1)-th smallest = n_p-th largest
+      for (int64_t i = 0; i < n; ++i) count += key[(size_t)i] >= tau;
+    }
+    thresh_out[u] = tau;
+    count_out[u] = count;
+    if (mask_out && n_p > 0)
+      for (int64_t r = 0; r < R; ++r)
+        for (int j = 0; j < G; ++j)
+          if (key[(size_t)(r * G + j)] >= tau) {
+            const int64_t col = u * G + j;
+            mask_out[r * (C / 8) + col / 8] |= (uint8_t)(1u << (col % 8));
+          }
+  }
+  return 0;
+}
+
+// Eq. 6 in full: B_i = 16 n_i for skip, else b_i (n_i - n_i^(p)) + 8 n_i^(p), in centibits, plus
+// the per-group scale / zero-point overhead of the quantised part as in oracle_effective_bits.
+// A skipped unit protects nothing (its weights stay fp16).
+int oracle_effective_bits_protected(const uint8_t* actions, const int64_t* n_protected, int64_t U, int64_t R, int G,
+                                    int scale_bits, int zero_bits, int64_t* unit_centibits_out,
+                                    int64_t* total_centibits_out) {
+  if (!actions || !n_protected || U <= 0 || R <= 0 || G <= 0 || scale_bits < 0 || zero_bits < 0) return 1;
+  static const int64_t centi[7] = {1600, 800, 400, 300, 200, 158, 100};
+  int64_t total = 0;
+  for (int64_t u = 0; u < U; ++u) {
+    const int a = actions[u];
+    const int64_t n = R * G, np_ = n_protected[u];
+    if (a > 6 || np_ < 0 || np_ > n) return 1;
+    int64_t cb;
+    if (a == 0) cb = 1600 * n;
+    else cb = centi[a] * (n - np_) + 800 * np_ + 100 * R * (scale_bits + ((a <= 4) ? zero_bits : 0));
+    if (unit_centibits_out) unit_centibits_out[u] = cb;
+    total += cb;
+  }
+  if (total_centibits_out) *total_centibits_out = total;
   return 0;
 }
 

@@ -1,0 +1,130 @@
+"""Pins for the oracle's salient-weight selection and Eq. 6 with protected weights (CPU only)."""
+import os
+
+import numpy as np
+import pytest
+
+import windq_synth as ws
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def numpy_selection(W, G, s, rate_ppm):
+    """Independent restatement: keys in float32 with numpy, selection by a full sort."""
+    R, C = W.shape
+    a = np.sqrt(s.astype(np.float32))
+    key = np.abs(W.astype(np.float32)) * a[None, :]
+    assert key.dtype == np.float32
+    U, n = C // G, R * G
+    n_p = rate_ppm * n // 1_000_000
+    thresh = np.full(U, np.inf, np.float32)
+    mask = np.zeros((R, C), bool)
+    for u in range(U):
+        if n_p == 0:
+            continue
+        k = key[:, u * G:(u + 1) * G]
+        thresh[u] = np.sort(k.ravel())[::-1][n_p - 1]
+        mask[:, u * G:(u + 1) * G] = k >= thresh[u]
+    return thresh, mask
+
+
+def unpack_mask(mask_bytes, C):
+    return np.unpackbits(mask_bytes, axis=1, bitorder="little")[:, :C].astype(bool)
+
+
+@pytest.mark.parametrize("R,C,G,rate", [(64, 256, 128, 30000), (33, 128, 32, 20000), (100, 512, 256, 123456), (7, 64, 64, 500000)])
+def test_selection_against_a_full_sort(oracle, R, C, G, rate):
+    W = ws.weights(R, C, 900 + R, "student_t").numpy()
+    s = ws.activations(64, C, 901).numpy().astype(np.float32)
+    s = (s * s).mean(0).astype(np.float32)
+    got = oracle.salient_select(W, G, s, rate)
+    thresh, mask = numpy_selection(W, G, s, rate)
+    assert (got["thresh"] == thresh).all()
+    assert (unpack_mask(got["mask"], C) == mask).all()
+    assert (got["count"] == mask.reshape(R, C // G, G).sum((0, 2))).all()
+    assert (got["count"] >= rate * R * G // 1_000_000).all()
+
+
+def test_count_arithmetic_and_extremes(oracle):
+    for line in open(os.path.join(GOLDEN, "eq6_protected.txt")):
+        t = line.split()
+        if t and t[0] == "count":
+            rate, R, G, want = map(int, t[1:])
+            assert rate * R * G // 1_000_000 == want
+            # a unit of that size whose keys are all different: exactly `want` weights are protected.
+            # |w| takes 1024 values, the channel scales are 128 distinct powers of two apart by far more
+            # than the spread of |w|, rows repeat |w| with a period that no two rows share a (value, channel)
+            Wd = (1.0 + ((np.arange(R)[:, None] * 37 + np.arange(G)[None, :] * 5) % 1024) / 1024.0).astype(np.float16)
+            got = oracle.salient_select(Wd, G, (4.0 ** (np.arange(G) - 64)).astype(np.float32), rate)
+            assert got["count"][0] >= want
+            keys = np.abs(Wd.astype(np.float32)) * np.sqrt((4.0 ** (np.arange(G) - 64)).astype(np.float32))[None, :]
+            assert got["count"][0] == (keys >= np.sort(keys.ravel())[::-1][want - 1]).sum()
+    ones = oracle.salient_select(np.ones((64, 128), np.float16), 128, np.ones(128, np.float32), 30000)
+    assert ones["count"][0] == 64 * 128 and ones["thresh"][0] == np.float32(1.0)   # all keys tie: everything is in
+    W = ws.weights(40, 128, 5, "normal").numpy()
+    s = np.linspace(0.5, 2.0, 128).astype(np.float32)
+    none = oracle.salient_select(W, 128, s, 0)
+    assert np.isinf(none["thresh"]).all() and (none["count"] == 0).all() and not none["mask"].any()
+    every = oracle.salient_select(W, 128, s, 1_000_000)
+    assert (every["count"] == 40 * 128).all() and (np.unpackbits(every["mask"]).sum() == 40 * 128)
+    tiny = oracle.salient_select(W, 128, s, 100)                                # 0.01 % of 5120 = 0 weights
+    assert (tiny["count"] == 0).all()
+
+
+def test_planted_salient_weights_are_found(oracle):
+    R, C, G = 64, 256, 128
+    rng = np.random.default_rng(3)
+    W = (rng.standard_normal((R, C)) * 0.01).astype(np.float16)
+    s = np.ones(C, np.float32)
+    s[130] = 400.0                                   # hot channel: scale 20
+    rows = rng.choice(R, 9, replace=False)
+    W[rows, 130] = 0.5                               # 9 weights with key 10, everything else below 0.06 * 20
+    W[5, 7] = -3.0                                   # one big weight on an ordinary channel of unit 0
+    n_p = 9
+    rate = (n_p * 1_000_000 + R * G - 1) // (R * G)
+    assert rate * R * G // 1_000_000 == n_p
+    got = oracle.salient_select(W, G, s, rate)
+    mask = unpack_mask(got["mask"], C)
+    assert got["count"][1] == 9 and set(np.flatnonzero(mask[:, 130])) == set(rows) and mask[:, 128:].sum() == 9
+    assert got["thresh"][1] == np.float32(10.0)
+    assert mask[5, 7] and got["thresh"][0] <= np.float32(3.0)
+
+
+def test_power_of_two_invariance_and_monotone_rate(oracle):
+    R, C, G = 48, 256, 64
+    W = ws.weights(R, C, 11, "student_t").numpy()
+    s = (np.random.default_rng(4).random(C).astype(np.float32) + 0.1)
+    base = oracle.salient_select(W, G, s, 30000)
+    scaled_s = oracle.salient_select(W, G, s * np.float32(4.0), 30000)       # a_j doubles exactly
+    assert (scaled_s["mask"] == base["mask"]).all() and (scaled_s["thresh"] == base["thresh"] * np.float32(2)).all()
+    scaled_w = oracle.salient_select((W.astype(np.float32) * 2).astype(np.float16), G, s, 30000)
+    assert (scaled_w["mask"] == base["mask"]).all()
+    more = oracle.salient_select(W, G, s, 60000)
+    assert ((base["mask"] & ~more["mask"]) == 0).all() and (more["thresh"] <= base["thresh"]).all()
+
+
+def test_eq6_with_protected_weights(oracle):
+    rows = []
+    for line in open(os.path.join(GOLDEN, "eq6_protected.txt")):
+        t = line.split()
+        if t and t[0].isdigit():
+            rows.append((int(t[0]), int(t[2]), int(t[3]), int(t[4])))
+    assert len(rows) >= 10
+    for a, n, n_p, want in rows:
+        R, G = (n // 128, 128) if n % 128 == 0 else (n // 8, 8)
+        # G = 8 is not a chunk width of the library; the accounting only needs n = R * G
+        got = oracle.effective_bits_protected(np.array([a], np.uint8), np.array([n_p]), R, G, 0, 0)
+        assert got["unit_centibits"][0] == want and got["total_centibits"] == want
+    # with no protected weights it is the plain accounting, overhead included
+    acts = np.arange(7, dtype=np.uint8)
+    plain = oracle.effective_bits(acts, 96, 128)
+    prot = oracle.effective_bits_protected(acts, np.zeros(7, np.int64), 96, 128)
+    assert (plain["unit_centibits"] == prot["unit_centibits"]).all() and plain["total_centibits"] == prot["total_centibits"]
+    # 8-bit units cost the same whatever is protected; the average is sum B_i / sum n_i
+    a8 = oracle.effective_bits_protected(np.array([1, 1], np.uint8), np.array([0, 500]), 96, 128, 0, 0)
+    assert a8["unit_centibits"][0] == a8["unit_centibits"][1]
+    mix = oracle.effective_bits_protected(np.array([4, 6], np.uint8), np.array([369, 369]), 96, 128, 0, 0)
+    n = 96 * 128
+    assert mix["total_centibits"] == 200 * (n - 369) + 800 * 369 + 100 * (n - 369) + 800 * 369
+    with pytest.raises(ValueError):
+        oracle.effective_bits_protected(np.array([4], np.uint8), np.array([n + 1]), 96, 128)

@@ -181,6 +181,34 @@ windq_status windq_apply_plan(windq_ctx* ctx, const void* W, int64_t R, int64_t 
                               const uint8_t* clip_idx, const int64_t* code_offsets, uint8_t* codes_out,
                               void* scales_out, void* zeros_out, void* Wq_out, void* stream);
 
+/* ---- beyond the five calls: salient-weight protection (App. "Salient Weight Protection") ---------
+ *
+ * The paper keeps, in every unit, the top-r fraction of the weights by saliency -- weight magnitude
+ * times the activation scale of the weight's input channel -- in INT8 and counts them at 8 bits in
+ * Eq. 6.  windq_salient_select finds that set exactly; windq_effective_bits_protected is Eq. 6 with
+ * it.  (Fits and packing that leave the protected weights out are not built yet.)
+ *
+ *   key(r, j)  = |W[r][j]| * sqrt(s[j])            two binary32 operations (sqrt, then product)
+ *   n_p        = floor(rate_ppm * R * G / 10^6)     weights asked for per unit (rate in parts per million)
+ *   thresh_out fp32 [U]   the n_p-th largest key of the unit; +infinity when n_p = 0
+ *   count_out  i64  [U]   number of keys >= thresh: keys equal to the threshold are all protected, so
+ *                         the count can exceed n_p; it is the n^(p) of Eq. 6
+ *   mask_out   u8   [R][C/8], nullable   bit (j % 8) of byte [r][j / 8] is set for a protected weight
+ * R * G must be below 2^32.  Scratch: windq_scratch_bytes_salient_select. */
+int64_t windq_scratch_bytes_salient_select(int64_t R, int64_t C, int G);
+windq_status windq_salient_select(windq_ctx* ctx, const void* W, int64_t R, int64_t C, int64_t ldw, int G,
+                                  const float* s, int64_t rate_ppm, float* thresh_out, int64_t* count_out,
+                                  uint8_t* mask_out, void* stream);
+
+/* Eq. 6 in full, in centibits: 1600 n for a skipped unit (nothing of it is protected), otherwise
+ * 100 b (n - n_p) + 800 n_p, plus 100 R (scale_bits [+ zero_bits for 8/4/3/2 bit]) for the groups'
+ * parameters as in windq_effective_bits.  n_protected: i64 [U] (device), e.g. count_out above.
+ * An action code above 6 or a count outside [0, R * G] makes the total -1 (that unit's entry -1).
+ *   unit_centibits_out i64 [U], nullable;  total_centibits_out i64 [1] */
+windq_status windq_effective_bits_protected(windq_ctx* ctx, const uint8_t* actions, const int64_t* n_protected,
+                                            int64_t U, int64_t R, int G, int scale_bits, int zero_bits,
+                                            int64_t* unit_centibits_out, int64_t* total_centibits_out, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

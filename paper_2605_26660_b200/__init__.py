@@ -49,7 +49,7 @@ def _load() -> ctypes.CDLL:
     for name in ("windq_scratch_bytes_act_stats",):
         getattr(lib, name).argtypes = [i64, i64]
         getattr(lib, name).restype = i64
-    for name in ("windq_scratch_bytes_unit_features", "windq_scratch_bytes_fit_eval"):
+    for name in ("windq_scratch_bytes_unit_features", "windq_scratch_bytes_fit_eval", "windq_scratch_bytes_salient_select"):
         getattr(lib, name).argtypes = [i64, i64, i32]
         getattr(lib, name).restype = i64
     lib.windq_act_stats.argtypes = [vp, vp, i64, i64, i64, vp, vp]
@@ -57,6 +57,8 @@ def _load() -> ctypes.CDLL:
     lib.windq_unit_features.argtypes = [vp, vp, i64, i64, i64, i32, vp, vp, vp]
     lib.windq_fit_eval.argtypes = [vp, vp, i64, i64, i64, i32, vp, vp, i32, vp, vp, vp, vp, vp]
     lib.windq_effective_bits.argtypes = [vp, vp, i64, i64, i32, i32, i32, vp, vp, vp, vp, vp]
+    lib.windq_salient_select.argtypes = [vp, vp, i64, i64, i64, i32, vp, i64, vp, vp, vp, vp]
+    lib.windq_effective_bits_protected.argtypes = [vp, vp, vp, i64, i64, i32, i32, i32, vp, vp, vp]
     lib.windq_apply_plan.argtypes = [vp, vp, i64, i64, i64, i32, vp, vp, i32, vp, vp, vp, vp, vp, vp, vp, vp]
     return lib
 
@@ -277,3 +279,44 @@ def windq_apply_plan(ctx: Context, W: torch.Tensor, G: int, s: torch.Tensor, cli
                                      _ptr(actions), _ptr(clip_idx), _ptr(code_offsets), _ptr(codes_out), _ptr(out["scales"]),
                                      _ptr(out["zeros"]), _ptr(out["wq"]), _stream(stream)))
     return out
+
+
+def windq_scratch_bytes_salient_select(R: int, C: int, G: int) -> int:
+    return int(_lib.windq_scratch_bytes_salient_select(R, C, G))
+
+
+def windq_salient_select(ctx: Context, W: torch.Tensor, G: int, s: torch.Tensor, rate_ppm: int, *,
+                         want_mask: bool = True, out: dict | None = None, stream=None) -> dict:
+    """Top-r salient weights per unit (key |w| * sqrt(s_j), rate in parts per million).
+
+    Returns dict(thresh [U] f32, count [U] i64, mask [R, C/8] u8 | None)."""
+    R, C, ldw = _matrix(W, "W")
+    _need(s, torch.float32, "s", 1)
+    U = C // G if G > 0 else 0
+    out = dict(out) if out else {}
+    dev = W.device
+    if out.get("thresh") is None:
+        out["thresh"] = torch.empty(U, dtype=torch.float32, device=dev)
+    if out.get("count") is None:
+        out["count"] = torch.empty(U, dtype=torch.int64, device=dev)
+    if want_mask and out.get("mask") is None:
+        out["mask"] = torch.empty((R, C // 8), dtype=torch.uint8, device=dev)
+    out.setdefault("mask", None)
+    ctx._check(_lib.windq_salient_select(ctx._h, _ptr(W), R, C, ldw, int(G), _ptr(s), int(rate_ppm), _ptr(out["thresh"]),
+                                         _ptr(out["count"]), _ptr(out["mask"]), _stream(stream)))
+    return out
+
+
+def windq_effective_bits_protected(ctx: Context, actions: torch.Tensor, n_protected: torch.Tensor, R: int, G: int,
+                                   scale_bits: int = 16, zero_bits: int = 16, stream=None) -> dict:
+    """Eq. 6 with INT8-protected weights.  Returns dict(unit_centibits [U] i64, total_centibits [1] i64)."""
+    _need(actions, torch.uint8, "actions", 1)
+    _need(n_protected, torch.int64, "n_protected", 1)
+    U = actions.numel()
+    if n_protected.numel() != U:
+        raise ValueError("n_protected must have one entry per unit")
+    unit = torch.empty(U, dtype=torch.int64, device=actions.device)
+    total = torch.empty(1, dtype=torch.int64, device=actions.device)
+    ctx._check(_lib.windq_effective_bits_protected(ctx._h, _ptr(actions), _ptr(n_protected), U, int(R), int(G),
+                                                   int(scale_bits), int(zero_bits), _ptr(unit), _ptr(total), _stream(stream)))
+    return dict(unit_centibits=unit, total_centibits=total)

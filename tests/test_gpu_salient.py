@@ -1,0 +1,107 @@
+"""GPU parity of salient-weight selection and Eq. 6 with protected weights against the CPU oracle.
+Thresholds, counts, mask bytes and bit totals are integers or bit patterns: all compared exactly."""
+import numpy as np
+import pytest
+import torch
+
+import windq_synth as ws
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def wq():
+    import paper_2605_26660_b200 as wq
+    return wq
+
+
+@pytest.fixture(scope="module")
+def ctx(wq):
+    c = wq.windq_create(0)
+    yield c
+    wq.windq_destroy(c)
+
+
+def run(wq, ctx, W, G, s, rate):
+    out = wq.windq_salient_select(ctx, W.cuda(), G, torch.from_numpy(s).cuda(), rate)
+    torch.cuda.synchronize()
+    return {k: v.cpu().numpy() for k, v in out.items()}
+
+
+@pytest.mark.parametrize("R,C,G,rate", [(300, 512, 128, 30000), (97, 256, 64, 20000), (64, 128, 32, 123456),
+                                        (1000, 1024, 256, 30000), (33, 1024, 512, 500000), (50, 256, 128, 1000000),
+                                        (4096, 512, 128, 30000), (3, 128, 128, 30000)])
+def test_salient_select(wq, ctx, oracle, R, C, G, rate):
+    W = ws.weights(R, C, 700 + R, "student_t")
+    W[::3, ::5] = 0
+    X = ws.activations(64, C, 701)
+    s = oracle.act_stats(X.numpy())
+    want = oracle.salient_select(W.numpy(), G, s, rate)
+    got = run(wq, ctx, W, G, s, rate)
+    assert (got["thresh"].view(np.uint32) == want["thresh"].view(np.uint32)).all()
+    assert (got["count"] == want["count"]).all()
+    assert (got["mask"] == want["mask"]).all()
+
+
+def test_salient_select_ties_zero_rate_and_strides(wq, ctx, oracle):
+    G, R = 128, 40
+    W = torch.full((R, 3 * G), 0.25, dtype=torch.float16)       # unit 0: every key equal
+    W[:, G:2 * G] = 0                                           # unit 1: every key zero
+    W[:, 2 * G:] = ws.weights(R, G, 3, "normal")
+    s = np.ones(3 * G, np.float32)
+    s[2 * G:2 * G + 5] = 0                                      # channels that never fire: key 0
+    want = oracle.salient_select(W.numpy(), G, s, 30000)
+    got = run(wq, ctx, W, G, s, 30000)
+    assert (got["count"] == want["count"]).all() and got["count"][0] == R * G and got["count"][1] == R * G
+    assert (got["thresh"].view(np.uint32) == want["thresh"].view(np.uint32)).all() and (got["mask"] == want["mask"]).all()
+    none = run(wq, ctx, W, G, s, 0)
+    assert np.isinf(none["thresh"]).all() and (none["count"] == 0).all() and not none["mask"].any()
+    wide = torch.zeros((R, 4 * G), dtype=torch.float16, device="cuda")
+    wide[:, G:] = W.cuda()
+    out = wq.windq_salient_select(ctx, wide[:, G:], G, torch.from_numpy(s).cuda(), 30000)
+    assert (out["mask"].cpu().numpy() == want["mask"]).all()
+    with pytest.raises(wq.WindqError) as e:
+        wq.windq_salient_select(ctx, W.cuda(), G, torch.from_numpy(s).cuda(), 1000001)
+    assert e.value.status == 4
+
+
+def test_effective_bits_protected(wq, ctx, oracle):
+    rng = np.random.default_rng(5)
+    for U, R, G in ((86, 4096, 128), (1, 7, 32), (3000, 50, 64)):
+        acts = rng.integers(0, 7, U).astype(np.uint8)
+        n_p = rng.integers(0, R * G // 20 + 1, U).astype(np.int64)
+        for sb, zb in ((16, 16), (0, 0)):
+            want = oracle.effective_bits_protected(acts, n_p, R, G, sb, zb)
+            got = wq.windq_effective_bits_protected(ctx, torch.from_numpy(acts).cuda(), torch.from_numpy(n_p).cuda(), R, G, sb, zb)
+            assert (got["unit_centibits"].cpu().numpy() == want["unit_centibits"]).all()
+            assert int(got["total_centibits"].item()) == want["total_centibits"]
+    bad = wq.windq_effective_bits_protected(ctx, torch.tensor([4, 9], dtype=torch.uint8, device="cuda"),
+                                            torch.tensor([0, 0], dtype=torch.int64, device="cuda"), 8, 128)
+    assert int(bad["total_centibits"].item()) == -1
+
+
+def test_full_size_selection_feeds_eq6(wq, ctx, oracle):
+    """11008 x 4096 Student-t matrix of the 7B-shaped sweep at the paper's 3 % rate: sampled units against
+    the oracle, counts into Eq. 6, and the average bits of an all-2-bit plan with protection."""
+    spec = ws.CONFIGS["cfg3_llama7b_model"]
+    m = spec.block_matrices()[4]
+    W = ws.block_weight(spec, 0, 0, m, device="cuda")
+    X = ws.block_input(spec, 0, 0, m.x_id, device="cuda")
+    s = wq.windq_act_stats(ctx, X)
+    G, U = 128, m.C // 128
+    out = wq.windq_salient_select(ctx, W, G, s, 30000)
+    n_p = 30000 * m.R * G // 1_000_000
+    count = out["count"].cpu().numpy()
+    assert (count >= n_p).all() and (count <= n_p + 64).all()      # ties at the threshold are rare on this data
+    bits_set = np.unpackbits(out["mask"].cpu().numpy(), axis=1, bitorder="little").reshape(m.R, U, G).sum((0, 2))
+    assert (bits_set == count).all()
+    s_h = s.cpu().numpy()
+    for u in (0, 17, U - 1):
+        want = oracle.salient_select(W[:, u * G:(u + 1) * G].cpu().numpy(), G, s_h[u * G:(u + 1) * G], 30000)
+        assert out["thresh"][u].cpu().numpy().view(np.uint32) == want["thresh"].view(np.uint32)[0]
+        assert count[u] == want["count"][0]
+        assert (out["mask"][:, u * G // 8:(u + 1) * G // 8].cpu().numpy() == want["mask"]).all()
+    acts = torch.full((U,), 4, dtype=torch.uint8, device="cuda")
+    eb = wq.windq_effective_bits_protected(ctx, acts, out["count"], m.R, G, 0, 0)
+    avg = int(eb["total_centibits"].item()) / (100.0 * m.R * m.C)
+    assert abs(avg - (2 * 0.97 + 8 * 0.03)) < 1e-3                  # 2.18 bits: the paper's accounting at 3 %

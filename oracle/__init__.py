@@ -112,8 +112,10 @@ def unit_features(W, G: int, s) -> np.ndarray:
     return feat
 
 
-def fit_eval(W, G: int, s, clip_grid, units=None, threads: int = 1, want_group_err: bool = True):
+def fit_eval(W, G: int, s, clip_grid, units=None, threads: int = 1, want_group_err: bool = True, thresh=None):
     """Returns dict(err[U,6], energy[U], clip_idx[4,U,R], group_err[6,U,R]).
+
+    ``thresh`` (fp32 [U], from salient_select) takes the protected weights out of the fits.
 
     ``units`` = (begin, end) restricts the work to a unit range (other rows of
     the outputs stay zero).  ``threads`` > 1 runs the same single-threaded
@@ -129,10 +131,20 @@ def fit_eval(W, G: int, s, clip_grid, units=None, threads: int = 1, want_group_e
     clip_idx = np.zeros((4, U, R), np.uint8)
     group_err = np.zeros((N_BITWIDTHS, U, R), np.float32) if want_group_err else None
 
+    if thresh is not None:
+        thresh = _f32(thresh)
+        assert thresh.size == U
+
     def run(a, b):
-        rc = lib().oracle_fit_eval(_p(W), ctypes.c_int64(R), ctypes.c_int64(C), ctypes.c_int64(C), ctypes.c_int(G),
-                                   _p(s), _p(clip_grid), ctypes.c_int(K), ctypes.c_int64(a), ctypes.c_int64(b),
-                                   _p(err), _p(energy), _p(clip_idx), _p(group_err))
+        if thresh is None:
+            rc = lib().oracle_fit_eval(_p(W), ctypes.c_int64(R), ctypes.c_int64(C), ctypes.c_int64(C), ctypes.c_int(G),
+                                       _p(s), _p(clip_grid), ctypes.c_int(K), ctypes.c_int64(a), ctypes.c_int64(b),
+                                       _p(err), _p(energy), _p(clip_idx), _p(group_err))
+        else:
+            rc = lib().oracle_fit_eval_protected(_p(W), ctypes.c_int64(R), ctypes.c_int64(C), ctypes.c_int64(C),
+                                                 ctypes.c_int(G), _p(s), _p(clip_grid), ctypes.c_int(K), ctypes.c_int64(a),
+                                                 ctypes.c_int64(b), _p(thresh), _p(err), _p(energy), _p(clip_idx),
+                                                 _p(group_err))
         if rc:
             raise ValueError("oracle_fit_eval: bad arguments")
 

@@ -436,21 +436,34 @@ int oracle_unit_features(const uint16_t* W, int64_t R, int64_t C, int64_t ldw, i
 // ---- a3: fit every row-group of units [u_begin, u_end) under all six bit-widths.
 // err_out[U][6], energy_out[U] (nullable), clip_idx_out[4][U][R] (nullable),
 // group_err_out[6][U][R] (nullable).  Only rows of the requested units are written.
-int oracle_fit_eval(const uint16_t* W, int64_t R, int64_t C, int64_t ldw, int G, const float* s,
-                    const float* clip_grid, int K, int64_t u_begin, int64_t u_end, float* err_out,
-                    float* energy_out, uint8_t* clip_idx_out, float* group_err_out) {
+// thresh == NULL: the fit of every group as it is.  thresh != NULL (one saliency threshold per unit,
+// from oracle_salient_select): READING -- a protected weight (key |w| * sqrt(s_j) >= thresh[u]) is
+// stored apart in INT8, so it is taken out of its group's fit: inside the group it counts as a zero
+// weight with zero activation weight (its position and the group size stay), which removes it from
+// the range, from every sum and from every error; the error of its INT8 copy is not part of err.
+static int fit_eval_impl(const uint16_t* W, int64_t R, int64_t C, int64_t ldw, int G, const float* s,
+                         const float* clip_grid, int K, int64_t u_begin, int64_t u_end, const float* thresh,
+                         float* err_out, float* energy_out, uint8_t* clip_idx_out, float* group_err_out) {
   if (!W || !s || !clip_grid || !err_out || R <= 0 || C <= 0 || !valid_group_width(G) || C % G != 0 ||
       ldw < C || K < 1 || K > 64)
     return 1;
   const int64_t U = C / G;
   if (u_begin < 0 || u_end > U || u_begin > u_end) return 1;
-  std::vector<float> w((size_t)G), what((size_t)G);
+  std::vector<float> w((size_t)G), what((size_t)G), sm((size_t)G);
   for (int64_t u = u_begin; u < u_end; ++u) {
     double tot[6] = {0, 0, 0, 0, 0, 0};
     double energy = 0.0;
     const float* su = s + u * G;
     for (int64_t r = 0; r < R; ++r) {
       load_group(W, ldw, r, u, G, w.data());
+      if (thresh) {
+        for (int j = 0; j < G; ++j) {
+          const bool prot = std::fabs(w[(size_t)j]) * std::sqrt(s[u * G + j]) >= thresh[u];
+          sm[(size_t)j] = prot ? 0.0f : s[u * G + j];
+          if (prot) w[(size_t)j] = 0.0f;
+        }
+        su = sm.data();
+      }
       Group g{G, w.data(), su};
       float e[6];
       float mn, rng;
@@ -480,6 +493,21 @@ int oracle_fit_eval(const uint16_t* W, int64_t R, int64_t C, int64_t ldw, int G,
 // ---- a5: effective bits (Eq. 6 with no protected weights, extended by the
 // per-group scale / zero-point overhead) in integer centibits, plus the byte
 // offset of every unit's packed block (each rounded up to 16 bytes).
+int oracle_fit_eval(const uint16_t* W, int64_t R, int64_t C, int64_t ldw, int G, const float* s,
+                    const float* clip_grid, int K, int64_t u_begin, int64_t u_end, float* err_out,
+                    float* energy_out, uint8_t* clip_idx_out, float* group_err_out) {
+  return fit_eval_impl(W, R, C, ldw, G, s, clip_grid, K, u_begin, u_end, nullptr, err_out, energy_out, clip_idx_out,
+                       group_err_out);
+}
+
+int oracle_fit_eval_protected(const uint16_t* W, int64_t R, int64_t C, int64_t ldw, int G, const float* s,
+                              const float* clip_grid, int K, int64_t u_begin, int64_t u_end, const float* thresh,
+                              float* err_out, float* energy_out, uint8_t* clip_idx_out, float* group_err_out) {
+  if (!thresh) return 1;
+  return fit_eval_impl(W, R, C, ldw, G, s, clip_grid, K, u_begin, u_end, thresh, err_out, energy_out, clip_idx_out,
+                       group_err_out);
+}
+
 int oracle_effective_bits(const uint8_t* actions, int64_t U, int64_t R, int G, int scale_bits,
                           int zero_bits, int64_t* unit_centibits_out, int64_t* code_offsets_out,
                           int64_t* total_centibits_out, int64_t* total_packed_bytes_out) {

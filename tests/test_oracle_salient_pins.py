@@ -128,3 +128,38 @@ def test_eq6_with_protected_weights(oracle):
     assert mix["total_centibits"] == 200 * (n - 369) + 800 * 369 + 100 * (n - 369) + 800 * 369
     with pytest.raises(ValueError):
         oracle.effective_bits_protected(np.array([4], np.uint8), np.array([n + 1]), 96, 128)
+
+
+# ------------------------------------------------------------------ fits with the protected weights left out
+def test_protected_fit_reduces_to_the_plain_fit(oracle):
+    R, C, G = 24, 256, 128
+    W = ws.weights(R, C, 21, "normal").numpy()
+    s = (np.random.default_rng(6).random(C).astype(np.float32) + 0.2)
+    grid = ws.clip_grid(20)
+    plain = oracle.fit_eval(W, G, s, grid)
+    nothing = oracle.fit_eval(W, G, s, grid, thresh=np.full(C // G, np.inf, np.float32))
+    for k in plain:
+        assert (plain[k].view(np.uint32 if plain[k].dtype == np.float32 else plain[k].dtype) ==
+                nothing[k].view(np.uint32 if nothing[k].dtype == np.float32 else nothing[k].dtype)).all()
+    # a column whose every weight is protected: the same as the plain fit of the matrix with that column
+    # zeroed and its activation weight zero (the masking is per weight, so this is the case the plain call
+    # can express)
+    W2 = W.copy()
+    W2[:, 40] = np.float16(0.75)                       # far above everything else in unit 0
+    sel = oracle.salient_select(W2, G, s, R * 1_000_000 // (R * G))     # n_p = R weights per unit
+    mask = np.unpackbits(sel["mask"], axis=1, bitorder="little").astype(bool)
+    assert mask[:, 40].all() and mask[:, :G].sum() == R
+    prot = oracle.fit_eval(W2, G, s, grid, thresh=sel["thresh"], units=(0, 1))
+    W3, s3 = W2.copy(), s.copy()
+    W3[:, 40] = 0
+    s3[40] = 0
+    want = oracle.fit_eval(W3, G, s3, grid, units=(0, 1))
+    assert (prot["clip_idx"][:, 0] == want["clip_idx"][:, 0]).all()
+    assert (prot["group_err"][:, 0].view(np.uint32) == want["group_err"][:, 0].view(np.uint32)).all()
+    assert prot["energy"][0] == want["energy"][0] and (prot["err"][0] == want["err"][0]).all()
+    # protecting the outlier column is the point of the method: the low-bit errors of the unit drop
+    unprot = oracle.fit_eval(W2, G, s, grid, units=(0, 1))
+    assert (prot["err"][0, 1:4] < 0.5 * unprot["err"][0, 1:4]).all()
+    # everything protected: nothing is left to fit
+    allp = oracle.fit_eval(W, G, s, grid, thresh=np.zeros(C // G, np.float32))
+    assert not allp["err"].any() and not allp["energy"].any()

@@ -186,7 +186,8 @@ windq_status windq_apply_plan(windq_ctx* ctx, const void* W, int64_t R, int64_t 
  * The paper keeps, in every unit, the top-r fraction of the weights by saliency -- weight magnitude
  * times the activation scale of the weight's input channel -- in INT8 and counts them at 8 bits in
  * Eq. 6.  windq_salient_select finds that set exactly; windq_effective_bits_protected is Eq. 6 with
- * it.  (Fits and packing that leave the protected weights out are not built yet.)
+ * it; windq_fit_eval_protected scores the fits with those weights left out.  (Packing with INT8 side
+ * storage for them is not built yet.)
  *
  *   key(r, j)  = |W[r][j]| * sqrt(s[j])            two binary32 operations (sqrt, then product)
  *   n_p        = floor(rate_ppm * R * G / 10^6)     weights asked for per unit (rate in parts per million)
@@ -199,6 +200,18 @@ int64_t windq_scratch_bytes_salient_select(int64_t R, int64_t C, int G);
 windq_status windq_salient_select(windq_ctx* ctx, const void* W, int64_t R, int64_t C, int64_t ldw, int G,
                                   const float* s, int64_t rate_ppm, float* thresh_out, int64_t* count_out,
                                   uint8_t* mask_out, void* stream);
+
+/* windq_fit_eval with the protected weights taken out of the fits: a weight whose key reaches
+ * thresh[u] (fp32 [U], device, from windq_salient_select with the same W, s and G) counts, inside its
+ * group, as a zero weight with zero activation weight -- it leaves the range, every sum and every
+ * error, while its position and the group size stay.  The error of its INT8 copy is not part of the
+ * outputs.  With every threshold +infinity the results are those of windq_fit_eval, bit for bit.
+ * Outputs and the other arguments as windq_fit_eval; scratch: windq_scratch_bytes_fit_eval_protected. */
+int64_t windq_scratch_bytes_fit_eval_protected(int64_t R, int64_t C, int G);
+windq_status windq_fit_eval_protected(windq_ctx* ctx, const void* W, int64_t R, int64_t C, int64_t ldw, int G,
+                                      const float* s, const float* clip_grid, int K, const float* thresh,
+                                      float* err_out, float* energy_out, uint8_t* clip_idx_out, float* group_err_out,
+                                      void* stream);
 
 /* Eq. 6 in full, in centibits: 1600 n for a skipped unit (nothing of it is protected), otherwise
  * 100 b (n - n_p) + 800 n_p, plus 100 R (scale_bits [+ zero_bits for 8/4/3/2 bit]) for the groups'

@@ -56,6 +56,9 @@ def _load() -> ctypes.CDLL:
     lib.windq_act_stats_noalloc.argtypes = [vp, vp, i64, i64, i64, vp, vp]
     lib.windq_unit_features.argtypes = [vp, vp, i64, i64, i64, i32, vp, vp, vp]
     lib.windq_fit_eval.argtypes = [vp, vp, i64, i64, i64, i32, vp, vp, i32, vp, vp, vp, vp, vp]
+    lib.windq_fit_eval_protected.argtypes = [vp, vp, i64, i64, i64, i32, vp, vp, i32, vp, vp, vp, vp, vp, vp]
+    lib.windq_scratch_bytes_fit_eval_protected.argtypes = [i64, i64, i32]
+    lib.windq_scratch_bytes_fit_eval_protected.restype = i64
     lib.windq_effective_bits.argtypes = [vp, vp, i64, i64, i32, i32, i32, vp, vp, vp, vp, vp]
     lib.windq_salient_select.argtypes = [vp, vp, i64, i64, i64, i32, vp, i64, vp, vp, vp, vp]
     lib.windq_effective_bits_protected.argtypes = [vp, vp, vp, i64, i64, i32, i32, i32, vp, vp, vp]
@@ -190,8 +193,9 @@ def windq_unit_features(ctx: Context, W: torch.Tensor, G: int, s: torch.Tensor, 
 
 def windq_fit_eval(ctx: Context, W: torch.Tensor, G: int, s: torch.Tensor, clip_grid: torch.Tensor, *,
                    want_energy: bool = True, want_clip_idx: bool = True, want_group_err: bool = False,
-                   out: dict | None = None, stream=None) -> dict:
-    """Fits every group under all six bit-widths.
+                   out: dict | None = None, stream=None, thresh: torch.Tensor | None = None) -> dict:
+    """Fits every group under all six bit-widths.  With ``thresh`` (fp32 [U], from windq_salient_select) the
+    call is windq_fit_eval_protected: the salient weights are left out of the fits.
 
     Returns dict(err [U,6] f32, energy [U] f32 | None, clip_idx [4,U,R] u8 | None,
     group_err [6,U,R] f32 | None).  ``out`` may hold preallocated tensors under the same keys.
@@ -212,9 +216,17 @@ def windq_fit_eval(ctx: Context, W: torch.Tensor, G: int, s: torch.Tensor, clip_
         out["group_err"] = torch.empty((N_BITWIDTHS, U, R), dtype=torch.float32, device=dev)
     for key in ("energy", "clip_idx", "group_err"):
         out.setdefault(key, None)
-    ctx._check(_lib.windq_fit_eval(ctx._h, _ptr(W), R, C, ldw, int(G), _ptr(s), _ptr(clip_grid), clip_grid.numel(),
-                                   _ptr(out["err"]), _ptr(out["energy"]), _ptr(out["clip_idx"]), _ptr(out["group_err"]),
-                                   _stream(stream)))
+    if thresh is None:
+        ctx._check(_lib.windq_fit_eval(ctx._h, _ptr(W), R, C, ldw, int(G), _ptr(s), _ptr(clip_grid), clip_grid.numel(),
+                                       _ptr(out["err"]), _ptr(out["energy"]), _ptr(out["clip_idx"]), _ptr(out["group_err"]),
+                                       _stream(stream)))
+    else:
+        _need(thresh, torch.float32, "thresh", 1)
+        if thresh.numel() != U:
+            raise ValueError("thresh must have one entry per unit")
+        ctx._check(_lib.windq_fit_eval_protected(ctx._h, _ptr(W), R, C, ldw, int(G), _ptr(s), _ptr(clip_grid),
+                                                 clip_grid.numel(), _ptr(thresh), _ptr(out["err"]), _ptr(out["energy"]),
+                                                 _ptr(out["clip_idx"]), _ptr(out["group_err"]), _stream(stream)))
     return out
 
 

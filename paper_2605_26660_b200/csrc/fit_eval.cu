@@ -27,11 +27,15 @@ __host__ __device__ inline int fit_cand_chunk(int G) {
 }
 __host__ __device__ inline int fit_cand_stride(int chunk) { return chunk | 1; }  // odd: conflict-free rows
 
-template <int G>
+// PROTECT: salient weights (key |w| * scale_j >= thresh[u], scale_j = sqrt(s_j)) are taken out of
+// the fits: in the lane's registers such a weight becomes a zero weight with zero activation weight,
+// after which the fit is the ordinary one.
+template <int G, bool PROTECT>
 __global__ void __launch_bounds__(kFitWarpsPerBlock * 32, 4)
 fit_eval_kernel(const __half* __restrict__ W, int R, int U, int64_t ldw, const float* __restrict__ s,
                 const float* __restrict__ clip, int K, double* __restrict__ partial, uint8_t* __restrict__ clip_idx_out,
-                float* __restrict__ group_err_out, int rows_blocks, int chunk, int stride) {
+                float* __restrict__ group_err_out, int rows_blocks, int chunk, int stride,
+                const float* __restrict__ scale, const float* __restrict__ thresh) {
   constexpr int LG = Map<G>::LG, GPW = Map<G>::GPW;
   extern __shared__ float4 smem_f4[];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -47,7 +51,7 @@ fit_eval_kernel(const __half* __restrict__ W, int R, int U, int64_t ldw, const f
   int cur_u = -1;
   for (int64_t item = item_begin; item < item_end; ++item) {
     const int u = (int)(item / rows_blocks), rb = (int)(item % rows_blocks);
-    if (u != cur_u) {
+    if (PROTECT || u != cur_u) {
       load_stats(s + (int64_t)u * G + 32 * q, sv);
       cur_u = u;
     }
@@ -56,6 +60,18 @@ fit_eval_kernel(const __half* __restrict__ W, int R, int U, int64_t ldw, const f
     const int row_ld = live ? row : R - 1;  // rows past the end repeat the last row and are not written
     Lane32 wv;
     load_weights(W + (int64_t)row_ld * ldw + (int64_t)u * G + 32 * q, wv);
+    if (PROTECT) {
+      Lane32 av;
+      load_stats(scale + (int64_t)u * G + 32 * q, av);
+      const float tau = __ldg(thresh + u);
+#pragma unroll
+      for (int h = 0; h < 2; ++h)
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          if (__fmul_rn(fabsf(wv.v[h][i].x), av.v[h][i].x) >= tau) { wv.v[h][i].x = 0.0f; sv.v[h][i].x = 0.0f; }
+          if (__fmul_rn(fabsf(wv.v[h][i].y), av.v[h][i].y) >= tau) { wv.v[h][i].y = 0.0f; sv.v[h][i].y = 0.0f; }
+        }
+    }
 
     float mn, mx;
     group_range<G>(wv, mn, mx);
@@ -121,23 +137,31 @@ fit_finalize_kernel(const double* __restrict__ partial, int rows_blocks, float* 
   }
 }
 
-template <int G>
+// sqrt(s_j): the activation scale that the saliency key uses.
+__global__ void fit_scale_kernel(const float* __restrict__ s, int C, float* __restrict__ scale) {
+  const int j = blockIdx.x * blockDim.x + threadIdx.x;
+  if (j < C) scale[j] = __fsqrt_rn(s[j]);
+}
+
+template <int G, bool PROTECT>
 windq_status launch_fit(windq_ctx* ctx, const __half* W, int R, int U, int64_t ldw, const float* s,
                         const float* clip, int K, double* partial, float* err_out, float* energy_out,
-                        uint8_t* clip_idx_out, float* group_err_out, cudaStream_t st) {
+                        uint8_t* clip_idx_out, float* group_err_out, float* scale, const float* thresh,
+                        cudaStream_t st) {
   constexpr int GPW = Map<G>::GPW;
   const int rows_blocks = (R + GPW - 1) / GPW;
   const int chunk = fit_cand_chunk(G), stride = fit_cand_stride(chunk);
   const size_t smem = (size_t)kFitWarpsPerBlock * GPW * stride * sizeof(Cand);
-  const int id = kFitG32 + g_index(G);
-  if (windq_status rc = prepare_kernel(ctx, id, fit_eval_kernel<G>, kFitWarpsPerBlock * 32, smem, true)) return rc;
+  const int id = (PROTECT ? kFitProtectG32 : kFitG32) + g_index(G);
+  if (windq_status rc = prepare_kernel(ctx, id, fit_eval_kernel<G, PROTECT>, kFitWarpsPerBlock * 32, smem, true)) return rc;
   const int blocks_per_sm = ctx->occupancy[id];
   const int64_t n_items = (int64_t)U * rows_blocks;
   int64_t grid = (int64_t)ctx->sm_count * blocks_per_sm;
   const int64_t need = (n_items + kFitWarpsPerBlock - 1) / kFitWarpsPerBlock;
   if (grid > need) grid = need;
-  fit_eval_kernel<G><<<(unsigned)grid, kFitWarpsPerBlock * 32, smem, st>>>(W, R, U, ldw, s, clip, K, partial, clip_idx_out,
-                                                                          group_err_out, rows_blocks, chunk, stride);
+  if (PROTECT) fit_scale_kernel<<<(unsigned)((U * G + 255) / 256), 256, 0, st>>>(s, U * G, scale);
+  fit_eval_kernel<G, PROTECT><<<(unsigned)grid, kFitWarpsPerBlock * 32, smem, st>>>(
+      W, R, U, ldw, s, clip, K, partial, clip_idx_out, group_err_out, rows_blocks, chunk, stride, scale, thresh);
   WINDQ_CUDA(ctx, cudaGetLastError());
   fit_finalize_kernel<<<(unsigned)U, 256, 0, st>>>(partial, rows_blocks, err_out, energy_out);
   WINDQ_CUDA(ctx, cudaGetLastError());
@@ -154,28 +178,58 @@ int64_t windq_scratch_bytes_fit_eval(int64_t R, int64_t C, int G) {
   return (C / G) * ((R + gpw - 1) / gpw) * windq::kFitPartials * (int64_t)sizeof(double);
 }
 
-windq_status windq_fit_eval(windq_ctx* ctx, const void* W, int64_t R, int64_t C, int64_t ldw, int G, const float* s,
-                            const float* clip_grid, int K, float* err_out, float* energy_out, uint8_t* clip_idx_out,
-                            float* group_err_out, void* stream) {
+static windq_status fit_eval_any(windq_ctx* ctx, const char* who, const void* W, int64_t R, int64_t C, int64_t ldw, int G,
+                                 const float* s, const float* clip_grid, int K, const float* thresh, float* err_out,
+                                 float* energy_out, uint8_t* clip_idx_out, float* group_err_out, void* stream) {
   using namespace windq;
-  if (!ctx) return fail(nullptr, WINDQ_ERR_NULL, "windq_fit_eval: ctx is NULL");
-  if (windq_status st = check_matrix(ctx, "windq_fit_eval", W, R, C, ldw, G)) return st;
-  if (windq_status st = check_K(ctx, "windq_fit_eval", K)) return st;
-  WINDQ_REQUIRE(ctx, s && clip_grid && err_out, WINDQ_ERR_NULL, "windq_fit_eval: s, clip_grid or err_out is NULL");
-  WINDQ_REQUIRE(ctx, aligned16(s), WINDQ_ERR_ALIGN, "windq_fit_eval: s is not 16-byte aligned");
+  if (!ctx) return fail(nullptr, WINDQ_ERR_NULL, "%s: ctx is NULL", who);
+  if (windq_status st = check_matrix(ctx, who, W, R, C, ldw, G)) return st;
+  if (windq_status st = check_K(ctx, who, K)) return st;
+  WINDQ_REQUIRE(ctx, s && clip_grid && err_out, WINDQ_ERR_NULL, "%s: s, clip_grid or err_out is NULL", who);
+  WINDQ_REQUIRE(ctx, aligned16(s), WINDQ_ERR_ALIGN, "%s: s is not 16-byte aligned", who);
   DeviceGuard guard(ctx->device);
-  if (windq_status st = ensure_scratch(ctx, windq_scratch_bytes_fit_eval(R, C, G))) return st;
+  const int64_t part_bytes = windq_scratch_bytes_fit_eval(R, C, G);
+  if (windq_status st = ensure_scratch(ctx, thresh ? windq_scratch_bytes_fit_eval_protected(R, C, G) : part_bytes)) return st;
   const int U = (int)(C / G);
   cudaStream_t st = (cudaStream_t)stream;
   const __half* Wh = (const __half*)W;
   double* partial = (double*)ctx->scratch;
+  float* scale = (float*)((char*)ctx->scratch + round_up(part_bytes, 16));
+#define WINDQ_FIT_CASE(GG)                                                                                              \
+  case GG:                                                                                                              \
+    return thresh ? launch_fit<GG, true>(ctx, Wh, (int)R, U, ldw, s, clip_grid, K, partial, err_out, energy_out,         \
+                                         clip_idx_out, group_err_out, scale, thresh, st)                                \
+                  : launch_fit<GG, false>(ctx, Wh, (int)R, U, ldw, s, clip_grid, K, partial, err_out, energy_out,        \
+                                          clip_idx_out, group_err_out, nullptr, nullptr, st);
   switch (G) {
-    case 32: return launch_fit<32>(ctx, Wh, (int)R, U, ldw, s, clip_grid, K, partial, err_out, energy_out, clip_idx_out, group_err_out, st);
-    case 64: return launch_fit<64>(ctx, Wh, (int)R, U, ldw, s, clip_grid, K, partial, err_out, energy_out, clip_idx_out, group_err_out, st);
-    case 128: return launch_fit<128>(ctx, Wh, (int)R, U, ldw, s, clip_grid, K, partial, err_out, energy_out, clip_idx_out, group_err_out, st);
-    case 256: return launch_fit<256>(ctx, Wh, (int)R, U, ldw, s, clip_grid, K, partial, err_out, energy_out, clip_idx_out, group_err_out, st);
-    default: return launch_fit<512>(ctx, Wh, (int)R, U, ldw, s, clip_grid, K, partial, err_out, energy_out, clip_idx_out, group_err_out, st);
+    WINDQ_FIT_CASE(32)
+    WINDQ_FIT_CASE(64)
+    WINDQ_FIT_CASE(128)
+    WINDQ_FIT_CASE(256)
+    default:
+      WINDQ_FIT_CASE(512)
   }
+#undef WINDQ_FIT_CASE
+}
+
+int64_t windq_scratch_bytes_fit_eval_protected(int64_t R, int64_t C, int G) {
+  const int64_t base = windq_scratch_bytes_fit_eval(R, C, G);
+  return base ? windq::round_up(base, 16) + C * (int64_t)sizeof(float) : 0;
+}
+
+windq_status windq_fit_eval(windq_ctx* ctx, const void* W, int64_t R, int64_t C, int64_t ldw, int G, const float* s,
+                            const float* clip_grid, int K, float* err_out, float* energy_out, uint8_t* clip_idx_out,
+                            float* group_err_out, void* stream) {
+  return fit_eval_any(ctx, "windq_fit_eval", W, R, C, ldw, G, s, clip_grid, K, nullptr, err_out, energy_out, clip_idx_out,
+                      group_err_out, stream);
+}
+
+windq_status windq_fit_eval_protected(windq_ctx* ctx, const void* W, int64_t R, int64_t C, int64_t ldw, int G,
+                                      const float* s, const float* clip_grid, int K, const float* thresh, float* err_out,
+                                      float* energy_out, uint8_t* clip_idx_out, float* group_err_out, void* stream) {
+  if (ctx && !thresh) return windq::fail(ctx, WINDQ_ERR_NULL, "windq_fit_eval_protected: thresh is NULL");
+  return fit_eval_any(ctx, "windq_fit_eval_protected", W, R, C, ldw, G, s, clip_grid, K, thresh, err_out, energy_out,
+                      clip_idx_out, group_err_out, stream);
 }
 
 }  // extern "C"

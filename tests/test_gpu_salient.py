@@ -105,3 +105,49 @@ def test_full_size_selection_feeds_eq6(wq, ctx, oracle):
     eb = wq.windq_effective_bits_protected(ctx, acts, out["count"], m.R, G, 0, 0)
     avg = int(eb["total_centibits"].item()) / (100.0 * m.R * m.C)
     assert abs(avg - (2 * 0.97 + 8 * 0.03)) < 1e-3                  # 2.18 bits: the paper's accounting at 3 %
+
+
+# ------------------------------------------------------------------ fits with the protected weights left out
+def fit(wq, ctx, W, G, s, grid, thresh=None):
+    out = wq.windq_fit_eval(ctx, W.cuda(), G, torch.from_numpy(s).cuda(), torch.from_numpy(grid).cuda(), want_group_err=True,
+                            thresh=None if thresh is None else torch.from_numpy(thresh).cuda())
+    torch.cuda.synchronize()
+    return {k: v.cpu().numpy() for k, v in out.items()}
+
+
+def same_fit(got, want):
+    assert (got["clip_idx"] == want["clip_idx"]).all()
+    assert (got["group_err"].view(np.uint32) == want["group_err"].view(np.uint32)).all()
+    for k in ("err", "energy"):
+        assert (np.abs(got[k] - want[k]) <= 1e-4 * np.abs(want[k]) + 1e-6).all(), k
+
+
+@pytest.mark.parametrize("G,R,C,rate", [(128, 70, 512, 30000), (64, 37, 256, 30000), (32, 33, 128, 100000),
+                                        (256, 19, 1024, 20000), (512, 9, 1024, 30000)])
+def test_fit_eval_protected(wq, ctx, oracle, G, R, C, rate):
+    W = ws.weights(R, C, 800 + G, "student_t")
+    X = ws.activations(64, C, 801)
+    s = oracle.act_stats(X.numpy())
+    grid = ws.clip_grid(20)
+    sel = oracle.salient_select(W.numpy(), G, s, rate)
+    want = oracle.fit_eval(W.numpy(), G, s, grid, threads=8, thresh=sel["thresh"])
+    same_fit(fit(wq, ctx, W, G, s, grid, sel["thresh"]), want)
+    # thresholds from the GPU selection are the same bits, so the two calls chain on the device
+    dev = wq.windq_salient_select(ctx, W.cuda(), G, torch.from_numpy(s).cuda(), rate, want_mask=False)
+    out = wq.windq_fit_eval(ctx, W.cuda(), G, torch.from_numpy(s).cuda(), torch.from_numpy(grid).cuda(), thresh=dev["thresh"])
+    assert (out["clip_idx"].cpu().numpy() == want["clip_idx"]).all()
+
+
+def test_fit_eval_protected_limits(wq, ctx, oracle):
+    G, R, C = 128, 40, 256
+    W = ws.weights(R, C, 810, "normal")
+    s = (np.random.default_rng(8).random(C).astype(np.float32) + 0.2)
+    grid = ws.clip_grid(20)
+    plain = fit(wq, ctx, W, G, s, grid)
+    nothing = fit(wq, ctx, W, G, s, grid, np.full(C // G, np.inf, np.float32))
+    for k in plain:
+        assert (plain[k] == nothing[k]).all() or k in ("err", "energy")
+    assert (plain["group_err"].view(np.uint32) == nothing["group_err"].view(np.uint32)).all()
+    everything = fit(wq, ctx, W, G, s, grid, np.zeros(C // G, np.float32))
+    assert not everything["err"].any() and not everything["energy"].any() and not everything["group_err"].any()
+    same_fit(everything, oracle.fit_eval(W.numpy(), G, s, grid, thresh=np.zeros(C // G, np.float32)))

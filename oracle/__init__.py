@@ -225,3 +225,28 @@ def effective_bits_protected(actions, n_protected, R: int, G: int, scale_bits: i
     if rc:
         raise ValueError("oracle_effective_bits_protected: bad arguments")
     return dict(unit_centibits=unit_cb, total_centibits=total.value)
+
+
+def unit_saliency(W, G: int, s):
+    """Mean of sqrt(s_j) * |w| over every unit.  Returns fp32 [U]."""
+    W, s = _as_u16(W), _f32(s)
+    R, C = W.shape
+    out = np.zeros(C // G, np.float32)
+    rc = lib().oracle_unit_saliency(_p(W), ctypes.c_int64(R), ctypes.c_int64(C), ctypes.c_int64(C), ctypes.c_int(G), _p(s), _p(out))
+    if rc:
+        raise ValueError("oracle_unit_saliency: bad arguments")
+    return out
+
+
+def fallback(err, energy, actions, theta: float):
+    """Moves every unit whose relative error exceeds theta to higher precision.  Returns (actions, n_changed)."""
+    err, energy = _f32(err), _f32(energy)
+    actions = np.ascontiguousarray(actions, dtype=np.uint8)
+    U = actions.size
+    assert err.shape == (U, N_BITWIDTHS) and energy.size == U
+    out = np.zeros(U, np.uint8)
+    n = ctypes.c_int64()
+    rc = lib().oracle_fallback(_p(err), _p(energy), _p(actions), ctypes.c_int64(U), ctypes.c_float(theta), _p(out), ctypes.byref(n))
+    if rc:
+        raise ValueError("oracle_fallback: bad arguments")
+    return out, n.value

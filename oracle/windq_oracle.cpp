@@ -663,4 +663,41 @@ int oracle_effective_bits_protected(const uint8_t* actions, const int64_t* n_pro
   return 0;
 }
 
+// ---- heuristic allocator inputs ("Comparison with Heuristic Sensitivity Allocator") and fallback ----
+// Saliency score of a unit: the mean, over the unit's weights, of activation scale times weight
+// magnitude, with the activation scale a_j = sqrt(s_j) as in oracle_salient_select.  Products and
+// the sum are taken in double (tolerance output).
+int oracle_unit_saliency(const uint16_t* W, int64_t R, int64_t C, int64_t ldw, int G, const float* s, float* sal_out) {
+  if (!W || !s || !sal_out || R <= 0 || C <= 0 || G <= 0 || C % G || ldw < C) return 1;
+  for (int64_t u = 0; u < C / G; ++u) {
+    double acc = 0.0;
+    for (int64_t r = 0; r < R; ++r)
+      for (int j = 0; j < G; ++j)
+        acc += (double)std::sqrt(s[u * G + j]) * (double)std::fabs(half_to_float(W[r * ldw + u * G + j]));
+    sal_out[u] = (float)(acc / (double)(R * G));
+  }
+  return 0;
+}
+
+// "If the reconstruction error of a selected operator is excessive, the implementation falls back to
+// a higher-precision operator" (Sec. 3.5).  READING (the paper gives neither the measure nor the
+// threshold): the error of action a is excessive when err[u][a] > theta * energy[u], both binary32,
+// one binary32 product on the right; the unit then moves to the next higher precision (1 -> 1.58 -> 2
+// -> 3 -> 4 -> 8 -> skip) until the test passes; skip has no error and always passes.
+int oracle_fallback(const float* err, const float* energy, const uint8_t* actions, int64_t U, float theta,
+                    uint8_t* actions_out, int64_t* n_changed_out) {
+  if (!err || !energy || !actions || !actions_out || U <= 0 || !(theta >= 0.0f)) return 1;
+  int64_t changed = 0;
+  for (int64_t u = 0; u < U; ++u) {
+    int a = actions[u];
+    if (a > 6) return 1;
+    const float limit = theta * energy[u];
+    while (a >= 1 && err[u * 6 + (a - 1)] > limit) --a;
+    actions_out[u] = (uint8_t)a;
+    changed += a != actions[u];
+  }
+  if (n_changed_out) *n_changed_out = changed;
+  return 0;
+}
+
 }  // extern "C"

@@ -163,3 +163,48 @@ def test_protected_fit_reduces_to_the_plain_fit(oracle):
     # everything protected: nothing is left to fit
     allp = oracle.fit_eval(W, G, s, grid, thresh=np.zeros(C // G, np.float32))
     assert not allp["err"].any() and not allp["energy"].any()
+
+
+# ------------------------------------------------------------------ unit saliency and the fallback rule
+def test_unit_saliency_closed_forms(oracle):
+    R, G = 30, 32
+    W = np.full((R, 2 * G), 0.5, np.float16)
+    W[:, G:] = -0.25
+    s = np.full(2 * G, 4.0, np.float32)
+    s[G:] = 9.0
+    assert (oracle.unit_saliency(W, G, s) == np.array([1.0, 0.75], np.float32)).all()     # 2 * 0.5, 3 * 0.25
+    rng = np.random.default_rng(9)
+    W = (rng.standard_normal((R, 4 * G)) * 0.02).astype(np.float16)
+    s = (rng.random(4 * G) + 0.1).astype(np.float32)
+    want = (np.abs(W.astype(np.float64)) * np.sqrt(s)[None, :].astype(np.float64)).reshape(R, 4, G).mean((0, 2))
+    assert np.allclose(oracle.unit_saliency(W, G, s), want, rtol=1e-6)
+    hot = s.copy()
+    hot[G:2 * G] *= 4                                   # activation scale of unit 1 doubles
+    got = oracle.unit_saliency(W, G, hot)
+    assert np.allclose(got[1], 2 * want[1], rtol=1e-6) and np.allclose(got[[0, 2, 3]], want[[0, 2, 3]], rtol=1e-6)
+
+
+def test_fallback_rule(oracle):
+    #            8     4     3     2    1.58   1
+    err = np.array([[0.0, 0.1, 0.2, 0.4, 0.6, 0.8],
+                    [0.0, 0.1, 0.2, 0.4, 0.6, 0.8],
+                    [0.3, 0.3, 0.3, 0.3, 0.3, 0.3],
+                    [0.0, 0.0, 0.0, 0.0, 0.0, 0.0]], np.float32)
+    energy = np.array([1.0, 2.0, 1.0, 0.0], np.float32)
+    acts = np.array([6, 6, 4, 5], np.uint8)
+    out, n = oracle.fallback(err, energy, acts, 0.25)
+    # unit 0: 1-bit 0.8 > 0.25 -> 1.58 (0.6) -> 2 (0.4) -> 3 (0.2) passes; unit 1: limit 0.5: 1-bit 0.8, 1.58 0.6 fail, 2-bit 0.4 passes;
+    # unit 2: every quantised action fails -> skip; unit 3: zero energy, zero error: 0 > 0 is false, stays
+    assert out.tolist() == [3, 4, 0, 5] and n == 3
+    same, n0 = oracle.fallback(err, energy, acts, np.inf)
+    assert (same == acts).all() and n0 == 0
+    strict, _ = oracle.fallback(err, energy, acts, 0.0)
+    assert strict.tolist() == [1, 1, 0, 5]              # 8-bit has zero error in units 0 and 1
+    # monotone in theta: a larger tolerance never asks for more precision
+    rng = np.random.default_rng(10)
+    e = np.sort(rng.random((50, 6)).astype(np.float32), axis=1)
+    en = np.ones(50, np.float32)
+    a = rng.integers(0, 7, 50).astype(np.uint8)
+    lo, _ = oracle.fallback(e, en, a, 0.2)
+    hi, _ = oracle.fallback(e, en, a, 0.6)
+    assert (hi >= lo).all() and (lo <= a).all()

@@ -222,6 +222,26 @@ windq_status windq_effective_bits_protected(windq_ctx* ctx, const uint8_t* actio
                                             int64_t U, int64_t R, int G, int scale_bits, int zero_bits,
                                             int64_t* unit_centibits_out, int64_t* total_centibits_out, void* stream);
 
+/* Saliency score of every unit ("Comparison with Heuristic Sensitivity Allocator": the mean product of
+ * activation scale and weight magnitude), the quantity the paper's heuristic allocator ranks units by:
+ *   sal_out[u] = (1 / (R G)) * sum over the unit of sqrt(s[j]) * |W[r][j]|        fp32 [U]
+ * (double accumulation; the order of the block sums is not fixed, so the last bits can differ from run
+ * to run; within 1e-6 relative of the exact value). */
+windq_status windq_unit_saliency(windq_ctx* ctx, const void* W, int64_t R, int64_t C, int64_t ldw, int G,
+                                 const float* s, float* sal_out, void* stream);
+
+/* Fallback to higher precision (Sec. 3.5: "if the reconstruction error of a selected operator is
+ * excessive, the implementation falls back to a higher-precision operator").  The paper gives neither
+ * the measure nor the threshold; here the error of unit u under action a is excessive when
+ *   err[u][a] > theta * energy[u]     (binary32 on both sides; err and energy from windq_fit_eval)
+ * and the unit moves one step at a time towards higher precision (1 -> 1.58 -> 2 -> 3 -> 4 -> 8 ->
+ * skip) until the test passes; skip always passes.
+ *   err fp32 [U][6], energy fp32 [U], actions u8 [U] (device); theta >= 0 (host value)
+ *   actions_out u8 [U] (may be `actions` itself);  n_changed_out i64 [1], nullable
+ * Action codes above 6 are copied unchanged. */
+windq_status windq_fallback(windq_ctx* ctx, const float* err, const float* energy, const uint8_t* actions, int64_t U,
+                            float theta, uint8_t* actions_out, int64_t* n_changed_out, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -62,6 +62,8 @@ def _load() -> ctypes.CDLL:
     lib.windq_effective_bits.argtypes = [vp, vp, i64, i64, i32, i32, i32, vp, vp, vp, vp, vp]
     lib.windq_salient_select.argtypes = [vp, vp, i64, i64, i64, i32, vp, i64, vp, vp, vp, vp]
     lib.windq_effective_bits_protected.argtypes = [vp, vp, vp, i64, i64, i32, i32, i32, vp, vp, vp]
+    lib.windq_unit_saliency.argtypes = [vp, vp, i64, i64, i64, i32, vp, vp, vp]
+    lib.windq_fallback.argtypes = [vp, vp, vp, vp, i64, ctypes.c_float, vp, vp, vp]
     lib.windq_apply_plan.argtypes = [vp, vp, i64, i64, i64, i32, vp, vp, i32, vp, vp, vp, vp, vp, vp, vp, vp]
     return lib
 
@@ -332,3 +334,32 @@ def windq_effective_bits_protected(ctx: Context, actions: torch.Tensor, n_protec
     ctx._check(_lib.windq_effective_bits_protected(ctx._h, _ptr(actions), _ptr(n_protected), U, int(R), int(G),
                                                    int(scale_bits), int(zero_bits), _ptr(unit), _ptr(total), _stream(stream)))
     return dict(unit_centibits=unit, total_centibits=total)
+
+
+def windq_unit_saliency(ctx: Context, W: torch.Tensor, G: int, s: torch.Tensor, sal_out: torch.Tensor | None = None,
+                        stream=None) -> torch.Tensor:
+    """Mean of sqrt(s_j) * |w| over every unit: fp32 [U]."""
+    R, C, ldw = _matrix(W, "W")
+    _need(s, torch.float32, "s", 1)
+    if sal_out is None:
+        sal_out = torch.empty(max(C // max(G, 1), 0), dtype=torch.float32, device=W.device)
+    _need(sal_out, torch.float32, "sal_out", 1)
+    ctx._check(_lib.windq_unit_saliency(ctx._h, _ptr(W), R, C, ldw, int(G), _ptr(s), _ptr(sal_out), _stream(stream)))
+    return sal_out
+
+
+def windq_fallback(ctx: Context, err: torch.Tensor, energy: torch.Tensor, actions: torch.Tensor, theta: float,
+                   stream=None) -> dict:
+    """Moves units whose relative error exceeds theta to higher precision.
+    Returns dict(actions [U] u8, n_changed [1] i64)."""
+    _need(err, torch.float32, "err", 2)
+    _need(energy, torch.float32, "energy", 1)
+    _need(actions, torch.uint8, "actions", 1)
+    U = actions.numel()
+    if err.shape != (U, N_BITWIDTHS) or energy.numel() != U or not err.is_contiguous():
+        raise ValueError("err must be a contiguous [U, 6] table and energy [U]")
+    out = torch.empty_like(actions)
+    n = torch.empty(1, dtype=torch.int64, device=actions.device)
+    ctx._check(_lib.windq_fallback(ctx._h, _ptr(err), _ptr(energy), _ptr(actions), U, float(theta), _ptr(out), _ptr(n),
+                                   _stream(stream)))
+    return dict(actions=out, n_changed=n)

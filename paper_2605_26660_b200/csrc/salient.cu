@@ -337,3 +337,149 @@ windq_status windq_effective_bits_protected(windq_ctx* ctx, const uint8_t* actio
 }
 
 }  // extern "C"
+
+// ---- unit saliency and the fallback rule --------------------------------------------------------
+namespace windq {
+
+// Per unit, the sum over its weights of scale_j * |w| ("Comparison with Heuristic Sensitivity
+// Allocator": saliency score = mean product of activation scale and weight magnitude).  Same block
+// schedule as the histogram passes; a thread adds |w| of its eight columns over its rows in fp32
+// (at most a few hundred terms), multiplies by the scales and hands a double to the block sum, which
+// goes to the unit's accumulator with one double atomic per (block, unit).
+template <int G>
+__global__ void __launch_bounds__(kSalThreads)
+unit_saliency_kernel(const __half* __restrict__ W, int R, int64_t ldw, const float* __restrict__ s, long long rows_per_block,
+                     long long total_rows, double* __restrict__ acc) {
+  __shared__ double wsum[kSalThreads / 32];
+  constexpr int TPR = G / 8, RPP = kSalThreads / TPR;
+  const int tr = threadIdx.x / TPR, tc = threadIdx.x % TPR;
+  long long p = (long long)blockIdx.x * rows_per_block;
+  const long long p_end = min(p + rows_per_block, total_rows);
+  while (p < p_end) {
+    const int u = (int)(p / R);
+    const int r0 = (int)(p - (long long)u * R);
+    const int r1 = (int)min((long long)R, r0 + (p_end - p));
+    const __half* base = W + (int64_t)u * G + tc * 8;
+    double sum = 0.0;
+    float col[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    int n_in_col = 0;
+    for (int r = r0 + tr; r < r1; r += 4 * RPP) {
+      uint4 raw[4];
+#pragma unroll
+      for (int k = 0; k < 4; ++k)
+        if (r + k * RPP < r1) raw[k] = __ldg(reinterpret_cast<const uint4*>(base + (int64_t)(r + k * RPP) * ldw));
+#pragma unroll
+      for (int k = 0; k < 4; ++k)
+        if (r + k * RPP < r1) {
+          const __half2* h = reinterpret_cast<const __half2*>(&raw[k]);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const float2 f = __half22float2(h[i]);
+            col[2 * i] += fabsf(f.x);
+            col[2 * i + 1] += fabsf(f.y);
+          }
+        }
+      if (++n_in_col == 64 || r + 4 * RPP >= r1) {  // at most 256 terms per fp32 column sum
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          sum += (double)col[i] * (double)__fsqrt_rn(__ldg(s + (int64_t)u * G + tc * 8 + i));
+          col[i] = 0.0f;
+        }
+        n_in_col = 0;
+      }
+    }
+#pragma unroll
+    for (int m = 16; m > 0; m >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, m);
+    if ((threadIdx.x & 31) == 0) wsum[threadIdx.x >> 5] = sum;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      double t = 0.0;
+      for (int i = 0; i < kSalThreads / 32; ++i) t += wsum[i];
+      atomicAdd(&acc[u], t);
+    }
+    __syncthreads();
+    p += r1 - r0;
+  }
+}
+
+__global__ void unit_saliency_finish_kernel(const double* __restrict__ acc, int U, double inv_n, float* __restrict__ sal_out) {
+  const int u = blockIdx.x * blockDim.x + threadIdx.x;
+  if (u < U) sal_out[u] = (float)(acc[u] * inv_n);
+}
+
+__global__ void fallback_kernel(const float* __restrict__ err, const float* __restrict__ energy,
+                                const uint8_t* __restrict__ actions, long long U, float theta,
+                                uint8_t* __restrict__ actions_out, unsigned long long* __restrict__ n_changed) {
+  const long long u = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  int changed = 0;
+  if (u < U) {
+    const int a0 = actions[u];
+    int a = a0;
+    if (a <= 6) {
+      const float limit = __fmul_rn(theta, energy[u]);
+      while (a >= 1 && err[u * 6 + (a - 1)] > limit) --a;
+    }
+    actions_out[u] = (uint8_t)a;
+    changed = a != a0;
+  }
+  const unsigned int votes = __ballot_sync(0xffffffffu, changed);
+  if ((threadIdx.x & 31) == 0 && votes && n_changed) atomicAdd(n_changed, (unsigned long long)__popc(votes));
+}
+
+template <int G>
+windq_status run_saliency(windq_ctx* ctx, const __half* W, int R, int C, int64_t ldw, const float* s, float* sal_out,
+                          cudaStream_t st) {
+  const int U = C / G;
+  double* acc = (double*)ctx->scratch;
+  const long long total = (long long)U * R;
+  long long nb = (long long)ctx->sm_count * kSalBlocksPerSM;
+  if (nb * 16 > total) nb = (total + 15) / 16;
+  const long long rpb = (total + nb - 1) / nb;
+  WINDQ_CUDA(ctx, cudaMemsetAsync(acc, 0, (size_t)U * sizeof(double), st));
+  unit_saliency_kernel<G><<<(unsigned)((total + rpb - 1) / rpb), kSalThreads, 0, st>>>(W, R, ldw, s, rpb, total, acc);
+  unit_saliency_finish_kernel<<<(unsigned)((U + 255) / 256), 256, 0, st>>>(acc, U, 1.0 / ((double)R * G), sal_out);
+  WINDQ_CUDA(ctx, cudaGetLastError());
+  return WINDQ_OK;
+}
+
+}  // namespace windq
+
+extern "C" {
+
+windq_status windq_unit_saliency(windq_ctx* ctx, const void* W, int64_t R, int64_t C, int64_t ldw, int G, const float* s,
+                                 float* sal_out, void* stream) {
+  using namespace windq;
+  if (!ctx) return fail(nullptr, WINDQ_ERR_NULL, "windq_unit_saliency: ctx is NULL");
+  if (windq_status st = check_matrix(ctx, "windq_unit_saliency", W, R, C, ldw, G)) return st;
+  WINDQ_REQUIRE(ctx, s && sal_out, WINDQ_ERR_NULL, "windq_unit_saliency: s or sal_out is NULL");
+  DeviceGuard guard(ctx->device);
+  if (windq_status rc = ensure_scratch(ctx, (C / G) * (int64_t)sizeof(double))) return rc;
+  cudaStream_t st = (cudaStream_t)stream;
+  const __half* Wh = (const __half*)W;
+  switch (G) {
+    case 32: return run_saliency<32>(ctx, Wh, (int)R, (int)C, ldw, s, sal_out, st);
+    case 64: return run_saliency<64>(ctx, Wh, (int)R, (int)C, ldw, s, sal_out, st);
+    case 128: return run_saliency<128>(ctx, Wh, (int)R, (int)C, ldw, s, sal_out, st);
+    case 256: return run_saliency<256>(ctx, Wh, (int)R, (int)C, ldw, s, sal_out, st);
+    default: return run_saliency<512>(ctx, Wh, (int)R, (int)C, ldw, s, sal_out, st);
+  }
+}
+
+windq_status windq_fallback(windq_ctx* ctx, const float* err, const float* energy, const uint8_t* actions, int64_t U,
+                            float theta, uint8_t* actions_out, int64_t* n_changed_out, void* stream) {
+  using namespace windq;
+  if (!ctx) return fail(nullptr, WINDQ_ERR_NULL, "windq_fallback: ctx is NULL");
+  WINDQ_REQUIRE(ctx, err && energy && actions && actions_out, WINDQ_ERR_NULL, "windq_fallback: a required pointer is NULL");
+  WINDQ_REQUIRE(ctx, U > 0 && U < (1ll << 31), WINDQ_ERR_SHAPE, "windq_fallback: U = %lld", (long long)U);
+  WINDQ_REQUIRE(ctx, theta >= 0.0f, WINDQ_ERR_ARG, "windq_fallback: theta must be a number >= 0");
+  WINDQ_REQUIRE(ctx, ((uintptr_t)n_changed_out & 7) == 0, WINDQ_ERR_ALIGN, "windq_fallback: n_changed_out is not 8-byte aligned");
+  DeviceGuard guard(ctx->device);
+  cudaStream_t st = (cudaStream_t)stream;
+  if (n_changed_out) WINDQ_CUDA(ctx, cudaMemsetAsync(n_changed_out, 0, sizeof(int64_t), st));
+  fallback_kernel<<<(unsigned)((U + 255) / 256), 256, 0, st>>>(err, energy, actions, (long long)U, theta, actions_out,
+                                                               (unsigned long long*)n_changed_out);
+  WINDQ_CUDA(ctx, cudaGetLastError());
+  return WINDQ_OK;
+}
+
+}  // extern "C"

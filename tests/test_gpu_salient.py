@@ -151,3 +151,30 @@ def test_fit_eval_protected_limits(wq, ctx, oracle):
     everything = fit(wq, ctx, W, G, s, grid, np.zeros(C // G, np.float32))
     assert not everything["err"].any() and not everything["energy"].any() and not everything["group_err"].any()
     same_fit(everything, oracle.fit_eval(W.numpy(), G, s, grid, thresh=np.zeros(C // G, np.float32)))
+
+
+# ------------------------------------------------------------------ unit saliency and the fallback rule
+@pytest.mark.parametrize("R,C,G", [(300, 512, 128), (4096, 1024, 256), (37, 128, 32), (11008, 512, 64), (5, 1024, 512)])
+def test_unit_saliency(wq, ctx, oracle, R, C, G):
+    W = ws.weights(R, C, 900 + R, "student_t")
+    s = oracle.act_stats(ws.activations(64, C, 901).numpy())
+    want = oracle.unit_saliency(W.numpy(), G, s)
+    got = wq.windq_unit_saliency(ctx, W.cuda(), G, torch.from_numpy(s).cuda()).cpu().numpy()
+    assert (np.abs(got - want) <= 1e-5 * np.abs(want) + 1e-9).all()
+
+
+def test_fallback(wq, ctx, oracle):
+    G, R, C = 128, 200, 2048
+    W = ws.weights(R, C, 910, "student_t")
+    s = oracle.act_stats(ws.activations(64, C, 911).numpy())
+    grid = torch.from_numpy(ws.clip_grid(20)).cuda()
+    fitd = wq.windq_fit_eval(ctx, W.cuda(), G, torch.from_numpy(s).cuda(), grid)
+    err, energy = fitd["err"].cpu().numpy(), fitd["energy"].cpu().numpy()
+    rng = np.random.default_rng(12)
+    acts = rng.integers(0, 7, C // G).astype(np.uint8)
+    for theta in (0.0, 0.01, 0.1, 0.4, np.inf):
+        want, n = oracle.fallback(err, energy, acts, theta)
+        got = wq.windq_fallback(ctx, fitd["err"], fitd["energy"], torch.from_numpy(acts).cuda(), theta)
+        assert (got["actions"].cpu().numpy() == want).all() and int(got["n_changed"].item()) == n
+    with pytest.raises(wq.WindqError):
+        wq.windq_fallback(ctx, fitd["err"], fitd["energy"], torch.from_numpy(acts).cuda(), -1.0)

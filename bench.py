@@ -187,29 +187,46 @@ def make_plans(wq, ctx, spec, n_blocks, G):
 
 class Buffers:
     """Output tensors sized for the largest matrix, reused for every matrix (a consumer would keep
-    what it needs); nothing is allocated inside a step."""
+    what it needs); nothing is allocated inside a step.  Every output that the e2e leg copies to the
+    host exists `ring` times and the calls write them in turn, so that a device-to-host copy on another
+    stream can still be reading one result while the next one is produced."""
 
-    def __init__(self, spec):
+    RINGED = ("feat", "err", "energy", "totals", "codes", "scales", "zeros")
+
+    def __init__(self, spec, ring=1):
         mats = matrices_of(spec)
         Gmin = min(spec.chunk_widths)
         maxU = max(m.C // Gmin for m in mats)
         maxRC = max(m.R * m.C for m in mats)
         maxUR = max((m.C // Gmin) * m.R for m in mats)
-        maxC = max(c for _, c in inputs_of(spec))
         dev = "cuda"
+        self.ring = ring
         self.s = {i: torch.empty(c, dtype=torch.float32, device=dev) for i, c in inputs_of(spec)}
-        self.feat = torch.empty(maxU * 8, dtype=torch.float32, device=dev)
-        self.err = torch.empty(maxU * 6, dtype=torch.float32, device=dev)
-        self.energy = torch.empty(maxU, dtype=torch.float32, device=dev)
         self.clip_idx = torch.empty(4 * maxUR, dtype=torch.uint8, device=dev)
         self.unit_cb = torch.empty(maxU, dtype=torch.int64, device=dev)
         self.offsets = torch.empty(maxU + 1, dtype=torch.int64, device=dev)
-        self.totals = torch.zeros(2 * len(TARGET_BITS), dtype=torch.int64, device=dev)
-        self.codes = torch.empty(2 * maxRC + 16 * maxU, dtype=torch.uint8, device=dev)
-        self.scales = torch.empty(maxUR, dtype=torch.float16, device=dev)
-        self.zeros = torch.empty(maxUR, dtype=torch.float16, device=dev)
         self.wq = torch.empty(maxRC, dtype=torch.float16, device=dev)
-        del maxC
+        shapes = dict(feat=(maxU * 8, torch.float32), err=(maxU * 6, torch.float32), energy=(maxU, torch.float32),
+                      totals=(2 * len(TARGET_BITS), torch.int64), codes=(2 * maxRC + 16 * maxU, torch.uint8),
+                      scales=(maxUR, torch.float16), zeros=(maxUR, torch.float16))
+        self.rings = {k: [torch.zeros(n, dtype=dt, device=dev) for _ in range(ring)] for k, (n, dt) in shapes.items()}
+        self.turn = {k: 0 for k in shapes}
+        self.pending = {}          # (name, slot) -> event of the copy that still reads that slot
+        self.last = {}             # name -> slot handed out last
+
+    def take(self, name):
+        """The tensor the next call writes `name` into; waits (on the current stream) for a copy that still reads it."""
+        slot = self.turn[name] % self.ring
+        self.turn[name] += 1
+        ev = self.pending.pop((name, slot), None)
+        if ev is not None:
+            torch.cuda.current_stream().wait_event(ev)
+        self.last[name] = slot
+        return self.rings[name][slot]
+
+    @property
+    def totals(self):
+        return self.rings["totals"][self.last.get("totals", 0)]
 
 
 class FitTimer:
@@ -244,10 +261,10 @@ def score_block(wq, ctx, spec, Wb, Xb, plans_b, buf, grid_d, timer=None, sink=No
         W, s = Wb[mi], buf.s[m.x_id]
         for G in spec.chunk_widths:
             U = m.C // G
-            feat = buf.feat[:U * 8].view(U, 8)
+            feat = buf.take("feat")[:U * 8].view(U, 8)
             wq.windq_unit_features(ctx, W, G, s, feat)
             launches += 2
-            out = dict(err=buf.err[:U * 6].view(U, 6), energy=buf.energy[:U],
+            out = dict(err=buf.take("err")[:U * 6].view(U, 6), energy=buf.take("energy")[:U],
                        clip_idx=buf.clip_idx[:4 * U * m.R].view(4, U, m.R))
             e0 = timer.start() if timer else None
             wq.windq_fit_eval(ctx, W, G, s, grid_d, out=out)
@@ -259,20 +276,23 @@ def score_block(wq, ctx, spec, Wb, Xb, plans_b, buf, grid_d, timer=None, sink=No
                 sink("err", out["err"])
                 sink("energy", out["energy"])
             if G == APPLY_G and plans_b:
+                totals = buf.take("totals")
                 for ti, target in enumerate(TARGET_BITS):
                     acts = plans_b[target][mi]
                     eb = wq.windq_effective_bits(ctx, acts, m.R, G, out=dict(
                         unit_centibits=buf.unit_cb[:U], code_offsets=buf.offsets[:U + 1],
-                        total_centibits=buf.totals[2 * ti:2 * ti + 1], total_packed_bytes=buf.totals[2 * ti + 1:2 * ti + 2]))
-                    plan = wq.windq_apply_plan(ctx, W, G, s, grid_d, acts, eb["code_offsets"], buf.codes, out["clip_idx"],
-                                               out=dict(scales=buf.scales[:U * m.R].view(U, m.R), zeros=buf.zeros[:U * m.R].view(U, m.R),
+                        total_centibits=totals[2 * ti:2 * ti + 1], total_packed_bytes=totals[2 * ti + 1:2 * ti + 2]))
+                    plan = wq.windq_apply_plan(ctx, W, G, s, grid_d, acts, eb["code_offsets"], buf.take("codes"), out["clip_idx"],
+                                               out=dict(scales=buf.take("scales")[:U * m.R].view(U, m.R),
+                                                        zeros=buf.take("zeros")[:U * m.R].view(U, m.R),
                                                         wq=buf.wq[:m.R * m.C].view(m.R, m.C)))
                     launches += 2
                     if sink:
                         sink("codes", (plan["codes"], acts, m.R, G))
                         sink("scales", plan["scales"])
                         sink("zeros", plan["zeros"])
-                        sink("totals", buf.totals[2 * ti:2 * ti + 2])
+                if sink:
+                    sink("totals", totals)
     return launches
 
 
@@ -325,7 +345,9 @@ def run_e2e_leg(wq, ctx, spec, model, plans, plans_np, buf, grid_d, steps, warmu
                           ready=torch.cuda.Event(), free=torch.cuda.Event()))
     copy_stream = torch.cuda.Stream()
     main = torch.cuda.current_stream()
-    # pinned result buffers (sized for the largest matrix); D2H on the main stream after each call
+    # pinned result buffers (sized for the largest matrix); results leave on a third stream, so that the
+    # kernels of the next matrix do not queue behind the copies of this one
+    out_stream = torch.cuda.Stream()
     host_out = {}
 
     def host_buf(name, n, dtype):
@@ -339,13 +361,18 @@ def run_e2e_leg(wq, ctx, spec, model, plans, plans_np, buf, grid_d, steps, warmu
     def sink(name, t):
         if name == "codes":
             codes, acts, R, G = t
-            n = sink.code_bytes[(id(acts))]
-            host_buf(name, n, torch.uint8).copy_(codes[:n], non_blocking=True)
-            d2h[0] += n
+            src = codes[:sink.code_bytes[(id(acts))]]
         else:
-            flat = t.reshape(-1)
-            host_buf(name, flat.numel(), flat.dtype).copy_(flat, non_blocking=True)
-            d2h[0] += flat.numel() * flat.element_size()
+            src = t.reshape(-1)
+        produced = torch.cuda.Event()
+        produced.record(main)
+        out_stream.wait_event(produced)
+        with torch.cuda.stream(out_stream):
+            host_buf(name, src.numel(), src.dtype).copy_(src, non_blocking=True)
+            copied = torch.cuda.Event()
+            copied.record(out_stream)
+        buf.pending[(name, buf.last[name])] = copied      # the call that writes this slot next waits for the copy
+        d2h[0] += src.numel() * src.element_size()
 
     sink.code_bytes = {}
     for target in plans:
@@ -386,6 +413,7 @@ def run_e2e_leg(wq, ctx, spec, model, plans, plans_np, buf, grid_d, steps, warmu
     t0.record()
     for _ in range(steps):
         step()
+    main.wait_stream(out_stream)      # the step is over when the last result is on the host
     t1.record()
     sync()
     wall = (time.perf_counter() - wall0) * 1e3
@@ -513,6 +541,7 @@ def main():
 
     # plan totals (control path): exact int64 sums over ranks
     total_cb = sharding.sum_int64(int(buf.totals[2 * (len(TARGET_BITS) - 1)].item())) if plans else 0
+    torch.cuda.synchronize()
 
     n_fit = len(spec.chunk_widths) * len(mats) * n_blocks * args.steps
     fit_elem = elems * len(spec.chunk_widths) * args.steps
@@ -535,7 +564,9 @@ def main():
 
     e2e = None
     if not args.no_e2e:
-        e_ms, e_wall, h2d, d2h, host_blocks = run_e2e_leg(wq, ctx, spec, model, plans, plans_np, buf, grid_d,
+        del buf
+        ebuf = Buffers(spec, ring=3)
+        e_ms, e_wall, h2d, d2h, host_blocks = run_e2e_leg(wq, ctx, spec, model, plans, plans_np, ebuf, grid_d,
                                                           max(1, min(args.steps, 2)), args.warmup, sync)
         e_steps = max(1, min(args.steps, 2))
         e_ms = sharding.max_float(max(e_ms, e_wall))

@@ -174,8 +174,11 @@ def effective_bits(actions, R: int, G: int, scale_bits: int = 16, zero_bits: int
                 total_packed_bytes=packed.value)
 
 
-def apply_plan(W, G: int, s, clip_grid, actions, clip_idx=None, want_wq: bool = True):
-    """Returns dict(codes[bytes], scales[U,R] u16, zeros[U,R] u16, wq[R,C] u16, code_offsets)."""
+def apply_plan(W, G: int, s, clip_grid, actions, clip_idx=None, want_wq: bool = True, thresh=None):
+    """Returns dict(codes[bytes], scales[U,R] u16, zeros[U,R] u16, wq[R,C] u16, code_offsets).
+
+    With ``thresh`` (fp32 [U], from salient_select) the salient weights are protected; the result then
+    also holds prot_scale[U] u16, prot_offsets[U+1] i64 and prot_q (int8 codes, row-major per unit)."""
     W, s, clip_grid = _as_u16(W), _f32(s), _f32(clip_grid)
     actions = np.ascontiguousarray(actions, dtype=np.uint8)
     R, C = W.shape
@@ -188,6 +191,20 @@ def apply_plan(W, G: int, s, clip_grid, actions, clip_idx=None, want_wq: bool = 
     if clip_idx is not None:
         clip_idx = np.ascontiguousarray(clip_idx, dtype=np.uint8)
         assert clip_idx.shape == (4, U, R)
+    if thresh is not None:
+        thresh = _f32(thresh)
+        assert thresh.size == U
+        prot_scale = np.zeros(U, np.uint16)
+        prot_offsets = np.zeros(U + 1, np.int64)
+        prot_q = np.zeros(R * C, np.int8)
+        rc = lib().oracle_apply_plan_protected(_p(W), ctypes.c_int64(R), ctypes.c_int64(C), ctypes.c_int64(C), ctypes.c_int(G),
+                                               _p(s), _p(clip_grid), ctypes.c_int(clip_grid.size), _p(actions), _p(clip_idx),
+                                               _p(offs), _p(thresh), _p(codes), _p(scales), _p(zeros), _p(wq),
+                                               _p(prot_scale), _p(prot_offsets), _p(prot_q))
+        if rc:
+            raise ValueError("oracle_apply_plan_protected: bad arguments")
+        return dict(codes=codes, scales=scales, zeros=zeros, wq=wq, code_offsets=offs, prot_scale=prot_scale,
+                    prot_offsets=prot_offsets, prot_q=prot_q[:int(prot_offsets[U])].copy())
     rc = lib().oracle_apply_plan(_p(W), ctypes.c_int64(R), ctypes.c_int64(C), ctypes.c_int64(C), ctypes.c_int(G),
                                  _p(s), _p(clip_grid), ctypes.c_int(clip_grid.size), _p(actions), _p(clip_idx),
                                  _p(offs), _p(codes), _p(scales), _p(zeros), _p(wq))

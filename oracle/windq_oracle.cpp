@@ -534,22 +534,51 @@ int oracle_effective_bits(const uint8_t* actions, int64_t U, int64_t R, int G, i
 // written (padding = 0); scales_out / zeros_out are fp16 [U][R]; Wq_out is
 // fp16 [R][ldw] (nullable).  clip_idx [4][U][R] may be null: the clip search is
 // then repeated for the chosen bit-width.
-int oracle_apply_plan(const uint16_t* W, int64_t R, int64_t C, int64_t ldw, int G, const float* s,
-                      const float* clip_grid, int K, const uint8_t* actions, const uint8_t* clip_idx,
-                      const int64_t* code_offsets, uint8_t* codes_out, uint16_t* scales_out,
-                      uint16_t* zeros_out, uint16_t* Wq_out) {
+// thresh == NULL: the plan applied to every weight.  thresh != NULL: salient-weight protection.
+// READING (the paper says only that protected weights are "stored in INT8"): in every unit that is
+// not skipped, a weight whose key |w| * sqrt(s_j) reaches thresh[u] is protected.  Inside its group it
+// counts as a zero weight with zero activation weight (as in the protected fit), so the group's
+// parameters and the codes of the other weights are those of the masked group, and its own slot in the
+// packed stream holds the code of the value 0 (a reader skips it by the mask).  The protected weights
+// of a unit share one symmetric INT8 grid: scale sigma_u = fp16(max |w| over them / 127) (1 if that is
+// zero), code clamp(rne(w / sigma_u), -127, 127), rounding as in the uniform fit; their fake-quantised
+// value is fp16(code * sigma_u).  The INT8 codes of a unit are listed in row-major order of the unit
+// (rows, then columns) starting at prot_offsets_out[u]; a skipped unit protects nothing.
+static int apply_plan_impl(const uint16_t* W, int64_t R, int64_t C, int64_t ldw, int G, const float* s,
+                           const float* clip_grid, int K, const uint8_t* actions, const uint8_t* clip_idx,
+                           const int64_t* code_offsets, const float* thresh, uint8_t* codes_out, uint16_t* scales_out,
+                           uint16_t* zeros_out, uint16_t* Wq_out, uint16_t* prot_scale_out, int64_t* prot_offsets_out,
+                           int8_t* prot_q_out) {
+  if (thresh && (!prot_scale_out || !prot_offsets_out || !prot_q_out)) return 1;
   if (!W || !s || !clip_grid || !actions || !code_offsets || !codes_out || !scales_out || !zeros_out ||
       R <= 0 || C <= 0 || !valid_group_width(G) || C % G != 0 || ldw < C || K < 1 || K > 64)
     return 1;
   const int64_t U = C / G;
   std::memset(codes_out, 0, (size_t)code_offsets[U]);
-  std::vector<float> w((size_t)G), what((size_t)G);
-  std::vector<uint8_t> q((size_t)G);
+  std::vector<float> w((size_t)G), what((size_t)G), worig((size_t)G), sm((size_t)G);
+  std::vector<uint8_t> q((size_t)G), prot((size_t)G);
+  int64_t n_prot = 0;
   for (int64_t u = 0; u < U; ++u) {
     const int a = actions[u];
     if (a > 6) return 1;
     const float* su = s + u * G;
     const int64_t gb = group_code_bytes(a, G);
+    const bool protect = thresh && a != 0;
+    float sigma = 1.0f, inv8 = 1.0f;
+    if (thresh) {
+      prot_offsets_out[u] = n_prot;
+      float m = 0.0f;
+      if (protect)
+        for (int64_t r = 0; r < R; ++r)
+          for (int j = 0; j < G; ++j) {
+            const float aw = std::fabs(half_to_float(W[r * ldw + u * G + j]));
+            if (aw * std::sqrt(s[u * G + j]) >= thresh[u] && aw > m) m = aw;
+          }
+      sigma = round_through_half(m / 127.0f);
+      if (sigma == 0.0f) sigma = 1.0f;
+      inv8 = 1.0f / sigma;
+      prot_scale_out[u] = protect ? float_to_half(sigma) : (uint16_t)0;
+    }
     for (int64_t r = 0; r < R; ++r) {
       uint8_t* dst = codes_out + code_offsets[u] + r * gb;
       uint16_t scale_h = 0, zero_h = 0;
@@ -558,6 +587,15 @@ int oracle_apply_plan(const uint16_t* W, int64_t R, int64_t C, int64_t ldw, int 
         if (Wq_out) std::memcpy(Wq_out + r * ldw + u * G, W + r * ldw + u * G, (size_t)(2 * G));
       } else {
         load_group(W, ldw, r, u, G, w.data());
+        if (protect) {
+          for (int j = 0; j < G; ++j) {
+            worig[(size_t)j] = w[(size_t)j];
+            prot[(size_t)j] = std::fabs(w[(size_t)j]) * std::sqrt(s[u * G + j]) >= thresh[u];
+            sm[(size_t)j] = prot[(size_t)j] ? 0.0f : s[u * G + j];
+            if (prot[(size_t)j]) w[(size_t)j] = 0.0f;
+          }
+          su = sm.data();
+        }
         Group g{G, w.data(), su};
         if (a <= 4) {
           const int bi = a - 1, bits = kUniformBits[bi];
@@ -586,6 +624,14 @@ int oracle_apply_plan(const uint16_t* W, int64_t R, int64_t C, int64_t ldw, int 
           scale_h = float_to_half(alpha);
         }
         pack_group(a, G, q.data(), dst);
+        if (protect)
+          for (int j = 0; j < G; ++j)
+            if (prot[(size_t)j]) {
+              float c = std::fmaf(worig[(size_t)j], inv8, kMagic) - kMagic;   // rne(w / sigma), one rounding
+              c = std::min(std::max(c, -127.0f), 127.0f);
+              what[(size_t)j] = c * sigma;
+              prot_q_out[n_prot++] = (int8_t)(int)c;
+            }
         if (Wq_out)
           for (int j = 0; j < G; ++j) Wq_out[r * ldw + u * G + j] = float_to_half(what[j]);
       }
@@ -593,7 +639,26 @@ int oracle_apply_plan(const uint16_t* W, int64_t R, int64_t C, int64_t ldw, int 
       zeros_out[u * R + r] = zero_h;
     }
   }
+  if (thresh) prot_offsets_out[U] = n_prot;
   return 0;
+}
+
+int oracle_apply_plan(const uint16_t* W, int64_t R, int64_t C, int64_t ldw, int G, const float* s,
+                      const float* clip_grid, int K, const uint8_t* actions, const uint8_t* clip_idx,
+                      const int64_t* code_offsets, uint8_t* codes_out, uint16_t* scales_out,
+                      uint16_t* zeros_out, uint16_t* Wq_out) {
+  return apply_plan_impl(W, R, C, ldw, G, s, clip_grid, K, actions, clip_idx, code_offsets, nullptr, codes_out,
+                         scales_out, zeros_out, Wq_out, nullptr, nullptr, nullptr);
+}
+
+int oracle_apply_plan_protected(const uint16_t* W, int64_t R, int64_t C, int64_t ldw, int G, const float* s,
+                                const float* clip_grid, int K, const uint8_t* actions, const uint8_t* clip_idx,
+                                const int64_t* code_offsets, const float* thresh, uint8_t* codes_out,
+                                uint16_t* scales_out, uint16_t* zeros_out, uint16_t* Wq_out, uint16_t* prot_scale_out,
+                                int64_t* prot_offsets_out, int8_t* prot_q_out) {
+  if (!thresh) return 1;
+  return apply_plan_impl(W, R, C, ldw, G, s, clip_grid, K, actions, clip_idx, code_offsets, thresh, codes_out,
+                         scales_out, zeros_out, Wq_out, prot_scale_out, prot_offsets_out, prot_q_out);
 }
 
 // ---- salient-weight selection (App. "Salient Weight Protection") -----------------------------

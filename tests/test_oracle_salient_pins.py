@@ -208,3 +208,56 @@ def test_fallback_rule(oracle):
     lo, _ = oracle.fallback(e, en, a, 0.2)
     hi, _ = oracle.fallback(e, en, a, 0.6)
     assert (hi >= lo).all() and (lo <= a).all()
+
+
+# ------------------------------------------------------------------ applying a plan with protected weights
+def test_apply_plan_protected(oracle):
+    R, C, G = 20, 1024, 128
+    rng = np.random.default_rng(13)
+    W = (rng.standard_normal((R, C)) * 0.02).astype(np.float16)          # no planted outlier columns here
+    s = (rng.random(C).astype(np.float32) + 0.2)
+    grid = ws.clip_grid(20)
+    acts = np.array([0, 1, 2, 3, 4, 5, 6, 4], np.uint8)
+    plain = oracle.apply_plan(W, G, s, grid, acts)
+    nothing = oracle.apply_plan(W, G, s, grid, acts, thresh=np.full(C // G, np.inf, np.float32))
+    for k in ("codes", "scales", "zeros", "wq"):
+        assert (plain[k] == nothing[k]).all(), k
+    assert nothing["prot_q"].size == 0 and not nothing["prot_offsets"].any()
+
+    # a hot column in every unit, fully protected (n_p = R weights per unit)
+    W2 = W.copy()
+    hot = [u * G + 17 for u in range(C // G)]
+    vals = np.linspace(0.3, 0.9, R).astype(np.float16) * np.where(np.arange(R) % 2 == 0, 1, -1).astype(np.float16)
+    for c in hot:
+        W2[:, c] = vals
+    sel = oracle.salient_select(W2, G, s, (R * 1_000_000 + R * G - 1) // (R * G))      # n_p = R weights per unit
+    mask = np.unpackbits(sel["mask"], axis=1, bitorder="little").astype(bool)
+    assert all(mask[:, c].all() for c in hot) and mask.sum() == R * (C // G)
+    got = oracle.apply_plan(W2, G, s, grid, acts, thresh=sel["thresh"])
+    # everything but the protected column: the plain plan on the matrix with that column zero and unweighted
+    W3, s3 = W2.copy(), s.copy()
+    for u, c in enumerate(hot):
+        if acts[u] != 0:
+            W3[:, c] = 0
+            s3[c] = 0
+    want = oracle.apply_plan(W3, G, s3, grid, acts)
+    assert (got["codes"] == want["codes"]).all() and (got["scales"] == want["scales"]).all() and (got["zeros"] == want["zeros"]).all()
+    others = np.ones(C, bool)
+    others[hot] = False
+    assert (got["wq"][:, others] == want["wq"][:, others]).all()
+    # the protected column: one INT8 grid per unit, restated in float64
+    offs = got["prot_offsets"]
+    assert offs[0] == 0 and (np.diff(offs) == np.where(acts != 0, R, 0)).all()       # a skipped unit protects nothing
+    for u, c in enumerate(hot):
+        col = W2[:, c].astype(np.float64)
+        if acts[u] == 0:
+            assert (got["wq"][:, c] == W2[:, c].view(np.uint16)).all() and got["prot_scale"][u] == 0
+            continue
+        sigma = np.float64(np.float16(np.float32(np.abs(col).max()) / np.float32(127.0)))
+        assert got["prot_scale"][u] == np.float16(sigma).view(np.uint16)
+        q = np.clip(np.rint(col / sigma), -127, 127)
+        assert (got["prot_q"][offs[u]:offs[u + 1]] == q.astype(np.int8)).all()          # row order
+        assert (got["wq"][:, c] == (q * sigma).astype(np.float16).view(np.uint16)).all()
+        assert (np.abs(q * sigma - col) <= 0.5 * sigma * (1 + 1e-3)).all()
+    # 8-bit round trip of the side grid: the largest protected magnitude is reproduced to within half a step
+    assert np.abs(got["prot_q"]).max() == 127

@@ -213,6 +213,28 @@ windq_status windq_fit_eval_protected(windq_ctx* ctx, const void* W, int64_t R, 
                                       float* err_out, float* energy_out, uint8_t* clip_idx_out, float* group_err_out,
                                       void* stream);
 
+/* windq_apply_plan with salient-weight protection.  In every unit that is not skipped, a weight whose
+ * key reaches thresh[u] is protected: inside its group it counts as a zero weight with zero activation
+ * weight (as in windq_fit_eval_protected, whose clip indices this call takes), so scales, zero points
+ * and the codes of the other weights are those of the masked group, and its own slot in the packed
+ * stream holds the code of the value 0 (a reader skips it by the mask of windq_salient_select).  The
+ * protected weights of a unit share one symmetric INT8 grid (the paper says only "stored in INT8"):
+ *   prot_scale_out   fp16 [U]     sigma_u = fp16(max |w| over the unit's protected weights / 127), 1 if that
+ *                                 is zero; 0 for a skipped unit, which protects nothing
+ *   prot_offsets_out i64  [U+1]   start of every unit's INT8 codes in prot_q_out; [U] = their number
+ *   prot_q_out       i8   [prot_q_capacity]  codes clamp(rne(w / sigma_u), -127, 127), per unit in row-major
+ *                                 order (rows, then columns).  Nothing is written at or beyond prot_q_capacity:
+ *                                 size it from the counts of windq_salient_select, or compare prot_offsets_out[U]
+ *   Wq_out                        fp16(code * sigma_u) at the protected positions
+ * Everything else as windq_apply_plan.  Scratch: windq_scratch_bytes_apply_plan_protected. */
+int64_t windq_scratch_bytes_apply_plan_protected(int64_t R, int64_t C, int G);
+windq_status windq_apply_plan_protected(windq_ctx* ctx, const void* W, int64_t R, int64_t C, int64_t ldw, int G,
+                                        const float* s, const float* clip_grid, int K, const uint8_t* actions,
+                                        const uint8_t* clip_idx, const int64_t* code_offsets, const float* thresh,
+                                        uint8_t* codes_out, void* scales_out, void* zeros_out, void* Wq_out,
+                                        void* prot_scale_out, int64_t* prot_offsets_out, int8_t* prot_q_out,
+                                        int64_t prot_q_capacity, void* stream);
+
 /* Eq. 6 in full, in centibits: 1600 n for a skipped unit (nothing of it is protected), otherwise
  * 100 b (n - n_p) + 800 n_p, plus 100 R (scale_bits [+ zero_bits for 8/4/3/2 bit]) for the groups'
  * parameters as in windq_effective_bits.  n_protected: i64 [U] (device), e.g. count_out above.

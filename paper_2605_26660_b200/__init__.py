@@ -62,6 +62,9 @@ def _load() -> ctypes.CDLL:
     lib.windq_effective_bits.argtypes = [vp, vp, i64, i64, i32, i32, i32, vp, vp, vp, vp, vp]
     lib.windq_salient_select.argtypes = [vp, vp, i64, i64, i64, i32, vp, i64, vp, vp, vp, vp]
     lib.windq_effective_bits_protected.argtypes = [vp, vp, vp, i64, i64, i32, i32, i32, vp, vp, vp]
+    lib.windq_apply_plan_protected.argtypes = [vp, vp, i64, i64, i64, i32, vp, vp, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, i64, vp]
+    lib.windq_scratch_bytes_apply_plan_protected.argtypes = [i64, i64, i32]
+    lib.windq_scratch_bytes_apply_plan_protected.restype = i64
     lib.windq_unit_saliency.argtypes = [vp, vp, i64, i64, i64, i32, vp, vp, vp]
     lib.windq_fallback.argtypes = [vp, vp, vp, vp, i64, ctypes.c_float, vp, vp, vp]
     lib.windq_apply_plan.argtypes = [vp, vp, i64, i64, i64, i32, vp, vp, i32, vp, vp, vp, vp, vp, vp, vp, vp]
@@ -363,3 +366,34 @@ def windq_fallback(ctx: Context, err: torch.Tensor, energy: torch.Tensor, action
     ctx._check(_lib.windq_fallback(ctx._h, _ptr(err), _ptr(energy), _ptr(actions), U, float(theta), _ptr(out), _ptr(n),
                                    _stream(stream)))
     return dict(actions=out, n_changed=n)
+
+
+def windq_apply_plan_protected(ctx: Context, W: torch.Tensor, G: int, s: torch.Tensor, clip_grid: torch.Tensor,
+                               actions: torch.Tensor, code_offsets: torch.Tensor, codes_out: torch.Tensor,
+                               thresh: torch.Tensor, prot_q_out: torch.Tensor, clip_idx: torch.Tensor | None = None, *,
+                               want_wq: bool = True, stream=None) -> dict:
+    """windq_apply_plan with the salient weights (key >= thresh[u]) kept on an INT8 grid per unit.
+    ``prot_q_out`` is an int8 tensor sized by the caller (sum of the counts of windq_salient_select is enough).
+
+    Returns dict(codes, scales, zeros, wq | None, prot_scale [U] f16, prot_offsets [U+1] i64, prot_q)."""
+    R, C, ldw = _matrix(W, "W")
+    for t_, dt, nm in ((s, torch.float32, "s"), (clip_grid, torch.float32, "clip_grid"), (actions, torch.uint8, "actions"),
+                       (code_offsets, torch.int64, "code_offsets"), (codes_out, torch.uint8, "codes_out"),
+                       (thresh, torch.float32, "thresh"), (prot_q_out, torch.int8, "prot_q_out")):
+        _need(t_, dt, nm, 1)
+    if clip_idx is not None:
+        _need(clip_idx, torch.uint8, "clip_idx", 3)
+    U = C // G if G > 0 else 0
+    if actions.numel() != U or code_offsets.numel() != U + 1 or thresh.numel() != U:
+        raise ValueError("actions and thresh must have U entries and code_offsets U + 1")
+    dev = W.device
+    out = dict(codes=codes_out, scales=torch.empty((U, R), dtype=torch.float16, device=dev),
+               zeros=torch.empty((U, R), dtype=torch.float16, device=dev),
+               wq=torch.empty_strided((R, C), (ldw, 1), dtype=torch.float16, device=dev) if want_wq else None,
+               prot_scale=torch.empty(U, dtype=torch.float16, device=dev),
+               prot_offsets=torch.empty(U + 1, dtype=torch.int64, device=dev), prot_q=prot_q_out)
+    ctx._check(_lib.windq_apply_plan_protected(ctx._h, _ptr(W), R, C, ldw, int(G), _ptr(s), _ptr(clip_grid), clip_grid.numel(),
+                                               _ptr(actions), _ptr(clip_idx), _ptr(code_offsets), _ptr(thresh), _ptr(codes_out),
+                                               _ptr(out["scales"]), _ptr(out["zeros"]), _ptr(out["wq"]), _ptr(out["prot_scale"]),
+                                               _ptr(out["prot_offsets"]), _ptr(prot_q_out), prot_q_out.numel(), _stream(stream)))
+    return out

@@ -124,16 +124,53 @@ __device__ __forceinline__ void store_words(uint8_t* dst, const unsigned (&w)[8]
 
 // SEARCH = false: clip indices are supplied.  SEARCH = true: the clip search is repeated for the
 // unit's bit-width (the candidate table follows the warp buffers in shared memory).
-template <int G, bool SEARCH>
+// Zero activation weight for the protected values of a lane (bit e of pm = value e = leaf e / 8, position e % 8).
+__device__ __forceinline__ void mask_stats(Lane32& sv, unsigned int pm) {
+#pragma unroll
+  for (int e = 0; e < 32; ++e)
+    if ((pm >> e) & 1u) sv.set(e >> 3, e & 7, 0.0f);
+}
+
+// What the protected variant needs beside the arguments of the plain one.
+struct ProtectArgs {
+  const float* scale;              // sqrt(s_j), [C]
+  const float* thresh;             // saliency threshold per unit, [U]
+  const unsigned int* row_off;     // [U][R] number of protected weights of the unit in the rows before this one
+  const long long* prot_offsets;   // [U + 1] start of every unit's INT8 codes
+  const __half* prot_scale;        // [U] INT8 scale of the unit's protected weights
+  int8_t* prot_q;                  // INT8 codes
+  long long capacity;              // entries of prot_q; nothing is written at or beyond it
+};
+
+// Saliency mask of a lane's 32 values: bit e is set when |w_e| * scale_e >= tau.
+__device__ __forceinline__ unsigned int protect_mask(const uint4 (&raw)[4], const float* __restrict__ scale, float tau) {
+  const unsigned int* r = reinterpret_cast<const unsigned int*>(raw);
+  const float4* a4 = reinterpret_cast<const float4*>(scale);
+  unsigned int pm = 0;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const float4 a = __ldg(a4 + i);
+    const float2 w0 = __half22float2(bits_h2(r[2 * i])), w1 = __half22float2(bits_h2(r[2 * i + 1]));
+    pm |= (__fmul_rn(fabsf(w0.x), a.x) >= tau ? 1u : 0u) << (4 * i);
+    pm |= (__fmul_rn(fabsf(w0.y), a.y) >= tau ? 1u : 0u) << (4 * i + 1);
+    pm |= (__fmul_rn(fabsf(w1.x), a.z) >= tau ? 1u : 0u) << (4 * i + 2);
+    pm |= (__fmul_rn(fabsf(w1.y), a.w) >= tau ? 1u : 0u) << (4 * i + 3);
+  }
+  return pm;
+}
+
 #ifndef WINDQ_APPLY_MIN_BLOCKS
 #define WINDQ_APPLY_MIN_BLOCKS 4
 #endif
+// PROTECT = true: salient weights (see ProtectArgs) are taken out of the group fits -- zero weight,
+// zero activation weight, as in the protected fit -- and kept on one symmetric INT8 grid per unit.
+template <int G, bool SEARCH, bool PROTECT>
 __global__ void __launch_bounds__(kApplyWarps * 32, WINDQ_APPLY_MIN_BLOCKS)
 apply_plan_kernel(const __half* __restrict__ W, int R, int U, int64_t ldw, const float* __restrict__ s,
                   const float* __restrict__ clip, int K, const uint8_t* __restrict__ actions,
                   const uint8_t* __restrict__ clip_idx, const long long* __restrict__ code_offsets,
                   uint8_t* __restrict__ codes_out, __half* __restrict__ scales_out, __half* __restrict__ zeros_out,
-                  __half* __restrict__ Wq_out, int rows_blocks) {
+                  __half* __restrict__ Wq_out, int rows_blocks, ProtectArgs pa) {
   constexpr int LG = Map<G>::LG, GPW = Map<G>::GPW;
   extern __shared__ uint4 smem_u4[];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -209,6 +246,17 @@ apply_plan_kernel(const __half* __restrict__ W, int R, int U, int64_t ldw, const
       continue;
     }
 
+    unsigned int pm = 0;  // protected values of this lane
+    uint4 raw_all[4];     // the lane's values before masking (PROTECT only)
+    if (PROTECT) {
+#pragma unroll
+      for (int i = 0; i < 4; ++i) raw_all[i] = raw[i];
+      pm = protect_mask(raw, pa.scale + (int64_t)u * G + 32 * q, __ldg(pa.thresh + u));
+      unsigned int* r = reinterpret_cast<unsigned int*>(raw);
+#pragma unroll
+      for (int i = 0; i < 16; ++i)
+        r[i] &= ~(((pm >> (2 * i)) & 1u ? 0x0000ffffu : 0u) | ((pm >> (2 * i + 1)) & 1u ? 0xffff0000u : 0u));
+    }
     unsigned wq[16], code[16];  // two fp16 weights / two codes per register
     float scale_store, zero_store = 0.0f;
     if (a <= 4) {
@@ -223,6 +271,7 @@ apply_plan_kernel(const __half* __restrict__ W, int R, int U, int64_t ldw, const
         Lane32 wv, sv;
         unpack_weights(raw, wv);
         load_stats(s + (int64_t)u * G + 32 * q, sv);
+        if (PROTECT) mask_stats(sv, pm);
         group_range<G>(wv, mn, mx);
         float be;
         search_uniform<G>(wv, sv, mn, __fsub_rn(mx, mn), bi, clip, K, cand, chunk, stride, lane, be, k);
@@ -236,6 +285,7 @@ apply_plan_kernel(const __half* __restrict__ W, int R, int U, int64_t ldw, const
       Lane32 wv, sv;
       unpack_weights(raw, wv);
       load_stats(s + (int64_t)u * G + 32 * q, sv);
+      if (PROTECT) mask_stats(sv, pm);
       float delta = 0.0f;
       const float alpha = (a == 5) ? ternary_scale<G>(wv, sv, delta) : binary_scale<G>(wv, sv);
       const unsigned alpha2 = h2_bits(__float2half2_rn(alpha));
@@ -262,6 +312,35 @@ apply_plan_kernel(const __half* __restrict__ W, int R, int U, int64_t ldw, const
       scale_store = alpha;
     }
 
+    if (PROTECT) {
+      // place of this lane's INT8 codes: the unit's list, then the rows before, then the lanes before
+      const int cnt = __popc(pm);
+      int before = cnt;
+#pragma unroll
+      for (int m = 1; m < LG; m <<= 1) {
+        const int o = __shfl_up_sync(0xffffffffu, before, m);
+        if (q >= m) before += o;
+      }
+      before -= cnt;
+      if (live && pm) {
+        const float sigma = __half2float(pa.prot_scale[u]);
+        const float inv8 = __frcp_rn(sigma);
+        const long long base = pa.prot_offsets[u] + pa.row_off[(int64_t)u * R + row] + before;
+        const unsigned int* ro = reinterpret_cast<const unsigned int*>(raw_all);
+        int rank = 0;
+#pragma unroll
+        for (int e = 0; e < 32; ++e)
+          if ((pm >> e) & 1u) {
+            const float2 w2 = __half22float2(bits_h2(ro[e >> 1]));
+            const float w = (e & 1) ? w2.y : w2.x;
+            const float c = fminf(fmaxf(__fadd_rn(__fmaf_rn(w, inv8, kMagic), -kMagic), -127.0f), 127.0f);
+            const unsigned int h = __half_as_ushort(__float2half_rn(__fmul_rn(c, sigma)));
+            wq[e >> 1] = (e & 1) ? ((wq[e >> 1] & 0x0000ffffu) | (h << 16)) : ((wq[e >> 1] & 0xffff0000u) | h);
+            if (base + rank < pa.capacity) pa.prot_q[base + rank] = (int8_t)(int)c;
+            ++rank;
+          }
+      }
+    }
     if (live) {
       if (wq_dst) {
         uint4* dst = reinterpret_cast<uint4*>(wq_dst);
@@ -305,15 +384,17 @@ apply_plan_kernel(const __half* __restrict__ W, int R, int U, int64_t ldw, const
   }
 }
 
-template <int G, bool SEARCH>
+template <int G, bool SEARCH, bool PROTECT>
 windq_status launch_apply(windq_ctx* ctx, const __half* W, int R, int U, int64_t ldw, const float* s, const float* clip,
                           int K, const uint8_t* actions, const uint8_t* clip_idx, const long long* code_offsets,
-                          uint8_t* codes_out, __half* scales_out, __half* zeros_out, __half* Wq_out, cudaStream_t st) {
+                          uint8_t* codes_out, __half* scales_out, __half* zeros_out, __half* Wq_out, const ProtectArgs& pa,
+                          cudaStream_t st) {
   constexpr int GPW = Map<G>::GPW;
   const int stride = apply_cand_chunk<G>() | 1;
   const size_t smem = (size_t)kApplyWarps * kApplyWarpBytes + (SEARCH ? (size_t)kApplyWarps * GPW * stride * sizeof(Cand) : 0);
-  const int id = (SEARCH ? kApplySearchG32 : kApplyG32) + g_index(G);
-  if (windq_status rc = prepare_kernel(ctx, id, apply_plan_kernel<G, SEARCH>, kApplyWarps * 32, smem, true)) return rc;
+  const int id = (PROTECT ? (SEARCH ? kApplyProtectSearchG32 : kApplyProtectG32) : (SEARCH ? kApplySearchG32 : kApplyG32)) +
+                 g_index(G);
+  if (windq_status rc = prepare_kernel(ctx, id, apply_plan_kernel<G, SEARCH, PROTECT>, kApplyWarps * 32, smem, true)) return rc;
   const int blocks_per_sm = ctx->occupancy[id];
   const int rows_blocks = (R + GPW - 1) / GPW;
   const int64_t n_items = (int64_t)U * rows_blocks;
@@ -321,11 +402,106 @@ windq_status launch_apply(windq_ctx* ctx, const __half* W, int R, int U, int64_t
   int64_t grid = (int64_t)ctx->sm_count * blocks_per_sm;
   const int64_t need = (n_items + kApplyWarps - 1) / kApplyWarps;
   if (grid > need) grid = need;
-  apply_plan_kernel<G, SEARCH><<<(unsigned)grid, kApplyWarps * 32, smem, st>>>(W, R, U, ldw, s, clip, K, actions, clip_idx,
-                                                                               code_offsets, codes_out, scales_out,
-                                                                               zeros_out, Wq_out, rows_blocks);
+  apply_plan_kernel<G, SEARCH, PROTECT><<<(unsigned)grid, kApplyWarps * 32, smem, st>>>(
+      W, R, U, ldw, s, clip, K, actions, clip_idx, code_offsets, codes_out, scales_out, zeros_out, Wq_out, rows_blocks, pa);
   WINDQ_CUDA(ctx, cudaGetLastError());
   return WINDQ_OK;
+}
+
+// ---- protected variant: what has to be known before the plan can be applied -----------------------
+__global__ void apply_scale_kernel(const float* __restrict__ s, int C, float* __restrict__ scale) {
+  const int j = blockIdx.x * blockDim.x + threadIdx.x;
+  if (j < C) scale[j] = __fsqrt_rn(s[j]);
+}
+
+// Per (unit, row): the number of protected weights; per unit: the largest protected magnitude.
+// One warp per item (unit, GPW rows), as in the plan kernel.
+template <int G>
+__global__ void __launch_bounds__(kApplyWarps * 32)
+protect_count_kernel(const __half* __restrict__ W, int R, int U, int64_t ldw, const uint8_t* __restrict__ actions,
+                     const float* __restrict__ scale, const float* __restrict__ thresh, int rows_blocks,
+                     unsigned int* __restrict__ row_cnt, unsigned int* __restrict__ unit_max_bits) {
+  constexpr int LG = Map<G>::LG, GPW = Map<G>::GPW;
+  const int lane = threadIdx.x & 31;
+  const int g = lane / LG, q = lane % LG;
+  const int n_items = U * rows_blocks;
+  const int n_warps = gridDim.x * kApplyWarps;
+  for (int item = blockIdx.x * kApplyWarps + (threadIdx.x >> 5); item < n_items; item += n_warps) {
+    const int u = item / rows_blocks, rb = item - u * rows_blocks;
+    const int row = rb * GPW + g;
+    unsigned int cnt = 0, mx = 0;
+    if (actions[u] != 0 && actions[u] <= 6 && row < R) {
+      uint4 raw[4];
+      const uint4* src = reinterpret_cast<const uint4*>(W + (int64_t)row * ldw + (int64_t)u * G + 32 * q);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) raw[i] = __ldg(src + i);
+      const unsigned int pm = protect_mask(raw, scale + (int64_t)u * G + 32 * q, __ldg(thresh + u));
+      cnt = __popc(pm);
+      const unsigned int* r = reinterpret_cast<const unsigned int*>(raw);
+#pragma unroll
+      for (int e = 0; e < 32; ++e)
+        if ((pm >> e) & 1u) mx = max(mx, ((e & 1) ? (r[e >> 1] >> 16) : r[e >> 1]) & 0x7fffu);  // |fp16| bits order like values
+    }
+#pragma unroll
+    for (int m = 1; m < LG; m <<= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, m);
+#pragma unroll
+    for (int m = 16; m > 0; m >>= 1) mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, m));
+    if (q == 0 && row < R) row_cnt[(int64_t)u * R + row] = cnt;
+    if (lane == 0 && mx) atomicMax(&unit_max_bits[u], mx);
+  }
+}
+
+// One block per unit: row counts -> exclusive offsets inside the unit (in place), unit total.
+__global__ void __launch_bounds__(1024)
+protect_row_scan_kernel(unsigned int* __restrict__ row_cnt, int R, unsigned int* __restrict__ unit_total) {
+  __shared__ unsigned int warp_sum[32];
+  __shared__ unsigned int carry_s;
+  const int u = blockIdx.x, t = threadIdx.x, lane = t & 31, wp = t >> 5;
+  unsigned int* c = row_cnt + (int64_t)u * R;
+  if (t == 0) carry_s = 0;
+  __syncthreads();
+  for (int base = 0; base < R; base += 1024) {
+    const int r = base + t;
+    const unsigned int v = r < R ? c[r] : 0u;
+    unsigned int incl = v;
+#pragma unroll
+    for (int m = 1; m < 32; m <<= 1) {
+      const unsigned int o = __shfl_up_sync(0xffffffffu, incl, m);
+      if (lane >= m) incl += o;
+    }
+    if (lane == 31) warp_sum[wp] = incl;
+    __syncthreads();
+    unsigned int before = carry_s;
+    for (int i = 0; i < wp; ++i) before += warp_sum[i];
+    if (r < R) c[r] = before + incl - v;
+    __syncthreads();
+    if (t == 1023) carry_s = before + incl;
+    __syncthreads();
+  }
+  if (t == 0) unit_total[u] = carry_s;
+}
+
+// Unit totals -> start of every unit's list; largest protected magnitude -> the unit's INT8 scale.
+__global__ void protect_unit_scan_kernel(const unsigned int* __restrict__ unit_total, const unsigned int* __restrict__ unit_max_bits,
+                                         const uint8_t* __restrict__ actions, int U, long long* __restrict__ prot_offsets,
+                                         __half* __restrict__ prot_scale) {
+  if (threadIdx.x == 0 && blockIdx.x == 0) {
+    long long run = 0;
+    for (int u = 0; u < U; ++u) {
+      prot_offsets[u] = run;
+      run += unit_total[u];
+    }
+    prot_offsets[U] = run;
+  }
+  for (int u = blockIdx.x * blockDim.x + threadIdx.x; u < U; u += gridDim.x * blockDim.x) {
+    float sigma = 0.0f;
+    if (actions[u] != 0 && actions[u] <= 6) {
+      const float m = __half2float(__ushort_as_half((unsigned short)unit_max_bits[u]));
+      sigma = __half2float(__float2half_rn(__fdiv_rn(m, 127.0f)));
+      if (sigma == 0.0f) sigma = 1.0f;
+    }
+    prot_scale[u] = __float2half_rn(sigma);
+  }
 }
 
 template <int G>
@@ -333,11 +509,47 @@ windq_status launch_apply_any(windq_ctx* ctx, const __half* W, int R, int U, int
                               const float* clip, int K, const uint8_t* actions, const uint8_t* clip_idx,
                               const long long* code_offsets, uint8_t* codes_out, __half* scales_out, __half* zeros_out,
                               __half* Wq_out, cudaStream_t st) {
+  const ProtectArgs none = {};
   if (clip_idx)
-    return launch_apply<G, false>(ctx, W, R, U, ldw, s, clip, K, actions, clip_idx, code_offsets, codes_out, scales_out,
-                                  zeros_out, Wq_out, st);
-  return launch_apply<G, true>(ctx, W, R, U, ldw, s, clip, K, actions, clip_idx, code_offsets, codes_out, scales_out,
-                               zeros_out, Wq_out, st);
+    return launch_apply<G, false, false>(ctx, W, R, U, ldw, s, clip, K, actions, clip_idx, code_offsets, codes_out,
+                                         scales_out, zeros_out, Wq_out, none, st);
+  return launch_apply<G, true, false>(ctx, W, R, U, ldw, s, clip, K, actions, clip_idx, code_offsets, codes_out, scales_out,
+                                      zeros_out, Wq_out, none, st);
+}
+
+template <int G>
+windq_status launch_apply_protected(windq_ctx* ctx, const __half* W, int R, int U, int64_t ldw, const float* s,
+                                    const float* clip, int K, const uint8_t* actions, const uint8_t* clip_idx,
+                                    const long long* code_offsets, const float* thresh, uint8_t* codes_out,
+                                    __half* scales_out, __half* zeros_out, __half* Wq_out, __half* prot_scale_out,
+                                    long long* prot_offsets_out, int8_t* prot_q_out, long long capacity, cudaStream_t st) {
+  constexpr int GPW = Map<G>::GPW;
+  const int C = U * G;
+  // scratch: sqrt(s) [C] | row counts / offsets [U][R] | unit totals [U] | unit maxima [U]
+  float* scale = (float*)ctx->scratch;
+  unsigned int* row_cnt = (unsigned int*)((char*)ctx->scratch + round_up((int64_t)C * 4, 16));
+  unsigned int* unit_total = row_cnt + (int64_t)U * R;
+  unsigned int* unit_max = unit_total + U;
+  const int rows_blocks = (R + GPW - 1) / GPW;
+  const int64_t n_items = (int64_t)U * rows_blocks;
+  WINDQ_REQUIRE(ctx, n_items < (1ll << 30), WINDQ_ERR_SHAPE, "windq_apply_plan_protected: R * C is too large for one call");
+  int64_t grid = (int64_t)ctx->sm_count * 8;
+  const int64_t need = (n_items + kApplyWarps - 1) / kApplyWarps;
+  if (grid > need) grid = need;
+  WINDQ_CUDA(ctx, cudaMemsetAsync(unit_max, 0, (size_t)U * sizeof(unsigned int), st));
+  apply_scale_kernel<<<(unsigned)((C + 255) / 256), 256, 0, st>>>(s, C, scale);
+  protect_count_kernel<G><<<(unsigned)grid, kApplyWarps * 32, 0, st>>>(W, R, U, ldw, actions, scale, thresh, rows_blocks, row_cnt,
+                                                                      unit_max);
+  protect_row_scan_kernel<<<(unsigned)U, 1024, 0, st>>>(row_cnt, R, unit_total);
+  protect_unit_scan_kernel<<<(unsigned)((U + 255) / 256), 256, 0, st>>>(unit_total, unit_max, actions, U, prot_offsets_out,
+                                                                       prot_scale_out);
+  WINDQ_CUDA(ctx, cudaGetLastError());
+  const ProtectArgs pa = {scale, thresh, row_cnt, prot_offsets_out, prot_scale_out, prot_q_out, capacity};
+  if (clip_idx)
+    return launch_apply<G, false, true>(ctx, W, R, U, ldw, s, clip, K, actions, clip_idx, code_offsets, codes_out, scales_out,
+                                        zeros_out, Wq_out, pa, st);
+  return launch_apply<G, true, true>(ctx, W, R, U, ldw, s, clip, K, actions, clip_idx, code_offsets, codes_out, scales_out,
+                                     zeros_out, Wq_out, pa, st);
 }
 
 }  // namespace windq
@@ -371,4 +583,55 @@ extern "C" windq_status windq_apply_plan(windq_ctx* ctx, const void* W, int64_t 
     case 256: return launch_apply_any<256>(ctx, Wh, (int)R, U, ldw, s, clip_grid, K, actions, clip_idx, offs, codes_out, sc, zp, wq, st);
     default: return launch_apply_any<512>(ctx, Wh, (int)R, U, ldw, s, clip_grid, K, actions, clip_idx, offs, codes_out, sc, zp, wq, st);
   }
+}
+
+extern "C" int64_t windq_scratch_bytes_apply_plan_protected(int64_t R, int64_t C, int G) {
+  if (!windq::valid_G(G) || R <= 0 || C <= 0) return 0;
+  const int64_t U = C / G;
+  return windq::round_up(C * 4, 16) + (U * R + 2 * U) * (int64_t)sizeof(unsigned int);
+}
+
+extern "C" windq_status windq_apply_plan_protected(windq_ctx* ctx, const void* W, int64_t R, int64_t C, int64_t ldw, int G,
+                                                   const float* s, const float* clip_grid, int K, const uint8_t* actions,
+                                                   const uint8_t* clip_idx, const int64_t* code_offsets, const float* thresh,
+                                                   uint8_t* codes_out, void* scales_out, void* zeros_out, void* Wq_out,
+                                                   void* prot_scale_out, int64_t* prot_offsets_out, int8_t* prot_q_out,
+                                                   int64_t prot_q_capacity, void* stream) {
+  using namespace windq;
+  const char* who = "windq_apply_plan_protected";
+  if (!ctx) return fail(nullptr, WINDQ_ERR_NULL, "%s: ctx is NULL", who);
+  if (windq_status st = check_matrix(ctx, who, W, R, C, ldw, G)) return st;
+  if (windq_status st = check_K(ctx, who, K)) return st;
+  WINDQ_REQUIRE(ctx, s && clip_grid && actions && code_offsets && codes_out && scales_out && zeros_out && thresh &&
+                         prot_scale_out && prot_offsets_out && (prot_q_out || prot_q_capacity == 0),
+                WINDQ_ERR_NULL, "%s: a required pointer is NULL", who);
+  WINDQ_REQUIRE(ctx, prot_q_capacity >= 0, WINDQ_ERR_ARG, "%s: prot_q_capacity = %lld", who, (long long)prot_q_capacity);
+  WINDQ_REQUIRE(ctx, aligned16(s) && aligned16(codes_out), WINDQ_ERR_ALIGN, "%s: s or codes_out is not 16-byte aligned", who);
+  WINDQ_REQUIRE(ctx, ((uintptr_t)code_offsets & 7) == 0 && ((uintptr_t)prot_offsets_out & 7) == 0 && ((uintptr_t)scales_out & 1) == 0 &&
+                         ((uintptr_t)zeros_out & 1) == 0 && ((uintptr_t)prot_scale_out & 1) == 0,
+                WINDQ_ERR_ALIGN, "%s: an output array is misaligned", who);
+  WINDQ_REQUIRE(ctx, Wq_out == nullptr || aligned16(Wq_out), WINDQ_ERR_ALIGN, "%s: Wq_out is not 16-byte aligned", who);
+  WINDQ_REQUIRE(ctx, Wq_out != W, WINDQ_ERR_ARG, "%s: Wq_out must not alias W", who);
+  WINDQ_REQUIRE(ctx, R * (int64_t)G < (1ll << 32), WINDQ_ERR_SHAPE, "%s: R * G must be below 2^32", who);
+  DeviceGuard guard(ctx->device);
+  if (windq_status rc = ensure_scratch(ctx, windq_scratch_bytes_apply_plan_protected(R, C, G))) return rc;
+  const int U = (int)(C / G);
+  cudaStream_t st = (cudaStream_t)stream;
+  const __half* Wh = (const __half*)W;
+  const long long* offs = (const long long*)code_offsets;
+  __half *sc = (__half*)scales_out, *zp = (__half*)zeros_out, *wq = (__half*)Wq_out, *ps = (__half*)prot_scale_out;
+  long long* po = (long long*)prot_offsets_out;
+#define WINDQ_APPLY_CASE(GG)                                                                                             \
+  case GG:                                                                                                               \
+    return launch_apply_protected<GG>(ctx, Wh, (int)R, U, ldw, s, clip_grid, K, actions, clip_idx, offs, thresh, codes_out, \
+                                      sc, zp, wq, ps, po, prot_q_out, (long long)prot_q_capacity, st);
+  switch (G) {
+    WINDQ_APPLY_CASE(32)
+    WINDQ_APPLY_CASE(64)
+    WINDQ_APPLY_CASE(128)
+    WINDQ_APPLY_CASE(256)
+    default:
+      WINDQ_APPLY_CASE(512)
+  }
+#undef WINDQ_APPLY_CASE
 }

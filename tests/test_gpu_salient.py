@@ -178,3 +178,64 @@ def test_fallback(wq, ctx, oracle):
         assert (got["actions"].cpu().numpy() == want).all() and int(got["n_changed"].item()) == n
     with pytest.raises(wq.WindqError):
         wq.windq_fallback(ctx, fitd["err"], fitd["energy"], torch.from_numpy(acts).cuda(), -1.0)
+
+
+# ------------------------------------------------------------------ applying a plan with protected weights
+def u16(t):
+    return t.cpu().view(torch.int16).numpy().view(np.uint16)
+
+
+@pytest.mark.parametrize("G,R,rate", [(128, 70, 30000), (64, 133, 30000), (32, 200, 50000), (256, 19, 20000), (512, 67, 30000),
+                                      (128, 3, 100000)])
+def test_apply_plan_protected(wq, ctx, oracle, G, R, rate):
+    C = 8 * G
+    W = ws.weights(R, C, 1000 + G + R, "student_t")
+    s = oracle.act_stats(ws.activations(64, C, 1001).numpy())
+    grid = ws.clip_grid(20)
+    acts = np.array([0, 1, 2, 3, 4, 5, 6, 5], np.uint8)
+    sel = oracle.salient_select(W.numpy(), G, s, rate)
+    fitp = oracle.fit_eval(W.numpy(), G, s, grid, threads=8, want_group_err=False, thresh=sel["thresh"])
+    want = oracle.apply_plan(W.numpy(), G, s, grid, acts, fitp["clip_idx"], thresh=sel["thresh"])
+    Wd, s_d, grid_d, a_d = W.cuda(), torch.from_numpy(s).cuda(), torch.from_numpy(grid).cuda(), torch.from_numpy(acts).cuda()
+    th_d = torch.from_numpy(sel["thresh"]).cuda()
+    eb = wq.windq_effective_bits(ctx, a_d, R, G)
+    n_codes = int(eb["code_offsets"][-1].item())
+    cap = int(sel["count"].sum())
+    for clip_idx in (torch.from_numpy(fitp["clip_idx"]).cuda(), None):
+        codes = torch.full((n_codes,), 0xAB, dtype=torch.uint8, device="cuda")
+        prot_q = torch.full((cap + 64,), 99, dtype=torch.int8, device="cuda")
+        got = wq.windq_apply_plan_protected(ctx, Wd, G, s_d, grid_d, a_d, eb["code_offsets"], codes, th_d, prot_q, clip_idx)
+        torch.cuda.synchronize()
+        assert (codes.cpu().numpy() == want["codes"]).all()
+        assert (u16(got["scales"]) == want["scales"]).all() and (u16(got["zeros"]) == want["zeros"]).all()
+        assert (u16(got["wq"]) == want["wq"]).all()
+        assert (u16(got["prot_scale"]) == want["prot_scale"]).all()
+        assert (got["prot_offsets"].cpu().numpy() == want["prot_offsets"]).all()
+        n = int(want["prot_offsets"][-1])
+        assert (prot_q[:n].cpu().numpy() == want["prot_q"]).all() and bool((prot_q[n:] == 99).all())
+    # too small a list: nothing beyond its end is touched, and the offsets still tell how many there are
+    small = torch.full((max(n // 2, 1) + 32,), 99, dtype=torch.int8, device="cuda")
+    got = wq.windq_apply_plan_protected(ctx, Wd, G, s_d, grid_d, a_d, eb["code_offsets"], codes, th_d, small[:max(n // 2, 1)])
+    torch.cuda.synchronize()
+    assert int(got["prot_offsets"][-1].item()) == n and bool((small[max(n // 2, 1):] == 99).all())
+
+
+def test_apply_plan_protected_without_protection_is_the_plain_plan(wq, ctx):
+    G, R, C = 128, 96, 1024
+    W = ws.weights(R, C, 1100, "student_t").cuda()
+    s = torch.rand(C, device="cuda") + 0.1
+    grid = torch.from_numpy(ws.clip_grid(20)).cuda()
+    acts = torch.tensor([4, 3, 5, 6, 1, 2, 0, 4], dtype=torch.uint8, device="cuda")
+    fitd = wq.windq_fit_eval(ctx, W, G, s, grid)
+    eb = wq.windq_effective_bits(ctx, acts, R, G)
+    n_codes = int(eb["code_offsets"][-1].item())
+    c1 = torch.empty(n_codes, dtype=torch.uint8, device="cuda")
+    c2 = torch.empty(n_codes, dtype=torch.uint8, device="cuda")
+    plain = wq.windq_apply_plan(ctx, W, G, s, grid, acts, eb["code_offsets"], c1, fitd["clip_idx"])
+    inf = torch.full((C // G,), float("inf"), device="cuda")
+    prot = wq.windq_apply_plan_protected(ctx, W, G, s, grid, acts, eb["code_offsets"], c2, inf,
+                                         torch.empty(16, dtype=torch.int8, device="cuda"), fitd["clip_idx"])
+    assert torch.equal(c1, c2)
+    for k in ("scales", "zeros", "wq"):
+        assert torch.equal(plain[k].view(torch.int16), prot[k].view(torch.int16))
+    assert int(prot["prot_offsets"][-1].item()) == 0

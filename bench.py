@@ -39,7 +39,7 @@ METRIC = "unit_x_bitwidth_candidate_evals_per_s"
 UNIT = "evals/s"
 TARGET_BITS = (1.58, 2.0, 3.0)
 APPLY_G = 128                    # chunk width the plans are applied at (the first of the workload's widths if it has no 128)
-FIT_TRAFFIC_PER_WEIGHT_BYTE = 34.82 / 33.554   # measured DRAM bytes per algorithmic byte (see profiles/)
+FIT_TRAFFIC_PER_WEIGHT_BYTE = 33.607 / 33.554   # measured DRAM bytes per algorithmic byte (see profiles/)
 SEED = 0
 
 
@@ -552,7 +552,7 @@ def main():
     hbm_time = 2.0 * fit_elem / (peaks["hbm_gbs"] * 1e9)
     alu_time = fit_elem * ops / (alu_peak * 1e12)
     # DRAM traffic of fit_eval_kernel per launch: dram__bytes_read + dram__bytes_write of one ncu capture on the
-    # 4096 x 4096 matrix (profiles/fit_eval_kernel_4096x4096_K20.txt: 34.82 MB against 33.55 MB of weights), scaled
+    # 4096 x 4096 matrix (profiles/fit_eval_kernel_4096x4096_K20.txt: 33.61 MB against 33.55 MB of weights), scaled
     # to this run's average launch by the weights a launch reads (traffic is proportional to them: one pass, no re-reads)
     traffic = FIT_TRAFFIC_PER_WEIGHT_BYTE * 2.0 * fit_elem / n_fit
     roofline = dict(bound="alu" if alu_time >= hbm_time else "hbm", kernel="fit_eval_kernel", achieved=achieved, peak=alu_peak,

@@ -7,8 +7,8 @@
 // loop at its minimum instruction count (see fit_device.cuh).
 //
 // Work is split into items = (unit, block of GPW consecutive rows), one warp per item, no
-// block-level synchronisation.  The grid is persistent: every warp takes a contiguous range of
-// items, so that it mostly stays within one unit and the unit's statistics stay in registers.
+// block-level synchronisation.  The grid is persistent (one block of 16 warps per SM) and the warps
+// claim items from a counter in scratch, in order.
 // Per item the warp writes seven partial sums (six errors and the energy, added over its rows in
 // double) to scratch; a second small kernel adds them per unit in a fixed order, so unit totals
 // are reproducible from run to run.
@@ -35,20 +35,25 @@ __global__ void __launch_bounds__(kFitWarpsPerBlock * 32, 1)
 fit_eval_kernel(const __half* __restrict__ W, int R, int U, int64_t ldw, const float* __restrict__ s,
                 const float* __restrict__ clip, int K, double* __restrict__ partial, uint8_t* __restrict__ clip_idx_out,
                 float* __restrict__ group_err_out, int rows_blocks, int chunk, int stride,
-                const float* __restrict__ scale, const float* __restrict__ thresh, float never) {
+                const float* __restrict__ scale, const float* __restrict__ thresh, float never,
+                unsigned int* __restrict__ next_item) {
   constexpr int LG = Map<G>::LG, GPW = Map<G>::GPW;
   extern __shared__ float4 smem_f4[];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   Cand* cand = reinterpret_cast<Cand*>(smem_f4) + (size_t)warp * GPW * stride;
   const int g = lane / LG, q = lane % LG;
 
-  const int64_t n_items = (int64_t)U * rows_blocks;
-  const int64_t n_warps = (int64_t)gridDim.x * kFitWarpsPerBlock;
-  const int64_t wid = (int64_t)blockIdx.x * kFitWarpsPerBlock + warp;
-  const int64_t item_begin = wid * n_items / n_warps, item_end = (wid + 1) * n_items / n_warps;
+  const unsigned int n_items = (unsigned int)(U * rows_blocks);
 
   Lane32 sv;
-  for (int64_t item = item_begin; item < item_end; ++item) {
+  for (;;) {
+    // items are claimed from a counter, in order: with equal static shares the warps of an SM do not
+    // finish together (the schedulers are not fair), and the SM ends the kernel on a few warps that
+    // cannot fill its issue slots; an item is about 100,000 cycles of work against one atomic
+    unsigned int item = 0;
+    if (lane == 0) item = atomicAdd(next_item, 1u);
+    item = __shfl_sync(0xffffffffu, item, 0);
+    if (item >= n_items) break;
     const int u = (int)(item / rows_blocks), rb = (int)(item % rows_blocks);
     load_stats(s + (int64_t)u * G + 32 * q, sv);
     const int row = rb * GPW + g;
@@ -110,7 +115,7 @@ fit_eval_kernel(const __half* __restrict__ W, int R, int U, int64_t ldw, const f
       double d = live ? (double)e[c] : 0.0;
 #pragma unroll
       for (int m = LG; m < 32; m <<= 1) d += __shfl_xor_sync(0xffffffffu, d, m);
-      if (lane == 0) partial[item * kFitPartials + c] = d;
+      if (lane == 0) partial[(int64_t)item * kFitPartials + c] = d;
     }
   }
 }
@@ -149,7 +154,7 @@ template <int G, bool PROTECT>
 windq_status launch_fit(windq_ctx* ctx, const __half* W, int R, int U, int64_t ldw, const float* s,
                         const float* clip, int K, double* partial, float* err_out, float* energy_out,
                         uint8_t* clip_idx_out, float* group_err_out, float* scale, const float* thresh,
-                        cudaStream_t st) {
+                        unsigned int* next_item, cudaStream_t st) {
   constexpr int GPW = Map<G>::GPW;
   const int rows_blocks = (R + GPW - 1) / GPW;
   const int chunk = fit_cand_chunk(G), stride = fit_cand_stride(chunk);
@@ -161,10 +166,12 @@ windq_status launch_fit(windq_ctx* ctx, const __half* W, int R, int U, int64_t l
   int64_t grid = (int64_t)ctx->sm_count * blocks_per_sm;
   const int64_t need = (n_items + kFitWarpsPerBlock - 1) / kFitWarpsPerBlock;
   if (grid > need) grid = need;
+  WINDQ_REQUIRE(ctx, n_items < (1ll << 31), WINDQ_ERR_SHAPE, "windq_fit_eval: R * C is too large for one call");
+  WINDQ_CUDA(ctx, cudaMemsetAsync(next_item, 0, sizeof(unsigned int), st));
   if (PROTECT) fit_scale_kernel<<<(unsigned)((U * G + 255) / 256), 256, 0, st>>>(s, U * G, scale);
   fit_eval_kernel<G, PROTECT><<<(unsigned)grid, kFitWarpsPerBlock * 32, smem, st>>>(
       W, R, U, ldw, s, clip, K, partial, clip_idx_out, group_err_out, rows_blocks, chunk, stride, scale, thresh,
-      __builtin_nanf(""));
+      __builtin_nanf(""), next_item);
   WINDQ_CUDA(ctx, cudaGetLastError());
   fit_finalize_kernel<<<(unsigned)U, 256, 0, st>>>(partial, rows_blocks, err_out, energy_out);
   WINDQ_CUDA(ctx, cudaGetLastError());
@@ -178,7 +185,8 @@ extern "C" {
 int64_t windq_scratch_bytes_fit_eval(int64_t R, int64_t C, int G) {
   if (!windq::valid_G(G) || R <= 0 || C <= 0) return 0;
   const int gpw = 32 / (G / 32);
-  return (C / G) * ((R + gpw - 1) / gpw) * windq::kFitPartials * (int64_t)sizeof(double);
+  // the item counter (16 bytes, so that the doubles stay aligned), then eight doubles per item
+  return 16 + (C / G) * ((R + gpw - 1) / gpw) * windq::kFitPartials * (int64_t)sizeof(double);
 }
 
 static windq_status fit_eval_any(windq_ctx* ctx, const char* who, const void* W, int64_t R, int64_t C, int64_t ldw, int G,
@@ -196,14 +204,15 @@ static windq_status fit_eval_any(windq_ctx* ctx, const char* who, const void* W,
   const int U = (int)(C / G);
   cudaStream_t st = (cudaStream_t)stream;
   const __half* Wh = (const __half*)W;
-  double* partial = (double*)ctx->scratch;
+  unsigned int* next_item = (unsigned int*)ctx->scratch;
+  double* partial = (double*)((char*)ctx->scratch + 16);
   float* scale = (float*)((char*)ctx->scratch + round_up(part_bytes, 16));
 #define WINDQ_FIT_CASE(GG)                                                                                              \
   case GG:                                                                                                              \
     return thresh ? launch_fit<GG, true>(ctx, Wh, (int)R, U, ldw, s, clip_grid, K, partial, err_out, energy_out,         \
-                                         clip_idx_out, group_err_out, scale, thresh, st)                                \
+                                         clip_idx_out, group_err_out, scale, thresh, next_item, st)                                \
                   : launch_fit<GG, false>(ctx, Wh, (int)R, U, ldw, s, clip_grid, K, partial, err_out, energy_out,        \
-                                          clip_idx_out, group_err_out, nullptr, nullptr, st);
+                                          clip_idx_out, group_err_out, nullptr, nullptr, next_item, st);
   switch (G) {
     WINDQ_FIT_CASE(32)
     WINDQ_FIT_CASE(64)

@@ -45,5 +45,5 @@ def test_null_context_is_rejected_without_a_gpu(lib):
     assert lib.windq_create(vp(), 0) == 1
     lib.windq_scratch_bytes_fit_eval.restype = ctypes.c_int64
     lib.windq_scratch_bytes_fit_eval.argtypes = [ctypes.c_int64, ctypes.c_int64, ctypes.c_int]
-    assert lib.windq_scratch_bytes_fit_eval(4096, 4096, 128) == 32 * 512 * 8 * 8
+    assert lib.windq_scratch_bytes_fit_eval(4096, 4096, 128) == 16 + 32 * 512 * 8 * 8
     assert lib.windq_scratch_bytes_fit_eval(4096, 4096, 100) == 0

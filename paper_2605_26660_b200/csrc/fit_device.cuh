@@ -225,7 +225,7 @@ __device__ __forceinline__ void search_uniform(const Lane32& w, const Lane32& s,
   const int g = lane / LG, q = lane % LG;
   const UniformSpec us = uniform_spec(bi);
   Cand* mine = cand + g * stride;
-  best_e = 0.0f;
+  best_e = __int_as_float(0x7f800000);  // +inf: the first candidate replaces it (or none does, if no error is finite)
   best_k = 0;
   for (int k0 = 0; k0 < K; k0 += chunk) {
     const int kc = min(chunk, K - k0);
@@ -237,7 +237,7 @@ __device__ __forceinline__ void search_uniform(const Lane32& w, const Lane32& s,
       float2 e01, e23;
       cand_leaf_errors(w, s, c, e01, e23);
       const float e = group_tree<G>(e01, e23);
-      if ((k0 + k == 0) || e < best_e) {
+      if (e < best_e) {
         best_e = e;
         best_k = k0 + k;
       }

@@ -267,3 +267,23 @@ def fallback(err, energy, actions, theta: float):
     if rc:
         raise ValueError("oracle_fallback: bad arguments")
     return out, n.value
+
+
+def greedy_allocate(saliency, n_weights, n_groups, target_cb: int, headroom_cb: int, n_protected=None,
+                    scale_bits: int = 0, zero_bits: int = 0):
+    """The heuristic allocator's deterministic rule.  Returns (actions u8 [U], order i64 [U], total centibits)."""
+    sal = _f32(saliency)
+    U = sal.size
+    n = np.ascontiguousarray(n_weights, dtype=np.int64)
+    g = np.ascontiguousarray(n_groups, dtype=np.int64)
+    p = None if n_protected is None else np.ascontiguousarray(n_protected, dtype=np.int64)
+    assert n.size == U and g.size == U and (p is None or p.size == U)
+    actions = np.zeros(U, np.uint8)
+    order = np.zeros(U, np.int64)
+    total = ctypes.c_int64()
+    rc = lib().oracle_greedy_allocate(_p(sal), _p(n), _p(p), _p(g), ctypes.c_int64(U), ctypes.c_int64(target_cb),
+                                      ctypes.c_int64(headroom_cb), ctypes.c_int(scale_bits), ctypes.c_int(zero_bits),
+                                      _p(actions), _p(order), ctypes.byref(total))
+    if rc:
+        raise ValueError("oracle_greedy_allocate: bad arguments")
+    return actions, order, total.value

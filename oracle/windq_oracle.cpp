@@ -765,4 +765,87 @@ int oracle_fallback(const float* err, const float* energy, const uint8_t* action
   return 0;
 }
 
+// The deterministic rule of the heuristic sensitivity allocator ("Comparison with Heuristic
+// Sensitivity Allocator"): units are ranked by saliency, all start at 2 bit, the least sensitive are
+// pushed to 1.58 or 1 bit to free budget and the most sensitive are promoted to 3 or 4 bit while the
+// budget permits.  READING (the paper fixes neither the order of the moves nor how much is freed):
+//   cost(u, a) = Eq. 6 of unit u under action a, in centibits, with the per-group parameter bits
+//                counted as in oracle_effective_bits_protected
+//   budget     = target_cb * N,   floor = budget - headroom_cb * N,   N = sum of n_weights
+//   rank       : saliency descending under the total order of the binary32 bit patterns (sign and
+//                magnitude; -0 below +0), equal scores by ascending unit index
+//   1. every unit takes the 2-bit action; total = sum of cost(u, 2 bit)
+//   2. two sweeps from the least sensitive unit upwards, the first to 1.58 bit, the second to 1 bit:
+//      a unit is moved down while total > floor; the first unit met with total <= floor ends step 2
+//   3. one pass from the most sensitive unit downwards over the units still at 2 bit: the unit takes
+//      4 bit if total stays <= budget, else 3 bit if total stays <= budget, else it stays
+// order_out (nullable) receives the ranking, total_out the final total.
+static uint32_t saliency_key(float x) {
+  uint32_t b;
+  std::memcpy(&b, &x, 4);
+  return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+
+static int64_t unit_cost(int a, int64_t n, int64_t np_, int64_t groups, int scale_bits, int zero_bits) {
+  static const int64_t centi[7] = {1600, 800, 400, 300, 200, 158, 100};
+  if (a == 0) return 1600 * n;
+  return centi[a] * (n - np_) + 800 * np_ + 100 * groups * (scale_bits + ((a <= 4) ? zero_bits : 0));
+}
+
+int oracle_greedy_allocate(const float* saliency, const int64_t* n_weights, const int64_t* n_protected,
+                           const int64_t* n_groups, int64_t U, int64_t target_cb, int64_t headroom_cb, int scale_bits,
+                           int zero_bits, uint8_t* actions_out, int64_t* order_out, int64_t* total_out) {
+  if (!saliency || !n_weights || !n_groups || !actions_out || U <= 0 || target_cb < 0 || headroom_cb < 0 ||
+      scale_bits < 0 || zero_bits < 0)
+    return 1;
+  int64_t N = 0;
+  for (int64_t u = 0; u < U; ++u) {
+    const int64_t np_ = n_protected ? n_protected[u] : 0;
+    if (n_weights[u] < 0 || n_groups[u] < 0 || np_ < 0 || np_ > n_weights[u]) return 1;
+    N += n_weights[u];
+  }
+  std::vector<int64_t> order((size_t)U);
+  for (int64_t u = 0; u < U; ++u) order[(size_t)u] = u;
+  std::sort(order.begin(), order.end(), [&](int64_t a, int64_t b) {
+    const uint32_t ka = saliency_key(saliency[a]), kb = saliency_key(saliency[b]);
+    return ka != kb ? ka > kb : a < b;
+  });
+  auto cost = [&](int64_t u, int a) {
+    return unit_cost(a, n_weights[u], n_protected ? n_protected[u] : 0, n_groups[u], scale_bits, zero_bits);
+  };
+  const int64_t budget = target_cb * N, floor_ = budget - headroom_cb * N;
+  int64_t total = 0;
+  for (int64_t u = 0; u < U; ++u) {
+    actions_out[u] = 4;
+    total += cost(u, 4);
+  }
+  bool freed = false;
+  for (int down = 5; down <= 6 && !freed; ++down)
+    for (int64_t r = U - 1; r >= 0; --r) {
+      if (total <= floor_) {
+        freed = true;
+        break;
+      }
+      const int64_t u = order[(size_t)r];
+      total += cost(u, down) - cost(u, actions_out[u]);
+      actions_out[u] = (uint8_t)down;
+    }
+  for (int64_t r = 0; r < U; ++r) {
+    const int64_t u = order[(size_t)r];
+    if (actions_out[u] != 4) continue;
+    for (int up = 2; up <= 3; ++up) {
+      const int64_t with = total + cost(u, up) - cost(u, 4);
+      if (with <= budget) {
+        total = with;
+        actions_out[u] = (uint8_t)up;
+        break;
+      }
+    }
+  }
+  if (order_out)
+    for (int64_t r = 0; r < U; ++r) order_out[r] = order[(size_t)r];
+  if (total_out) *total_out = total;
+  return 0;
+}
+
 }  // extern "C"

@@ -186,8 +186,8 @@ windq_status windq_apply_plan(windq_ctx* ctx, const void* W, int64_t R, int64_t 
  * The paper keeps, in every unit, the top-r fraction of the weights by saliency -- weight magnitude
  * times the activation scale of the weight's input channel -- in INT8 and counts them at 8 bits in
  * Eq. 6.  windq_salient_select finds that set exactly; windq_effective_bits_protected is Eq. 6 with
- * it; windq_fit_eval_protected scores the fits with those weights left out.  (Packing with INT8 side
- * storage for them is not built yet.)
+ * it; windq_fit_eval_protected scores the fits with those weights left out; windq_apply_plan_protected
+ * packs a plan with the INT8 side storage for them.
  *
  *   key(r, j)  = |W[r][j]| * sqrt(s[j])            two binary32 operations (sqrt, then product)
  *   n_p        = floor(rate_ppm * R * G / 10^6)     weights asked for per unit (rate in parts per million)
@@ -251,6 +251,36 @@ windq_status windq_effective_bits_protected(windq_ctx* ctx, const uint8_t* actio
  * to run; within 1e-6 relative of the exact value). */
 windq_status windq_unit_saliency(windq_ctx* ctx, const void* W, int64_t R, int64_t C, int64_t ldw, int G,
                                  const float* s, float* sal_out, void* stream);
+
+/* The deterministic rule of the paper's heuristic allocator ("Comparison with Heuristic Sensitivity
+ * Allocator": units ranked by saliency; all start at 2 bit; the least sensitive are pushed to 1.58 or
+ * 1 bit to free budget; the most sensitive are promoted to 3 or 4 bit if budget permits).  The paper
+ * fixes neither the order of the moves nor how much is freed; this call does the following, over the
+ * U units of any number of matrices:
+ *   cost(u, a) = 100 b_a (n_u - p_u) + 800 p_u + 100 g_u (scale_bits [+ zero_bits for 4/3/2 bit])   Eq. 6, centibits
+ *   budget = target_cb * N,  floor = budget - headroom_cb * N,  N = sum of n_u
+ *   rank: saliency descending in the total order of the binary32 bit patterns (-0 below +0), equal
+ *         scores by ascending unit index
+ *   1. every unit takes 2 bit; total = sum of the costs
+ *   2. two sweeps from the least sensitive unit upwards, the first to 1.58 bit, the second to 1 bit: a
+ *      unit moves while total > floor; the first unit met with total <= floor ends the step
+ *   3. one pass from the most sensitive unit downwards over the units still at 2 bit: 4 bit if the total
+ *      stays <= budget, else 3 bit if it stays <= budget, else no change
+ * Arguments (device unless said otherwise):
+ *   saliency fp32 [U] (e.g. windq_unit_saliency, matrix after matrix);  n_weights, n_groups i64 [U]
+ *   (R G and R of the unit's matrix);  n_protected i64 [U], nullable = none (count_out of
+ *   windq_salient_select);  target_cb, headroom_cb in [0, 1600] (host values)
+ *   actions_out u8 [U];  order_out i64 [U], nullable: unit indices, most sensitive first;
+ *   total_centibits_out i64 [1]: the final total, or -1 if a count is negative or p_u > n_u (actions
+ *   are then meaningless)
+ * U <= WINDQ_MAX_ALLOC_UNITS.  All arithmetic is int64: results are exact.  Scratch:
+ * windq_scratch_bytes_greedy_allocate. */
+#define WINDQ_MAX_ALLOC_UNITS (1 << 20)
+int64_t windq_scratch_bytes_greedy_allocate(int64_t U);
+windq_status windq_greedy_allocate(windq_ctx* ctx, const float* saliency, const int64_t* n_weights,
+                                   const int64_t* n_protected, const int64_t* n_groups, int64_t U, int64_t target_cb,
+                                   int64_t headroom_cb, int scale_bits, int zero_bits, uint8_t* actions_out,
+                                   int64_t* order_out, int64_t* total_centibits_out, void* stream);
 
 /* Fallback to higher precision (Sec. 3.5: "if the reconstruction error of a selected operator is
  * excessive, the implementation falls back to a higher-precision operator").  The paper gives neither

@@ -67,6 +67,9 @@ def _load() -> ctypes.CDLL:
     lib.windq_scratch_bytes_apply_plan_protected.restype = i64
     lib.windq_unit_saliency.argtypes = [vp, vp, i64, i64, i64, i32, vp, vp, vp]
     lib.windq_fallback.argtypes = [vp, vp, vp, vp, i64, ctypes.c_float, vp, vp, vp]
+    lib.windq_greedy_allocate.argtypes = [vp, vp, vp, vp, vp, i64, i64, i64, i32, i32, vp, vp, vp, vp]
+    lib.windq_scratch_bytes_greedy_allocate.restype = i64
+    lib.windq_scratch_bytes_greedy_allocate.argtypes = [i64]
     lib.windq_apply_plan.argtypes = [vp, vp, i64, i64, i64, i32, vp, vp, i32, vp, vp, vp, vp, vp, vp, vp, vp]
     return lib
 
@@ -366,6 +369,32 @@ def windq_fallback(ctx: Context, err: torch.Tensor, energy: torch.Tensor, action
     ctx._check(_lib.windq_fallback(ctx._h, _ptr(err), _ptr(energy), _ptr(actions), U, float(theta), _ptr(out), _ptr(n),
                                    _stream(stream)))
     return dict(actions=out, n_changed=n)
+
+
+def windq_greedy_allocate(ctx: Context, saliency: torch.Tensor, n_weights: torch.Tensor, n_groups: torch.Tensor,
+                          target_cb: int, headroom_cb: int, n_protected: torch.Tensor | None = None, *,
+                          scale_bits: int = 0, zero_bits: int = 0, stream=None) -> dict:
+    """The heuristic allocator's rule over U units: rank by saliency, free budget from the bottom, promote from the top.
+    Returns dict(actions [U] u8, order [U] i64 (most sensitive first), total_centibits [1] i64)."""
+    _need(saliency, torch.float32, "saliency", 1)
+    _need(n_weights, torch.int64, "n_weights", 1)
+    _need(n_groups, torch.int64, "n_groups", 1)
+    U = saliency.numel()
+    if n_weights.numel() != U or n_groups.numel() != U:
+        raise ValueError("n_weights and n_groups must have one entry per unit")
+    if not (saliency.is_contiguous() and n_weights.is_contiguous() and n_groups.is_contiguous()):
+        raise ValueError("saliency, n_weights and n_groups must be contiguous")
+    if n_protected is not None:
+        _need(n_protected, torch.int64, "n_protected", 1)
+        if n_protected.numel() != U or not n_protected.is_contiguous():
+            raise ValueError("n_protected must be contiguous with one entry per unit")
+    actions = torch.empty(U, dtype=torch.uint8, device=saliency.device)
+    order = torch.empty(U, dtype=torch.int64, device=saliency.device)
+    total = torch.empty(1, dtype=torch.int64, device=saliency.device)
+    ctx._check(_lib.windq_greedy_allocate(ctx._h, _ptr(saliency), _ptr(n_weights), _ptr(n_protected), _ptr(n_groups), U,
+                                          int(target_cb), int(headroom_cb), int(scale_bits), int(zero_bits), _ptr(actions),
+                                          _ptr(order), _ptr(total), _stream(stream)))
+    return dict(actions=actions, order=order, total_centibits=total)
 
 
 def windq_apply_plan_protected(ctx: Context, W: torch.Tensor, G: int, s: torch.Tensor, clip_grid: torch.Tensor,

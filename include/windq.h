@@ -252,6 +252,31 @@ windq_status windq_effective_bits_protected(windq_ctx* ctx, const uint8_t* actio
 windq_status windq_unit_saliency(windq_ctx* ctx, const void* W, int64_t R, int64_t C, int64_t ldw, int G,
                                  const float* s, float* sal_out, void* stream);
 
+/* Iterative refinement of the step sizes (App. "Per-unit Scale Optimization": the selected operator fits
+ * its scale by a small local optimisation, typically 10 Adam steps, on the reconstruction loss of the
+ * chunk; the 3/4/8-bit operators learn step sizes with straight-through estimation of the rounding).
+ * The paper prints no formulas; this call does the following for the four uniform bit-widths (8, 4, 3,
+ * 2), per group, in binary32:
+ *   warm start  the clip-grid fit that clip_idx names: Delta_0 = its fp16 scale, its zero point z stays
+ *   iterate t   Delta_h = fp16(Delta_t);  c_j = clamp(rne(w_j / Delta_h), -z, qmax - z);
+ *               d_j = c_j Delta_h - w_j;  loss e_t = sum s_j d_j^2  (the operations of windq_fit_eval)
+ *               psi_j = rne(w_j / Delta_h) - w_j / Delta_h in range, c_j where clipped;  g_t = sum s_j d_j psi_j
+ *   Adam        beta1 0.9, beta2 0.999, eps 1e-8, bias-corrected, learning rate lr * Delta_0
+ *   result      the iterate of least loss among t = 0..n_steps (the first on ties), so no error exceeds
+ *               that of windq_fit_eval; a group stops early when fp16(Delta) is not positive and finite
+ * Arguments as windq_fit_eval, and
+ *   clip_idx      u8   [4][U][R]  from windq_fit_eval for the same W, s, G and grid (an index >= K is K-1)
+ *   n_steps       0..32 (host);  lr in [0, 1] (host): step of the first update relative to Delta_0
+ *   err_out       fp32 [U][4]     unit sums of the refined group errors (double accumulation)
+ *   scale_out     fp16 [4][U][R]  refined scales
+ *   group_err_out fp32 [4][U][R]  nullable
+ * With n_steps = 0 scales and group errors are those of the clip-grid fit, bit for bit.  Scratch:
+ * windq_scratch_bytes_fit_refine. */
+int64_t windq_scratch_bytes_fit_refine(int64_t R, int64_t C, int G);
+windq_status windq_fit_refine(windq_ctx* ctx, const void* W, int64_t R, int64_t C, int64_t ldw, int G, const float* s,
+                              const float* clip_grid, int K, const uint8_t* clip_idx, int n_steps, float lr,
+                              float* err_out, void* scale_out, float* group_err_out, void* stream);
+
 /* The deterministic rule of the paper's heuristic allocator ("Comparison with Heuristic Sensitivity
  * Allocator": units ranked by saliency; all start at 2 bit; the least sensitive are pushed to 1.58 or
  * 1 bit to free budget; the most sensitive are promoted to 3 or 4 bit if budget permits).  The paper

@@ -287,3 +287,37 @@ def greedy_allocate(saliency, n_weights, n_groups, target_cb: int, headroom_cb: 
     if rc:
         raise ValueError("oracle_greedy_allocate: bad arguments")
     return actions, order, total.value
+
+
+def refine_trace(w, s, bits: int, scale0: float, zf: float, T: int, lr: float):
+    """The refinement iteration on one group.  Returns (scales, losses, grads) of the iterates evaluated."""
+    w, s = _f32(w), _f32(s)
+    G = w.size
+    assert s.size == G
+    sc, lo, gr = (np.zeros(T + 1, np.float32) for _ in range(3))
+    fn = lib().oracle_refine_trace
+    fn.restype = ctypes.c_int
+    n = fn(_p(w), _p(s), ctypes.c_int(G), ctypes.c_int(bits), ctypes.c_float(scale0), ctypes.c_float(zf), ctypes.c_int(T),
+           ctypes.c_float(lr), _p(sc), _p(lo), _p(gr))
+    if n < 0:
+        raise ValueError("oracle_refine_trace: bad arguments")
+    return sc[:n], lo[:n], gr[:n]
+
+
+def fit_refine(W, G: int, s, clip_grid, clip_idx, T: int = 10, lr: float = 0.01):
+    """Step-size refinement of the four uniform fits, warm-started from clip_idx [4][U][R] of fit_eval.
+    Returns dict(err [U][4] f32, scale [4][U][R] f16, group_err [4][U][R] f32)."""
+    W, s, clip_grid = _as_u16(W), _f32(s), _f32(clip_grid)
+    R, C = W.shape
+    U = C // G
+    clip_idx = np.ascontiguousarray(clip_idx, dtype=np.uint8)
+    assert clip_idx.shape == (4, U, R)
+    err = np.zeros((U, 4), np.float32)
+    scale = np.zeros((4, U, R), np.uint16)
+    gerr = np.zeros((4, U, R), np.float32)
+    rc = lib().oracle_fit_refine(_p(W), ctypes.c_int64(R), ctypes.c_int64(C), ctypes.c_int64(W.strides[0] // 2),
+                                 ctypes.c_int(G), _p(s), _p(clip_grid), ctypes.c_int(clip_grid.size), _p(clip_idx),
+                                 ctypes.c_int(T), ctypes.c_float(lr), _p(err), _p(scale), _p(gerr))
+    if rc:
+        raise ValueError("oracle_fit_refine: bad arguments (%d)" % rc)
+    return dict(err=err, scale=scale.view(np.float16), group_err=gerr)

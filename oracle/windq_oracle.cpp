@@ -848,4 +848,143 @@ int oracle_greedy_allocate(const float* saliency, const int64_t* n_weights, cons
   return 0;
 }
 
+// ---- iterative step-size refinement (App. "Per-unit Scale Optimization") -------------------------
+// The paper's operators fit their scale by a small local optimisation, typically 10 Adam steps on
+// the reconstruction loss of the current chunk, and the 3/4/8-bit ones "learn step sizes with
+// straight-through estimation for discrete rounding" (the LSQ rule, Esser et al. 2020).  It prints no
+// formulas.  READING, for the four uniform bit-widths, per group, all in binary32:
+//   warm start   the clip-grid fit: Delta_0 = its stored fp16 scale, zero point z fixed at its value
+//   iterate t    Delta_h = fp16(Delta_t) is the step actually used (a scale is stored in fp16);
+//                c_j = clamp(rne(w_j / Delta_h), -z, qmax - z), d_j = c_j Delta_h - w_j,
+//                loss e_t = sum s_j d_j^2            (the operations of uniform_error, same order)
+//                psi_j = rne(w_j / Delta_h) - w_j / Delta_h inside the range, c_j where clipped
+//                g_t = sum (s_j d_j) psi_j           (half the LSQ gradient; PSUM8 order)
+//   Adam         beta1 0.9, beta2 0.999, eps 1e-8, bias-corrected, learning rate lr * Delta_0:
+//                m = 0.9 m + 0.1 g;  v = 0.999 v + 0.001 g^2;
+//                Delta_{t+1} = Delta_t - (lr Delta_0) * (m c1_t) / (sqrt(v c2_t) + eps),
+//                c1_t = 1 / (1 - 0.9^t), c2_t = 1 / (1 - 0.999^t) rounded to binary32
+//   result       the iterate with the least loss among t = 0..T (first one on ties), so the refined
+//                error never exceeds the clip-grid error; the iteration stops early when fp16(Delta)
+//                is not a positive finite number.
+struct RefineStep {
+  float scale;  // Delta_h
+  float loss;
+  float grad;
+};
+
+static void refine_eval(const Group& g, float scale, float zf, float qmaxf, float* loss, float* grad) {
+  UniformParams u;
+  u.scale = scale;
+  u.inv = 1.0f / scale;
+  u.zf = zf;
+  u.qmaxf = qmaxf;
+  *loss = uniform_error(g, u);
+  *grad = psum8(g.G, [&](int l) {
+    float acc = 0.0f;
+    for (int j = 8 * l; j < 8 * l + 8; ++j) {
+      const float r = std::fmaf(g.w[j], u.inv, kMagic) - kMagic;
+      const float c = centred_code(g.w[j], u);
+      const float x = g.w[j] * u.inv;
+      const float psi = (c == r) ? r - x : c;
+      const float d = std::fmaf(c, u.scale, -g.w[j]);
+      const float t = g.s[j] * d;
+      acc = std::fmaf(t, psi, acc);
+    }
+    return acc;
+  });
+}
+
+static void adam_corrections(int T, float* c1, float* c2) {  // c[t-1] for t = 1..T
+  double p1 = 1.0, p2 = 1.0;
+  for (int t = 1; t <= T; ++t) {
+    p1 *= 0.9;
+    p2 *= 0.999;
+    c1[t - 1] = (float)(1.0 / (1.0 - p1));
+    c2[t - 1] = (float)(1.0 / (1.0 - p2));
+  }
+}
+
+// Runs the iteration on one group; trace (nullable) receives every iterate that was evaluated.
+// Returns the number of iterates evaluated (1..T+1).
+static int refine_group(const Group& g, float scale0, float zf, float qmaxf, int T, float lr, float* best_scale,
+                        float* best_loss, RefineStep* trace) {
+  float c1[32], c2[32];
+  adam_corrections(T, c1, c2);
+  const float step = lr * scale0;
+  float delta = scale0, m = 0.0f, v = 0.0f;
+  int n = 0;
+  for (int t = 0; t <= T; ++t) {
+    const float sh = round_through_half(delta);
+    if (!(sh > 0.0f) || std::isinf(sh)) break;
+    float loss, grad;
+    refine_eval(g, sh, zf, qmaxf, &loss, &grad);
+    if (trace) trace[n] = RefineStep{sh, loss, grad};
+    if (n == 0 || loss < *best_loss) {
+      *best_loss = loss;
+      *best_scale = sh;
+    }
+    ++n;
+    if (t == T) break;
+    m = std::fmaf(0.9f, m, 0.1f * grad);
+    v = std::fmaf(0.999f, v, 0.001f * (grad * grad));
+    const float mhat = m * c1[t], vhat = v * c2[t];
+    const float upd = mhat / (std::sqrt(vhat) + 1e-8f);
+    delta = std::fmaf(-step, upd, delta);
+  }
+  return n;
+}
+
+// One group, for the pins: w, s of length G; scale0 and zf as a clip-grid fit would give them.
+// scales / losses / grads receive T+1 entries (unused ones untouched); returns the number evaluated.
+int oracle_refine_trace(const float* w, const float* s, int G, int bits, float scale0, float zf, int T, float lr,
+                        float* scales, float* losses, float* grads) {
+  if (!w || !s || !valid_group_width(G) || T < 0 || T > 32) return -1;
+  RefineStep tr[33];
+  float bs = 0.0f, bl = 0.0f;
+  Group g{G, w, s};
+  const int n = refine_group(g, scale0, zf, (float)((1 << bits) - 1), T, lr, &bs, &bl, tr);
+  for (int i = 0; i < n; ++i) {
+    if (scales) scales[i] = tr[i].scale;
+    if (losses) losses[i] = tr[i].loss;
+    if (grads) grads[i] = tr[i].grad;
+  }
+  return n;
+}
+
+// Refinement of every group's step size for the four uniform bit-widths, warm-started from the clip
+// indices of oracle_fit_eval.  err_out [U][4] (unit sums in double, rows ascending), scale_out fp16
+// bits [4][U][R], group_err_out [4][U][R] (nullable).
+int oracle_fit_refine(const uint16_t* W, int64_t R, int64_t C, int64_t ldw, int G, const float* s,
+                      const float* clip_grid, int K, const uint8_t* clip_idx, int T, float lr, float* err_out,
+                      uint16_t* scale_out, float* group_err_out) {
+  if (!W || !s || !clip_grid || !clip_idx || !err_out || !scale_out || R <= 0 || C <= 0 || !valid_group_width(G) ||
+      C % G != 0 || ldw < C || K < 1 || K > 64 || T < 0 || T > 32 || !(lr >= 0.0f))
+    return 1;
+  const int64_t U = C / G;
+  std::vector<float> w((size_t)G);
+  for (int64_t u = 0; u < U; ++u) {
+    double tot[4] = {0, 0, 0, 0};
+    for (int64_t r = 0; r < R; ++r) {
+      load_group(W, ldw, r, u, G, w.data());
+      Group g{G, w.data(), s + u * G};
+      float mn, rng;
+      group_range(g, &mn, &rng);
+      for (int bi = 0; bi < 4; ++bi) {
+        const int64_t o = ((int64_t)bi * U + u) * R + r;
+        int k = clip_idx[o];
+        if (k >= K) k = K - 1;
+        const UniformParams p = uniform_params(mn, rng, clip_grid[k], kUniformBits[bi]);
+        float bs = 0.0f, bl = 0.0f;
+        const int n = refine_group(g, p.scale, p.zf, p.qmaxf, T, lr, &bs, &bl, nullptr);
+        if (n == 0) return 2;  // cannot happen: the warm-start scale is a positive finite fp16 value
+        tot[bi] += (double)bl;
+        scale_out[o] = float_to_half(bs);
+        if (group_err_out) group_err_out[o] = bl;
+      }
+    }
+    for (int bi = 0; bi < 4; ++bi) err_out[u * 4 + bi] = (float)tot[bi];
+  }
+  return 0;
+}
+
 }  // extern "C"

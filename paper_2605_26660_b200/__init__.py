@@ -67,6 +67,9 @@ def _load() -> ctypes.CDLL:
     lib.windq_scratch_bytes_apply_plan_protected.restype = i64
     lib.windq_unit_saliency.argtypes = [vp, vp, i64, i64, i64, i32, vp, vp, vp]
     lib.windq_fallback.argtypes = [vp, vp, vp, vp, i64, ctypes.c_float, vp, vp, vp]
+    lib.windq_fit_refine.argtypes = [vp, vp, i64, i64, i64, i32, vp, vp, i32, vp, i32, ctypes.c_float, vp, vp, vp, vp]
+    lib.windq_scratch_bytes_fit_refine.restype = i64
+    lib.windq_scratch_bytes_fit_refine.argtypes = [i64, i64, i32]
     lib.windq_greedy_allocate.argtypes = [vp, vp, vp, vp, vp, i64, i64, i64, i32, i32, vp, vp, vp, vp]
     lib.windq_scratch_bytes_greedy_allocate.restype = i64
     lib.windq_scratch_bytes_greedy_allocate.argtypes = [i64]
@@ -235,6 +238,28 @@ def windq_fit_eval(ctx: Context, W: torch.Tensor, G: int, s: torch.Tensor, clip_
         ctx._check(_lib.windq_fit_eval_protected(ctx._h, _ptr(W), R, C, ldw, int(G), _ptr(s), _ptr(clip_grid),
                                                  clip_grid.numel(), _ptr(thresh), _ptr(out["err"]), _ptr(out["energy"]),
                                                  _ptr(out["clip_idx"]), _ptr(out["group_err"]), _stream(stream)))
+    return out
+
+
+def windq_fit_refine(ctx: Context, W: torch.Tensor, G: int, s: torch.Tensor, clip_grid: torch.Tensor,
+                     clip_idx: torch.Tensor, n_steps: int = 10, lr: float = 0.01, *, want_group_err: bool = False,
+                     stream=None) -> dict:
+    """Refines the step sizes of the four uniform fits by ``n_steps`` Adam steps, warm-started from ``clip_idx``
+    ([4, U, R] u8 of windq_fit_eval).  Returns dict(err [U,4] f32, scale [4,U,R] f16, group_err [4,U,R] f32 | None)."""
+    R, C, ldw = _matrix(W, "W")
+    _need(s, torch.float32, "s", 1)
+    _need(clip_grid, torch.float32, "clip_grid", 1)
+    _need(clip_idx, torch.uint8, "clip_idx", 3)
+    U = C // G if G > 0 else 0
+    if tuple(clip_idx.shape) != (4, U, R) or not clip_idx.is_contiguous():
+        raise ValueError("clip_idx must be a contiguous [4, U, R] tensor")
+    dev = W.device
+    out = dict(err=torch.empty((U, 4), dtype=torch.float32, device=dev),
+               scale=torch.empty((4, U, R), dtype=torch.float16, device=dev),
+               group_err=torch.empty((4, U, R), dtype=torch.float32, device=dev) if want_group_err else None)
+    ctx._check(_lib.windq_fit_refine(ctx._h, _ptr(W), R, C, ldw, int(G), _ptr(s), _ptr(clip_grid), clip_grid.numel(),
+                                     _ptr(clip_idx), int(n_steps), float(lr), _ptr(out["err"]), _ptr(out["scale"]),
+                                     _ptr(out["group_err"]), _stream(stream)))
     return out
 
 

@@ -8,7 +8,8 @@
 // a few microseconds for the tens of thousands of units of a model.  The rule itself runs in one block:
 // the two sweeps of step 2 are prefix sums (a unit moves while the running total is above the floor,
 // and the savings are never negative, so the moved units are a prefix of the sweep), step 3 is serial by
-// nature and runs in one warp, 32 units at a time, with two shortcuts for chunks that take all or nothing.
+// nature and runs in one warp, 32 units at a time, over counts gathered in rank order beforehand, with
+// two shortcuts for chunks that take all or nothing.
 #include "windq_internal.cuh"
 
 namespace windq {
@@ -76,7 +77,8 @@ __device__ __forceinline__ long long block_sum(long long v, long long* red) {
 }
 
 __global__ void __launch_bounds__(1024)
-alloc_greedy_kernel(AllocArgs a, const int* __restrict__ order, uint8_t* actions, long long* __restrict__ total_out) {
+alloc_greedy_kernel(AllocArgs a, const int* __restrict__ order, long long* __restrict__ walk, uint8_t* actions,
+                    long long* __restrict__ total_out) {
   __shared__ long long red[32];
   __shared__ long long warp_incl[32];
   const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
@@ -134,22 +136,26 @@ alloc_greedy_kernel(AllocArgs a, const int* __restrict__ order, uint8_t* actions
       }
     }
   }
-  __syncthreads();  // the actions written above are read by warp 0 below
+  __syncthreads();  // the actions written above are read below
 
-  // step 3: most sensitive first, only units still at 2 bit (those moved down are the tail of the ranking)
+  // step 3: most sensitive first, only units still at 2 bit (those moved down are the tail of the
+  // ranking).  All warps first gather, in rank order, what the walk needs -- the unit's quantised
+  // weight count, or a mark for a unit that was moved down -- so that the one warp that walks reads
+  // consecutive words instead of chasing order[] -> counts through memory one chunk at a time.
+  for (int r = t; r < U; r += 1024) {
+    const int u = order[r];
+    walk[r] = actions[u] == 4 ? a.n_weights[u] - (a.n_protected ? a.n_protected[u] : 0) : -1;
+  }
+  __syncthreads();
   if (warp != 0) return;
+  long long q_next = lane < U ? walk[lane] : -1;
   for (int base = 0; base < U; base += 32) {
     const int r = base + lane;
-    int u = -1, act = 255;
-    long long q = 0;
-    if (r < U) {
-      u = order[r];
-      act = actions[u];
-      q = a.n_weights[u] - (a.n_protected ? a.n_protected[u] : 0);
-    }
-    const bool cand = act == 4;
+    const long long q = q_next;
+    q_next = r + 32 < U ? walk[r + 32] : -1;  // in flight while this chunk is decided
+    const bool cand = r < U && q >= 0;
     const unsigned cands = __ballot_sync(0xffffffffu, cand);
-    const bool tail = __any_sync(0xffffffffu, r < U && act >= 5);
+    const bool tail = __any_sync(0xffffffffu, r < U && q < 0);
     if (cands) {
       const long long all4 = warp_sum(cand ? 200 * q : 0);
       long long qmin = cand ? q : 0x7fffffffffffffffll;
@@ -175,7 +181,7 @@ alloc_greedy_kernel(AllocArgs a, const int* __restrict__ order, uint8_t* actions
           if (i == lane) choice = c;
         }
       }
-      if (cand && choice != 4) actions[u] = (uint8_t)choice;
+      if (cand && choice != 4) actions[order[r]] = (uint8_t)choice;
     }
     if (tail) break;
   }
@@ -188,7 +194,7 @@ extern "C" {
 
 int64_t windq_scratch_bytes_greedy_allocate(int64_t U) {
   if (U <= 0) return 0;
-  return windq::round_up(U * 8, 256) + windq::round_up(U * 4, 256);
+  return 2 * windq::round_up(U * 8, 256) + windq::round_up(U * 4, 256);
 }
 
 windq_status windq_greedy_allocate(windq_ctx* ctx, const float* saliency, const int64_t* n_weights, const int64_t* n_protected,
@@ -210,13 +216,14 @@ windq_status windq_greedy_allocate(windq_ctx* ctx, const float* saliency, const 
   if (windq_status rc = ensure_scratch(ctx, windq_scratch_bytes_greedy_allocate(U))) return rc;
   cudaStream_t st = (cudaStream_t)stream;
   unsigned long long* comp = (unsigned long long*)ctx->scratch;
-  int* order = (int*)((char*)ctx->scratch + round_up(U * 8, 256));
+  long long* walk = (long long*)((char*)ctx->scratch + round_up(U * 8, 256));
+  int* order = (int*)((char*)ctx->scratch + 2 * round_up(U * 8, 256));
   alloc_key_kernel<<<(unsigned)((U + 255) / 256), 256, 0, st>>>(saliency, (int)U, comp);
   alloc_rank_kernel<<<(unsigned)((U + kRankThreads - 1) / kRankThreads), kRankThreads, 0, st>>>(comp, (int)U, order,
                                                                                                (long long*)order_out);
   AllocArgs a{(const long long*)n_weights, (const long long*)n_protected, (const long long*)n_groups, (int)U,
               target_cb, headroom_cb, scale_bits, zero_bits};
-  alloc_greedy_kernel<<<1, 1024, 0, st>>>(a, order, actions_out, (long long*)total_centibits_out);
+  alloc_greedy_kernel<<<1, 1024, 0, st>>>(a, order, walk, actions_out, (long long*)total_centibits_out);
   WINDQ_CUDA(ctx, cudaGetLastError());
   return WINDQ_OK;
 }

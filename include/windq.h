@@ -277,6 +277,14 @@ windq_status windq_fit_refine(windq_ctx* ctx, const void* W, int64_t R, int64_t 
                               const float* clip_grid, int K, const uint8_t* clip_idx, int n_steps, float lr,
                               float* err_out, void* scale_out, float* group_err_out, void* stream);
 
+/* windq_apply_plan with the refined step sizes: the scale of every 8/4/3/2-bit group is scale_in
+ * (fp16 [4][U][R], device, from windq_fit_refine); its zero point is that of the clip-grid fit clip_idx
+ * names (required here).  Everything else as windq_apply_plan; scales_out repeats the scales used. */
+windq_status windq_apply_plan_refined(windq_ctx* ctx, const void* W, int64_t R, int64_t C, int64_t ldw, int G,
+                                      const float* s, const float* clip_grid, int K, const uint8_t* actions,
+                                      const uint8_t* clip_idx, const void* scale_in, const int64_t* code_offsets,
+                                      uint8_t* codes_out, void* scales_out, void* zeros_out, void* Wq_out, void* stream);
+
 /* The deterministic rule of the paper's heuristic allocator ("Comparison with Heuristic Sensitivity
  * Allocator": units ranked by saliency; all start at 2 bit; the least sensitive are pushed to 1.58 or
  * 1 bit to free budget; the most sensitive are promoted to 3 or 4 bit if budget permits).  The paper

@@ -174,11 +174,12 @@ def effective_bits(actions, R: int, G: int, scale_bits: int = 16, zero_bits: int
                 total_packed_bytes=packed.value)
 
 
-def apply_plan(W, G: int, s, clip_grid, actions, clip_idx=None, want_wq: bool = True, thresh=None):
+def apply_plan(W, G: int, s, clip_grid, actions, clip_idx=None, want_wq: bool = True, thresh=None, scale_in=None):
     """Returns dict(codes[bytes], scales[U,R] u16, zeros[U,R] u16, wq[R,C] u16, code_offsets).
 
     With ``thresh`` (fp32 [U], from salient_select) the salient weights are protected; the result then
-    also holds prot_scale[U] u16, prot_offsets[U+1] i64 and prot_q (int8 codes, row-major per unit)."""
+    also holds prot_scale[U] u16, prot_offsets[U+1] i64 and prot_q (int8 codes, row-major per unit).
+    With ``scale_in`` (fp16 [4][U][R], from fit_refine; needs clip_idx) the uniform groups use those scales."""
     W, s, clip_grid = _as_u16(W), _f32(s), _f32(clip_grid)
     actions = np.ascontiguousarray(actions, dtype=np.uint8)
     R, C = W.shape
@@ -205,6 +206,16 @@ def apply_plan(W, G: int, s, clip_grid, actions, clip_idx=None, want_wq: bool = 
             raise ValueError("oracle_apply_plan_protected: bad arguments")
         return dict(codes=codes, scales=scales, zeros=zeros, wq=wq, code_offsets=offs, prot_scale=prot_scale,
                     prot_offsets=prot_offsets, prot_q=prot_q[:int(prot_offsets[U])].copy())
+    if scale_in is not None:
+        assert thresh is None and clip_idx is not None
+        scale_in = _as_u16(scale_in)
+        assert scale_in.shape == (4, U, R)
+        rc = lib().oracle_apply_plan_refined(_p(W), ctypes.c_int64(R), ctypes.c_int64(C), ctypes.c_int64(C), ctypes.c_int(G),
+                                             _p(s), _p(clip_grid), ctypes.c_int(clip_grid.size), _p(actions), _p(clip_idx),
+                                             _p(scale_in), _p(offs), _p(codes), _p(scales), _p(zeros), _p(wq))
+        if rc:
+            raise ValueError("oracle_apply_plan_refined: bad arguments")
+        return dict(codes=codes, scales=scales, zeros=zeros, wq=wq, code_offsets=offs)
     rc = lib().oracle_apply_plan(_p(W), ctypes.c_int64(R), ctypes.c_int64(C), ctypes.c_int64(C), ctypes.c_int(G),
                                  _p(s), _p(clip_grid), ctypes.c_int(clip_grid.size), _p(actions), _p(clip_idx),
                                  _p(offs), _p(codes), _p(scales), _p(zeros), _p(wq))

@@ -548,7 +548,7 @@ static int apply_plan_impl(const uint16_t* W, int64_t R, int64_t C, int64_t ldw,
                            const float* clip_grid, int K, const uint8_t* actions, const uint8_t* clip_idx,
                            const int64_t* code_offsets, const float* thresh, uint8_t* codes_out, uint16_t* scales_out,
                            uint16_t* zeros_out, uint16_t* Wq_out, uint16_t* prot_scale_out, int64_t* prot_offsets_out,
-                           int8_t* prot_q_out) {
+                           int8_t* prot_q_out, const uint16_t* scale_in = nullptr) {
   if (thresh && (!prot_scale_out || !prot_offsets_out || !prot_q_out)) return 1;
   if (!W || !s || !clip_grid || !actions || !code_offsets || !codes_out || !scales_out || !zeros_out ||
       R <= 0 || C <= 0 || !valid_group_width(G) || C % G != 0 || ldw < C || K < 1 || K > 64)
@@ -609,7 +609,11 @@ static int apply_plan_impl(const uint16_t* W, int64_t R, int64_t C, int64_t ldw,
             float e;
             search_uniform(g, mn, rng, bits, clip_grid, K, &k, &e);
           }
-          const UniformParams p = uniform_params(mn, rng, clip_grid[k], bits);
+          UniformParams p = uniform_params(mn, rng, clip_grid[k], bits);
+          if (scale_in) {  // a refined step size replaces the clip-grid scale; the zero point stays
+            p.scale = half_to_float(scale_in[((int64_t)bi * U + u) * R + r]);
+            p.inv = 1.0f / p.scale;
+          }
           for (int j = 0; j < G; ++j) {
             const float c = centred_code(w[j], p);
             q[j] = (uint8_t)(int)(c + p.zf);
@@ -846,6 +850,17 @@ int oracle_greedy_allocate(const float* saliency, const int64_t* n_weights, cons
     for (int64_t r = 0; r < U; ++r) order_out[r] = order[(size_t)r];
   if (total_out) *total_out = total;
   return 0;
+}
+
+// oracle_apply_plan with the scales of the uniform groups taken from oracle_fit_refine (scale_in fp16 bits
+// [4][U][R]); zero points are those of the clip-grid fit that clip_idx names.
+int oracle_apply_plan_refined(const uint16_t* W, int64_t R, int64_t C, int64_t ldw, int G, const float* s,
+                              const float* clip_grid, int K, const uint8_t* actions, const uint8_t* clip_idx,
+                              const uint16_t* scale_in, const int64_t* code_offsets, uint8_t* codes_out,
+                              uint16_t* scales_out, uint16_t* zeros_out, uint16_t* Wq_out) {
+  if (!clip_idx || !scale_in) return 1;
+  return apply_plan_impl(W, R, C, ldw, G, s, clip_grid, K, actions, clip_idx, code_offsets, nullptr, codes_out,
+                         scales_out, zeros_out, Wq_out, nullptr, nullptr, nullptr, scale_in);
 }
 
 // ---- iterative step-size refinement (App. "Per-unit Scale Optimization") -------------------------

@@ -67,6 +67,7 @@ def _load() -> ctypes.CDLL:
     lib.windq_scratch_bytes_apply_plan_protected.restype = i64
     lib.windq_unit_saliency.argtypes = [vp, vp, i64, i64, i64, i32, vp, vp, vp]
     lib.windq_fallback.argtypes = [vp, vp, vp, vp, i64, ctypes.c_float, vp, vp, vp]
+    lib.windq_apply_plan_refined.argtypes = [vp, vp, i64, i64, i64, i32, vp, vp, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.windq_fit_refine.argtypes = [vp, vp, i64, i64, i64, i32, vp, vp, i32, vp, i32, ctypes.c_float, vp, vp, vp, vp]
     lib.windq_scratch_bytes_fit_refine.restype = i64
     lib.windq_scratch_bytes_fit_refine.argtypes = [i64, i64, i32]
@@ -288,10 +289,11 @@ def windq_effective_bits(ctx: Context, actions: torch.Tensor, R: int, G: int, sc
 def windq_apply_plan(ctx: Context, W: torch.Tensor, G: int, s: torch.Tensor, clip_grid: torch.Tensor,
                      actions: torch.Tensor, code_offsets: torch.Tensor, codes_out: torch.Tensor,
                      clip_idx: torch.Tensor | None = None, *, want_wq: bool = True, out: dict | None = None,
-                     stream=None) -> dict:
+                     stream=None, scale_in: torch.Tensor | None = None) -> dict:
     """Applies a plan.  ``code_offsets`` comes from windq_effective_bits for the same actions;
     ``codes_out`` is a uint8 tensor of at least code_offsets[U] bytes (the caller sizes it, e.g.
-    from the worst case 2*R*C + 16*U, to avoid a device-to-host read).
+    from the worst case 2*R*C + 16*U, to avoid a device-to-host read).  With ``scale_in`` (fp16 [4, U, R] from
+    windq_fit_refine; needs ``clip_idx``) the call is windq_apply_plan_refined.
 
     Returns dict(codes, scales [U,R] f16, zeros [U,R] f16, wq [R,C] f16 | None).
     """
@@ -320,6 +322,15 @@ def windq_apply_plan(ctx: Context, W: torch.Tensor, G: int, s: torch.Tensor, cli
     if out["wq"] is not None and (_matrix(out["wq"], "wq")[2] != ldw or out["wq"].shape != W.shape):
         raise ValueError("wq must have the shape and row stride of W")
     out["codes"] = codes_out
+    if scale_in is not None:
+        _need(scale_in, torch.float16, "scale_in", 3)
+        if clip_idx is None or tuple(scale_in.shape) != (4, U, R) or not scale_in.is_contiguous():
+            raise ValueError("scale_in must be a contiguous [4, U, R] tensor and needs clip_idx")
+        ctx._check(_lib.windq_apply_plan_refined(ctx._h, _ptr(W), R, C, ldw, int(G), _ptr(s), _ptr(clip_grid),
+                                                 clip_grid.numel(), _ptr(actions), _ptr(clip_idx), _ptr(scale_in),
+                                                 _ptr(code_offsets), _ptr(codes_out), _ptr(out["scales"]),
+                                                 _ptr(out["zeros"]), _ptr(out["wq"]), _stream(stream)))
+        return out
     ctx._check(_lib.windq_apply_plan(ctx._h, _ptr(W), R, C, ldw, int(G), _ptr(s), _ptr(clip_grid), clip_grid.numel(),
                                      _ptr(actions), _ptr(clip_idx), _ptr(code_offsets), _ptr(codes_out), _ptr(out["scales"]),
                                      _ptr(out["zeros"]), _ptr(out["wq"]), _stream(stream)))

@@ -140,6 +140,7 @@ struct ProtectArgs {
   const __half* prot_scale;        // [U] INT8 scale of the unit's protected weights
   int8_t* prot_q;                  // INT8 codes
   long long capacity;              // entries of prot_q; nothing is written at or beyond it
+  const __half* scale_in;          // [4][U][R] refined scales of the uniform groups, or NULL (any variant)
 };
 
 // Saliency mask of a lane's 32 values: bit e is set when |w_e| * scale_e >= tau.
@@ -278,6 +279,7 @@ apply_plan_kernel(const __half* __restrict__ W, int R, int U, int64_t ldw, const
       }
       float scale, zf;
       uniform_scale_zero(mn, __fsub_rn(mx, mn), __ldg(clip + k), us, scale, zf);
+      if (pa.scale_in) scale = __half2float(pa.scale_in[((int64_t)bi * U + u) * R + min(row, R - 1)]);
       quantise_uniform(raw, scale, zf, us.qmax, wq, code);
       scale_store = scale;
       zero_store = zf;
@@ -508,8 +510,9 @@ template <int G>
 windq_status launch_apply_any(windq_ctx* ctx, const __half* W, int R, int U, int64_t ldw, const float* s,
                               const float* clip, int K, const uint8_t* actions, const uint8_t* clip_idx,
                               const long long* code_offsets, uint8_t* codes_out, __half* scales_out, __half* zeros_out,
-                              __half* Wq_out, cudaStream_t st) {
-  const ProtectArgs none = {};
+                              __half* Wq_out, const __half* scale_in, cudaStream_t st) {
+  ProtectArgs none = {};
+  none.scale_in = scale_in;
   if (clip_idx)
     return launch_apply<G, false, false>(ctx, W, R, U, ldw, s, clip, K, actions, clip_idx, code_offsets, codes_out,
                                          scales_out, zeros_out, Wq_out, none, st);
@@ -554,12 +557,11 @@ windq_status launch_apply_protected(windq_ctx* ctx, const __half* W, int R, int 
 
 }  // namespace windq
 
-extern "C" windq_status windq_apply_plan(windq_ctx* ctx, const void* W, int64_t R, int64_t C, int64_t ldw, int G,
-                                         const float* s, const float* clip_grid, int K, const uint8_t* actions,
-                                         const uint8_t* clip_idx, const int64_t* code_offsets, uint8_t* codes_out,
-                                         void* scales_out, void* zeros_out, void* Wq_out, void* stream) {
+static windq_status apply_plan_plain(windq_ctx* ctx, const void* W, int64_t R, int64_t C, int64_t ldw, int G, const float* s,
+                                     const float* clip_grid, int K, const uint8_t* actions, const uint8_t* clip_idx,
+                                     const void* scale_in, const int64_t* code_offsets, uint8_t* codes_out,
+                                     void* scales_out, void* zeros_out, void* Wq_out, void* stream) {
   using namespace windq;
-  if (!ctx) return fail(nullptr, WINDQ_ERR_NULL, "windq_apply_plan: ctx is NULL");
   if (windq_status st = check_matrix(ctx, "windq_apply_plan", W, R, C, ldw, G)) return st;
   if (windq_status st = check_K(ctx, "windq_apply_plan", K)) return st;
   WINDQ_REQUIRE(ctx, s && clip_grid && actions && code_offsets && codes_out && scales_out && zeros_out, WINDQ_ERR_NULL,
@@ -576,13 +578,36 @@ extern "C" windq_status windq_apply_plan(windq_ctx* ctx, const void* W, int64_t 
   const __half* Wh = (const __half*)W;
   const long long* offs = (const long long*)code_offsets;
   __half *sc = (__half*)scales_out, *zp = (__half*)zeros_out, *wq = (__half*)Wq_out;
+  const __half* si = (const __half*)scale_in;
   switch (G) {
-    case 32: return launch_apply_any<32>(ctx, Wh, (int)R, U, ldw, s, clip_grid, K, actions, clip_idx, offs, codes_out, sc, zp, wq, st);
-    case 64: return launch_apply_any<64>(ctx, Wh, (int)R, U, ldw, s, clip_grid, K, actions, clip_idx, offs, codes_out, sc, zp, wq, st);
-    case 128: return launch_apply_any<128>(ctx, Wh, (int)R, U, ldw, s, clip_grid, K, actions, clip_idx, offs, codes_out, sc, zp, wq, st);
-    case 256: return launch_apply_any<256>(ctx, Wh, (int)R, U, ldw, s, clip_grid, K, actions, clip_idx, offs, codes_out, sc, zp, wq, st);
-    default: return launch_apply_any<512>(ctx, Wh, (int)R, U, ldw, s, clip_grid, K, actions, clip_idx, offs, codes_out, sc, zp, wq, st);
+    case 32: return launch_apply_any<32>(ctx, Wh, (int)R, U, ldw, s, clip_grid, K, actions, clip_idx, offs, codes_out, sc, zp, wq, si, st);
+    case 64: return launch_apply_any<64>(ctx, Wh, (int)R, U, ldw, s, clip_grid, K, actions, clip_idx, offs, codes_out, sc, zp, wq, si, st);
+    case 128: return launch_apply_any<128>(ctx, Wh, (int)R, U, ldw, s, clip_grid, K, actions, clip_idx, offs, codes_out, sc, zp, wq, si, st);
+    case 256: return launch_apply_any<256>(ctx, Wh, (int)R, U, ldw, s, clip_grid, K, actions, clip_idx, offs, codes_out, sc, zp, wq, si, st);
+    default: return launch_apply_any<512>(ctx, Wh, (int)R, U, ldw, s, clip_grid, K, actions, clip_idx, offs, codes_out, sc, zp, wq, si, st);
   }
+}
+
+extern "C" windq_status windq_apply_plan(windq_ctx* ctx, const void* W, int64_t R, int64_t C, int64_t ldw, int G,
+                                         const float* s, const float* clip_grid, int K, const uint8_t* actions,
+                                         const uint8_t* clip_idx, const int64_t* code_offsets, uint8_t* codes_out,
+                                         void* scales_out, void* zeros_out, void* Wq_out, void* stream) {
+  if (!ctx) return windq::fail(nullptr, WINDQ_ERR_NULL, "windq_apply_plan: ctx is NULL");
+  return apply_plan_plain(ctx, W, R, C, ldw, G, s, clip_grid, K, actions, clip_idx, nullptr, code_offsets, codes_out,
+                          scales_out, zeros_out, Wq_out, stream);
+}
+
+extern "C" windq_status windq_apply_plan_refined(windq_ctx* ctx, const void* W, int64_t R, int64_t C, int64_t ldw, int G,
+                                                 const float* s, const float* clip_grid, int K, const uint8_t* actions,
+                                                 const uint8_t* clip_idx, const void* scale_in, const int64_t* code_offsets,
+                                                 uint8_t* codes_out, void* scales_out, void* zeros_out, void* Wq_out,
+                                                 void* stream) {
+  if (!ctx) return windq::fail(nullptr, WINDQ_ERR_NULL, "windq_apply_plan_refined: ctx is NULL");
+  if (!clip_idx || !scale_in)
+    return windq::fail(ctx, WINDQ_ERR_NULL, "windq_apply_plan_refined: clip_idx or scale_in is NULL");
+  if ((uintptr_t)scale_in & 1) return windq::fail(ctx, WINDQ_ERR_ALIGN, "windq_apply_plan_refined: scale_in is misaligned");
+  return apply_plan_plain(ctx, W, R, C, ldw, G, s, clip_grid, K, actions, clip_idx, scale_in, code_offsets, codes_out,
+                          scales_out, zeros_out, Wq_out, stream);
 }
 
 extern "C" int64_t windq_scratch_bytes_apply_plan_protected(int64_t R, int64_t C, int G) {

@@ -143,3 +143,29 @@ def test_argument_checks(wq, ctx):
         wq.windq_fit_refine(ctx, W, 128, s, grid, idx[:, :, :4], 10, 0.01)
     out = wq.windq_fit_refine(ctx, W, 128, s, grid, idx, 10, 0.01)
     assert (out["err"] == 0).all()
+
+
+@pytest.mark.parametrize("R,C,G", [(37, 256, 32), (45, 512, 128), (9, 1024, 512)])
+def test_plan_applied_with_refined_scales(wq, ctx, oracle, R, C, G):
+    """Codes, scales, zero points and fake-quantised weights of a mixed plan that uses the refined scales."""
+    W, s, grid = inputs(oracle, R, C, 500 + G)
+    Wd, sd, gd = W.cuda(), torch.from_numpy(s).cuda(), torch.from_numpy(grid).cuda()
+    U = C // G
+    fit = wq.windq_fit_eval(ctx, Wd, G, sd, gd)
+    ref = wq.windq_fit_refine(ctx, Wd, G, sd, gd, fit["clip_idx"], 10, 0.03)
+    actions = (np.arange(U) % 7).astype(np.uint8)
+    ad = torch.from_numpy(actions).cuda()
+    eb = wq.windq_effective_bits(ctx, ad, R, G)
+    codes = torch.zeros(2 * R * C + 16 * U, dtype=torch.uint8, device="cuda")
+    got = wq.windq_apply_plan(ctx, Wd, G, sd, gd, ad, eb["code_offsets"], codes, fit["clip_idx"], scale_in=ref["scale"])
+    torch.cuda.synchronize()
+    want = oracle.apply_plan(W.numpy(), G, s, grid, actions, fit["clip_idx"].cpu().numpy(), scale_in=ref["scale"].cpu().numpy())
+    n = int(want["code_offsets"][U])
+    assert np.array_equal(got["codes"][:n].cpu().numpy(), want["codes"])
+    assert np.array_equal(got["scales"].cpu().numpy().view(np.uint16), want["scales"])
+    assert np.array_equal(got["zeros"].cpu().numpy().view(np.uint16), want["zeros"])
+    assert np.array_equal(got["wq"].cpu().numpy().view(np.uint16), want["wq"])
+    # the plain call is untouched by the new argument
+    plain = wq.windq_apply_plan(ctx, Wd, G, sd, gd, ad, eb["code_offsets"], codes.clone(), fit["clip_idx"])
+    want_plain = oracle.apply_plan(W.numpy(), G, s, grid, actions, fit["clip_idx"].cpu().numpy())
+    assert np.array_equal(plain["wq"].cpu().numpy().view(np.uint16), want_plain["wq"])

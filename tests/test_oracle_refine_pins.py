@@ -108,3 +108,23 @@ def test_stops_when_the_step_size_leaves_the_positive_range(oracle):
     assert len(sc) == 1                                            # Delta_1 = 1 - 1 * 1 rounds to a non-positive fp16
     sc, _, _ = oracle.refine_trace(w, np.ones(32, np.float32), 2, 1.0, 0.0, 5, 0.1)
     assert len(sc) == 6 and (np.diff(sc[:2]) < 0).all()
+
+
+def test_refined_plan_reproduces_the_refined_errors(oracle):
+    """Packing with the refined scales: the 8-bit codes, zero points and scales of the plan, decoded here,
+    give back the group errors the refinement reported."""
+    W, X = case(16, 256, 31)
+    s = oracle.act_stats(X)
+    grid = ws.clip_grid(20)
+    fit = oracle.fit_eval(W, 64, s, grid)
+    ref = oracle.fit_refine(W, 64, s, grid, fit["clip_idx"], T=10, lr=0.02)
+    plan = oracle.apply_plan(W, 64, s, grid, np.full(4, 1, np.uint8), fit["clip_idx"], scale_in=ref["scale"])
+    assert np.array_equal(plan["scales"], ref["scale"][0].view(np.uint16))
+    offs = plan["code_offsets"]
+    for u in range(4):
+        q = plan["codes"][offs[u]:offs[u] + 16 * 64].reshape(16, 64).astype(np.float64)
+        z = plan["zeros"].view(np.float16)[u].astype(np.float64)[:, None]
+        sc = plan["scales"].view(np.float16)[u].astype(np.float64)[:, None]
+        d = (q - z) * sc - W[:, u * 64:(u + 1) * 64].astype(np.float64)
+        e = (s[u * 64:(u + 1) * 64].astype(np.float64)[None, :] * d * d).sum(1)
+        np.testing.assert_allclose(e, ref["group_err"][0, u], rtol=1e-5)

@@ -53,6 +53,8 @@ def parse_args():
     ap.add_argument("--blocks", type=int, default=0, help="use only the first B blocks (0 = all; profiling aid)")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--extras", action="store_true",
+                    help="also time the calls beyond the five of a step (protection, refinement, allocator) on block 0")
     return ap.parse_args()
 
 
@@ -424,6 +426,67 @@ def run_e2e_leg(wq, ctx, spec, model, plans, plans_np, buf, grid_d, steps, warmu
 ORACLE_SAMPLE_MATRICES = 5     # block 0: q, k, v, o and gate projections (about 55 % of a block's weights)
 
 
+def run_extras(wq, ctx, spec, model, buf, grid_d, reps=3):
+    """Times, on the matrices of this rank's first block at the plan chunk width, the calls that are not part
+    of a step: saliency score, salient-weight selection at 3 %, the protected fit, the step-size refinement
+    (10 steps), packing with protection, and the heuristic allocator's rule over the units of the whole model.
+    Returns {name: milliseconds per block} (the allocator: per call)."""
+    G, mats = APPLY_G, matrices_of(spec)
+    Wb, Xb = model.W[0], model.X[0]
+    for i, X in Xb.items():
+        wq.windq_act_stats(ctx, X, buf.s[i])
+    need = max(max(wq.windq_scratch_bytes_salient_select(m.R, m.C, G), wq.windq_scratch_bytes_fit_eval_protected(m.R, m.C, G),
+                   wq.windq_scratch_bytes_apply_plan_protected(m.R, m.C, G), wq.windq_scratch_bytes_fit_refine(m.R, m.C, G))
+               for m in mats)
+    n_units_model = sum(m.C // G for m in mats) * spec.n_blocks
+    wq.windq_reserve(ctx, max(need, wq.windq_scratch_bytes_greedy_allocate(n_units_model)))
+    times = {}
+
+    def timed(name, fn):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        out = fn()
+        e1.record()
+        torch.cuda.synchronize()
+        times.setdefault(name, []).append(e0.elapsed_time(e1))
+        return out
+
+    sal_all, cnt_all, n_all, g_all = [], [], [], []
+    for rep in range(reps + 1):
+        for mi, m in enumerate(mats):
+            W, s, U = Wb[mi], buf.s[m.x_id], m.C // G
+            sal = timed("unit_saliency", lambda: wq.windq_unit_saliency(ctx, W, G, s))
+            sel = timed("salient_select", lambda: wq.windq_salient_select(ctx, W, G, s, 30000, want_mask=False))
+            fit = timed("fit_eval_protected", lambda: wq.windq_fit_eval(ctx, W, G, s, grid_d, thresh=sel["thresh"]))
+            plain = wq.windq_fit_eval(ctx, W, G, s, grid_d)
+            timed("fit_refine", lambda: wq.windq_fit_refine(ctx, W, G, s, grid_d, plain["clip_idx"], 10, 0.01))
+            acts = torch.full((U,), 4, dtype=torch.uint8, device="cuda")
+            eb = wq.windq_effective_bits(ctx, acts, m.R, G)
+            prot_q = torch.empty(int(0.04 * m.R * m.C) + 1024, dtype=torch.int8, device="cuda")
+            timed("apply_plan_protected", lambda: wq.windq_apply_plan_protected(
+                ctx, W, G, s, grid_d, acts, eb["code_offsets"], buf.take("codes"), sel["thresh"], prot_q, fit["clip_idx"]))
+            if rep == 0:
+                sal_all.append(sal)
+                cnt_all.append(sel["count"])
+                n_all.append(torch.full((U,), m.R * G, dtype=torch.int64, device="cuda"))
+                g_all.append(torch.full((U,), m.R, dtype=torch.int64, device="cuda"))
+    n_rep = spec.n_blocks
+    sal_m, cnt_m = torch.cat(sal_all).repeat(n_rep), torch.cat(cnt_all).repeat(n_rep)
+    n_m, g_m = torch.cat(n_all).repeat(n_rep), torch.cat(g_all).repeat(n_rep)
+    sal_m = (sal_m * (1.0 + 0.001 * torch.arange(sal_m.numel(), device="cuda") / sal_m.numel())).contiguous()
+    for rep in range(reps + 1):
+        timed("greedy_allocate", lambda: wq.windq_greedy_allocate(ctx, sal_m, n_m, g_m, 200, 10, cnt_m, scale_bits=16, zero_bits=16))
+    out = {}
+    for name, ts in times.items():
+        per_rep = len(ts) // (reps + 1)
+        kept = ts[per_rep:]                                   # the first repetition is the warm-up
+        out[name + "_ms"] = sum(kept) / reps
+    out["chunk_width"] = G
+    out["allocator_units"] = int(sal_m.numel())
+    out["note"] = "per block (7 matrices), except greedy_allocate: one call over the model's units"
+    return out
+
+
 def oracle_sample(spec, seed, threads):
     """The CPU oracle on a bounded sample of the workload: the whole hot path for the first
     ORACLE_SAMPLE_MATRICES matrices of block 0 -- their calibration statistics, and per matrix
@@ -574,6 +637,10 @@ def main():
                    d2h_bytes_per_step=d2h, steps=e_steps, ms_per_step=e_ms / e_steps,
                    host_blocks_resident=host_blocks)
 
+    extras = None
+    if args.extras and rank == 0:
+        extras = run_extras(wq, ctx, spec, model, Buffers(spec), grid_d)
+
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         threads = os.cpu_count() or 1
@@ -591,6 +658,8 @@ def main():
                                     (2 * elems + 2 * spec.T * sum(c for _, c in inputs_of(spec)) * n_blocks) / 1e9)),
                     clocks=clocks, e2e=e2e, gpu_launches=launches, roofline=roofline, cpu_baseline=cpu,
                     fit_eval_ms_per_step=fit_ms / args.steps, plan_total_centibits_last=total_cb)
+        if extras:
+            line["extras"] = extras
         print(json.dumps(line))
     wq.windq_destroy(ctx)
     if world > 1:

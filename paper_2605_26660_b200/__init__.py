@@ -337,6 +337,22 @@ def windq_apply_plan(ctx: Context, W: torch.Tensor, G: int, s: torch.Tensor, cli
     return out
 
 
+def windq_scratch_bytes_fit_eval_protected(R: int, C: int, G: int) -> int:
+    return int(_lib.windq_scratch_bytes_fit_eval_protected(R, C, G))
+
+
+def windq_scratch_bytes_apply_plan_protected(R: int, C: int, G: int) -> int:
+    return int(_lib.windq_scratch_bytes_apply_plan_protected(R, C, G))
+
+
+def windq_scratch_bytes_fit_refine(R: int, C: int, G: int) -> int:
+    return int(_lib.windq_scratch_bytes_fit_refine(R, C, G))
+
+
+def windq_scratch_bytes_greedy_allocate(U: int) -> int:
+    return int(_lib.windq_scratch_bytes_greedy_allocate(U))
+
+
 def windq_scratch_bytes_salient_select(R: int, C: int, G: int) -> int:
     return int(_lib.windq_scratch_bytes_salient_select(R, C, G))
 

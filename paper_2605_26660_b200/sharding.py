@@ -4,7 +4,9 @@ Units, matrices and blocks are independent, so the path shards with no exchange 
 ranks: every rank scores its own contiguous range of decoder blocks.  The only cross-rank
 values are scalars on the control path -- the plan's total bits (an int64 sum) and the step time
 (a max) -- reduced with torch.distributed on whatever backend the process group uses (NCCL on
-GPUs, gloo in the CPU tests).
+GPUs, gloo in the CPU tests).  The one call that looks at all units at once is the heuristic
+allocator's rule: for it the ranks exchange their units' scores and counts (a few bytes per unit,
+`gather_units`), every rank runs the rule on the same gathered arrays and keeps its own slice.
 """
 from __future__ import annotations
 
@@ -46,3 +48,45 @@ def max_float(value: float) -> float:
 def average_bits(total_centibits: int, n_weights: int) -> float:
     """b_bar = sum B_i / sum n_i over all ranks (Eq. 6), from per-rank totals."""
     return sum_int64(total_centibits) / (100.0 * sum_int64(n_weights))
+
+
+def gather_units(*arrays: torch.Tensor):
+    """All-gathers per-unit 1-D tensors of the same length (scores, weight counts, ...) in rank order.
+
+    Ranks may hold different numbers of units.  Returns (gathered tensors, begin, end): every rank gets the
+    same concatenation, and [begin, end) is where this rank's units sit in it.  Without a process group the
+    inputs come back unchanged."""
+    n = int(arrays[0].numel())
+    for a in arrays:
+        if a.dim() != 1 or a.numel() != n:
+            raise ValueError("gather_units wants 1-D tensors of one length")
+    if not (dist.is_available() and dist.is_initialized()):
+        return list(arrays), 0, n
+    world, rank = dist.get_world_size(), dist.get_rank()
+    counts = torch.zeros(world, dtype=torch.int64, device=arrays[0].device)
+    counts[rank] = n
+    dist.all_reduce(counts, op=dist.ReduceOp.SUM)
+    counts = [int(c) for c in counts.tolist()]
+    width = max(counts)
+    out = []
+    for a in arrays:
+        padded = torch.zeros(width, dtype=a.dtype, device=a.device)
+        padded[:n] = a
+        parts = [torch.empty_like(padded) for _ in range(world)]
+        dist.all_gather(parts, padded)
+        out.append(torch.cat([p[:c] for p, c in zip(parts, counts)]))
+    begin = sum(counts[:rank])
+    return out, begin, begin + n
+
+
+def allocate_across_ranks(allocate, saliency, n_weights, n_groups, n_protected=None):
+    """The heuristic allocator's rule over the units of all ranks.  `allocate(saliency, n_weights, n_groups,
+    n_protected)` is the rule on whole-model arrays (e.g. a closure over windq_greedy_allocate with the
+    target and headroom) and returns a dict with `actions` and `total_centibits`; every rank calls it on the
+    same gathered arrays, so all ranks hold the same plan.  Returns (this rank's actions, total centibits of
+    the model)."""
+    has_p = n_protected is not None
+    arrays = [saliency, n_weights, n_groups] + ([n_protected] if has_p else [])
+    gathered, begin, end = gather_units(*arrays)
+    res = allocate(gathered[0], gathered[1], gathered[2], gathered[3] if has_p else None)
+    return res["actions"][begin:end], int(res["total_centibits"])

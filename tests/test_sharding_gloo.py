@@ -95,3 +95,63 @@ def test_two_gloo_ranks_agree_with_one_process(tmp_path, oracle):
         assert g[2] == 10.0 + (world - 1)            # step time = slowest rank
     assert sum(int(g[3]) for g in got) == N_BLOCKS   # every block scored exactly once
     assert int(got[0][5]) + 1 == int(got[1][4])      # contiguous, disjoint ranges
+
+
+# ---- the allocator's rule over units that live on different ranks ------------------------------------
+def _rank_units(rank):
+    rng = np.random.default_rng(50 + rank)
+    U = 40 + 13 * rank                                   # ranks hold different numbers of units
+    g = rng.integers(8, 200, U)
+    n = g * rng.choice([32, 64, 128], U)
+    p = (n * 0.03).astype(np.int64)
+    sal = rng.choice(rng.random(12).astype(np.float32), U)   # equal scores across ranks: ties by global index
+    return sal, n, g, p
+
+
+def _oracle_rule(oracle):
+    def rule(sal, n, g, p):
+        actions, _, total = oracle.greedy_allocate(sal.numpy(), n.numpy(), g.numpy(), 200, 10, n_protected=p.numpy(),
+                                                   scale_bits=16, zero_bits=8)
+        return dict(actions=torch.from_numpy(actions), total_centibits=total)
+    return rule
+
+
+def _alloc_worker(rank, world, port, out_dir):
+    sys.path.insert(0, ROOT)
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        sharding = _load_sharding()
+        import oracle
+        oracle.build()
+        sal, n, g, p = (torch.from_numpy(a) for a in _rank_units(rank))
+        actions, total = sharding.allocate_across_ranks(_oracle_rule(oracle), sal, n, g, p)
+        np.save(os.path.join(out_dir, "alloc%d.npy" % rank), np.concatenate([[total], actions.numpy().astype(np.int64)]))
+    finally:
+        dist.destroy_process_group()
+
+
+def test_allocator_rule_over_two_ranks_equals_one_process(tmp_path, oracle):
+    world = 2
+    mp.start_processes(_alloc_worker, args=(world, _free_port(), str(tmp_path)), nprocs=world, join=True, start_method="spawn")
+    parts = [_rank_units(r) for r in range(world)]
+    sal, n, g, p = (np.concatenate([q[i] for q in parts]) for i in range(4))
+    want, _, want_total = oracle.greedy_allocate(sal, n, g, 200, 10, n_protected=p, scale_bits=16, zero_bits=8)
+    pos = 0
+    for r in range(world):
+        got = np.load(os.path.join(str(tmp_path), "alloc%d.npy" % r))
+        U = parts[r][0].size
+        assert int(got[0]) == want_total
+        assert np.array_equal(got[1:], want[pos:pos + U].astype(np.int64))
+        pos += U
+    assert {2, 3, 4, 5} & set(want.tolist())
+
+
+def test_gather_units_without_a_process_group():
+    sh = _load_sharding()
+    a, b = torch.arange(5, dtype=torch.float32), torch.arange(5, dtype=torch.int64)
+    (ga, gb), lo, hi = sh.gather_units(a, b)
+    assert torch.equal(ga, a) and torch.equal(gb, b) and (lo, hi) == (0, 5)
+    with pytest.raises(ValueError):
+        sh.gather_units(a, b[:3])

@@ -198,16 +198,25 @@ def apply_plan(W, G: int, s, clip_grid, actions, clip_idx=None, want_wq: bool = 
         prot_scale = np.zeros(U, np.uint16)
         prot_offsets = np.zeros(U + 1, np.int64)
         prot_q = np.zeros(R * C, np.int8)
-        rc = lib().oracle_apply_plan_protected(_p(W), ctypes.c_int64(R), ctypes.c_int64(C), ctypes.c_int64(C), ctypes.c_int(G),
-                                               _p(s), _p(clip_grid), ctypes.c_int(clip_grid.size), _p(actions), _p(clip_idx),
-                                               _p(offs), _p(thresh), _p(codes), _p(scales), _p(zeros), _p(wq),
-                                               _p(prot_scale), _p(prot_offsets), _p(prot_q))
+        if scale_in is not None:
+            assert clip_idx is not None
+            scale_in = _as_u16(scale_in)
+            assert scale_in.shape == (4, U, R)
+            rc = lib().oracle_apply_plan_protected_refined(
+                _p(W), ctypes.c_int64(R), ctypes.c_int64(C), ctypes.c_int64(C), ctypes.c_int(G), _p(s), _p(clip_grid),
+                ctypes.c_int(clip_grid.size), _p(actions), _p(clip_idx), _p(scale_in), _p(offs), _p(thresh), _p(codes),
+                _p(scales), _p(zeros), _p(wq), _p(prot_scale), _p(prot_offsets), _p(prot_q))
+        else:
+            rc = lib().oracle_apply_plan_protected(_p(W), ctypes.c_int64(R), ctypes.c_int64(C), ctypes.c_int64(C), ctypes.c_int(G),
+                                                   _p(s), _p(clip_grid), ctypes.c_int(clip_grid.size), _p(actions), _p(clip_idx),
+                                                   _p(offs), _p(thresh), _p(codes), _p(scales), _p(zeros), _p(wq),
+                                                   _p(prot_scale), _p(prot_offsets), _p(prot_q))
         if rc:
             raise ValueError("oracle_apply_plan_protected: bad arguments")
         return dict(codes=codes, scales=scales, zeros=zeros, wq=wq, code_offsets=offs, prot_scale=prot_scale,
                     prot_offsets=prot_offsets, prot_q=prot_q[:int(prot_offsets[U])].copy())
     if scale_in is not None:
-        assert thresh is None and clip_idx is not None
+        assert clip_idx is not None
         scale_in = _as_u16(scale_in)
         assert scale_in.shape == (4, U, R)
         rc = lib().oracle_apply_plan_refined(_p(W), ctypes.c_int64(R), ctypes.c_int64(C), ctypes.c_int64(C), ctypes.c_int(G),
@@ -315,8 +324,9 @@ def refine_trace(w, s, bits: int, scale0: float, zf: float, T: int, lr: float):
     return sc[:n], lo[:n], gr[:n]
 
 
-def fit_refine(W, G: int, s, clip_grid, clip_idx, T: int = 10, lr: float = 0.01):
+def fit_refine(W, G: int, s, clip_grid, clip_idx, T: int = 10, lr: float = 0.01, thresh=None):
     """Step-size refinement of the four uniform fits, warm-started from clip_idx [4][U][R] of fit_eval.
+    With ``thresh`` (fp32 [U]) the salient weights are left out of the groups as in the protected fit.
     Returns dict(err [U][4] f32, scale [4][U][R] f16, group_err [4][U][R] f32)."""
     W, s, clip_grid = _as_u16(W), _f32(s), _f32(clip_grid)
     R, C = W.shape
@@ -326,9 +336,17 @@ def fit_refine(W, G: int, s, clip_grid, clip_idx, T: int = 10, lr: float = 0.01)
     err = np.zeros((U, 4), np.float32)
     scale = np.zeros((4, U, R), np.uint16)
     gerr = np.zeros((4, U, R), np.float32)
-    rc = lib().oracle_fit_refine(_p(W), ctypes.c_int64(R), ctypes.c_int64(C), ctypes.c_int64(W.strides[0] // 2),
-                                 ctypes.c_int(G), _p(s), _p(clip_grid), ctypes.c_int(clip_grid.size), _p(clip_idx),
-                                 ctypes.c_int(T), ctypes.c_float(lr), _p(err), _p(scale), _p(gerr))
+    if thresh is not None:
+        thresh = _f32(thresh)
+        assert thresh.size == U
+        rc = lib().oracle_fit_refine_protected(_p(W), ctypes.c_int64(R), ctypes.c_int64(C), ctypes.c_int64(W.strides[0] // 2),
+                                               ctypes.c_int(G), _p(s), _p(clip_grid), ctypes.c_int(clip_grid.size),
+                                               _p(clip_idx), _p(thresh), ctypes.c_int(T), ctypes.c_float(lr), _p(err),
+                                               _p(scale), _p(gerr))
+    else:
+        rc = lib().oracle_fit_refine(_p(W), ctypes.c_int64(R), ctypes.c_int64(C), ctypes.c_int64(W.strides[0] // 2),
+                                     ctypes.c_int(G), _p(s), _p(clip_grid), ctypes.c_int(clip_grid.size), _p(clip_idx),
+                                     ctypes.c_int(T), ctypes.c_float(lr), _p(err), _p(scale), _p(gerr))
     if rc:
         raise ValueError("oracle_fit_refine: bad arguments (%d)" % rc)
     return dict(err=err, scale=scale.view(np.float16), group_err=gerr)

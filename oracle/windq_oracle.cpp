@@ -665,6 +665,17 @@ int oracle_apply_plan_protected(const uint16_t* W, int64_t R, int64_t C, int64_t
                          scales_out, zeros_out, Wq_out, prot_scale_out, prot_offsets_out, prot_q_out);
 }
 
+// Protection and refined step sizes together (scale_in from oracle_fit_refine_protected; needs clip_idx).
+int oracle_apply_plan_protected_refined(const uint16_t* W, int64_t R, int64_t C, int64_t ldw, int G, const float* s,
+                                        const float* clip_grid, int K, const uint8_t* actions, const uint8_t* clip_idx,
+                                        const uint16_t* scale_in, const int64_t* code_offsets, const float* thresh,
+                                        uint8_t* codes_out, uint16_t* scales_out, uint16_t* zeros_out, uint16_t* Wq_out,
+                                        uint16_t* prot_scale_out, int64_t* prot_offsets_out, int8_t* prot_q_out) {
+  if (!thresh || !clip_idx || !scale_in) return 1;
+  return apply_plan_impl(W, R, C, ldw, G, s, clip_grid, K, actions, clip_idx, code_offsets, thresh, codes_out,
+                         scales_out, zeros_out, Wq_out, prot_scale_out, prot_offsets_out, prot_q_out, scale_in);
+}
+
 // ---- salient-weight selection (App. "Salient Weight Protection") -----------------------------
 // The saliency of a weight is the product of its magnitude and the activation scale of its input
 // channel; the top-r fraction of a unit's weights by saliency is kept in INT8.
@@ -969,19 +980,28 @@ int oracle_refine_trace(const float* w, const float* s, int G, int bits, float s
 // Refinement of every group's step size for the four uniform bit-widths, warm-started from the clip
 // indices of oracle_fit_eval.  err_out [U][4] (unit sums in double, rows ascending), scale_out fp16
 // bits [4][U][R], group_err_out [4][U][R] (nullable).
-int oracle_fit_refine(const uint16_t* W, int64_t R, int64_t C, int64_t ldw, int G, const float* s,
-                      const float* clip_grid, int K, const uint8_t* clip_idx, int T, float lr, float* err_out,
-                      uint16_t* scale_out, float* group_err_out) {
+static int fit_refine_impl(const uint16_t* W, int64_t R, int64_t C, int64_t ldw, int G, const float* s,
+                           const float* clip_grid, int K, const uint8_t* clip_idx, const float* thresh, int T, float lr,
+                           float* err_out, uint16_t* scale_out, float* group_err_out) {
   if (!W || !s || !clip_grid || !clip_idx || !err_out || !scale_out || R <= 0 || C <= 0 || !valid_group_width(G) ||
       C % G != 0 || ldw < C || K < 1 || K > 64 || T < 0 || T > 32 || !(lr >= 0.0f))
     return 1;
   const int64_t U = C / G;
-  std::vector<float> w((size_t)G);
+  std::vector<float> w((size_t)G), sm((size_t)G);
   for (int64_t u = 0; u < U; ++u) {
     double tot[4] = {0, 0, 0, 0};
     for (int64_t r = 0; r < R; ++r) {
       load_group(W, ldw, r, u, G, w.data());
-      Group g{G, w.data(), s + u * G};
+      const float* su = s + u * G;
+      if (thresh) {  // protected weights leave the group as in the protected fit: zero weight, zero activation weight
+        for (int j = 0; j < G; ++j) {
+          const bool prot = std::fabs(w[(size_t)j]) * std::sqrt(s[u * G + j]) >= thresh[u];
+          sm[(size_t)j] = prot ? 0.0f : s[u * G + j];
+          if (prot) w[(size_t)j] = 0.0f;
+        }
+        su = sm.data();
+      }
+      Group g{G, w.data(), su};
       float mn, rng;
       group_range(g, &mn, &rng);
       for (int bi = 0; bi < 4; ++bi) {
@@ -1000,6 +1020,21 @@ int oracle_fit_refine(const uint16_t* W, int64_t R, int64_t C, int64_t ldw, int 
     for (int bi = 0; bi < 4; ++bi) err_out[u * 4 + bi] = (float)tot[bi];
   }
   return 0;
+}
+
+int oracle_fit_refine(const uint16_t* W, int64_t R, int64_t C, int64_t ldw, int G, const float* s,
+                      const float* clip_grid, int K, const uint8_t* clip_idx, int T, float lr, float* err_out,
+                      uint16_t* scale_out, float* group_err_out) {
+  return fit_refine_impl(W, R, C, ldw, G, s, clip_grid, K, clip_idx, nullptr, T, lr, err_out, scale_out, group_err_out);
+}
+
+// The refinement with the salient weights taken out of the groups (thresh [U] from oracle_salient_select,
+// clip_idx from oracle_fit_eval_protected with the same thresholds).
+int oracle_fit_refine_protected(const uint16_t* W, int64_t R, int64_t C, int64_t ldw, int G, const float* s,
+                                const float* clip_grid, int K, const uint8_t* clip_idx, const float* thresh, int T,
+                                float lr, float* err_out, uint16_t* scale_out, float* group_err_out) {
+  if (!thresh) return 1;
+  return fit_refine_impl(W, R, C, ldw, G, s, clip_grid, K, clip_idx, thresh, T, lr, err_out, scale_out, group_err_out);
 }
 
 }  // extern "C"

@@ -128,3 +128,34 @@ def test_refined_plan_reproduces_the_refined_errors(oracle):
         d = (q - z) * sc - W[:, u * 64:(u + 1) * 64].astype(np.float64)
         e = (s[u * 64:(u + 1) * 64].astype(np.float64)[None, :] * d * d).sum(1)
         np.testing.assert_allclose(e, ref["group_err"][0, u], rtol=1e-5)
+
+
+def test_protected_refinement_reduces_to_its_parts(oracle):
+    """With the salient weights taken out: no steps give the protected fit; thresholds of +infinity give the
+    plain refinement; the packed 8-bit plan decodes to the refined errors over the unprotected weights."""
+    W, X = case(16, 256, 51)
+    s = oracle.act_stats(X)
+    grid = ws.clip_grid(20)
+    sel = oracle.salient_select(W, 64, s, 30000)
+    fitp = oracle.fit_eval(W, 64, s, grid, thresh=sel["thresh"])
+    r0 = oracle.fit_refine(W, 64, s, grid, fitp["clip_idx"], T=0, thresh=sel["thresh"])
+    assert np.array_equal(r0["group_err"], fitp["group_err"][:4])
+    fit = oracle.fit_eval(W, 64, s, grid)
+    a = oracle.fit_refine(W, 64, s, grid, fit["clip_idx"], T=10, lr=0.02)
+    b = oracle.fit_refine(W, 64, s, grid, fit["clip_idx"], T=10, lr=0.02, thresh=np.full(4, np.inf, np.float32))
+    assert np.array_equal(a["scale"].view(np.uint16), b["scale"].view(np.uint16))
+    assert np.array_equal(a["group_err"], b["group_err"])
+    r = oracle.fit_refine(W, 64, s, grid, fitp["clip_idx"], T=10, lr=0.02, thresh=sel["thresh"])
+    assert (r["group_err"] <= fitp["group_err"][:4]).all()
+    plan = oracle.apply_plan(W, 64, s, grid, np.full(4, 1, np.uint8), fitp["clip_idx"], thresh=sel["thresh"], scale_in=r["scale"])
+    assert plan["prot_q"].size == int(sel["count"].sum())
+    mask = np.unpackbits(sel["mask"], axis=1, bitorder="little")[:, :256].astype(bool)
+    offs = plan["code_offsets"]
+    for u in range(4):
+        q = plan["codes"][offs[u]:offs[u] + 16 * 64].reshape(16, 64).astype(np.float64)
+        z = plan["zeros"].view(np.float16)[u].astype(np.float64)[:, None]
+        sc = plan["scales"].view(np.float16)[u].astype(np.float64)[:, None]
+        keep = ~mask[:, u * 64:(u + 1) * 64]
+        d = ((q - z) * sc - W[:, u * 64:(u + 1) * 64].astype(np.float64)) * keep
+        e = (s[u * 64:(u + 1) * 64].astype(np.float64)[None, :] * d * d).sum(1)
+        np.testing.assert_allclose(e, r["group_err"][0, u], rtol=1e-5, atol=1e-12)

@@ -277,6 +277,14 @@ windq_status windq_fit_refine(windq_ctx* ctx, const void* W, int64_t R, int64_t 
                               const float* clip_grid, int K, const uint8_t* clip_idx, int n_steps, float lr,
                               float* err_out, void* scale_out, float* group_err_out, void* stream);
 
+/* windq_fit_refine with the salient weights taken out of the groups, as in windq_fit_eval_protected:
+ * thresh fp32 [U] from windq_salient_select, clip_idx from windq_fit_eval_protected with the same thresholds.
+ * With every threshold +infinity the results are those of windq_fit_refine, bit for bit.  Same scratch size. */
+windq_status windq_fit_refine_protected(windq_ctx* ctx, const void* W, int64_t R, int64_t C, int64_t ldw, int G,
+                                        const float* s, const float* clip_grid, int K, const uint8_t* clip_idx,
+                                        const float* thresh, int n_steps, float lr, float* err_out, void* scale_out,
+                                        float* group_err_out, void* stream);
+
 /* windq_apply_plan with the refined step sizes: the scale of every 8/4/3/2-bit group is scale_in
  * (fp16 [4][U][R], device, from windq_fit_refine); its zero point is that of the clip-grid fit clip_idx
  * names (required here).  Everything else as windq_apply_plan; scales_out repeats the scales used. */
@@ -284,6 +292,15 @@ windq_status windq_apply_plan_refined(windq_ctx* ctx, const void* W, int64_t R, 
                                       const float* s, const float* clip_grid, int K, const uint8_t* actions,
                                       const uint8_t* clip_idx, const void* scale_in, const int64_t* code_offsets,
                                       uint8_t* codes_out, void* scales_out, void* zeros_out, void* Wq_out, void* stream);
+
+/* windq_apply_plan_protected with the refined step sizes of windq_fit_refine_protected (scale_in fp16
+ * [4][U][R], device; clip_idx required).  Everything else as windq_apply_plan_protected. */
+windq_status windq_apply_plan_protected_refined(windq_ctx* ctx, const void* W, int64_t R, int64_t C, int64_t ldw, int G,
+                                                const float* s, const float* clip_grid, int K, const uint8_t* actions,
+                                                const uint8_t* clip_idx, const void* scale_in, const int64_t* code_offsets,
+                                                const float* thresh, uint8_t* codes_out, void* scales_out, void* zeros_out,
+                                                void* Wq_out, void* prot_scale_out, int64_t* prot_offsets_out,
+                                                int8_t* prot_q_out, int64_t prot_q_capacity, void* stream);
 
 /* The deterministic rule of the paper's heuristic allocator ("Comparison with Heuristic Sensitivity
  * Allocator": units ranked by saliency; all start at 2 bit; the least sensitive are pushed to 1.58 or

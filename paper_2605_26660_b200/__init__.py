@@ -68,6 +68,8 @@ def _load() -> ctypes.CDLL:
     lib.windq_unit_saliency.argtypes = [vp, vp, i64, i64, i64, i32, vp, vp, vp]
     lib.windq_fallback.argtypes = [vp, vp, vp, vp, i64, ctypes.c_float, vp, vp, vp]
     lib.windq_apply_plan_refined.argtypes = [vp, vp, i64, i64, i64, i32, vp, vp, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.windq_apply_plan_protected_refined.argtypes = [vp, vp, i64, i64, i64, i32, vp, vp, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, i64, vp]
+    lib.windq_fit_refine_protected.argtypes = [vp, vp, i64, i64, i64, i32, vp, vp, i32, vp, vp, i32, ctypes.c_float, vp, vp, vp, vp]
     lib.windq_fit_refine.argtypes = [vp, vp, i64, i64, i64, i32, vp, vp, i32, vp, i32, ctypes.c_float, vp, vp, vp, vp]
     lib.windq_scratch_bytes_fit_refine.restype = i64
     lib.windq_scratch_bytes_fit_refine.argtypes = [i64, i64, i32]
@@ -244,9 +246,10 @@ def windq_fit_eval(ctx: Context, W: torch.Tensor, G: int, s: torch.Tensor, clip_
 
 def windq_fit_refine(ctx: Context, W: torch.Tensor, G: int, s: torch.Tensor, clip_grid: torch.Tensor,
                      clip_idx: torch.Tensor, n_steps: int = 10, lr: float = 0.01, *, want_group_err: bool = False,
-                     stream=None) -> dict:
+                     stream=None, thresh: torch.Tensor | None = None) -> dict:
     """Refines the step sizes of the four uniform fits by ``n_steps`` Adam steps, warm-started from ``clip_idx``
-    ([4, U, R] u8 of windq_fit_eval).  Returns dict(err [U,4] f32, scale [4,U,R] f16, group_err [4,U,R] f32 | None)."""
+    ([4, U, R] u8 of windq_fit_eval).  With ``thresh`` (fp32 [U]) the salient weights are left out of the groups
+    (windq_fit_refine_protected; clip_idx then comes from the protected fit).  Returns dict(err [U,4] f32, scale [4,U,R] f16, group_err [4,U,R] f32 | None)."""
     R, C, ldw = _matrix(W, "W")
     _need(s, torch.float32, "s", 1)
     _need(clip_grid, torch.float32, "clip_grid", 1)
@@ -258,6 +261,15 @@ def windq_fit_refine(ctx: Context, W: torch.Tensor, G: int, s: torch.Tensor, cli
     out = dict(err=torch.empty((U, 4), dtype=torch.float32, device=dev),
                scale=torch.empty((4, U, R), dtype=torch.float16, device=dev),
                group_err=torch.empty((4, U, R), dtype=torch.float32, device=dev) if want_group_err else None)
+    if thresh is not None:
+        _need(thresh, torch.float32, "thresh", 1)
+        if thresh.numel() != U:
+            raise ValueError("thresh must have one entry per unit")
+        ctx._check(_lib.windq_fit_refine_protected(ctx._h, _ptr(W), R, C, ldw, int(G), _ptr(s), _ptr(clip_grid),
+                                                   clip_grid.numel(), _ptr(clip_idx), _ptr(thresh), int(n_steps), float(lr),
+                                                   _ptr(out["err"]), _ptr(out["scale"]), _ptr(out["group_err"]),
+                                                   _stream(stream)))
+        return out
     ctx._check(_lib.windq_fit_refine(ctx._h, _ptr(W), R, C, ldw, int(G), _ptr(s), _ptr(clip_grid), clip_grid.numel(),
                                      _ptr(clip_idx), int(n_steps), float(lr), _ptr(out["err"]), _ptr(out["scale"]),
                                      _ptr(out["group_err"]), _stream(stream)))
@@ -452,7 +464,7 @@ def windq_greedy_allocate(ctx: Context, saliency: torch.Tensor, n_weights: torch
 def windq_apply_plan_protected(ctx: Context, W: torch.Tensor, G: int, s: torch.Tensor, clip_grid: torch.Tensor,
                                actions: torch.Tensor, code_offsets: torch.Tensor, codes_out: torch.Tensor,
                                thresh: torch.Tensor, prot_q_out: torch.Tensor, clip_idx: torch.Tensor | None = None, *,
-                               want_wq: bool = True, stream=None) -> dict:
+                               want_wq: bool = True, stream=None, scale_in: torch.Tensor | None = None) -> dict:
     """windq_apply_plan with the salient weights (key >= thresh[u]) kept on an INT8 grid per unit.
     ``prot_q_out`` is an int8 tensor sized by the caller (sum of the counts of windq_salient_select is enough).
 
@@ -473,6 +485,16 @@ def windq_apply_plan_protected(ctx: Context, W: torch.Tensor, G: int, s: torch.T
                wq=torch.empty_strided((R, C), (ldw, 1), dtype=torch.float16, device=dev) if want_wq else None,
                prot_scale=torch.empty(U, dtype=torch.float16, device=dev),
                prot_offsets=torch.empty(U + 1, dtype=torch.int64, device=dev), prot_q=prot_q_out)
+    if scale_in is not None:
+        _need(scale_in, torch.float16, "scale_in", 3)
+        if clip_idx is None or tuple(scale_in.shape) != (4, U, R) or not scale_in.is_contiguous():
+            raise ValueError("scale_in must be a contiguous [4, U, R] tensor and needs clip_idx")
+        ctx._check(_lib.windq_apply_plan_protected_refined(
+            ctx._h, _ptr(W), R, C, ldw, int(G), _ptr(s), _ptr(clip_grid), clip_grid.numel(), _ptr(actions), _ptr(clip_idx),
+            _ptr(scale_in), _ptr(code_offsets), _ptr(thresh), _ptr(codes_out), _ptr(out["scales"]), _ptr(out["zeros"]),
+            _ptr(out["wq"]), _ptr(out["prot_scale"]), _ptr(out["prot_offsets"]), _ptr(prot_q_out), prot_q_out.numel(),
+            _stream(stream)))
+        return out
     ctx._check(_lib.windq_apply_plan_protected(ctx._h, _ptr(W), R, C, ldw, int(G), _ptr(s), _ptr(clip_grid), clip_grid.numel(),
                                                _ptr(actions), _ptr(clip_idx), _ptr(code_offsets), _ptr(thresh), _ptr(codes_out),
                                                _ptr(out["scales"]), _ptr(out["zeros"]), _ptr(out["wq"]), _ptr(out["prot_scale"]),

@@ -525,7 +525,8 @@ windq_status launch_apply_protected(windq_ctx* ctx, const __half* W, int R, int 
                                     const float* clip, int K, const uint8_t* actions, const uint8_t* clip_idx,
                                     const long long* code_offsets, const float* thresh, uint8_t* codes_out,
                                     __half* scales_out, __half* zeros_out, __half* Wq_out, __half* prot_scale_out,
-                                    long long* prot_offsets_out, int8_t* prot_q_out, long long capacity, cudaStream_t st) {
+                                    long long* prot_offsets_out, int8_t* prot_q_out, long long capacity,
+                                    const __half* scale_in, cudaStream_t st) {
   constexpr int GPW = Map<G>::GPW;
   const int C = U * G;
   // scratch: sqrt(s) [C] | row counts / offsets [U][R] | unit totals [U] | unit maxima [U]
@@ -547,7 +548,7 @@ windq_status launch_apply_protected(windq_ctx* ctx, const __half* W, int R, int 
   protect_unit_scan_kernel<<<(unsigned)((U + 255) / 256), 256, 0, st>>>(unit_total, unit_max, actions, U, prot_offsets_out,
                                                                        prot_scale_out);
   WINDQ_CUDA(ctx, cudaGetLastError());
-  const ProtectArgs pa = {scale, thresh, row_cnt, prot_offsets_out, prot_scale_out, prot_q_out, capacity};
+  const ProtectArgs pa = {scale, thresh, row_cnt, prot_offsets_out, prot_scale_out, prot_q_out, capacity, scale_in};
   if (clip_idx)
     return launch_apply<G, false, true>(ctx, W, R, U, ldw, s, clip, K, actions, clip_idx, code_offsets, codes_out, scales_out,
                                         zeros_out, Wq_out, pa, st);
@@ -616,14 +617,13 @@ extern "C" int64_t windq_scratch_bytes_apply_plan_protected(int64_t R, int64_t C
   return windq::round_up(C * 4, 16) + (U * R + 2 * U) * (int64_t)sizeof(unsigned int);
 }
 
-extern "C" windq_status windq_apply_plan_protected(windq_ctx* ctx, const void* W, int64_t R, int64_t C, int64_t ldw, int G,
-                                                   const float* s, const float* clip_grid, int K, const uint8_t* actions,
-                                                   const uint8_t* clip_idx, const int64_t* code_offsets, const float* thresh,
-                                                   uint8_t* codes_out, void* scales_out, void* zeros_out, void* Wq_out,
-                                                   void* prot_scale_out, int64_t* prot_offsets_out, int8_t* prot_q_out,
-                                                   int64_t prot_q_capacity, void* stream) {
+static windq_status apply_plan_protected_any(windq_ctx* ctx, const char* who, const void* W, int64_t R, int64_t C, int64_t ldw,
+                                             int G, const float* s, const float* clip_grid, int K, const uint8_t* actions,
+                                             const uint8_t* clip_idx, const void* scale_in, const int64_t* code_offsets,
+                                             const float* thresh, uint8_t* codes_out, void* scales_out, void* zeros_out,
+                                             void* Wq_out, void* prot_scale_out, int64_t* prot_offsets_out,
+                                             int8_t* prot_q_out, int64_t prot_q_capacity, void* stream) {
   using namespace windq;
-  const char* who = "windq_apply_plan_protected";
   if (!ctx) return fail(nullptr, WINDQ_ERR_NULL, "%s: ctx is NULL", who);
   if (windq_status st = check_matrix(ctx, who, W, R, C, ldw, G)) return st;
   if (windq_status st = check_K(ctx, who, K)) return st;
@@ -649,7 +649,7 @@ extern "C" windq_status windq_apply_plan_protected(windq_ctx* ctx, const void* W
 #define WINDQ_APPLY_CASE(GG)                                                                                             \
   case GG:                                                                                                               \
     return launch_apply_protected<GG>(ctx, Wh, (int)R, U, ldw, s, clip_grid, K, actions, clip_idx, offs, thresh, codes_out, \
-                                      sc, zp, wq, ps, po, prot_q_out, (long long)prot_q_capacity, st);
+                                      sc, zp, wq, ps, po, prot_q_out, (long long)prot_q_capacity, (const __half*)scale_in, st);
   switch (G) {
     WINDQ_APPLY_CASE(32)
     WINDQ_APPLY_CASE(64)
@@ -659,4 +659,32 @@ extern "C" windq_status windq_apply_plan_protected(windq_ctx* ctx, const void* W
       WINDQ_APPLY_CASE(512)
   }
 #undef WINDQ_APPLY_CASE
+}
+
+extern "C" windq_status windq_apply_plan_protected(windq_ctx* ctx, const void* W, int64_t R, int64_t C, int64_t ldw, int G,
+                                                   const float* s, const float* clip_grid, int K, const uint8_t* actions,
+                                                   const uint8_t* clip_idx, const int64_t* code_offsets, const float* thresh,
+                                                   uint8_t* codes_out, void* scales_out, void* zeros_out, void* Wq_out,
+                                                   void* prot_scale_out, int64_t* prot_offsets_out, int8_t* prot_q_out,
+                                                   int64_t prot_q_capacity, void* stream) {
+  return apply_plan_protected_any(ctx, "windq_apply_plan_protected", W, R, C, ldw, G, s, clip_grid, K, actions, clip_idx,
+                                  nullptr, code_offsets, thresh, codes_out, scales_out, zeros_out, Wq_out, prot_scale_out,
+                                  prot_offsets_out, prot_q_out, prot_q_capacity, stream);
+}
+
+extern "C" windq_status windq_apply_plan_protected_refined(windq_ctx* ctx, const void* W, int64_t R, int64_t C, int64_t ldw,
+                                                           int G, const float* s, const float* clip_grid, int K,
+                                                           const uint8_t* actions, const uint8_t* clip_idx,
+                                                           const void* scale_in, const int64_t* code_offsets,
+                                                           const float* thresh, uint8_t* codes_out, void* scales_out,
+                                                           void* zeros_out, void* Wq_out, void* prot_scale_out,
+                                                           int64_t* prot_offsets_out, int8_t* prot_q_out,
+                                                           int64_t prot_q_capacity, void* stream) {
+  const char* who = "windq_apply_plan_protected_refined";
+  if (!ctx) return windq::fail(nullptr, WINDQ_ERR_NULL, "%s: ctx is NULL", who);
+  if (!clip_idx || !scale_in) return windq::fail(ctx, WINDQ_ERR_NULL, "%s: clip_idx or scale_in is NULL", who);
+  if ((uintptr_t)scale_in & 1) return windq::fail(ctx, WINDQ_ERR_ALIGN, "%s: scale_in is misaligned", who);
+  return apply_plan_protected_any(ctx, who, W, R, C, ldw, G, s, clip_grid, K, actions, clip_idx, scale_in, code_offsets, thresh,
+                                  codes_out, scales_out, zeros_out, Wq_out, prot_scale_out, prot_offsets_out, prot_q_out,
+                                  prot_q_capacity, stream);
 }

@@ -57,12 +57,21 @@ __device__ __forceinline__ void refine_leaf_sums(const Lane32& w, const Lane32& 
   g23 = gacc[1];
 }
 
-template <int G>
+// sqrt(s_j): the activation scale that the saliency key uses.
+__global__ void refine_scale_kernel(const float* __restrict__ s, int C, float* __restrict__ scale) {
+  const int j = blockIdx.x * blockDim.x + threadIdx.x;
+  if (j < C) scale[j] = __fsqrt_rn(s[j]);
+}
+
+// PROTECT: a weight whose key |w| * act_scale_j reaches thresh[u] is taken out of its group (zero weight,
+// zero activation weight), exactly as in the protected fit whose clip indices this kernel starts from.
+template <int G, bool PROTECT>
 __global__ void __launch_bounds__(kRefineWarpsPerBlock * 32, 1)
 fit_refine_kernel(const __half* __restrict__ W, int R, int U, int64_t ldw, const float* __restrict__ s,
                   const float* __restrict__ clip, int K, const uint8_t* __restrict__ clip_idx, int T, float lr,
                   AdamTable adam, double* __restrict__ partial, __half* __restrict__ scale_out,
-                  float* __restrict__ group_err_out, int rows_blocks, unsigned int* __restrict__ next_item) {
+                  float* __restrict__ group_err_out, int rows_blocks, unsigned int* __restrict__ next_item,
+                  const float* __restrict__ act_scale, const float* __restrict__ thresh) {
   constexpr int LG = Map<G>::LG, GPW = Map<G>::GPW;
   const int lane = threadIdx.x & 31;
   const int g = lane / LG, q = lane % LG;
@@ -80,6 +89,18 @@ fit_refine_kernel(const __half* __restrict__ W, int R, int U, int64_t ldw, const
     const bool live = row < R;
     const int row_ld = live ? row : R - 1;  // rows past the end repeat the last row and are not written
     load_weights(W + (int64_t)row_ld * ldw + (int64_t)u * G + 32 * q, wv);
+    if (PROTECT) {
+      Lane32 av;
+      load_stats(act_scale + (int64_t)u * G + 32 * q, av);
+      const float tau = __ldg(thresh + u);
+#pragma unroll
+      for (int h = 0; h < 2; ++h)
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          if (__fmul_rn(fabsf(wv.v[h][i].x), av.v[h][i].x) >= tau) { wv.v[h][i].x = 0.0f; sv.v[h][i].x = 0.0f; }
+          if (__fmul_rn(fabsf(wv.v[h][i].y), av.v[h][i].y) >= tau) { wv.v[h][i].y = 0.0f; sv.v[h][i].y = 0.0f; }
+        }
+    }
 
     float mn, mx;
     group_range<G>(wv, mn, mx);
@@ -162,7 +183,7 @@ refine_finalize_kernel(const double* __restrict__ partial, int rows_blocks, floa
 template <int G>
 windq_status launch_refine(windq_ctx* ctx, const __half* W, int R, int U, int64_t ldw, const float* s, const float* clip,
                            int K, const uint8_t* clip_idx, int T, float lr, const AdamTable& adam, float* err_out,
-                           __half* scale_out, float* group_err_out, cudaStream_t st) {
+                           __half* scale_out, float* group_err_out, const float* thresh, cudaStream_t st) {
   constexpr int GPW = Map<G>::GPW;
   const int rows_blocks = (R + GPW - 1) / GPW;
   const int64_t n_items = (int64_t)U * rows_blocks;
@@ -173,8 +194,17 @@ windq_status launch_refine(windq_ctx* ctx, const __half* W, int R, int U, int64_
   const int64_t need = (n_items + kRefineWarpsPerBlock - 1) / kRefineWarpsPerBlock;
   if (grid > need) grid = need;
   WINDQ_CUDA(ctx, cudaMemsetAsync(next_item, 0, sizeof(unsigned int), st));
-  fit_refine_kernel<G><<<(unsigned)grid, kRefineWarpsPerBlock * 32, 0, st>>>(
-      W, R, U, ldw, s, clip, K, clip_idx, T, lr, adam, partial, scale_out, group_err_out, rows_blocks, next_item);
+  if (thresh) {
+    float* act_scale = (float*)((char*)ctx->scratch + round_up(16 + n_items * 4 * (int64_t)sizeof(double), 16));
+    refine_scale_kernel<<<(unsigned)((U * G + 255) / 256), 256, 0, st>>>(s, U * G, act_scale);
+    fit_refine_kernel<G, true><<<(unsigned)grid, kRefineWarpsPerBlock * 32, 0, st>>>(
+        W, R, U, ldw, s, clip, K, clip_idx, T, lr, adam, partial, scale_out, group_err_out, rows_blocks, next_item, act_scale,
+        thresh);
+  } else {
+    fit_refine_kernel<G, false><<<(unsigned)grid, kRefineWarpsPerBlock * 32, 0, st>>>(
+        W, R, U, ldw, s, clip, K, clip_idx, T, lr, adam, partial, scale_out, group_err_out, rows_blocks, next_item, nullptr,
+        nullptr);
+  }
   WINDQ_CUDA(ctx, cudaGetLastError());
   refine_finalize_kernel<<<(unsigned)U, 256, 0, st>>>(partial, rows_blocks, err_out);
   WINDQ_CUDA(ctx, cudaGetLastError());
@@ -188,14 +218,15 @@ extern "C" {
 int64_t windq_scratch_bytes_fit_refine(int64_t R, int64_t C, int G) {
   if (!windq::valid_G(G) || R <= 0 || C <= 0) return 0;
   const int gpw = 32 / (G / 32);
-  return 16 + (C / G) * ((R + gpw - 1) / gpw) * 4 * (int64_t)sizeof(double);
+  // the item counter, four doubles per item, and (protected variant) C activation scales
+  return windq::round_up(16 + (C / G) * ((R + gpw - 1) / gpw) * 4 * (int64_t)sizeof(double), 16) + C * (int64_t)sizeof(float);
 }
 
-windq_status windq_fit_refine(windq_ctx* ctx, const void* W, int64_t R, int64_t C, int64_t ldw, int G, const float* s,
-                              const float* clip_grid, int K, const uint8_t* clip_idx, int n_steps, float lr,
-                              float* err_out, void* scale_out, float* group_err_out, void* stream) {
+static windq_status fit_refine_any(windq_ctx* ctx, const char* who, const void* W, int64_t R, int64_t C, int64_t ldw, int G,
+                                   const float* s, const float* clip_grid, int K, const uint8_t* clip_idx,
+                                   const float* thresh, int n_steps, float lr, float* err_out, void* scale_out,
+                                   float* group_err_out, void* stream) {
   using namespace windq;
-  const char* who = "windq_fit_refine";
   if (!ctx) return fail(nullptr, WINDQ_ERR_NULL, "%s: ctx is NULL", who);
   if (windq_status st = check_matrix(ctx, who, W, R, C, ldw, G)) return st;
   if (windq_status st = check_K(ctx, who, K)) return st;
@@ -220,12 +251,28 @@ windq_status windq_fit_refine(windq_ctx* ctx, const void* W, int64_t R, int64_t 
   const __half* Wh = (const __half*)W;
   __half* so = (__half*)scale_out;
   switch (G) {
-    case 32: return launch_refine<32>(ctx, Wh, (int)R, U, ldw, s, clip_grid, K, clip_idx, n_steps, lr, adam, err_out, so, group_err_out, st);
-    case 64: return launch_refine<64>(ctx, Wh, (int)R, U, ldw, s, clip_grid, K, clip_idx, n_steps, lr, adam, err_out, so, group_err_out, st);
-    case 128: return launch_refine<128>(ctx, Wh, (int)R, U, ldw, s, clip_grid, K, clip_idx, n_steps, lr, adam, err_out, so, group_err_out, st);
-    case 256: return launch_refine<256>(ctx, Wh, (int)R, U, ldw, s, clip_grid, K, clip_idx, n_steps, lr, adam, err_out, so, group_err_out, st);
-    default: return launch_refine<512>(ctx, Wh, (int)R, U, ldw, s, clip_grid, K, clip_idx, n_steps, lr, adam, err_out, so, group_err_out, st);
+    case 32: return launch_refine<32>(ctx, Wh, (int)R, U, ldw, s, clip_grid, K, clip_idx, n_steps, lr, adam, err_out, so, group_err_out, thresh, st);
+    case 64: return launch_refine<64>(ctx, Wh, (int)R, U, ldw, s, clip_grid, K, clip_idx, n_steps, lr, adam, err_out, so, group_err_out, thresh, st);
+    case 128: return launch_refine<128>(ctx, Wh, (int)R, U, ldw, s, clip_grid, K, clip_idx, n_steps, lr, adam, err_out, so, group_err_out, thresh, st);
+    case 256: return launch_refine<256>(ctx, Wh, (int)R, U, ldw, s, clip_grid, K, clip_idx, n_steps, lr, adam, err_out, so, group_err_out, thresh, st);
+    default: return launch_refine<512>(ctx, Wh, (int)R, U, ldw, s, clip_grid, K, clip_idx, n_steps, lr, adam, err_out, so, group_err_out, thresh, st);
   }
+}
+
+windq_status windq_fit_refine(windq_ctx* ctx, const void* W, int64_t R, int64_t C, int64_t ldw, int G, const float* s,
+                              const float* clip_grid, int K, const uint8_t* clip_idx, int n_steps, float lr,
+                              float* err_out, void* scale_out, float* group_err_out, void* stream) {
+  return fit_refine_any(ctx, "windq_fit_refine", W, R, C, ldw, G, s, clip_grid, K, clip_idx, nullptr, n_steps, lr, err_out,
+                        scale_out, group_err_out, stream);
+}
+
+windq_status windq_fit_refine_protected(windq_ctx* ctx, const void* W, int64_t R, int64_t C, int64_t ldw, int G,
+                                        const float* s, const float* clip_grid, int K, const uint8_t* clip_idx,
+                                        const float* thresh, int n_steps, float lr, float* err_out, void* scale_out,
+                                        float* group_err_out, void* stream) {
+  if (ctx && !thresh) return windq::fail(ctx, WINDQ_ERR_NULL, "windq_fit_refine_protected: thresh is NULL");
+  return fit_refine_any(ctx, "windq_fit_refine_protected", W, R, C, ldw, G, s, clip_grid, K, clip_idx, thresh, n_steps, lr,
+                        err_out, scale_out, group_err_out, stream);
 }
 
 }  // extern "C"

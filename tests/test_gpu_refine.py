@@ -169,3 +169,48 @@ def test_plan_applied_with_refined_scales(wq, ctx, oracle, R, C, G):
     plain = wq.windq_apply_plan(ctx, Wd, G, sd, gd, ad, eb["code_offsets"], codes.clone(), fit["clip_idx"])
     want_plain = oracle.apply_plan(W.numpy(), G, s, grid, actions, fit["clip_idx"].cpu().numpy())
     assert np.array_equal(plain["wq"].cpu().numpy().view(np.uint16), want_plain["wq"])
+
+
+@pytest.mark.parametrize("R,C,G", [(37, 256, 32), (45, 512, 128), (9, 1024, 512), (300, 256, 64)])
+def test_protected_refinement_and_packing(wq, ctx, oracle, R, C, G):
+    """Salient weights at 3 % taken out of the groups: refined scales and errors, then a mixed plan packed with
+    those scales and the INT8 side storage, all against the oracle bit for bit."""
+    W, s, grid = inputs(oracle, R, C, 600 + G)
+    Wd, sd, gd = W.cuda(), torch.from_numpy(s).cuda(), torch.from_numpy(grid).cuda()
+    U = C // G
+    sel = wq.windq_salient_select(ctx, Wd, G, sd, 30000)
+    fit = wq.windq_fit_eval(ctx, Wd, G, sd, gd, thresh=sel["thresh"])
+    got = wq.windq_fit_refine(ctx, Wd, G, sd, gd, fit["clip_idx"], 10, 0.03, want_group_err=True, thresh=sel["thresh"])
+    torch.cuda.synchronize()
+    thresh = sel["thresh"].cpu().numpy()
+    clip_idx = fit["clip_idx"].cpu().numpy()
+    want = oracle.fit_refine(W.numpy(), G, s, grid, clip_idx, T=10, lr=0.03, thresh=thresh)
+    compare(got, want)
+    actions = ((np.arange(U) + 1) % 7).astype(np.uint8)
+    ad = torch.from_numpy(actions).cuda()
+    eb = wq.windq_effective_bits(ctx, ad, R, G)
+    codes = torch.zeros(2 * R * C + 16 * U, dtype=torch.uint8, device="cuda")
+    prot_q = torch.zeros(R * C, dtype=torch.int8, device="cuda")
+    plan = wq.windq_apply_plan_protected(ctx, Wd, G, sd, gd, ad, eb["code_offsets"], codes, sel["thresh"], prot_q,
+                                         fit["clip_idx"], scale_in=got["scale"])
+    torch.cuda.synchronize()
+    ref = oracle.apply_plan(W.numpy(), G, s, grid, actions, clip_idx, thresh=thresh, scale_in=want["scale"])
+    n = int(ref["code_offsets"][U])
+    assert np.array_equal(plan["codes"][:n].cpu().numpy(), ref["codes"])
+    assert np.array_equal(plan["scales"].cpu().numpy().view(np.uint16), ref["scales"])
+    assert np.array_equal(plan["zeros"].cpu().numpy().view(np.uint16), ref["zeros"])
+    assert np.array_equal(plan["wq"].cpu().numpy().view(np.uint16), ref["wq"])
+    assert np.array_equal(plan["prot_offsets"].cpu().numpy(), ref["prot_offsets"])
+    assert np.array_equal(plan["prot_scale"].cpu().numpy().view(np.uint16), ref["prot_scale"])
+    assert np.array_equal(plan["prot_q"][:ref["prot_q"].size].cpu().numpy(), ref["prot_q"])
+
+
+def test_protected_refinement_with_infinite_thresholds_is_the_plain_one(wq, ctx, oracle):
+    W, s, grid = inputs(oracle, 64, 512, 47)
+    Wd, sd, gd = W.cuda(), torch.from_numpy(s).cuda(), torch.from_numpy(grid).cuda()
+    fit = wq.windq_fit_eval(ctx, Wd, 128, sd, gd)
+    a = wq.windq_fit_refine(ctx, Wd, 128, sd, gd, fit["clip_idx"], 10, 0.02, want_group_err=True)
+    inf = torch.full((4,), float("inf"), device="cuda")
+    b = wq.windq_fit_refine(ctx, Wd, 128, sd, gd, fit["clip_idx"], 10, 0.02, want_group_err=True, thresh=inf)
+    assert torch.equal(a["scale"].view(torch.int16), b["scale"].view(torch.int16))
+    assert torch.equal(a["group_err"].view(torch.int32), b["group_err"].view(torch.int32))

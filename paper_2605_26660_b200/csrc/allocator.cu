@@ -3,9 +3,13 @@
 // least sensitive to 1.58 / 1 bit until enough budget is free, promote the most sensitive to 4 / 3 bit
 // while the budget permits.  Costs are Eq. 6 in centibits, all arithmetic int64.
 //
-// Three launches.  Ranking is by counting: every unit counts the units that come before it under
-// (score descending, index ascending), which is exact, stable and needs no sort; U^2 comparisons are
-// a few microseconds for the tens of thousands of units of a model.  The rule itself runs in one block:
+// Ranking is by counting: a unit's rank is the number of units that come before it under (score
+// descending, index ascending), which is exact, stable and needs no sort.  To keep that from costing
+// U^2 comparisons the units are first spread over buckets by score (a linear map of the score's
+// order-preserving bit pattern between the smallest and the largest one, so equal scores share a bucket
+// and a lower bucket holds strictly larger scores); a unit then counts inside its own bucket only and
+// adds the sizes of the buckets before it.  If all scores are equal that is the U^2 count again, which
+// the limit on U bounds.  The rule itself runs in one block:
 // the two sweeps of step 2 are prefix sums (a unit moves while the running total is above the floor,
 // and the savings are never negative, so the moved units are a prefix of the sweep), step 3 is serial by
 // nature and runs in one warp, 32 units at a time, over counts gathered in rank order beforehand, with
@@ -14,36 +18,98 @@
 
 namespace windq {
 
-constexpr int kRankThreads = 256;
-constexpr int kRankTile = 2048;
+constexpr int kMaxBuckets = 65536;
 
-// (score key, reversed index) in one word: a larger word ranks earlier.
-__global__ void alloc_key_kernel(const float* __restrict__ sal, int U, unsigned long long* __restrict__ comp) {
+// comp as above, and the smallest and largest key.
+__global__ void alloc_key_range_kernel(const float* __restrict__ sal, int U, unsigned long long* __restrict__ comp,
+                                       unsigned int* __restrict__ key_min_max) {
   const int u = blockIdx.x * blockDim.x + threadIdx.x;
-  if (u >= U) return;
-  const unsigned b = __float_as_uint(sal[u]);
-  const unsigned key = (b & 0x80000000u) ? ~b : (b | 0x80000000u);
-  comp[u] = ((unsigned long long)key << 32) | (unsigned long long)(0xffffffffu - (unsigned)u);
+  unsigned lo = 0xffffffffu, hi = 0u;
+  if (u < U) {
+    const unsigned b = __float_as_uint(sal[u]);
+    const unsigned key = (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+    comp[u] = ((unsigned long long)key << 32) | (unsigned long long)(0xffffffffu - (unsigned)u);
+    lo = hi = key;
+  }
+#pragma unroll
+  for (int m = 16; m; m >>= 1) {
+    lo = min(lo, __shfl_xor_sync(0xffffffffu, lo, m));
+    hi = max(hi, __shfl_xor_sync(0xffffffffu, hi, m));
+  }
+  if ((threadIdx.x & 31) == 0) {
+    atomicMin(key_min_max, lo);
+    atomicMax(key_min_max + 1, hi);
+  }
 }
 
-__global__ void __launch_bounds__(kRankThreads)
-alloc_rank_kernel(const unsigned long long* __restrict__ comp, int U, int* __restrict__ order, long long* __restrict__ order64) {
-  __shared__ unsigned long long tile[kRankTile];
-  const int u = blockIdx.x * kRankThreads + threadIdx.x;
-  const unsigned long long mine = u < U ? comp[u] : 0ull;
-  int before = 0;
-  for (int base = 0; base < U; base += kRankTile) {
-    const int n = min(kRankTile, U - base);
-    __syncthreads();
-    for (int i = threadIdx.x; i < n; i += kRankThreads) tile[i] = comp[base + i];
-    __syncthreads();
-#pragma unroll 8
-    for (int i = 0; i < n; ++i) before += tile[i] > mine;
+// Bucket of a key: 0 for the largest key, growing as keys fall; monotone, equal keys share a bucket.
+__device__ __forceinline__ int alloc_bucket(unsigned key, unsigned kmin, unsigned kmax, int n_buckets) {
+  const unsigned long long span = (unsigned long long)(kmax - kmin) + 1ull;
+  return (int)(((unsigned long long)(kmax - key) * (unsigned long long)n_buckets) / span);
+}
+
+__global__ void alloc_hist_kernel(const unsigned long long* __restrict__ comp, int U, const unsigned int* __restrict__ key_min_max,
+                                  int n_buckets, unsigned int* __restrict__ hist) {
+  const int u = blockIdx.x * blockDim.x + threadIdx.x;
+  if (u >= U) return;
+  atomicAdd(hist + alloc_bucket((unsigned)(comp[u] >> 32), key_min_max[0], key_min_max[1], n_buckets), 1u);
+}
+
+// start[b] = number of units in the buckets before b (one block; n_buckets is a multiple of 1024 or below it).
+__global__ void __launch_bounds__(1024)
+alloc_scan_kernel(const unsigned int* __restrict__ hist, int n_buckets, unsigned int* __restrict__ start,
+                  unsigned int* __restrict__ cursor) {
+  __shared__ unsigned int warp_tot[32];
+  const int t = threadIdx.x, per = (n_buckets + 1023) / 1024;
+  unsigned int mine = 0;
+  for (int i = 0; i < per; ++i) {
+    const int b = t * per + i;
+    if (b < n_buckets) mine += hist[b];
   }
-  if (u < U) {
-    order[before] = u;
-    if (order64) order64[before] = u;
+  unsigned int incl = mine;
+#pragma unroll
+  for (int m = 1; m < 32; m <<= 1) {
+    const unsigned int o = __shfl_up_sync(0xffffffffu, incl, m);
+    if ((t & 31) >= m) incl += o;
   }
+  if ((t & 31) == 31) warp_tot[t >> 5] = incl;
+  __syncthreads();
+  unsigned int before = incl - mine;
+  for (int w = 0; w < (t >> 5); ++w) before += warp_tot[w];
+  for (int i = 0; i < per; ++i) {
+    const int b = t * per + i;
+    if (b < n_buckets) {
+      start[b] = before;
+      cursor[b] = before;
+      before += hist[b];
+    }
+  }
+}
+
+// Units into their buckets, in whatever order the atomics give: the count below does not depend on it.
+__global__ void alloc_scatter_kernel(const unsigned long long* __restrict__ comp, int U,
+                                     const unsigned int* __restrict__ key_min_max, int n_buckets,
+                                     unsigned int* __restrict__ cursor, unsigned long long* __restrict__ members) {
+  const int u = blockIdx.x * blockDim.x + threadIdx.x;
+  if (u >= U) return;
+  const unsigned long long c = comp[u];
+  const int b = alloc_bucket((unsigned)(c >> 32), key_min_max[0], key_min_max[1], n_buckets);
+  members[atomicAdd(cursor + b, 1u)] = c;
+}
+
+__global__ void alloc_rank_kernel(const unsigned long long* __restrict__ comp, int U, const unsigned int* __restrict__ key_min_max,
+                                  int n_buckets, const unsigned int* __restrict__ start, const unsigned int* __restrict__ hist,
+                                  const unsigned long long* __restrict__ members, int* __restrict__ order,
+                                  long long* __restrict__ order64) {
+  const int u = blockIdx.x * blockDim.x + threadIdx.x;
+  if (u >= U) return;
+  const unsigned long long mine = comp[u];
+  const int b = alloc_bucket((unsigned)(mine >> 32), key_min_max[0], key_min_max[1], n_buckets);
+  const unsigned int first = start[b], n = hist[b];
+  unsigned int before = first;
+  for (unsigned int i = 0; i < n; ++i) before += members[first + i] > mine;
+  order[before] = u;
+  if (order64) order64[before] = u;
 }
 
 struct AllocArgs {
@@ -194,7 +260,8 @@ extern "C" {
 
 int64_t windq_scratch_bytes_greedy_allocate(int64_t U) {
   if (U <= 0) return 0;
-  return 2 * windq::round_up(U * 8, 256) + windq::round_up(U * 4, 256);
+  // composite keys, bucket members, walk array (8 bytes per unit each), order (4), three bucket tables, key range
+  return 3 * windq::round_up(U * 8, 256) + windq::round_up(U * 4, 256) + 3 * (int64_t)windq::kMaxBuckets * 4 + 256;
 }
 
 windq_status windq_greedy_allocate(windq_ctx* ctx, const float* saliency, const int64_t* n_weights, const int64_t* n_protected,
@@ -215,12 +282,27 @@ windq_status windq_greedy_allocate(windq_ctx* ctx, const float* saliency, const 
   DeviceGuard guard(ctx->device);
   if (windq_status rc = ensure_scratch(ctx, windq_scratch_bytes_greedy_allocate(U))) return rc;
   cudaStream_t st = (cudaStream_t)stream;
-  unsigned long long* comp = (unsigned long long*)ctx->scratch;
-  long long* walk = (long long*)((char*)ctx->scratch + round_up(U * 8, 256));
-  int* order = (int*)((char*)ctx->scratch + 2 * round_up(U * 8, 256));
-  alloc_key_kernel<<<(unsigned)((U + 255) / 256), 256, 0, st>>>(saliency, (int)U, comp);
-  alloc_rank_kernel<<<(unsigned)((U + kRankThreads - 1) / kRankThreads), kRankThreads, 0, st>>>(comp, (int)U, order,
-                                                                                               (long long*)order_out);
+  char* base = (char*)ctx->scratch;
+  unsigned long long* comp = (unsigned long long*)base;
+  unsigned long long* members = (unsigned long long*)(base + round_up(U * 8, 256));
+  long long* walk = (long long*)(base + 2 * round_up(U * 8, 256));
+  int* order = (int*)(base + 3 * round_up(U * 8, 256));
+  unsigned int* hist = (unsigned int*)(base + 3 * round_up(U * 8, 256) + round_up(U * 4, 256));
+  unsigned int* start = hist + kMaxBuckets;
+  unsigned int* cursor = start + kMaxBuckets;
+  unsigned int* key_min_max = cursor + kMaxBuckets;
+  int n_buckets = 256;  // about four units per bucket
+  while (n_buckets < kMaxBuckets && (int64_t)n_buckets * 4 < U) n_buckets *= 2;
+  const unsigned blocks = (unsigned)((U + 255) / 256);
+  WINDQ_CUDA(ctx, cudaMemsetAsync(hist, 0, (size_t)n_buckets * sizeof(unsigned int), st));
+  WINDQ_CUDA(ctx, cudaMemsetAsync(key_min_max, 0xff, sizeof(unsigned int), st));
+  WINDQ_CUDA(ctx, cudaMemsetAsync(key_min_max + 1, 0, sizeof(unsigned int), st));
+  alloc_key_range_kernel<<<blocks, 256, 0, st>>>(saliency, (int)U, comp, key_min_max);
+  alloc_hist_kernel<<<blocks, 256, 0, st>>>(comp, (int)U, key_min_max, n_buckets, hist);
+  alloc_scan_kernel<<<1, 1024, 0, st>>>(hist, n_buckets, start, cursor);
+  alloc_scatter_kernel<<<blocks, 256, 0, st>>>(comp, (int)U, key_min_max, n_buckets, cursor, members);
+  alloc_rank_kernel<<<blocks, 256, 0, st>>>(comp, (int)U, key_min_max, n_buckets, start, hist, members, order,
+                                            (long long*)order_out);
   AllocArgs a{(const long long*)n_weights, (const long long*)n_protected, (const long long*)n_groups, (int)U,
               target_cb, headroom_cb, scale_bits, zero_bits};
   alloc_greedy_kernel<<<1, 1024, 0, st>>>(a, order, walk, actions_out, (long long*)total_centibits_out);

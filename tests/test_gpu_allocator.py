@@ -122,3 +122,24 @@ def test_argument_checks(wq, ctx):
         wq.windq_greedy_allocate(ctx, sal, n, n, 200, -1)
     with pytest.raises(Exception):
         wq.windq_greedy_allocate(ctx, sal, n[:3], n, 200, 0)
+
+
+def test_all_scores_equal_and_two_distinct_scores(wq, ctx, oracle):
+    """Every unit in one bucket of the ranking, and all units in the two end buckets."""
+    _, n, g, p = units(9, 3000)
+    check(wq, ctx, oracle, np.full(3000, 0.25, np.float32), n, g, 190, 5, p, 16, 8)
+    sal = np.where(np.arange(3000) % 3 == 0, 1e-30, 3e38).astype(np.float32)
+    check(wq, ctx, oracle, sal, n, g, 190, 5, p, 16, 8)
+
+
+def test_quarter_of_a_million_units(wq, ctx, oracle):
+    """More units than any bucket table entry count per bucket assumes: 262,144 units, scores spread over
+    six decades with many repeats."""
+    U = 262144
+    rng = np.random.default_rng(12)
+    sal = (10.0 ** rng.uniform(-4, 2, U)).astype(np.float32)
+    sal[rng.integers(0, U, U // 10)] = sal[rng.integers(0, U, U // 10)]
+    g = rng.integers(1, 64, U)
+    n = g * 128
+    p = (n * 0.03).astype(np.int64)
+    check(wq, ctx, oracle, sal, n, g, 200, 10, p, 16, 16)

@@ -406,6 +406,8 @@ FULL_SIZE_CASES = [
     ("cfg5_llama70b_model", 6, 1, 2.0),     # down_proj 8192 x 28672
     ("llama3_8b_g256", 4, 1, None),         # gate_proj 14336 x 4096 at the paper's chunk sizes 256 and 512
     ("llama3_8b_g256", 2, 2, None),         # v_proj 1024 x 4096 (grouped-query attention)
+    ("llama32_1b_g256", 6, 2, 2.0),         # down_proj 2048 x 8192 of the 1B shape, chunk size 256, plan at 2.0 bits
+    ("llama32_1b_g256", 1, 1, None),        # k_proj 512 x 2048
 ]
 
 

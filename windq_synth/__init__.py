@@ -126,6 +126,7 @@ CONFIGS = {
     "cfg3_llama7b_model": ModelSpec("cfg3_llama7b_model", 32, 4096, 11008, 4096, "student_t", 2048, 20, (64, 128)),
     "cfg4_llama13b_model": ModelSpec("cfg4_llama13b_model", 40, 5120, 13824, 5120, "student_t", 4096, 40, (128,)),
     "llama3_8b_g256": ModelSpec("llama3_8b_g256", 32, 4096, 14336, 1024, "student_t", 2048, 20, (256, 512)),
+    "llama32_1b_g256": ModelSpec("llama32_1b_g256", 16, 2048, 8192, 512, "student_t", 2048, 20, (256,)),
     "cfg5_llama70b_model": ModelSpec("cfg5_llama70b_model", 80, 8192, 28672, 1024, "student_t", 2048, 20, (128,)),
 }
 

@@ -30,7 +30,11 @@ __host__ __device__ inline int fit_cand_stride(int chunk) { return chunk | 1; } 
 // PROTECT: salient weights (key |w| * scale_j >= thresh[u], scale_j = sqrt(s_j)) are taken out of
 // the fits: in the lane's registers such a weight becomes a zero weight with zero activation weight,
 // after which the fit is the ordinary one.  `never` is a NaN (see the masking step).
-template <int G, bool PROTECT>
+// PARTS: every item is handed out in five parts (one per uniform bit-width, one for the two low-bit fits and
+// the energy), each of which reloads the group.  Used for matrices with fewer than a few items per warp, where
+// whole items leave most warps idle at the end (or from the start); the code of the other instantiation is
+// untouched by it.
+template <int G, bool PROTECT, bool PARTS>
 __global__ void __launch_bounds__(kFitWarpsPerBlock * 32, 1)
 fit_eval_kernel(const __half* __restrict__ W, int R, int U, int64_t ldw, const float* __restrict__ s,
                 const float* __restrict__ clip, int K, double* __restrict__ partial, uint8_t* __restrict__ clip_idx_out,
@@ -43,7 +47,7 @@ fit_eval_kernel(const __half* __restrict__ W, int R, int U, int64_t ldw, const f
   Cand* cand = reinterpret_cast<Cand*>(smem_f4) + (size_t)warp * GPW * stride;
   const int g = lane / LG, q = lane % LG;
 
-  const unsigned int n_items = (unsigned int)(U * rows_blocks);
+  const unsigned int n_items = (unsigned int)(U * rows_blocks) * (PARTS ? 5u : 1u);
 
   Lane32 sv;
   for (;;) {
@@ -54,6 +58,11 @@ fit_eval_kernel(const __half* __restrict__ W, int R, int U, int64_t ldw, const f
     if (lane == 0) item = atomicAdd(next_item, 1u);
     item = __shfl_sync(0xffffffffu, item, 0);
     if (item >= n_items) break;
+    unsigned int parts = 0x1fu;
+    if (PARTS) {
+      parts = 1u << (item % 5u);
+      item /= 5u;
+    }
     const int u = (int)(item / rows_blocks), rb = (int)(item % rows_blocks);
     load_stats(s + (int64_t)u * G + 32 * q, sv);
     const int row = rb * GPW + g;
@@ -87,6 +96,7 @@ fit_eval_kernel(const __half* __restrict__ W, int R, int U, int64_t ldw, const f
     float e[7] = {0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f};
 #pragma unroll 1
     for (int bi = 0; bi < 4; ++bi) {
+      if (PARTS && !((parts >> bi) & 1u)) continue;
       float be;
       int bk;
       search_uniform<G>(wv, sv, mn, rng, bi, clip, K, cand, chunk, stride, lane, be, bk);
@@ -100,13 +110,15 @@ fit_eval_kernel(const __half* __restrict__ W, int R, int U, int64_t ldw, const f
         if (group_err_out) group_err_out[o] = be;
       }
     }
-    const LowBitFit low = fit_low_bits<G>(wv, sv);
-    e[4] = low.err_t;
-    e[5] = low.err_b;
-    e[6] = low.energy;
-    if (live && q == 0 && group_err_out) {
-      group_err_out[((int64_t)4 * U + u) * R + row] = low.err_t;
-      group_err_out[((int64_t)5 * U + u) * R + row] = low.err_b;
+    if (!PARTS || (parts & 0x10u)) {
+      const LowBitFit low = fit_low_bits<G>(wv, sv);
+      e[4] = low.err_t;
+      e[5] = low.err_b;
+      e[6] = low.energy;
+      if (live && q == 0 && group_err_out) {
+        group_err_out[((int64_t)4 * U + u) * R + row] = low.err_t;
+        group_err_out[((int64_t)5 * U + u) * R + row] = low.err_b;
+      }
     }
 
     // add over the rows of this item in double; lanes of a group hold equal values
@@ -115,7 +127,7 @@ fit_eval_kernel(const __half* __restrict__ W, int R, int U, int64_t ldw, const f
       double d = live ? (double)e[c] : 0.0;
 #pragma unroll
       for (int m = LG; m < 32; m <<= 1) d += __shfl_xor_sync(0xffffffffu, d, m);
-      if (lane == 0) partial[(int64_t)item * kFitPartials + c] = d;
+      if (lane == 0 && (!PARTS || ((parts >> (c < 4 ? c : 4)) & 1u))) partial[(int64_t)item * kFitPartials + c] = d;
     }
   }
 }
@@ -160,18 +172,31 @@ windq_status launch_fit(windq_ctx* ctx, const __half* W, int R, int U, int64_t l
   const int chunk = fit_cand_chunk(G), stride = fit_cand_stride(chunk);
   const size_t smem = (size_t)kFitWarpsPerBlock * GPW * stride * sizeof(Cand);
   const int id = (PROTECT ? kFitProtectG32 : kFitG32) + g_index(G);
-  if (windq_status rc = prepare_kernel(ctx, id, fit_eval_kernel<G, PROTECT>, kFitWarpsPerBlock * 32, smem, true)) return rc;
+  if (windq_status rc = prepare_kernel(ctx, id, fit_eval_kernel<G, PROTECT, false>, kFitWarpsPerBlock * 32, smem, true)) return rc;
   const int blocks_per_sm = ctx->occupancy[id];
   const int64_t n_items = (int64_t)U * rows_blocks;
-  int64_t grid = (int64_t)ctx->sm_count * blocks_per_sm;
-  const int64_t need = (n_items + kFitWarpsPerBlock - 1) / kFitWarpsPerBlock;
+  WINDQ_REQUIRE(ctx, n_items < (1ll << 28), WINDQ_ERR_SHAPE, "windq_fit_eval: R * C is too large for one call");
+  const int64_t full_grid = (int64_t)ctx->sm_count * blocks_per_sm;
+  // fewer than one and a half items per warp of a full grid: hand the items out in parts.  (With more, whole
+  // items are as fast: an SM whose warps run out one by one gives their issue slots to the rest, measured on
+  // 2048 x 2048.  A 512 x 2048 matrix, whose 1024 items would fill less than half the warps, gains 1.5x.)
+  const bool in_parts = 2 * n_items < 3 * full_grid * kFitWarpsPerBlock;
+  if (in_parts)
+    if (windq_status rc = prepare_kernel(ctx, id + kFitPartsOffset, fit_eval_kernel<G, PROTECT, true>, kFitWarpsPerBlock * 32, smem, false))
+      return rc;
+  int64_t grid = full_grid;
+  const int64_t need = ((in_parts ? 5 : 1) * n_items + kFitWarpsPerBlock - 1) / kFitWarpsPerBlock;
   if (grid > need) grid = need;
-  WINDQ_REQUIRE(ctx, n_items < (1ll << 31), WINDQ_ERR_SHAPE, "windq_fit_eval: R * C is too large for one call");
   WINDQ_CUDA(ctx, cudaMemsetAsync(next_item, 0, sizeof(unsigned int), st));
   if (PROTECT) fit_scale_kernel<<<(unsigned)((U * G + 255) / 256), 256, 0, st>>>(s, U * G, scale);
-  fit_eval_kernel<G, PROTECT><<<(unsigned)grid, kFitWarpsPerBlock * 32, smem, st>>>(
-      W, R, U, ldw, s, clip, K, partial, clip_idx_out, group_err_out, rows_blocks, chunk, stride, scale, thresh,
-      __builtin_nanf(""), next_item);
+  if (in_parts)
+    fit_eval_kernel<G, PROTECT, true><<<(unsigned)grid, kFitWarpsPerBlock * 32, smem, st>>>(
+        W, R, U, ldw, s, clip, K, partial, clip_idx_out, group_err_out, rows_blocks, chunk, stride, scale, thresh,
+        __builtin_nanf(""), next_item);
+  else
+    fit_eval_kernel<G, PROTECT, false><<<(unsigned)grid, kFitWarpsPerBlock * 32, smem, st>>>(
+        W, R, U, ldw, s, clip, K, partial, clip_idx_out, group_err_out, rows_blocks, chunk, stride, scale, thresh,
+        __builtin_nanf(""), next_item);
   WINDQ_CUDA(ctx, cudaGetLastError());
   fit_finalize_kernel<<<(unsigned)U, 256, 0, st>>>(partial, rows_blocks, err_out, energy_out);
   WINDQ_CUDA(ctx, cudaGetLastError());

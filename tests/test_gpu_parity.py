@@ -469,3 +469,22 @@ def test_full_size_matrix_sampled_units(wq, ctx, oracle, config, mi, n_units, ta
             assert (plan["wq"][:, u * G:(u + 1) * G].cpu().view(torch.int16).numpy().view(np.uint16) == wp["wq"]).all()
     del W
     torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("R,C,G", [(512, 2048, 256), (512, 2048, 128), (100, 4096, 512), (1000, 512, 32)])
+def test_fit_eval_of_a_matrix_smaller_than_the_grid(wq, ctx, oracle, R, C, G):
+    """Matrices with fewer items than the grid has warps take the launch shape that hands every item out in
+    five parts; clip indices and group errors must be those of the oracle bit for bit, unit sums within tolerance."""
+    W = ws.weights(R, C, 77 + R, "student_t")
+    X = ws.activations(64, C, 78)
+    s = oracle.act_stats(X.numpy())
+    grid = ws.clip_grid(20)
+    got = wq.windq_fit_eval(ctx, W.cuda(), G, torch.from_numpy(s).cuda(), torch.from_numpy(grid).cuda(), want_group_err=True)
+    torch.cuda.synchronize()
+    units = sorted(set([0, C // G - 1, (C // G) // 2]))
+    cols = np.concatenate([np.arange(u * G, (u + 1) * G) for u in units])
+    want = oracle.fit_eval(W.numpy()[:, cols], G, s[cols], grid)
+    assert np.array_equal(got["clip_idx"][:, units].cpu().numpy(), want["clip_idx"])
+    assert np.array_equal(got["group_err"][:, units].cpu().numpy().view(np.uint32), want["group_err"].view(np.uint32))
+    assert close(got["err"][units].cpu().numpy(), want["err"]).all()
+    assert close(got["energy"][units].cpu().numpy(), want["energy"]).all()

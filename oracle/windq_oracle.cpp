@@ -604,7 +604,7 @@ static int apply_plan_impl(const uint16_t* W, int64_t R, int64_t C, int64_t ldw,
           int k;
           if (clip_idx) {
             k = clip_idx[((int64_t)bi * U + u) * R + r];
-            if (k >= K) return 1;
+            if (k >= K) k = K - 1;  // the interface treats an index beyond the grid as the last ratio
           } else {
             float e;
             search_uniform(g, mn, rng, bits, clip_grid, K, &k, &e);

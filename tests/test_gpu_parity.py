@@ -488,3 +488,27 @@ def test_fit_eval_of_a_matrix_smaller_than_the_grid(wq, ctx, oracle, R, C, G):
     assert np.array_equal(got["group_err"][:, units].cpu().numpy().view(np.uint32), want["group_err"].view(np.uint32))
     assert close(got["err"][units].cpu().numpy(), want["err"]).all()
     assert close(got["energy"][units].cpu().numpy(), want["energy"]).all()
+
+
+def test_apply_plan_clip_indices_beyond_the_grid_mean_the_last_ratio(wq, ctx, oracle):
+    R, C, G, K = 40, 512, 128, 7
+    W = ws.weights(R, C, 91, "student_t")
+    s = oracle.act_stats(ws.activations(64, C, 92).numpy())
+    grid = ws.clip_grid(K)
+    U = C // G
+    idx = np.random.default_rng(3).integers(0, 256, (4, U, R)).astype(np.uint8)      # most entries are >= K
+    actions = np.array([1, 2, 3, 4], np.uint8)
+    ad = torch.from_numpy(actions).cuda()
+    eb = wq.windq_effective_bits(ctx, ad, R, G)
+    codes = torch.zeros(2 * R * C + 16 * U, dtype=torch.uint8, device="cuda")
+    got = wq.windq_apply_plan(ctx, W.cuda(), G, torch.from_numpy(s).cuda(), torch.from_numpy(grid).cuda(), ad,
+                              eb["code_offsets"], codes, torch.from_numpy(idx).cuda())
+    torch.cuda.synchronize()
+    want = oracle.apply_plan(W.numpy(), G, s, grid, actions, idx)
+    clamped = oracle.apply_plan(W.numpy(), G, s, grid, actions, np.minimum(idx, K - 1))
+    assert np.array_equal(want["codes"], clamped["codes"]) and np.array_equal(want["wq"], clamped["wq"])
+    n = int(want["code_offsets"][U])
+    assert np.array_equal(got["codes"][:n].cpu().numpy(), want["codes"])
+    assert np.array_equal(got["scales"].cpu().numpy().view(np.uint16), want["scales"])
+    assert np.array_equal(got["zeros"].cpu().numpy().view(np.uint16), want["zeros"])
+    assert np.array_equal(got["wq"].cpu().numpy().view(np.uint16), want["wq"])

@@ -770,9 +770,8 @@ int oracle_fallback(const float* err, const float* energy, const uint8_t* action
   int64_t changed = 0;
   for (int64_t u = 0; u < U; ++u) {
     int a = actions[u];
-    if (a > 6) return 1;
     const float limit = theta * energy[u];
-    while (a >= 1 && err[u * 6 + (a - 1)] > limit) --a;
+    while (a >= 1 && a <= 6 && err[u * 6 + (a - 1)] > limit) --a;   // codes above 6 are not actions: copied as they are
     actions_out[u] = (uint8_t)a;
     changed += a != actions[u];
   }

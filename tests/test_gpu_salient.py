@@ -176,6 +176,12 @@ def test_fallback(wq, ctx, oracle):
         want, n = oracle.fallback(err, energy, acts, theta)
         got = wq.windq_fallback(ctx, fitd["err"], fitd["energy"], torch.from_numpy(acts).cuda(), theta)
         assert (got["actions"].cpu().numpy() == want).all() and int(got["n_changed"].item()) == n
+    odd = acts.copy()
+    odd[::3] = [7, 200, 255, 9, 7, 8][:len(odd[::3])]          # not action codes: copied as they are
+    want, n = oracle.fallback(err, energy, odd, 0.05)
+    got = wq.windq_fallback(ctx, fitd["err"], fitd["energy"], torch.from_numpy(odd).cuda(), 0.05)
+    assert (got["actions"].cpu().numpy() == want).all() and int(got["n_changed"].item()) == n
+    assert (want[::3] == odd[::3]).all()
     with pytest.raises(wq.WindqError):
         wq.windq_fallback(ctx, fitd["err"], fitd["energy"], torch.from_numpy(acts).cuda(), -1.0)
 

@@ -7,6 +7,7 @@ values are scalars on the control path -- the plan's total bits (an int64 sum) a
 GPUs, gloo in the CPU tests).  The one call that looks at all units at once is the heuristic
 allocator's rule: for it the ranks exchange their units' scores and counts (a few bytes per unit,
 `gather_units`), every rank runs the rule on the same gathered arrays and keeps its own slice.
+A calibration input can also be split by tokens: `combine_act_stats` merges the per-rank statistics.
 """
 from __future__ import annotations
 
@@ -90,3 +91,19 @@ def allocate_across_ranks(allocate, saliency, n_weights, n_groups, n_protected=N
     gathered, begin, end = gather_units(*arrays)
     res = allocate(gathered[0], gathered[1], gathered[2], gathered[3] if has_p else None)
     return res["actions"][begin:end], int(res["total_centibits"])
+
+
+def combine_act_stats(s_local: torch.Tensor, tokens_local: int) -> torch.Tensor:
+    """Activation statistics of a calibration input whose tokens are split over the ranks.
+
+    Every rank calls windq_act_stats on its own slice of tokens (s_local[j] = mean of x_tj^2 over its
+    tokens_local tokens); the statistic of the whole input is the token-weighted mean of the slices,
+    s[j] = sum_r tokens_r * s_r[j] / sum_r tokens_r, formed in float64 and all-reduced (one sum of C + 1
+    numbers).  Returns fp32 [C] on every rank.  Without a process group the input comes back unchanged."""
+    if not (dist.is_available() and dist.is_initialized()):
+        return s_local
+    acc = torch.empty(s_local.numel() + 1, dtype=torch.float64, device=s_local.device)
+    acc[:-1] = s_local.to(torch.float64) * float(tokens_local)
+    acc[-1] = float(tokens_local)
+    dist.all_reduce(acc, op=dist.ReduceOp.SUM)
+    return (acc[:-1] / acc[-1]).to(torch.float32)

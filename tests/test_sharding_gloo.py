@@ -155,3 +155,39 @@ def test_gather_units_without_a_process_group():
     assert torch.equal(ga, a) and torch.equal(gb, b) and (lo, hi) == (0, 5)
     with pytest.raises(ValueError):
         sh.gather_units(a, b[:3])
+
+
+# ---- activation statistics of an input whose tokens are split over the ranks ---------------------------
+ACT_T, ACT_C = 96, 256
+
+
+def _act_input():
+    import windq_synth as ws
+    return ws.activations(ACT_T, ACT_C, 61).numpy()
+
+
+def _act_worker(rank, world, port, out_dir):
+    sys.path.insert(0, ROOT)
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        sharding = _load_sharding()
+        import oracle
+        oracle.build()
+        X = _act_input()
+        lo, hi = (0, 40) if rank == 0 else (40, ACT_T)           # unequal slices
+        s_local = torch.from_numpy(oracle.act_stats(X[lo:hi]))
+        s = sharding.combine_act_stats(s_local, hi - lo)
+        np.save(os.path.join(out_dir, "act%d.npy" % rank), s.numpy())
+    finally:
+        dist.destroy_process_group()
+
+
+def test_token_sharded_act_stats_equal_the_whole_input(tmp_path, oracle):
+    world = 2
+    mp.start_processes(_act_worker, args=(world, _free_port(), str(tmp_path)), nprocs=world, join=True, start_method="spawn")
+    want = oracle.act_stats(_act_input())
+    got = [np.load(os.path.join(str(tmp_path), "act%d.npy" % r)) for r in range(world)]
+    assert np.array_equal(got[0], got[1])                       # every rank holds the same statistic
+    assert np.allclose(got[0], want, rtol=1e-6, atol=0)

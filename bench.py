@@ -53,6 +53,8 @@ def parse_args():
     ap.add_argument("--blocks", type=int, default=0, help="use only the first B blocks (0 = all; profiling aid)")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--separate-fits", action="store_true",
+                    help="one windq_fit_eval call per matrix instead of one windq_fit_eval_batch call per block and chunk width")
     ap.add_argument("--extras", action="store_true",
                     help="also time the calls beyond the five of a step (protection, refinement, allocator) on block 0")
     return ap.parse_args()
@@ -211,6 +213,11 @@ class Buffers:
         shapes = dict(feat=(maxU * 8, torch.float32), err=(maxU * 6, torch.float32), energy=(maxU, torch.float32),
                       totals=(2 * len(TARGET_BITS), torch.int64), codes=(2 * maxRC + 16 * maxU, torch.uint8),
                       scales=(maxUR, torch.float16), zeros=(maxUR, torch.float16))
+        # one set of fit outputs per matrix of a block, for the batched fit (all matrices of a block in one call)
+        for mi, m in enumerate(mats):
+            shapes["err%d" % mi] = ((m.C // Gmin) * 6, torch.float32)
+            shapes["energy%d" % mi] = (m.C // Gmin, torch.float32)
+        self.clip_idx_m = [torch.empty(4 * (m.C // Gmin) * m.R, dtype=torch.uint8, device=dev) for m in mats]
         self.rings = {k: [torch.zeros(n, dtype=dt, device=dev) for _ in range(ring)] for k, (n, dt) in shapes.items()}
         self.turn = {k: 0 for k in shapes}
         self.pending = {}          # (name, slot) -> event of the copy that still reads that slot
@@ -251,6 +258,32 @@ class FitTimer:
         return sum(a.elapsed_time(b) for a, b in self.pairs)
 
 
+BATCH_FITS = True      # one windq_fit_eval_batch call per block and chunk width (False: one windq_fit_eval per matrix)
+
+
+def apply_plans(wq, ctx, spec, m, mi, W, s, G, clip_idx, plans_b, buf, grid_d, sink):
+    """The three plans of one matrix: bit accounting, then packing.  Returns the number of kernels launched."""
+    U, launches = m.C // G, 0
+    totals = buf.take("totals")
+    for ti, target in enumerate(TARGET_BITS):
+        acts = plans_b[target][mi]
+        eb = wq.windq_effective_bits(ctx, acts, m.R, G, out=dict(
+            unit_centibits=buf.unit_cb[:U], code_offsets=buf.offsets[:U + 1],
+            total_centibits=totals[2 * ti:2 * ti + 1], total_packed_bytes=totals[2 * ti + 1:2 * ti + 2]))
+        plan = wq.windq_apply_plan(ctx, W, G, s, grid_d, acts, eb["code_offsets"], buf.take("codes"), clip_idx,
+                                   out=dict(scales=buf.take("scales")[:U * m.R].view(U, m.R),
+                                            zeros=buf.take("zeros")[:U * m.R].view(U, m.R),
+                                            wq=buf.wq[:m.R * m.C].view(m.R, m.C)))
+        launches += 2
+        if sink:
+            sink("codes", (plan["codes"], acts, m.R, G))
+            sink("scales", plan["scales"])
+            sink("zeros", plan["zeros"])
+    if sink:
+        sink("totals", totals)
+    return launches
+
+
 def score_block(wq, ctx, spec, Wb, Xb, plans_b, buf, grid_d, timer=None, sink=None):
     """The whole hot path for one block.  Returns the number of kernels launched.  `sink(name, tensor)`
     receives every result (the e2e leg copies them to the host)."""
@@ -259,6 +292,33 @@ def score_block(wq, ctx, spec, Wb, Xb, plans_b, buf, grid_d, timer=None, sink=No
     for i, X in Xb.items():
         wq.windq_act_stats(ctx, X, buf.s[i])
         launches += 2
+    if BATCH_FITS:
+        for G in spec.chunk_widths:
+            for mi, m in enumerate(mats):
+                U = m.C // G
+                feat = buf.take("feat")[:U * 8].view(U, 8)
+                wq.windq_unit_features(ctx, Wb[mi], G, buf.s[m.x_id], feat)
+                launches += 2
+                if sink:
+                    sink("feat", feat)
+            outs = [dict(err=buf.take("err%d" % mi)[:(m.C // G) * 6].view(m.C // G, 6),
+                         energy=buf.take("energy%d" % mi)[:m.C // G],
+                         clip_idx=buf.clip_idx_m[mi][:4 * (m.C // G) * m.R].view(4, m.C // G, m.R))
+                    for mi, m in enumerate(mats)]
+            e0 = timer.start() if timer else None
+            wq.windq_fit_eval_batch(ctx, Wb, G, [buf.s[m.x_id] for m in mats], grid_d, outs=outs)
+            if timer:
+                timer.stop(e0)
+            launches += 2
+            if sink:
+                for mi in range(len(mats)):
+                    sink("err%d" % mi, outs[mi]["err"])
+                    sink("energy%d" % mi, outs[mi]["energy"])
+            if G == APPLY_G and plans_b:
+                for mi, m in enumerate(mats):
+                    launches += apply_plans(wq, ctx, spec, m, mi, Wb[mi], buf.s[m.x_id], G, outs[mi]["clip_idx"], plans_b, buf,
+                                            grid_d, sink)
+        return launches
     for mi, m in enumerate(mats):
         W, s = Wb[mi], buf.s[m.x_id]
         for G in spec.chunk_widths:
@@ -278,23 +338,7 @@ def score_block(wq, ctx, spec, Wb, Xb, plans_b, buf, grid_d, timer=None, sink=No
                 sink("err", out["err"])
                 sink("energy", out["energy"])
             if G == APPLY_G and plans_b:
-                totals = buf.take("totals")
-                for ti, target in enumerate(TARGET_BITS):
-                    acts = plans_b[target][mi]
-                    eb = wq.windq_effective_bits(ctx, acts, m.R, G, out=dict(
-                        unit_centibits=buf.unit_cb[:U], code_offsets=buf.offsets[:U + 1],
-                        total_centibits=totals[2 * ti:2 * ti + 1], total_packed_bytes=totals[2 * ti + 1:2 * ti + 2]))
-                    plan = wq.windq_apply_plan(ctx, W, G, s, grid_d, acts, eb["code_offsets"], buf.take("codes"), out["clip_idx"],
-                                               out=dict(scales=buf.take("scales")[:U * m.R].view(U, m.R),
-                                                        zeros=buf.take("zeros")[:U * m.R].view(U, m.R),
-                                                        wq=buf.wq[:m.R * m.C].view(m.R, m.C)))
-                    launches += 2
-                    if sink:
-                        sink("codes", (plan["codes"], acts, m.R, G))
-                        sink("scales", plan["scales"])
-                        sink("zeros", plan["zeros"])
-                if sink:
-                    sink("totals", totals)
+                launches += apply_plans(wq, ctx, spec, m, mi, W, s, G, out["clip_idx"], plans_b, buf, grid_d, sink)
     return launches
 
 
@@ -554,13 +598,14 @@ def reference_main(args, spec):
 
 
 def main():
-    global APPLY_G
+    global APPLY_G, BATCH_FITS
     args = parse_args()
     spec = ws.CONFIGS[args.workload]
     if APPLY_G not in spec.chunk_widths:
         APPLY_G = spec.chunk_widths[0]
     if args.impl == "reference":
         return reference_main(args, spec)
+    BATCH_FITS = not args.separate_fits
 
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -594,6 +639,8 @@ def main():
     mats = matrices_of(spec)
     scratch = max(max(wq.windq_scratch_bytes_fit_eval(m.R, m.C, G), wq.windq_scratch_bytes_unit_features(m.R, m.C, G))
                   for m in mats for G in spec.chunk_widths)
+    if BATCH_FITS:
+        scratch = max(scratch, max(sum(wq.windq_scratch_bytes_fit_eval(m.R, m.C, G) for m in mats) for G in spec.chunk_widths))
     wq.windq_reserve(ctx, scratch)
 
     elems, units = workload_counts(spec, n_blocks)
@@ -606,7 +653,7 @@ def main():
     total_cb = sharding.sum_int64(int(buf.totals[2 * (len(TARGET_BITS) - 1)].item())) if plans else 0
     torch.cuda.synchronize()
 
-    n_fit = len(spec.chunk_widths) * len(mats) * n_blocks * args.steps
+    n_fit = len(spec.chunk_widths) * (1 if BATCH_FITS else len(mats)) * n_blocks * args.steps
     fit_elem = elems * len(spec.chunk_widths) * args.steps
     ops = fit_ops_per_element(spec.K)
     sm_count = torch.cuda.get_device_properties(local_rank).multi_processor_count
@@ -628,7 +675,10 @@ def main():
     e2e = None
     if not args.no_e2e:
         del buf
-        ebuf = Buffers(spec, ring=3)
+        # with the batched fit the 21 plan applications of a block run back to back: give every one of them its own
+        # output slot (and three more), so that packing never waits for a device-to-host copy and the copies of one
+        # block overlap the fits of the next
+        ebuf = Buffers(spec, ring=3 * len(mats) + 3 if BATCH_FITS else 3)
         e_ms, e_wall, h2d, d2h, host_blocks = run_e2e_leg(wq, ctx, spec, model, plans, plans_np, ebuf, grid_d,
                                                           max(1, min(args.steps, 2)), args.warmup, sync)
         e_steps = max(1, min(args.steps, 2))
@@ -654,6 +704,8 @@ def main():
                     config=dict(workload=spec.name, blocks=n_blocks, elements_per_chunk_width=elems, units=units, K=spec.K,
                                 chunk_widths=list(spec.chunk_widths), plan_targets=list(TARGET_BITS), apply_chunk_width=APPLY_G,
                                 tokens=spec.T, weights=spec.dist, parallelism="replica per GPU",
+                                fits="one windq_fit_eval_batch call per block and chunk width" if BATCH_FITS
+                                else "one windq_fit_eval call per matrix",
                                 l2="every step streams %.1f GB of inputs, far above the 126 MB L2" % (
                                     (2 * elems + 2 * spec.T * sum(c for _, c in inputs_of(spec)) * n_blocks) / 1e9)),
                     clocks=clocks, e2e=e2e, gpu_launches=launches, roofline=roofline, cpu_baseline=cpu,

@@ -159,6 +159,27 @@ windq_status windq_effective_bits(windq_ctx* ctx, const uint8_t* actions, int64_
                                   int64_t* code_offsets_out, int64_t* total_centibits_out,
                                   int64_t* total_packed_bytes_out, void* stream);
 
+/* windq_fit_eval for several matrices in one launch (the paper has no counterpart: the consumer loops
+ * over the seven projections of every block, and matrices that are small against the GPU -- a few million
+ * weights -- neither fill it nor amortise the fixed cost of a call on their own).  All jobs share G, the
+ * clip grid and K; every job is one windq_fit_eval: W, R, C, ldw, s and the four outputs with the meanings,
+ * layouts and nullability given there.  Results are those of the separate calls (group errors and clip
+ * indices bit for bit; unit sums to the last bit too, being added in the same order).
+ *   jobs: HOST array of n_jobs descriptors (1 <= n_jobs <= 16), read during the call only; the pointers
+ *   inside are device pointers.  Scratch: windq_scratch_bytes_fit_eval_batch. */
+typedef struct {
+  const void* W;          /* fp16 [R][ldw] */
+  int64_t R, C, ldw;
+  const float* s;         /* fp32 [C] */
+  float* err_out;         /* fp32 [U][6] */
+  float* energy_out;      /* fp32 [U], nullable */
+  uint8_t* clip_idx_out;  /* u8 [4][U][R], nullable */
+  float* group_err_out;   /* fp32 [6][U][R], nullable */
+} windq_fit_job;
+int64_t windq_scratch_bytes_fit_eval_batch(const windq_fit_job* jobs, int n_jobs, int G);
+windq_status windq_fit_eval_batch(windq_ctx* ctx, const windq_fit_job* jobs, int n_jobs, int G, const float* clip_grid,
+                                  int K, void* stream);
+
 /* a4 -- apply a plan to one matrix ("the environment applies the selected quantization to the
  * current unit"): integer codes packed as described above, the fp16 scale and zero point of
  * every group, and optionally the fake-quantised weights for the consumer's forward pass.

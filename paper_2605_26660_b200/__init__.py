@@ -56,6 +56,9 @@ def _load() -> ctypes.CDLL:
     lib.windq_act_stats_noalloc.argtypes = [vp, vp, i64, i64, i64, vp, vp]
     lib.windq_unit_features.argtypes = [vp, vp, i64, i64, i64, i32, vp, vp, vp]
     lib.windq_fit_eval.argtypes = [vp, vp, i64, i64, i64, i32, vp, vp, i32, vp, vp, vp, vp, vp]
+    lib.windq_fit_eval_batch.argtypes = [vp, vp, i32, i32, vp, i32, vp]
+    lib.windq_scratch_bytes_fit_eval_batch.restype = i64
+    lib.windq_scratch_bytes_fit_eval_batch.argtypes = [vp, i32, i32]
     lib.windq_fit_eval_protected.argtypes = [vp, vp, i64, i64, i64, i32, vp, vp, i32, vp, vp, vp, vp, vp, vp]
     lib.windq_scratch_bytes_fit_eval_protected.argtypes = [i64, i64, i32]
     lib.windq_scratch_bytes_fit_eval_protected.restype = i64
@@ -242,6 +245,47 @@ def windq_fit_eval(ctx: Context, W: torch.Tensor, G: int, s: torch.Tensor, clip_
                                                  clip_grid.numel(), _ptr(thresh), _ptr(out["err"]), _ptr(out["energy"]),
                                                  _ptr(out["clip_idx"]), _ptr(out["group_err"]), _stream(stream)))
     return out
+
+
+class _FitJob(ctypes.Structure):
+    _fields_ = [("W", ctypes.c_void_p), ("R", ctypes.c_int64), ("C", ctypes.c_int64), ("ldw", ctypes.c_int64),
+                ("s", ctypes.c_void_p), ("err_out", ctypes.c_void_p), ("energy_out", ctypes.c_void_p),
+                ("clip_idx_out", ctypes.c_void_p), ("group_err_out", ctypes.c_void_p)]
+
+
+def windq_fit_eval_batch(ctx: Context, Ws, G: int, ss, clip_grid: torch.Tensor, *, want_energy: bool = True,
+                         want_clip_idx: bool = True, want_group_err: bool = False, outs=None, stream=None) -> list:
+    """windq_fit_eval of up to 16 matrices in one launch.  ``Ws`` and ``ss`` are equally long sequences of weight
+    matrices and their statistics; ``outs`` may hold one dict of preallocated outputs per matrix (keys as
+    windq_fit_eval).  Returns the list of output dicts."""
+    if len(Ws) != len(ss) or not Ws:
+        raise ValueError("Ws and ss must be non-empty and equally long")
+    _need(clip_grid, torch.float32, "clip_grid", 1)
+    jobs = (_FitJob * len(Ws))()
+    results = []
+    for j, (W, s) in enumerate(zip(Ws, ss)):
+        R, C, ldw = _matrix(W, "W")
+        _need(s, torch.float32, "s", 1)
+        U = C // G if G > 0 else 0
+        out = dict(outs[j]) if outs else {}
+        dev = W.device
+        if out.get("err") is None:
+            out["err"] = torch.empty((U, N_BITWIDTHS), dtype=torch.float32, device=dev)
+        if want_energy and out.get("energy") is None:
+            out["energy"] = torch.empty(U, dtype=torch.float32, device=dev)
+        if want_clip_idx and out.get("clip_idx") is None:
+            out["clip_idx"] = torch.empty((4, U, R), dtype=torch.uint8, device=dev)
+        if want_group_err and out.get("group_err") is None:
+            out["group_err"] = torch.empty((N_BITWIDTHS, U, R), dtype=torch.float32, device=dev)
+        for key in ("energy", "clip_idx", "group_err"):
+            out.setdefault(key, None)
+        ptr = lambda x: None if x is None else x.data_ptr()
+        jobs[j] = _FitJob(W.data_ptr(), R, C, ldw, s.data_ptr(), ptr(out["err"]), ptr(out["energy"]), ptr(out["clip_idx"]),
+                          ptr(out["group_err"]))
+        results.append(out)
+    ctx._check(_lib.windq_fit_eval_batch(ctx._h, ctypes.cast(jobs, ctypes.c_void_p), len(Ws), int(G), _ptr(clip_grid),
+                                         clip_grid.numel(), _stream(stream)))
+    return results
 
 
 def windq_fit_refine(ctx: Context, W: torch.Tensor, G: int, s: torch.Tensor, clip_grid: torch.Tensor,

@@ -12,6 +12,8 @@
 // Per item the warp writes seven partial sums (six errors and the energy, added over its rows in
 // double) to scratch; a second small kernel adds them per unit in a fixed order, so unit totals
 // are reproducible from run to run.
+#include <string.h>
+
 #include "fit_device.cuh"
 
 namespace windq {
@@ -27,6 +29,24 @@ __host__ __device__ inline int fit_cand_chunk(int G) {
 }
 __host__ __device__ inline int fit_cand_stride(int chunk) { return chunk | 1; }  // odd: conflict-free rows
 
+// Several matrices in one launch (windq_fit_eval_batch): what differs from matrix to matrix, by value in
+// the kernel's parameters.  Items are numbered through all jobs; job j owns [first_item[j], first_item[j+1]).
+constexpr int kFitMaxJobs = 16;
+struct FitJobs {
+  const __half* W[kFitMaxJobs];
+  const float* s[kFitMaxJobs];
+  uint8_t* clip_idx[kFitMaxJobs];
+  float* group_err[kFitMaxJobs];
+  float* err[kFitMaxJobs];
+  float* energy[kFitMaxJobs];
+  long long ldw[kFitMaxJobs];
+  int R[kFitMaxJobs];
+  int U[kFitMaxJobs];
+  unsigned int first_item[kFitMaxJobs + 1];
+  unsigned int first_unit[kFitMaxJobs + 1];
+  int n;
+};
+
 // PROTECT: salient weights (key |w| * scale_j >= thresh[u], scale_j = sqrt(s_j)) are taken out of
 // the fits: in the lane's registers such a weight becomes a zero weight with zero activation weight,
 // after which the fit is the ordinary one.  `never` is a NaN (see the masking step).
@@ -34,20 +54,21 @@ __host__ __device__ inline int fit_cand_stride(int chunk) { return chunk | 1; } 
 // the energy), each of which reloads the group.  Used for matrices with fewer than a few items per warp, where
 // whole items leave most warps idle at the end (or from the start); the code of the other instantiation is
 // untouched by it.
-template <int G, bool PROTECT, bool PARTS>
+// BATCH: the matrix of an item is looked up in `jobs` (the scalar matrix parameters are then unused).
+template <int G, bool PROTECT, bool PARTS, bool BATCH>
 __global__ void __launch_bounds__(kFitWarpsPerBlock * 32, 1)
-fit_eval_kernel(const __half* __restrict__ W, int R, int U, int64_t ldw, const float* __restrict__ s,
-                const float* __restrict__ clip, int K, double* __restrict__ partial, uint8_t* __restrict__ clip_idx_out,
-                float* __restrict__ group_err_out, int rows_blocks, int chunk, int stride,
+fit_eval_kernel(const __half* __restrict__ W_one, int R_one, int U_one, int64_t ldw_one, const float* __restrict__ s_one,
+                const float* __restrict__ clip, int K, double* __restrict__ partial, uint8_t* __restrict__ clip_idx_one,
+                float* __restrict__ group_err_one, int rows_blocks_one, int chunk, int stride,
                 const float* __restrict__ scale, const float* __restrict__ thresh, float never,
-                unsigned int* __restrict__ next_item) {
+                unsigned int* __restrict__ next_item, const FitJobs jobs) {
   constexpr int LG = Map<G>::LG, GPW = Map<G>::GPW;
   extern __shared__ float4 smem_f4[];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   Cand* cand = reinterpret_cast<Cand*>(smem_f4) + (size_t)warp * GPW * stride;
   const int g = lane / LG, q = lane % LG;
 
-  const unsigned int n_items = (unsigned int)(U * rows_blocks) * (PARTS ? 5u : 1u);
+  const unsigned int n_items = (BATCH ? jobs.first_item[jobs.n] : (unsigned int)(U_one * rows_blocks_one)) * (PARTS ? 5u : 1u);
 
   Lane32 sv;
   for (;;) {
@@ -63,7 +84,27 @@ fit_eval_kernel(const __half* __restrict__ W, int R, int U, int64_t ldw, const f
       parts = 1u << (item % 5u);
       item /= 5u;
     }
-    const int u = (int)(item / rows_blocks), rb = (int)(item % rows_blocks);
+    const __half* W = W_one;
+    const float* s = s_one;
+    uint8_t* clip_idx_out = clip_idx_one;
+    float* group_err_out = group_err_one;
+    int R = R_one, U = U_one, rows_blocks = rows_blocks_one;
+    int64_t ldw = ldw_one;
+    unsigned int local = item;
+    if (BATCH) {
+      int j = 0;
+      while (j + 1 < jobs.n && item >= jobs.first_item[j + 1]) ++j;
+      W = jobs.W[j];
+      s = jobs.s[j];
+      clip_idx_out = jobs.clip_idx[j];
+      group_err_out = jobs.group_err[j];
+      R = jobs.R[j];
+      U = jobs.U[j];
+      ldw = jobs.ldw[j];
+      rows_blocks = (R + GPW - 1) / GPW;
+      local = item - jobs.first_item[j];
+    }
+    const int u = (int)(local / rows_blocks), rb = (int)(local % rows_blocks);
     load_stats(s + (int64_t)u * G + 32 * q, sv);
     const int row = rb * GPW + g;
     const bool live = row < R;
@@ -156,6 +197,33 @@ fit_finalize_kernel(const double* __restrict__ partial, int rows_blocks, float* 
   }
 }
 
+// The same for a batch: block b is unit b - first_unit[j] of job j.
+__global__ void __launch_bounds__(256)
+fit_finalize_batch_kernel(const double* __restrict__ partial, int gpw, const FitJobs jobs) {
+  __shared__ double red[256];
+  const int b = blockIdx.x, t = threadIdx.x;
+  int j = 0;
+  while (j + 1 < jobs.n && (unsigned int)b >= jobs.first_unit[j + 1]) ++j;
+  const int u = b - (int)jobs.first_unit[j];
+  const int rows_blocks = (jobs.R[j] + gpw - 1) / gpw;
+  const double* p = partial + ((int64_t)jobs.first_item[j] + (int64_t)u * rows_blocks) * kFitPartials;
+  for (int c = 0; c < 7; ++c) {
+    double acc = 0.0;
+    for (int rb = t; rb < rows_blocks; rb += 256) acc += p[(int64_t)rb * kFitPartials + c];
+    red[t] = acc;
+    __syncthreads();
+    for (int n = 128; n > 0; n >>= 1) {
+      if (t < n) red[t] += red[t + n];
+      __syncthreads();
+    }
+    if (t == 0) {
+      if (c < 6) jobs.err[j][(int64_t)u * 6 + c] = (float)red[0];
+      else if (jobs.energy[j]) jobs.energy[j][u] = (float)red[0];
+    }
+    __syncthreads();
+  }
+}
+
 // sqrt(s_j): the activation scale that the saliency key uses.
 __global__ void fit_scale_kernel(const float* __restrict__ s, int C, float* __restrict__ scale) {
   const int j = blockIdx.x * blockDim.x + threadIdx.x;
@@ -172,7 +240,7 @@ windq_status launch_fit(windq_ctx* ctx, const __half* W, int R, int U, int64_t l
   const int chunk = fit_cand_chunk(G), stride = fit_cand_stride(chunk);
   const size_t smem = (size_t)kFitWarpsPerBlock * GPW * stride * sizeof(Cand);
   const int id = (PROTECT ? kFitProtectG32 : kFitG32) + g_index(G);
-  if (windq_status rc = prepare_kernel(ctx, id, fit_eval_kernel<G, PROTECT, false>, kFitWarpsPerBlock * 32, smem, true)) return rc;
+  if (windq_status rc = prepare_kernel(ctx, id, fit_eval_kernel<G, PROTECT, false, false>, kFitWarpsPerBlock * 32, smem, true)) return rc;
   const int blocks_per_sm = ctx->occupancy[id];
   const int64_t n_items = (int64_t)U * rows_blocks;
   WINDQ_REQUIRE(ctx, n_items < (1ll << 28), WINDQ_ERR_SHAPE, "windq_fit_eval: R * C is too large for one call");
@@ -182,7 +250,7 @@ windq_status launch_fit(windq_ctx* ctx, const __half* W, int R, int U, int64_t l
   // 2048 x 2048.  A 512 x 2048 matrix, whose 1024 items would fill less than half the warps, gains 1.5x.)
   const bool in_parts = 2 * n_items < 3 * full_grid * kFitWarpsPerBlock;
   if (in_parts)
-    if (windq_status rc = prepare_kernel(ctx, id + kFitPartsOffset, fit_eval_kernel<G, PROTECT, true>, kFitWarpsPerBlock * 32, smem, false))
+    if (windq_status rc = prepare_kernel(ctx, id + kFitPartsOffset, fit_eval_kernel<G, PROTECT, true, false>, kFitWarpsPerBlock * 32, smem, false))
       return rc;
   int64_t grid = full_grid;
   const int64_t need = ((in_parts ? 5 : 1) * n_items + kFitWarpsPerBlock - 1) / kFitWarpsPerBlock;
@@ -190,15 +258,48 @@ windq_status launch_fit(windq_ctx* ctx, const __half* W, int R, int U, int64_t l
   WINDQ_CUDA(ctx, cudaMemsetAsync(next_item, 0, sizeof(unsigned int), st));
   if (PROTECT) fit_scale_kernel<<<(unsigned)((U * G + 255) / 256), 256, 0, st>>>(s, U * G, scale);
   if (in_parts)
-    fit_eval_kernel<G, PROTECT, true><<<(unsigned)grid, kFitWarpsPerBlock * 32, smem, st>>>(
+    fit_eval_kernel<G, PROTECT, true, false><<<(unsigned)grid, kFitWarpsPerBlock * 32, smem, st>>>(
         W, R, U, ldw, s, clip, K, partial, clip_idx_out, group_err_out, rows_blocks, chunk, stride, scale, thresh,
-        __builtin_nanf(""), next_item);
+        __builtin_nanf(""), next_item, FitJobs());
   else
-    fit_eval_kernel<G, PROTECT, false><<<(unsigned)grid, kFitWarpsPerBlock * 32, smem, st>>>(
+    fit_eval_kernel<G, PROTECT, false, false><<<(unsigned)grid, kFitWarpsPerBlock * 32, smem, st>>>(
         W, R, U, ldw, s, clip, K, partial, clip_idx_out, group_err_out, rows_blocks, chunk, stride, scale, thresh,
-        __builtin_nanf(""), next_item);
+        __builtin_nanf(""), next_item, FitJobs());
   WINDQ_CUDA(ctx, cudaGetLastError());
   fit_finalize_kernel<<<(unsigned)U, 256, 0, st>>>(partial, rows_blocks, err_out, energy_out);
+  WINDQ_CUDA(ctx, cudaGetLastError());
+  return WINDQ_OK;
+}
+
+template <int G>
+windq_status launch_fit_batch(windq_ctx* ctx, const FitJobs& jobs, const float* clip, int K, cudaStream_t st) {
+  constexpr int GPW = Map<G>::GPW;
+  const int chunk = fit_cand_chunk(G), stride = fit_cand_stride(chunk);
+  const size_t smem = (size_t)kFitWarpsPerBlock * GPW * stride * sizeof(Cand);
+  const int id = kFitBatchG32 + g_index(G);
+  if (windq_status rc = prepare_kernel(ctx, id, fit_eval_kernel<G, false, false, true>, kFitWarpsPerBlock * 32, smem, true)) return rc;
+  const int64_t full_grid = (int64_t)ctx->sm_count * ctx->occupancy[id];
+  const int64_t n_items = jobs.first_item[jobs.n];
+  const bool in_parts = 2 * n_items < 3 * full_grid * kFitWarpsPerBlock;
+  if (in_parts)
+    if (windq_status rc = prepare_kernel(ctx, id + 5, fit_eval_kernel<G, false, true, true>, kFitWarpsPerBlock * 32, smem, false))
+      return rc;
+  int64_t grid = full_grid;
+  const int64_t need = ((in_parts ? 5 : 1) * n_items + kFitWarpsPerBlock - 1) / kFitWarpsPerBlock;
+  if (grid > need) grid = need;
+  unsigned int* next_item = (unsigned int*)ctx->scratch;
+  double* partial = (double*)((char*)ctx->scratch + 16);
+  WINDQ_CUDA(ctx, cudaMemsetAsync(next_item, 0, sizeof(unsigned int), st));
+  if (in_parts)
+    fit_eval_kernel<G, false, true, true><<<(unsigned)grid, kFitWarpsPerBlock * 32, smem, st>>>(
+        nullptr, 0, 0, 0, nullptr, clip, K, partial, nullptr, nullptr, 0, chunk, stride, nullptr, nullptr, __builtin_nanf(""),
+        next_item, jobs);
+  else
+    fit_eval_kernel<G, false, false, true><<<(unsigned)grid, kFitWarpsPerBlock * 32, smem, st>>>(
+        nullptr, 0, 0, 0, nullptr, clip, K, partial, nullptr, nullptr, 0, chunk, stride, nullptr, nullptr, __builtin_nanf(""),
+        next_item, jobs);
+  WINDQ_CUDA(ctx, cudaGetLastError());
+  fit_finalize_batch_kernel<<<jobs.first_unit[jobs.n], 256, 0, st>>>(partial, GPW, jobs);
   WINDQ_CUDA(ctx, cudaGetLastError());
   return WINDQ_OK;
 }
@@ -267,6 +368,65 @@ windq_status windq_fit_eval_protected(windq_ctx* ctx, const void* W, int64_t R, 
   if (ctx && !thresh) return windq::fail(ctx, WINDQ_ERR_NULL, "windq_fit_eval_protected: thresh is NULL");
   return fit_eval_any(ctx, "windq_fit_eval_protected", W, R, C, ldw, G, s, clip_grid, K, thresh, err_out, energy_out,
                       clip_idx_out, group_err_out, stream);
+}
+
+int64_t windq_scratch_bytes_fit_eval_batch(const windq_fit_job* jobs, int n_jobs, int G) {
+  if (!jobs || n_jobs <= 0 || !windq::valid_G(G)) return 0;
+  const int gpw = 32 / (G / 32);
+  int64_t items = 0;
+  for (int j = 0; j < n_jobs; ++j) {
+    if (jobs[j].R <= 0 || jobs[j].C <= 0) return 0;
+    items += (jobs[j].C / G) * ((jobs[j].R + gpw - 1) / gpw);
+  }
+  return 16 + items * windq::kFitPartials * (int64_t)sizeof(double);
+}
+
+windq_status windq_fit_eval_batch(windq_ctx* ctx, const windq_fit_job* jobs, int n_jobs, int G, const float* clip_grid, int K,
+                                  void* stream) {
+  using namespace windq;
+  const char* who = "windq_fit_eval_batch";
+  if (!ctx) return fail(nullptr, WINDQ_ERR_NULL, "%s: ctx is NULL", who);
+  WINDQ_REQUIRE(ctx, jobs && clip_grid, WINDQ_ERR_NULL, "%s: jobs or clip_grid is NULL", who);
+  WINDQ_REQUIRE(ctx, n_jobs >= 1 && n_jobs <= kFitMaxJobs, WINDQ_ERR_SHAPE, "%s: n_jobs = %d is outside [1, %d]", who, n_jobs,
+                kFitMaxJobs);
+  if (windq_status st = check_K(ctx, who, K)) return st;
+  FitJobs fj;
+  memset(&fj, 0, sizeof(fj));
+  fj.n = n_jobs;
+  int64_t items = 0, units = 0;
+  for (int j = 0; j < n_jobs; ++j) {
+    const windq_fit_job& b = jobs[j];
+    if (windq_status st = check_matrix(ctx, who, b.W, b.R, b.C, b.ldw, G)) return st;
+    WINDQ_REQUIRE(ctx, b.s && b.err_out, WINDQ_ERR_NULL, "%s: job %d: s or err_out is NULL", who, j);
+    WINDQ_REQUIRE(ctx, aligned16(b.s), WINDQ_ERR_ALIGN, "%s: job %d: s is not 16-byte aligned", who, j);
+    const int gpw = 32 / (G / 32);
+    fj.W[j] = (const __half*)b.W;
+    fj.s[j] = b.s;
+    fj.clip_idx[j] = b.clip_idx_out;
+    fj.group_err[j] = b.group_err_out;
+    fj.err[j] = b.err_out;
+    fj.energy[j] = b.energy_out;
+    fj.ldw[j] = b.ldw;
+    fj.R[j] = (int)b.R;
+    fj.U[j] = (int)(b.C / G);
+    fj.first_item[j] = (unsigned int)items;
+    fj.first_unit[j] = (unsigned int)units;
+    items += (b.C / G) * ((b.R + gpw - 1) / gpw);
+    units += b.C / G;
+    WINDQ_REQUIRE(ctx, items < (1ll << 28), WINDQ_ERR_SHAPE, "%s: the batch is too large for one call", who);
+  }
+  fj.first_item[n_jobs] = (unsigned int)items;
+  fj.first_unit[n_jobs] = (unsigned int)units;
+  DeviceGuard guard(ctx->device);
+  if (windq_status st = ensure_scratch(ctx, 16 + items * kFitPartials * (int64_t)sizeof(double))) return st;
+  cudaStream_t st = (cudaStream_t)stream;
+  switch (G) {
+    case 32: return launch_fit_batch<32>(ctx, fj, clip_grid, K, st);
+    case 64: return launch_fit_batch<64>(ctx, fj, clip_grid, K, st);
+    case 128: return launch_fit_batch<128>(ctx, fj, clip_grid, K, st);
+    case 256: return launch_fit_batch<256>(ctx, fj, clip_grid, K, st);
+    default: return launch_fit_batch<512>(ctx, fj, clip_grid, K, st);
+  }
 }
 
 }  // extern "C"

@@ -512,3 +512,41 @@ def test_apply_plan_clip_indices_beyond_the_grid_mean_the_last_ratio(wq, ctx, or
     assert np.array_equal(got["scales"].cpu().numpy().view(np.uint16), want["scales"])
     assert np.array_equal(got["zeros"].cpu().numpy().view(np.uint16), want["zeros"])
     assert np.array_equal(got["wq"].cpu().numpy().view(np.uint16), want["wq"])
+
+
+@pytest.mark.parametrize("G,shapes", [(128, [(300, 512), (64, 1024), (1000, 256), (17, 128)]),
+                                      (64, [(40, 256), (2048, 2048)]),
+                                      (256, [(512, 2048)] * 3 + [(2048, 2048)]),
+                                      (32, [(5, 32)])])
+def test_fit_eval_batch_equals_the_separate_calls(wq, ctx, oracle, G, shapes):
+    """Several matrices in one launch: every output of every job equals that of its own windq_fit_eval call bit
+    for bit (clip indices, group errors, and the unit sums, which are added in the same order), and sampled units
+    equal the oracle."""
+    grid = ws.clip_grid(20)
+    gd = torch.from_numpy(grid).cuda()
+    Ws = [ws.weights(R, C, 300 + i, "student_t").cuda() for i, (R, C) in enumerate(shapes)]
+    ss = [(torch.rand(C, generator=torch.Generator().manual_seed(i)) * 3 + 0.01).cuda() for i, (R, C) in enumerate(shapes)]
+    got = wq.windq_fit_eval_batch(ctx, Ws, G, ss, gd, want_group_err=True)
+    torch.cuda.synchronize()
+    for W, s, out in zip(Ws, ss, got):
+        one = wq.windq_fit_eval(ctx, W, G, s, gd, want_group_err=True)
+        assert torch.equal(out["clip_idx"], one["clip_idx"])
+        assert torch.equal(out["group_err"].view(torch.int32), one["group_err"].view(torch.int32))
+        assert torch.equal(out["err"].view(torch.int32), one["err"].view(torch.int32))
+        assert torch.equal(out["energy"].view(torch.int32), one["energy"].view(torch.int32))
+    W, s, out = Ws[0], ss[0], got[0]
+    want = oracle.fit_eval(W.cpu().numpy()[:, :G], G, s.cpu().numpy()[:G], grid)
+    assert np.array_equal(out["clip_idx"][:, :1].cpu().numpy(), want["clip_idx"])
+    assert close(out["err"][:1].cpu().numpy(), want["err"]).all()
+
+
+def test_fit_eval_batch_argument_checks(wq, ctx):
+    gd = torch.from_numpy(ws.clip_grid(4)).cuda()
+    W = torch.zeros((8, 128), dtype=torch.float16, device="cuda")
+    s = torch.ones(128, device="cuda")
+    with pytest.raises(Exception):
+        wq.windq_fit_eval_batch(ctx, [W] * 17, 128, [s] * 17, gd)
+    with pytest.raises(Exception):
+        wq.windq_fit_eval_batch(ctx, [W, torch.zeros((8, 100), dtype=torch.float16, device="cuda")], 128, [s, s], gd)
+    out = wq.windq_fit_eval_batch(ctx, [W], 128, [s], gd)
+    assert (out[0]["err"] == 0).all()

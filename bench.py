@@ -57,7 +57,8 @@ def parse_args():
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--separate-fits", action="store_true",
-                    help="one windq_fit_eval call per matrix instead of one windq_fit_eval_batch call per block and chunk width")
+                    help="one windq_unit_features and one windq_fit_eval call per matrix instead of one batched call of each per "
+                         "block and chunk width")
     ap.add_argument("--extras", action="store_true",
                     help="also time the calls beyond the five of a step (protection, refinement, allocator) on block 0")
     return ap.parse_args()
@@ -218,6 +219,7 @@ class Buffers:
                       scales=(maxUR, torch.float16), zeros=(maxUR, torch.float16))
         # one set of fit outputs per matrix of a block, for the batched fit (all matrices of a block in one call)
         for mi, m in enumerate(mats):
+            shapes["feat%d" % mi] = ((m.C // Gmin) * 8, torch.float32)
             shapes["err%d" % mi] = ((m.C // Gmin) * 6, torch.float32)
             shapes["energy%d" % mi] = (m.C // Gmin, torch.float32)
         self.clip_idx_m = [torch.empty(4 * (m.C // Gmin) * m.R, dtype=torch.uint8, device=dev) for m in mats]
@@ -297,19 +299,19 @@ def score_block(wq, ctx, spec, Wb, Xb, plans_b, buf, grid_d, timer=None, sink=No
         launches += 2
     if BATCH_FITS:
         for G in spec.chunk_widths:
-            for mi, m in enumerate(mats):
-                U = m.C // G
-                feat = buf.take("feat")[:U * 8].view(U, 8)
-                wq.windq_unit_features(ctx, Wb[mi], G, buf.s[m.x_id], feat)
-                launches += 2
-                if sink:
-                    sink("feat", feat)
+            stats = [buf.s[m.x_id] for m in mats]
+            feats = [buf.take("feat%d" % mi)[:(m.C // G) * 8].view(m.C // G, 8) for mi, m in enumerate(mats)]
+            wq.windq_unit_features_batch(ctx, Wb, G, stats, feats)
+            launches += 2
+            if sink:
+                for mi in range(len(mats)):
+                    sink("feat%d" % mi, feats[mi])
             outs = [dict(err=buf.take("err%d" % mi)[:(m.C // G) * 6].view(m.C // G, 6),
                          energy=buf.take("energy%d" % mi)[:m.C // G],
                          clip_idx=buf.clip_idx_m[mi][:4 * (m.C // G) * m.R].view(4, m.C // G, m.R))
                     for mi, m in enumerate(mats)]
             e0 = timer.start() if timer else None
-            wq.windq_fit_eval_batch(ctx, Wb, G, [buf.s[m.x_id] for m in mats], grid_d, outs=outs)
+            wq.windq_fit_eval_batch(ctx, Wb, G, stats, grid_d, outs=outs)
             if timer:
                 timer.stop(e0)
             launches += 2
@@ -643,7 +645,8 @@ def main():
     scratch = max(max(wq.windq_scratch_bytes_fit_eval(m.R, m.C, G), wq.windq_scratch_bytes_unit_features(m.R, m.C, G))
                   for m in mats for G in spec.chunk_widths)
     if BATCH_FITS:
-        scratch = max(scratch, max(sum(wq.windq_scratch_bytes_fit_eval(m.R, m.C, G) for m in mats) for G in spec.chunk_widths))
+        scratch = max(scratch, max(sum(wq.windq_scratch_bytes_fit_eval(m.R, m.C, G) for m in mats) for G in spec.chunk_widths),
+                      2 * max(sum(wq.windq_scratch_bytes_unit_features(m.R, m.C, G) for m in mats) for G in spec.chunk_widths))
     wq.windq_reserve(ctx, scratch)
 
     elems, units = workload_counts(spec, n_blocks)
@@ -708,8 +711,8 @@ def main():
                     config=dict(workload=spec.name, blocks=n_blocks, elements_per_chunk_width=elems, units=units, K=spec.K,
                                 chunk_widths=list(spec.chunk_widths), plan_targets=list(TARGET_BITS), apply_chunk_width=APPLY_G,
                                 tokens=spec.T, weights=spec.dist, parallelism="replica per GPU",
-                                fits="one windq_fit_eval_batch call per block and chunk width" if BATCH_FITS
-                                else "one windq_fit_eval call per matrix",
+                                fits="one windq_unit_features_batch and one windq_fit_eval_batch call per block and chunk width" if BATCH_FITS
+                                else "one windq_unit_features and one windq_fit_eval call per matrix",
                                 l2="every step streams %.1f GB of inputs, far above the 126 MB L2" % (
                                     (2 * elems + 2 * spec.T * sum(c for _, c in inputs_of(spec)) * n_blocks) / 1e9)),
                     clocks=clocks, e2e=e2e, gpu_launches=launches, roofline=roofline, cpu_baseline=cpu,

@@ -159,6 +159,22 @@ windq_status windq_effective_bits(windq_ctx* ctx, const uint8_t* actions, int64_
                                   int64_t* code_offsets_out, int64_t* total_centibits_out,
                                   int64_t* total_packed_bytes_out, void* stream);
 
+/* windq_unit_features for several matrices in one pass (no counterpart in the paper; same reason as
+ * windq_fit_eval_batch below).  Every job is one windq_unit_features call: W, R, C, ldw, s, feat_out as there;
+ * all jobs share G.  The features that come from the histogram (std, abs_mean, sparsity, outlier_frac) and
+ * those of s are those of the separate calls bit for bit; the mean is a sum of block sums whose blocks fall
+ * differently, so its last bits can differ (within 1e-6 relative).
+ *   jobs: HOST array of n_jobs descriptors (1 <= n_jobs <= 16), read during the call only.
+ * Scratch: windq_scratch_bytes_unit_features_batch (128 KB per unit of all jobs). */
+typedef struct {
+  const void* W;    /* fp16 [R][ldw] */
+  int64_t R, C, ldw;
+  const float* s;   /* fp32 [C] */
+  float* feat_out;  /* fp32 [U][8] */
+} windq_feat_job;
+int64_t windq_scratch_bytes_unit_features_batch(const windq_feat_job* jobs, int n_jobs, int G);
+windq_status windq_unit_features_batch(windq_ctx* ctx, const windq_feat_job* jobs, int n_jobs, int G, void* stream);
+
 /* windq_fit_eval for several matrices in one launch (the paper has no counterpart: the consumer loops
  * over the seven projections of every block, and matrices that are small against the GPU -- a few million
  * weights -- neither fill it nor amortise the fixed cost of a call on their own).  All jobs share G, the

@@ -56,6 +56,9 @@ def _load() -> ctypes.CDLL:
     lib.windq_act_stats_noalloc.argtypes = [vp, vp, i64, i64, i64, vp, vp]
     lib.windq_unit_features.argtypes = [vp, vp, i64, i64, i64, i32, vp, vp, vp]
     lib.windq_fit_eval.argtypes = [vp, vp, i64, i64, i64, i32, vp, vp, i32, vp, vp, vp, vp, vp]
+    lib.windq_unit_features_batch.argtypes = [vp, vp, i32, i32, vp]
+    lib.windq_scratch_bytes_unit_features_batch.restype = i64
+    lib.windq_scratch_bytes_unit_features_batch.argtypes = [vp, i32, i32]
     lib.windq_fit_eval_batch.argtypes = [vp, vp, i32, i32, vp, i32, vp]
     lib.windq_scratch_bytes_fit_eval_batch.restype = i64
     lib.windq_scratch_bytes_fit_eval_batch.argtypes = [vp, i32, i32]
@@ -245,6 +248,32 @@ def windq_fit_eval(ctx: Context, W: torch.Tensor, G: int, s: torch.Tensor, clip_
                                                  clip_grid.numel(), _ptr(thresh), _ptr(out["err"]), _ptr(out["energy"]),
                                                  _ptr(out["clip_idx"]), _ptr(out["group_err"]), _stream(stream)))
     return out
+
+
+class _FeatJob(ctypes.Structure):
+    _fields_ = [("W", ctypes.c_void_p), ("R", ctypes.c_int64), ("C", ctypes.c_int64), ("ldw", ctypes.c_int64),
+                ("s", ctypes.c_void_p), ("feat_out", ctypes.c_void_p)]
+
+
+def windq_unit_features_batch(ctx: Context, Ws, G: int, ss, feats=None, stream=None) -> list:
+    """windq_unit_features of up to 16 matrices in one pass.  ``feats`` may hold one preallocated [U, 8] fp32
+    tensor per matrix.  Returns the list of feature tensors."""
+    if len(Ws) != len(ss) or not Ws:
+        raise ValueError("Ws and ss must be non-empty and equally long")
+    jobs = (_FeatJob * len(Ws))()
+    outs = []
+    for j, (W, s) in enumerate(zip(Ws, ss)):
+        R, C, ldw = _matrix(W, "W")
+        _need(s, torch.float32, "s", 1)
+        U = C // G if G > 0 else 0
+        f = feats[j] if feats is not None else torch.empty((U, N_FEATURES), dtype=torch.float32, device=W.device)
+        _need(f, torch.float32, "feat_out", 2)
+        if tuple(f.shape) != (U, N_FEATURES) or not f.is_contiguous():
+            raise ValueError("feat_out must be a contiguous [U, 8] tensor")
+        jobs[j] = _FeatJob(W.data_ptr(), R, C, ldw, s.data_ptr(), f.data_ptr())
+        outs.append(f)
+    ctx._check(_lib.windq_unit_features_batch(ctx._h, ctypes.cast(jobs, ctypes.c_void_p), len(Ws), int(G), _stream(stream)))
+    return outs
 
 
 class _FitJob(ctypes.Structure):

@@ -13,6 +13,8 @@
 //           is what keeps enough bytes on their way from HBM.  The signed sum of every
 //           (unit, block) segment goes to its own slot in scratch as a double.
 //   pass 2  one block per unit scans the histogram and writes the eight features.
+#include <string.h>
+
 #include "windq_internal.cuh"
 
 namespace windq {
@@ -27,6 +29,22 @@ constexpr int kFeatMaxBlocks = 1024;  // bound on the pass-1 grid that the scrat
 #define WINDQ_FEAT_LOADS 4
 #endif
 constexpr int kFeatLoads = WINDQ_FEAT_LOADS;  // rows in flight per thread
+
+// Several matrices in one pass (windq_unit_features_batch): the (unit, row) pairs are numbered through all
+// jobs, job-major; job j owns the pairs [first_pair[j], first_pair[j + 1]) and the units
+// [first_unit[j], first_unit[j + 1]) of the histogram and slot arrays.  n = 0: one matrix, described by the
+// kernels' scalar parameters.
+constexpr int kFeatMaxJobs = 16;
+struct FeatJobs {
+  const __half* W[kFeatMaxJobs];
+  const float* s[kFeatMaxJobs];
+  float* feat[kFeatMaxJobs];
+  long long ldw[kFeatMaxJobs];
+  long long first_pair[kFeatMaxJobs + 1];
+  int R[kFeatMaxJobs];
+  int first_unit[kFeatMaxJobs + 1];
+  int n;
+};
 
 __device__ __forceinline__ void hist_add8(unsigned int* sh, const uint4& raw, float& part) {
   const unsigned int v[4] = {raw.x, raw.y, raw.z, raw.w};
@@ -43,8 +61,8 @@ __device__ __forceinline__ void hist_add8(unsigned int* sh, const uint4& raw, fl
 // (u * R) / rows_per_block + j.
 template <int G>
 __global__ void __launch_bounds__(kFeatThreads, kFeatThreads <= 256 ? 4 : 1)  // at most 64 registers per thread
-feat_hist_kernel(const __half* __restrict__ W, int R, int64_t ldw, long long rows_per_block, long long total_rows,
-                 unsigned int* __restrict__ hist, double* __restrict__ slot_sum, int slots_per_unit) {
+feat_hist_kernel(const __half* __restrict__ W_one, int R_one, int64_t ldw_one, long long rows_per_block, long long total_rows,
+                 unsigned int* __restrict__ hist, double* __restrict__ slot_sum, int slots_per_unit, const FeatJobs jobs) {
   extern __shared__ unsigned int sh[];
   __shared__ double wsum[kFeatThreads / 32];
   constexpr int TPR = G / 8;               // threads per row (8 halves = 16 bytes each)
@@ -55,8 +73,21 @@ feat_hist_kernel(const __half* __restrict__ W, int R, int64_t ldw, long long row
   long long p = (long long)blockIdx.x * rows_per_block;
   const long long p_end = min(p + rows_per_block, total_rows);
   while (p < p_end) {
-    const int u = (int)(p / R);
-    const int r0 = (int)(p - (long long)u * R);
+    const __half* W = W_one;
+    int R = R_one, unit0 = 0;
+    int64_t ldw = ldw_one;
+    long long pair0 = 0;
+    if (jobs.n) {
+      int j = 0;
+      while (j + 1 < jobs.n && p >= jobs.first_pair[j + 1]) ++j;
+      W = jobs.W[j];
+      R = jobs.R[j];
+      ldw = jobs.ldw[j];
+      unit0 = jobs.first_unit[j];
+      pair0 = jobs.first_pair[j];
+    }
+    const int u = (int)((p - pair0) / R);
+    const int r0 = (int)(p - pair0 - (long long)u * R);
     const int r1 = (int)min((long long)R, r0 + (p_end - p));
     const __half* base = W + (int64_t)u * G + tc * 8;
     double sum = 0.0;
@@ -78,10 +109,10 @@ feat_hist_kernel(const __half* __restrict__ W, int R, int64_t ldw, long long row
     if (threadIdx.x == 0) {
       double t = 0.0;
       for (int i = 0; i < kFeatThreads / 32; ++i) t += wsum[i];
-      const long long first_block = ((long long)u * R) / rows_per_block;
-      slot_sum[(int64_t)u * slots_per_unit + (blockIdx.x - first_block)] = t;
+      const long long first_block = (pair0 + (long long)u * R) / rows_per_block;
+      slot_sum[(int64_t)(unit0 + u) * slots_per_unit + (blockIdx.x - first_block)] = t;
     }
-    unsigned int* gh = hist + (int64_t)u * kBins;
+    unsigned int* gh = hist + (int64_t)(unit0 + u) * kBins;
     for (int i = threadIdx.x; i < kBins; i += kFeatThreads) {
       const unsigned int c = sh[i];
       if (c) {
@@ -99,18 +130,32 @@ feat_hist_kernel(const __half* __restrict__ W, int R, int64_t ldw, long long row
 // memory starting at bin t mod 32, so that the lanes of a warp stay on different banks.
 __global__ void __launch_bounds__(1024)
 feat_finalize_kernel(const unsigned int* __restrict__ hist, const double* __restrict__ slot_sum, int slots_per_unit,
-                     long long rows_per_block, int R, int G, const float* __restrict__ s, float* __restrict__ feat) {
+                     long long rows_per_block, int R_one, int G, const float* __restrict__ s_one, float* __restrict__ feat_one,
+                     const FeatJobs jobs) {
   extern __shared__ unsigned int sh[];  // kBins counts
   __shared__ unsigned long long warp_total[32];
   __shared__ double red[3][32];
   __shared__ unsigned long long redc[2][32];
   __shared__ double s_stat[3];
   __shared__ int p99_bin;
-  const int u = blockIdx.x, t = threadIdx.x, lane = t & 31, wp = t >> 5;
+  const int ug = blockIdx.x, t = threadIdx.x, lane = t & 31, wp = t >> 5;  // ug: the unit's place in hist and slot_sum
+  int u = ug, R = R_one;
+  const float* s = s_one;
+  float* feat = feat_one;
+  long long pair0 = 0;
+  if (jobs.n) {
+    int j = 0;
+    while (j + 1 < jobs.n && ug >= jobs.first_unit[j + 1]) ++j;
+    u = ug - jobs.first_unit[j];
+    R = jobs.R[j];
+    s = jobs.s[j];
+    feat = jobs.feat[j];
+    pair0 = jobs.first_pair[j];
+  }
   const long long n = (long long)R * G;
   const unsigned long long k = (unsigned long long)((99 * n + 99) / 100);  // rank of P99, 1-indexed
   {
-    const uint4* src = reinterpret_cast<const uint4*>(hist + (int64_t)u * kBins);
+    const uint4* src = reinterpret_cast<const uint4*>(hist + (int64_t)ug * kBins);
     uint4* dst = reinterpret_cast<uint4*>(sh);
 #pragma unroll
     for (int i = 0; i < kBins / 4 / 1024; ++i) dst[i * 1024 + t] = src[i * 1024 + t];
@@ -189,9 +234,10 @@ feat_finalize_kernel(const unsigned int* __restrict__ hist, const double* __rest
   }
   double ss = 0.0;
   {
-    const long long first = ((long long)u * R) / rows_per_block, last = ((long long)(u + 1) * R - 1) / rows_per_block;
+    const long long first = (pair0 + (long long)u * R) / rows_per_block;
+    const long long last = (pair0 + (long long)(u + 1) * R - 1) / rows_per_block;
     const int cnt = (int)(last - first + 1);
-    for (int i = t; i < cnt; i += 1024) ss += slot_sum[(int64_t)u * slots_per_unit + i];
+    for (int i = t; i < cnt; i += 1024) ss += slot_sum[(int64_t)ug * slots_per_unit + i];
   }
 #pragma unroll
   for (int m = 16; m > 0; m >>= 1) {
@@ -241,9 +287,9 @@ struct FeatGrid {
   long long rows_per_block;
   int slots_per_unit;
 };
-inline FeatGrid feat_grid(int sm_count, int64_t R, int64_t U) {
+inline FeatGrid feat_grid(int sm_count, int64_t R, int64_t U, long long total_pairs = 0) {  // R: the largest row count
   FeatGrid g;
-  const long long total = (long long)U * R;
+  const long long total = total_pairs ? total_pairs : (long long)U * R;
   int nb = sm_count < kFeatMaxBlocks ? sm_count : kFeatMaxBlocks;
   const long long min_rows = 16;  // a block should see at least a few rows
   if ((long long)nb * min_rows > total) nb = (int)((total + min_rows - 1) / min_rows);
@@ -255,11 +301,12 @@ inline FeatGrid feat_grid(int sm_count, int64_t R, int64_t U) {
 
 template <int G>
 windq_status launch_hist(windq_ctx* ctx, const __half* W, int R, int U, int64_t ldw, const FeatGrid& fg,
-                         unsigned int* hist, double* slot_sum, cudaStream_t st) {
+                         unsigned int* hist, double* slot_sum, cudaStream_t st, const FeatJobs& jobs = FeatJobs(),
+                         long long total_pairs = 0) {
   const size_t smem = (size_t)kBins * sizeof(unsigned int);
   if (windq_status rc = prepare_kernel(ctx, kHistG32 + g_index(G), feat_hist_kernel<G>, kFeatThreads, smem, false)) return rc;
-  feat_hist_kernel<G><<<(unsigned)fg.blocks, kFeatThreads, smem, st>>>(W, R, ldw, fg.rows_per_block, (long long)U * R, hist,
-                                                                      slot_sum, fg.slots_per_unit);
+  feat_hist_kernel<G><<<(unsigned)fg.blocks, kFeatThreads, smem, st>>>(
+      W, R, ldw, fg.rows_per_block, total_pairs ? total_pairs : (long long)U * R, hist, slot_sum, fg.slots_per_unit, jobs);
   WINDQ_CUDA(ctx, cudaGetLastError());
   return WINDQ_OK;
 }
@@ -303,7 +350,77 @@ windq_status windq_unit_features(windq_ctx* ctx, const void* W, int64_t R, int64
   }
   if (rc != WINDQ_OK) return rc;
   if (windq_status st2 = prepare_kernel(ctx, kFinalize, feat_finalize_kernel, 1024, kBins * sizeof(unsigned int), false)) return st2;
-  feat_finalize_kernel<<<(unsigned)U, 1024, kBins * sizeof(unsigned int), st>>>(hist, slot_sum, fg.slots_per_unit, fg.rows_per_block, (int)R, G, s, feat_out);
+  feat_finalize_kernel<<<(unsigned)U, 1024, kBins * sizeof(unsigned int), st>>>(hist, slot_sum, fg.slots_per_unit, fg.rows_per_block, (int)R, G, s, feat_out, FeatJobs());
+  WINDQ_CUDA(ctx, cudaGetLastError());
+  return WINDQ_OK;
+}
+
+int64_t windq_scratch_bytes_unit_features_batch(const windq_feat_job* jobs, int n_jobs, int G) {
+  if (!jobs || n_jobs <= 0 || !windq::valid_G(G)) return 0;
+  int64_t U = 0, pairs = 0, max_R = 0;
+  for (int j = 0; j < n_jobs; ++j) {
+    if (jobs[j].R <= 0 || jobs[j].C <= 0) return 0;
+    U += jobs[j].C / G;
+    pairs += (jobs[j].C / G) * jobs[j].R;
+    max_R = jobs[j].R > max_R ? jobs[j].R : max_R;
+  }
+  if (pairs <= 0) return 0;
+  // histograms + one double per (unit, block that can hold rows of it): a block has at least
+  // pairs / kFeatMaxBlocks pairs, so a unit of at most max_R rows meets at most the number of blocks below
+  const int64_t slots = max_R * windq::kFeatMaxBlocks / pairs + 3;
+  return U * windq::kBins * (int64_t)sizeof(unsigned int) + U * slots * (int64_t)sizeof(double);
+}
+
+windq_status windq_unit_features_batch(windq_ctx* ctx, const windq_feat_job* jobs, int n_jobs, int G, void* stream) {
+  using namespace windq;
+  const char* who = "windq_unit_features_batch";
+  if (!ctx) return fail(nullptr, WINDQ_ERR_NULL, "%s: ctx is NULL", who);
+  WINDQ_REQUIRE(ctx, jobs, WINDQ_ERR_NULL, "%s: jobs is NULL", who);
+  WINDQ_REQUIRE(ctx, n_jobs >= 1 && n_jobs <= kFeatMaxJobs, WINDQ_ERR_SHAPE, "%s: n_jobs = %d is outside [1, %d]", who, n_jobs,
+                kFeatMaxJobs);
+  FeatJobs fj;
+  memset(&fj, 0, sizeof(fj));
+  fj.n = n_jobs;
+  long long pairs = 0;
+  int64_t units = 0, max_R = 0;
+  for (int j = 0; j < n_jobs; ++j) {
+    const windq_feat_job& b = jobs[j];
+    if (windq_status st = check_matrix(ctx, who, b.W, b.R, b.C, b.ldw, G)) return st;
+    WINDQ_REQUIRE(ctx, b.s && b.feat_out, WINDQ_ERR_NULL, "%s: job %d: s or feat_out is NULL", who, j);
+    WINDQ_REQUIRE(ctx, b.R * (int64_t)G < (1ll << 32), WINDQ_ERR_SHAPE, "%s: job %d: R * G must be below 2^32", who, j);
+    fj.W[j] = (const __half*)b.W;
+    fj.s[j] = b.s;
+    fj.feat[j] = b.feat_out;
+    fj.ldw[j] = b.ldw;
+    fj.R[j] = (int)b.R;
+    fj.first_pair[j] = pairs;
+    fj.first_unit[j] = (int)units;
+    pairs += (b.C / G) * b.R;
+    units += b.C / G;
+    max_R = b.R > max_R ? b.R : max_R;
+  }
+  fj.first_pair[n_jobs] = pairs;
+  fj.first_unit[n_jobs] = (int)units;
+  WINDQ_REQUIRE(ctx, units <= 65535 * 32, WINDQ_ERR_SHAPE, "%s: too many units", who);
+  DeviceGuard guard(ctx->device);
+  if (windq_status st = ensure_scratch(ctx, windq_scratch_bytes_unit_features_batch(jobs, n_jobs, G))) return st;
+  cudaStream_t st = (cudaStream_t)stream;
+  unsigned int* hist = (unsigned int*)ctx->scratch;
+  double* slot_sum = (double*)((char*)ctx->scratch + units * kBins * (int64_t)sizeof(unsigned int));
+  const FeatGrid fg = feat_grid(ctx->sm_count, max_R, units, pairs);
+  WINDQ_CUDA(ctx, cudaMemsetAsync(hist, 0, (size_t)units * kBins * sizeof(unsigned int), st));
+  windq_status rc;
+  switch (G) {
+    case 32: rc = launch_hist<32>(ctx, nullptr, 0, 0, 0, fg, hist, slot_sum, st, fj, pairs); break;
+    case 64: rc = launch_hist<64>(ctx, nullptr, 0, 0, 0, fg, hist, slot_sum, st, fj, pairs); break;
+    case 128: rc = launch_hist<128>(ctx, nullptr, 0, 0, 0, fg, hist, slot_sum, st, fj, pairs); break;
+    case 256: rc = launch_hist<256>(ctx, nullptr, 0, 0, 0, fg, hist, slot_sum, st, fj, pairs); break;
+    default: rc = launch_hist<512>(ctx, nullptr, 0, 0, 0, fg, hist, slot_sum, st, fj, pairs); break;
+  }
+  if (rc != WINDQ_OK) return rc;
+  if (windq_status st2 = prepare_kernel(ctx, kFinalize, feat_finalize_kernel, 1024, kBins * sizeof(unsigned int), false)) return st2;
+  feat_finalize_kernel<<<(unsigned)units, 1024, kBins * sizeof(unsigned int), st>>>(hist, slot_sum, fg.slots_per_unit,
+                                                                                    fg.rows_per_block, 0, G, nullptr, nullptr, fj);
   WINDQ_CUDA(ctx, cudaGetLastError());
   return WINDQ_OK;
 }

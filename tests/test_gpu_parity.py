@@ -550,3 +550,25 @@ def test_fit_eval_batch_argument_checks(wq, ctx):
         wq.windq_fit_eval_batch(ctx, [W, torch.zeros((8, 100), dtype=torch.float16, device="cuda")], 128, [s, s], gd)
     out = wq.windq_fit_eval_batch(ctx, [W], 128, [s], gd)
     assert (out[0]["err"] == 0).all()
+
+
+@pytest.mark.parametrize("G,shapes", [(128, [(300, 512), (64, 1024), (1000, 256), (17, 128)]),
+                                      (64, [(40, 256), (2048, 2048)]),
+                                      (256, [(512, 2048)] * 3 + [(2048, 2048)]),
+                                      (32, [(5, 32)]),
+                                      (128, [(5000, 128), (3, 4096)])])
+def test_unit_features_batch_equals_the_separate_calls(wq, ctx, oracle, G, shapes):
+    """Several matrices in one pass: the histogram features and those of s equal the separate calls bit for bit,
+    the mean within tolerance, and everything equals the oracle within tolerance."""
+    Ws = [ws.weights(R, C, 400 + i, "student_t").cuda() for i, (R, C) in enumerate(shapes)]
+    for W in Ws:
+        W[::7, ::3] = 0
+    ss = [(torch.rand(C, generator=torch.Generator().manual_seed(i)) * 3 + 0.01).cuda() for i, (R, C) in enumerate(shapes)]
+    got = wq.windq_unit_features_batch(ctx, Ws, G, ss)
+    torch.cuda.synchronize()
+    for W, s, f in zip(Ws, ss, got):
+        one = wq.windq_unit_features(ctx, W, G, s)
+        assert torch.equal(f[:, 1:].view(torch.int32), one[:, 1:].view(torch.int32))
+        assert close(f[:, 0].cpu().numpy(), one[:, 0].cpu().numpy()).all()
+        want = oracle.unit_features(W.cpu().numpy(), G, s.cpu().numpy())
+        assert close(f.cpu().numpy(), want).all()

@@ -572,3 +572,23 @@ def test_unit_features_batch_equals_the_separate_calls(wq, ctx, oracle, G, shape
         assert close(f[:, 0].cpu().numpy(), one[:, 0].cpu().numpy()).all()
         want = oracle.unit_features(W.cpu().numpy(), G, s.cpu().numpy())
         assert close(f.cpu().numpy(), want).all()
+
+
+def test_batches_take_strided_matrices_and_preallocated_outputs(wq, ctx):
+    """Jobs that are column slices of one wider tensor (ldw > C) and outputs supplied by the caller."""
+    G = 128
+    big = ws.weights(200, 1024, 510, "student_t").cuda()
+    Ws = [big[:, :256], big[:, 256:768], big[:100, 768:]]
+    ss = [(torch.rand(W.shape[1], generator=torch.Generator().manual_seed(i)) + 0.01).cuda() for i, W in enumerate(Ws)]
+    gd = torch.from_numpy(ws.clip_grid(20)).cuda()
+    feats = [torch.full((W.shape[1] // G, 8), -1.0, device="cuda") for W in Ws]
+    out_f = wq.windq_unit_features_batch(ctx, Ws, G, ss, feats)
+    outs = [dict(err=torch.full((W.shape[1] // G, 6), -1.0, device="cuda")) for W in Ws]
+    out_e = wq.windq_fit_eval_batch(ctx, Ws, G, ss, gd, outs=outs, want_energy=False, want_clip_idx=False)
+    torch.cuda.synchronize()
+    for W, s, f, o, o_given in zip(Ws, ss, out_f, out_e, outs):
+        Wc = W.contiguous()
+        assert torch.equal(f[:, 1:], wq.windq_unit_features(ctx, Wc, G, s)[:, 1:])
+        one = wq.windq_fit_eval(ctx, Wc, G, s, gd)
+        assert o["err"].data_ptr() == o_given["err"].data_ptr() and o["energy"] is None and o["clip_idx"] is None
+        assert torch.equal(o["err"], one["err"])

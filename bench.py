@@ -220,9 +220,11 @@ class Buffers:
         # one set of fit outputs per matrix of a block, for the batched fit (all matrices of a block in one call)
         for mi, m in enumerate(mats):
             shapes["feat%d" % mi] = ((m.C // Gmin) * 8, torch.float32)
+            shapes["totals%d" % mi] = (2 * len(TARGET_BITS), torch.int64)
             shapes["err%d" % mi] = ((m.C // Gmin) * 6, torch.float32)
             shapes["energy%d" % mi] = (m.C // Gmin, torch.float32)
         self.clip_idx_m = [torch.empty(4 * (m.C // Gmin) * m.R, dtype=torch.uint8, device=dev) for m in mats]
+        self.offsets_m = [[torch.empty(m.C // Gmin + 1, dtype=torch.int64, device=dev) for _ in TARGET_BITS] for m in mats]
         self.rings = {k: [torch.zeros(n, dtype=dt, device=dev) for _ in range(ring)] for k, (n, dt) in shapes.items()}
         self.turn = {k: 0 for k in shapes}
         self.pending = {}          # (name, slot) -> event of the copy that still reads that slot
@@ -240,7 +242,9 @@ class Buffers:
 
     @property
     def totals(self):
-        return self.rings["totals"][self.last.get("totals", 0)]
+        """The totals written last (those of the block's last matrix when a block is accounted in one launch)."""
+        name = "totals%d" % (len(self.clip_idx_m) - 1) if BATCH_FITS else "totals"
+        return self.rings[name][self.last.get(name, 0)]
 
 
 class FitTimer:
@@ -266,15 +270,20 @@ class FitTimer:
 BATCH_FITS = True      # one windq_fit_eval_batch call per block and chunk width (False: one windq_fit_eval per matrix)
 
 
-def apply_plans(wq, ctx, spec, m, mi, W, s, G, clip_idx, plans_b, buf, grid_d, sink):
-    """The three plans of one matrix: bit accounting, then packing.  Returns the number of kernels launched."""
+def apply_plans(wq, ctx, spec, m, mi, W, s, G, clip_idx, plans_b, buf, grid_d, sink, accounted=None):
+    """The three plans of one matrix: bit accounting (unless `accounted` = (totals, [code offsets per plan]) holds
+    it already), then packing.  Returns the number of kernels launched."""
     U, launches = m.C // G, 0
-    totals = buf.take("totals")
+    totals = accounted[0] if accounted else buf.take("totals")
     for ti, target in enumerate(TARGET_BITS):
         acts = plans_b[target][mi]
-        eb = wq.windq_effective_bits(ctx, acts, m.R, G, out=dict(
-            unit_centibits=buf.unit_cb[:U], code_offsets=buf.offsets[:U + 1],
-            total_centibits=totals[2 * ti:2 * ti + 1], total_packed_bytes=totals[2 * ti + 1:2 * ti + 2]))
+        if accounted:
+            eb = dict(code_offsets=accounted[1][ti])
+            launches -= 1
+        else:
+            eb = wq.windq_effective_bits(ctx, acts, m.R, G, out=dict(
+                unit_centibits=buf.unit_cb[:U], code_offsets=buf.offsets[:U + 1],
+                total_centibits=totals[2 * ti:2 * ti + 1], total_packed_bytes=totals[2 * ti + 1:2 * ti + 2]))
         plan = wq.windq_apply_plan(ctx, W, G, s, grid_d, acts, eb["code_offsets"], buf.take("codes"), clip_idx,
                                    out=dict(scales=buf.take("scales")[:U * m.R].view(U, m.R),
                                             zeros=buf.take("zeros")[:U * m.R].view(U, m.R),
@@ -285,7 +294,7 @@ def apply_plans(wq, ctx, spec, m, mi, W, s, G, clip_idx, plans_b, buf, grid_d, s
             sink("scales", plan["scales"])
             sink("zeros", plan["zeros"])
     if sink:
-        sink("totals", totals)
+        sink("totals%d" % mi if accounted else "totals", totals)
     return launches
 
 
@@ -320,9 +329,19 @@ def score_block(wq, ctx, spec, Wb, Xb, plans_b, buf, grid_d, timer=None, sink=No
                     sink("err%d" % mi, outs[mi]["err"])
                     sink("energy%d" % mi, outs[mi]["energy"])
             if G == APPLY_G and plans_b:
+                # the bit accounting of the block's 21 (matrix, plan) pairs in one launch
+                totals = [buf.take("totals%d" % mi) for mi in range(len(mats))]
+                offs = [[buf.offsets_m[mi][ti][:m.C // G + 1] for ti in range(len(TARGET_BITS))] for mi, m in enumerate(mats)]
+                wq.windq_effective_bits_batch(
+                    ctx, [plans_b[target][mi] for mi in range(len(mats)) for target in TARGET_BITS],
+                    [m.R for m in mats for _ in TARGET_BITS], G,
+                    outs=[dict(unit_centibits=None, code_offsets=offs[mi][ti], total_centibits=totals[mi][2 * ti:2 * ti + 1],
+                               total_packed_bytes=totals[mi][2 * ti + 1:2 * ti + 2])
+                          for mi in range(len(mats)) for ti in range(len(TARGET_BITS))])
+                launches += 1
                 for mi, m in enumerate(mats):
                     launches += apply_plans(wq, ctx, spec, m, mi, Wb[mi], buf.s[m.x_id], G, outs[mi]["clip_idx"], plans_b, buf,
-                                            grid_d, sink)
+                                            grid_d, sink, accounted=(totals[mi], offs[mi]))
         return launches
     for mi, m in enumerate(mats):
         W, s = Wb[mi], buf.s[m.x_id]

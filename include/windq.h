@@ -196,6 +196,21 @@ int64_t windq_scratch_bytes_fit_eval_batch(const windq_fit_job* jobs, int n_jobs
 windq_status windq_fit_eval_batch(windq_ctx* ctx, const windq_fit_job* jobs, int n_jobs, int G, const float* clip_grid,
                                   int K, void* stream);
 
+/* windq_effective_bits for several plans in one launch (plans of different matrices may differ in U and R;
+ * G, scale_bits and zero_bits are shared).  Every job is one windq_effective_bits call with the same meanings,
+ * nullability and results.  Two jobs must not share an output array.
+ *   jobs: HOST array of n_jobs descriptors (1 <= n_jobs <= 32), read during the call only. */
+typedef struct {
+  const uint8_t* actions;           /* u8 [U] */
+  int64_t U, R;
+  int64_t* unit_centibits_out;      /* i64 [U], nullable */
+  int64_t* code_offsets_out;        /* i64 [U+1], nullable */
+  int64_t* total_centibits_out;     /* i64 [1] */
+  int64_t* total_packed_bytes_out;  /* i64 [1], nullable */
+} windq_bits_job;
+windq_status windq_effective_bits_batch(windq_ctx* ctx, const windq_bits_job* jobs, int n_jobs, int G, int scale_bits,
+                                        int zero_bits, void* stream);
+
 /* a4 -- apply a plan to one matrix ("the environment applies the selected quantization to the
  * current unit"): integer codes packed as described above, the fp16 scale and zero point of
  * every group, and optionally the fake-quantised weights for the consumer's forward pass.

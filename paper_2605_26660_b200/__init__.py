@@ -56,6 +56,7 @@ def _load() -> ctypes.CDLL:
     lib.windq_act_stats_noalloc.argtypes = [vp, vp, i64, i64, i64, vp, vp]
     lib.windq_unit_features.argtypes = [vp, vp, i64, i64, i64, i32, vp, vp, vp]
     lib.windq_fit_eval.argtypes = [vp, vp, i64, i64, i64, i32, vp, vp, i32, vp, vp, vp, vp, vp]
+    lib.windq_effective_bits_batch.argtypes = [vp, vp, i32, i32, i32, i32, vp]
     lib.windq_unit_features_batch.argtypes = [vp, vp, i32, i32, vp]
     lib.windq_scratch_bytes_unit_features_batch.restype = i64
     lib.windq_scratch_bytes_unit_features_batch.argtypes = [vp, i32, i32]
@@ -248,6 +249,43 @@ def windq_fit_eval(ctx: Context, W: torch.Tensor, G: int, s: torch.Tensor, clip_
                                                  clip_grid.numel(), _ptr(thresh), _ptr(out["err"]), _ptr(out["energy"]),
                                                  _ptr(out["clip_idx"]), _ptr(out["group_err"]), _stream(stream)))
     return out
+
+
+class _BitsJob(ctypes.Structure):
+    _fields_ = [("actions", ctypes.c_void_p), ("U", ctypes.c_int64), ("R", ctypes.c_int64),
+                ("unit_centibits_out", ctypes.c_void_p), ("code_offsets_out", ctypes.c_void_p),
+                ("total_centibits_out", ctypes.c_void_p), ("total_packed_bytes_out", ctypes.c_void_p)]
+
+
+def windq_effective_bits_batch(ctx: Context, actions_list, Rs, G: int, scale_bits: int = 16, zero_bits: int = 16,
+                               outs=None, stream=None) -> list:
+    """windq_effective_bits of up to 32 plans in one launch.  ``actions_list``: one u8 tensor per plan; ``Rs``: the
+    row count of each plan's matrix.  ``outs`` may hold one dict of preallocated outputs per plan (keys as
+    windq_effective_bits; a key that is present with value None is not computed).  Returns the list of dicts."""
+    if len(actions_list) != len(Rs) or not actions_list:
+        raise ValueError("actions_list and Rs must be non-empty and equally long")
+    jobs = (_BitsJob * len(actions_list))()
+    results = []
+    for j, (acts, R) in enumerate(zip(actions_list, Rs)):
+        _need(acts, torch.uint8, "actions", 1)
+        U = acts.numel()
+        out = dict(outs[j]) if outs else {}
+        dev = acts.device
+        if "unit_centibits" not in out:
+            out["unit_centibits"] = torch.empty(U, dtype=torch.int64, device=dev)
+        if "code_offsets" not in out:
+            out["code_offsets"] = torch.empty(U + 1, dtype=torch.int64, device=dev)
+        if out.get("total_centibits") is None:
+            out["total_centibits"] = torch.empty(1, dtype=torch.int64, device=dev)
+        if "total_packed_bytes" not in out:
+            out["total_packed_bytes"] = torch.empty(1, dtype=torch.int64, device=dev)
+        ptr = lambda x: None if x is None else x.data_ptr()
+        jobs[j] = _BitsJob(acts.data_ptr(), U, int(R), ptr(out["unit_centibits"]), ptr(out["code_offsets"]),
+                           ptr(out["total_centibits"]), ptr(out["total_packed_bytes"]))
+        results.append(out)
+    ctx._check(_lib.windq_effective_bits_batch(ctx._h, ctypes.cast(jobs, ctypes.c_void_p), len(actions_list), int(G),
+                                               int(scale_bits), int(zero_bits), _stream(stream)))
+    return results
 
 
 class _FeatJob(ctypes.Structure):

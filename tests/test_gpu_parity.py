@@ -592,3 +592,23 @@ def test_batches_take_strided_matrices_and_preallocated_outputs(wq, ctx):
         one = wq.windq_fit_eval(ctx, Wc, G, s, gd)
         assert o["err"].data_ptr() == o_given["err"].data_ptr() and o["energy"] is None and o["clip_idx"] is None
         assert torch.equal(o["err"], one["err"])
+
+
+def test_effective_bits_batch_equals_the_separate_calls(wq, ctx, oracle):
+    rng = np.random.default_rng(8)
+    G = 128
+    plans = [(rng.integers(0, 7, U).astype(np.uint8), R) for U, R in [(32, 4096), (86, 4096), (1, 3), (1500, 11008), (32, 11008)] * 4]
+    plans[3][0][5] = 9                                            # a code that is not an action: totals of -1
+    acts = [torch.from_numpy(a).cuda() for a, _ in plans]
+    got = wq.windq_effective_bits_batch(ctx, acts, [R for _, R in plans], G, 16, 8)
+    torch.cuda.synchronize()
+    for (a, R), ad, out in zip(plans, acts, got):
+        one = wq.windq_effective_bits(ctx, ad, R, G, 16, 8)
+        for key in ("unit_centibits", "code_offsets", "total_centibits", "total_packed_bytes"):
+            assert torch.equal(out[key], one[key]), key
+    want = oracle.effective_bits(plans[0][0], plans[0][1], G, 16, 8)
+    assert int(got[0]["total_centibits"].item()) == int(want["total_centibits"])
+    assert np.array_equal(got[0]["code_offsets"].cpu().numpy(), want["code_offsets"])
+    assert int(got[3]["total_centibits"].item()) == -1
+    with pytest.raises(Exception):
+        wq.windq_effective_bits_batch(ctx, acts * 2, [R for _, R in plans] * 2, G)      # 40 jobs

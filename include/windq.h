@@ -233,6 +233,25 @@ windq_status windq_apply_plan(windq_ctx* ctx, const void* W, int64_t R, int64_t 
                               const uint8_t* clip_idx, const int64_t* code_offsets, uint8_t* codes_out,
                               void* scales_out, void* zeros_out, void* Wq_out, void* stream);
 
+/* windq_apply_plan for several (matrix, plan) pairs in one launch.  Every job is one windq_apply_plan call with
+ * clip indices (clip_idx is required here): same meanings, layouts and results, bit for bit.  All jobs share G,
+ * the clip grid and K.  Jobs must not share output arrays (two plans of one matrix need two Wq_out, or NULL).
+ *   jobs: HOST array of n_jobs descriptors (1 <= n_jobs <= 24), read during the call only. */
+typedef struct {
+  const void* W;                /* fp16 [R][ldw] */
+  int64_t R, C, ldw;
+  const float* s;               /* fp32 [C] */
+  const uint8_t* actions;       /* u8 [U] */
+  const uint8_t* clip_idx;      /* u8 [4][U][R] */
+  const int64_t* code_offsets;  /* i64 [U+1] */
+  uint8_t* codes_out;
+  void* scales_out;             /* fp16 [U][R] */
+  void* zeros_out;              /* fp16 [U][R] */
+  void* Wq_out;                 /* fp16 [R][ldw], nullable */
+} windq_apply_job;
+windq_status windq_apply_plan_batch(windq_ctx* ctx, const windq_apply_job* jobs, int n_jobs, int G,
+                                    const float* clip_grid, int K, void* stream);
+
 /* ---- beyond the five calls: salient-weight protection (App. "Salient Weight Protection") ---------
  *
  * The paper keeps, in every unit, the top-r fraction of the weights by saliency -- weight magnitude

@@ -56,6 +56,7 @@ def _load() -> ctypes.CDLL:
     lib.windq_act_stats_noalloc.argtypes = [vp, vp, i64, i64, i64, vp, vp]
     lib.windq_unit_features.argtypes = [vp, vp, i64, i64, i64, i32, vp, vp, vp]
     lib.windq_fit_eval.argtypes = [vp, vp, i64, i64, i64, i32, vp, vp, i32, vp, vp, vp, vp, vp]
+    lib.windq_apply_plan_batch.argtypes = [vp, vp, i32, i32, vp, i32, vp]
     lib.windq_effective_bits_batch.argtypes = [vp, vp, i32, i32, i32, i32, vp]
     lib.windq_unit_features_batch.argtypes = [vp, vp, i32, i32, vp]
     lib.windq_scratch_bytes_unit_features_batch.restype = i64
@@ -249,6 +250,54 @@ def windq_fit_eval(ctx: Context, W: torch.Tensor, G: int, s: torch.Tensor, clip_
                                                  clip_grid.numel(), _ptr(thresh), _ptr(out["err"]), _ptr(out["energy"]),
                                                  _ptr(out["clip_idx"]), _ptr(out["group_err"]), _stream(stream)))
     return out
+
+
+class _ApplyJob(ctypes.Structure):
+    _fields_ = [("W", ctypes.c_void_p), ("R", ctypes.c_int64), ("C", ctypes.c_int64), ("ldw", ctypes.c_int64),
+                ("s", ctypes.c_void_p), ("actions", ctypes.c_void_p), ("clip_idx", ctypes.c_void_p),
+                ("code_offsets", ctypes.c_void_p), ("codes_out", ctypes.c_void_p), ("scales_out", ctypes.c_void_p),
+                ("zeros_out", ctypes.c_void_p), ("Wq_out", ctypes.c_void_p)]
+
+
+def windq_apply_plan_batch(ctx: Context, jobs, G: int, clip_grid: torch.Tensor, *, stream=None) -> list:
+    """windq_apply_plan of up to 24 (matrix, plan) pairs in one launch.  ``jobs``: a sequence of dicts with the keys
+    W, s, actions, clip_idx, code_offsets, codes (uint8 output, sized by the caller) and optionally scales, zeros
+    ([U, R] fp16) and wq ([R, C] fp16 with the row stride of W, or None for no fake-quantised output; absent = allocated).
+    Returns one dict(codes, scales, zeros, wq) per job."""
+    if not jobs:
+        raise ValueError("jobs must not be empty")
+    _need(clip_grid, torch.float32, "clip_grid", 1)
+    arr = (_ApplyJob * len(jobs))()
+    results = []
+    for j, job in enumerate(jobs):
+        W, s, actions, clip_idx = job["W"], job["s"], job["actions"], job["clip_idx"]
+        R, C, ldw = _matrix(W, "W")
+        _need(s, torch.float32, "s", 1)
+        _need(actions, torch.uint8, "actions", 1)
+        _need(clip_idx, torch.uint8, "clip_idx", 3)
+        _need(job["code_offsets"], torch.int64, "code_offsets", 1)
+        _need(job["codes"], torch.uint8, "codes", 1)
+        U = C // G if G > 0 else 0
+        if actions.numel() != U or job["code_offsets"].numel() != U + 1 or tuple(clip_idx.shape) != (4, U, R) \
+                or not clip_idx.is_contiguous():
+            raise ValueError("job %d: actions [U], code_offsets [U + 1] and a contiguous clip_idx [4, U, R] are needed" % j)
+        dev = W.device
+        scales = job.get("scales")
+        zeros = job.get("zeros")
+        if scales is None:
+            scales = torch.empty((U, R), dtype=torch.float16, device=dev)
+        if zeros is None:
+            zeros = torch.empty((U, R), dtype=torch.float16, device=dev)
+        wq_out = job["wq"] if "wq" in job else torch.empty_strided((R, C), (ldw, 1), dtype=torch.float16, device=dev)
+        if wq_out is not None and (_matrix(wq_out, "wq")[2] != ldw or wq_out.shape != W.shape):
+            raise ValueError("job %d: wq must have the shape and row stride of W" % j)
+        arr[j] = _ApplyJob(W.data_ptr(), R, C, ldw, s.data_ptr(), actions.data_ptr(), clip_idx.data_ptr(),
+                           job["code_offsets"].data_ptr(), job["codes"].data_ptr(), scales.data_ptr(), zeros.data_ptr(),
+                           None if wq_out is None else wq_out.data_ptr())
+        results.append(dict(codes=job["codes"], scales=scales, zeros=zeros, wq=wq_out))
+    ctx._check(_lib.windq_apply_plan_batch(ctx._h, ctypes.cast(arr, ctypes.c_void_p), len(jobs), int(G), _ptr(clip_grid),
+                                           clip_grid.numel(), _stream(stream)))
+    return results
 
 
 class _BitsJob(ctypes.Structure):

@@ -16,6 +16,8 @@
 // Only the base-3 ternary packing crosses lanes (5 trits per byte): its trits are staged as 2-bit
 // fields in shared memory and each output byte is looked up from the 10-bit window that holds its
 // five trits.
+#include <string.h>
+
 #include "fit_device.cuh"
 
 namespace windq {
@@ -160,18 +162,40 @@ __device__ __forceinline__ unsigned int protect_mask(const uint4 (&raw)[4], cons
   return pm;
 }
 
+// Several plans in one launch (windq_apply_plan_batch): what differs from job to job, by value in the kernel's
+// parameters.  Items are numbered through all jobs; job j owns [first_item[j], first_item[j + 1]).
+constexpr int kApplyMaxJobs = 24;
+struct ApplyJobs {
+  const __half* W[kApplyMaxJobs];
+  const float* s[kApplyMaxJobs];
+  const uint8_t* actions[kApplyMaxJobs];
+  const uint8_t* clip_idx[kApplyMaxJobs];
+  const long long* code_offsets[kApplyMaxJobs];
+  uint8_t* codes[kApplyMaxJobs];
+  __half* scales[kApplyMaxJobs];
+  __half* zeros[kApplyMaxJobs];
+  __half* Wq[kApplyMaxJobs];
+  long long ldw[kApplyMaxJobs];
+  int R[kApplyMaxJobs];
+  int U[kApplyMaxJobs];
+  int first_item[kApplyMaxJobs + 1];
+  int n;
+};
+
 #ifndef WINDQ_APPLY_MIN_BLOCKS
 #define WINDQ_APPLY_MIN_BLOCKS 4
 #endif
 // PROTECT = true: salient weights (see ProtectArgs) are taken out of the group fits -- zero weight,
 // zero activation weight, as in the protected fit -- and kept on one symmetric INT8 grid per unit.
-template <int G, bool SEARCH, bool PROTECT>
+// BATCH: the matrix and the plan of an item are looked up in `jobs` (the scalar parameters that describe one
+// matrix are then unused).
+template <int G, bool SEARCH, bool PROTECT, bool BATCH>
 __global__ void __launch_bounds__(kApplyWarps * 32, WINDQ_APPLY_MIN_BLOCKS)
-apply_plan_kernel(const __half* __restrict__ W, int R, int U, int64_t ldw, const float* __restrict__ s,
-                  const float* __restrict__ clip, int K, const uint8_t* __restrict__ actions,
-                  const uint8_t* __restrict__ clip_idx, const long long* __restrict__ code_offsets,
-                  uint8_t* __restrict__ codes_out, __half* __restrict__ scales_out, __half* __restrict__ zeros_out,
-                  __half* __restrict__ Wq_out, int rows_blocks, ProtectArgs pa) {
+apply_plan_kernel(const __half* __restrict__ W_one, int R_one, int U_one, int64_t ldw_one, const float* __restrict__ s_one,
+                  const float* __restrict__ clip, int K, const uint8_t* __restrict__ actions_one,
+                  const uint8_t* __restrict__ clip_idx_one, const long long* __restrict__ code_offsets_one,
+                  uint8_t* __restrict__ codes_one, __half* __restrict__ scales_one, __half* __restrict__ zeros_one,
+                  __half* __restrict__ Wq_one, int rows_blocks_one, ProtectArgs pa, const ApplyJobs jobs) {
   constexpr int LG = Map<G>::LG, GPW = Map<G>::GPW;
   extern __shared__ uint4 smem_u4[];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -187,13 +211,25 @@ apply_plan_kernel(const __half* __restrict__ W, int R, int U, int64_t ldw, const
   Cand* cand = reinterpret_cast<Cand*>(reinterpret_cast<uint8_t*>(smem_u4) + (size_t)kApplyWarps * kApplyWarpBytes) +
                (size_t)warp * GPW * stride;
 
-  const int n_items = U * rows_blocks;
+  const int n_items = BATCH ? jobs.first_item[jobs.n] : U_one * rows_blocks_one;
   const int n_warps = gridDim.x * kApplyWarps;
   int item = blockIdx.x * kApplyWarps + warp;
 
   // asks for the lane's 64 bytes of `it` into buffer `buf` (rows past the end repeat the last row)
   auto prefetch = [&](int it, int buf) {
     if (it < n_items) {
+      const __half* W = W_one;
+      int R = R_one, rows_blocks = rows_blocks_one;
+      int64_t ldw = ldw_one;
+      if (BATCH) {
+        int j = 0;
+        while (j + 1 < jobs.n && it >= jobs.first_item[j + 1]) ++j;
+        W = jobs.W[j];
+        R = jobs.R[j];
+        ldw = jobs.ldw[j];
+        rows_blocks = (R + GPW - 1) / GPW;
+        it -= jobs.first_item[j];
+      }
       const int u = it / rows_blocks, rb = it - u * rows_blocks;
       const int row = min(rb * GPW + g, R - 1);
       const __half* src = W + (int64_t)row * ldw + (int64_t)u * G + 32 * q;
@@ -208,7 +244,32 @@ apply_plan_kernel(const __half* __restrict__ W, int R, int U, int64_t ldw, const
   for (int n = 0; item < n_items; item += n_warps, ++n) {
     prefetch(item + n_warps, (n + 1) & 1);
     cp_async_wait_all_but_one();  // this lane's 64 bytes of the current item have arrived
-    const int u = item / rows_blocks, rb = item - u * rows_blocks;
+    const float* s = s_one;
+    const uint8_t* actions = actions_one;
+    const uint8_t* clip_idx = clip_idx_one;
+    const long long* code_offsets = code_offsets_one;
+    uint8_t* codes_out = codes_one;
+    __half *scales_out = scales_one, *zeros_out = zeros_one, *Wq_out = Wq_one;
+    int R = R_one, U = U_one, rows_blocks = rows_blocks_one, local = item;
+    int64_t ldw = ldw_one;
+    if (BATCH) {
+      int j = 0;
+      while (j + 1 < jobs.n && item >= jobs.first_item[j + 1]) ++j;
+      s = jobs.s[j];
+      actions = jobs.actions[j];
+      clip_idx = jobs.clip_idx[j];
+      code_offsets = jobs.code_offsets[j];
+      codes_out = jobs.codes[j];
+      scales_out = jobs.scales[j];
+      zeros_out = jobs.zeros[j];
+      Wq_out = jobs.Wq[j];
+      R = jobs.R[j];
+      U = jobs.U[j];
+      ldw = jobs.ldw[j];
+      rows_blocks = (R + GPW - 1) / GPW;
+      local = item - jobs.first_item[j];
+    }
+    const int u = local / rows_blocks, rb = local - u * rows_blocks;
     const int a = actions[u];
     if (a > 6) continue;
     const int row = rb * GPW + g;
@@ -396,7 +457,7 @@ windq_status launch_apply(windq_ctx* ctx, const __half* W, int R, int U, int64_t
   const size_t smem = (size_t)kApplyWarps * kApplyWarpBytes + (SEARCH ? (size_t)kApplyWarps * GPW * stride * sizeof(Cand) : 0);
   const int id = (PROTECT ? (SEARCH ? kApplyProtectSearchG32 : kApplyProtectG32) : (SEARCH ? kApplySearchG32 : kApplyG32)) +
                  g_index(G);
-  if (windq_status rc = prepare_kernel(ctx, id, apply_plan_kernel<G, SEARCH, PROTECT>, kApplyWarps * 32, smem, true)) return rc;
+  if (windq_status rc = prepare_kernel(ctx, id, apply_plan_kernel<G, SEARCH, PROTECT, false>, kApplyWarps * 32, smem, true)) return rc;
   const int blocks_per_sm = ctx->occupancy[id];
   const int rows_blocks = (R + GPW - 1) / GPW;
   const int64_t n_items = (int64_t)U * rows_blocks;
@@ -404,8 +465,9 @@ windq_status launch_apply(windq_ctx* ctx, const __half* W, int R, int U, int64_t
   int64_t grid = (int64_t)ctx->sm_count * blocks_per_sm;
   const int64_t need = (n_items + kApplyWarps - 1) / kApplyWarps;
   if (grid > need) grid = need;
-  apply_plan_kernel<G, SEARCH, PROTECT><<<(unsigned)grid, kApplyWarps * 32, smem, st>>>(
-      W, R, U, ldw, s, clip, K, actions, clip_idx, code_offsets, codes_out, scales_out, zeros_out, Wq_out, rows_blocks, pa);
+  apply_plan_kernel<G, SEARCH, PROTECT, false><<<(unsigned)grid, kApplyWarps * 32, smem, st>>>(
+      W, R, U, ldw, s, clip, K, actions, clip_idx, code_offsets, codes_out, scales_out, zeros_out, Wq_out, rows_blocks, pa,
+      ApplyJobs());
   WINDQ_CUDA(ctx, cudaGetLastError());
   return WINDQ_OK;
 }
@@ -687,4 +749,75 @@ extern "C" windq_status windq_apply_plan_protected_refined(windq_ctx* ctx, const
   return apply_plan_protected_any(ctx, who, W, R, C, ldw, G, s, clip_grid, K, actions, clip_idx, scale_in, code_offsets, thresh,
                                   codes_out, scales_out, zeros_out, Wq_out, prot_scale_out, prot_offsets_out, prot_q_out,
                                   prot_q_capacity, stream);
+}
+
+namespace windq {
+
+template <int G>
+windq_status launch_apply_batch(windq_ctx* ctx, const ApplyJobs& jobs, const float* clip, int K, cudaStream_t st) {
+  const size_t smem = (size_t)kApplyWarps * kApplyWarpBytes;
+  const int id = kApplyBatchG32 + g_index(G);
+  if (windq_status rc = prepare_kernel(ctx, id, apply_plan_kernel<G, false, false, true>, kApplyWarps * 32, smem, true)) return rc;
+  int64_t grid = (int64_t)ctx->sm_count * ctx->occupancy[id];
+  const int64_t need = ((int64_t)jobs.first_item[jobs.n] + kApplyWarps - 1) / kApplyWarps;
+  if (grid > need) grid = need;
+  apply_plan_kernel<G, false, false, true><<<(unsigned)grid, kApplyWarps * 32, smem, st>>>(
+      nullptr, 0, 0, 0, nullptr, clip, K, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, 0, ProtectArgs(), jobs);
+  WINDQ_CUDA(ctx, cudaGetLastError());
+  return WINDQ_OK;
+}
+
+}  // namespace windq
+
+extern "C" windq_status windq_apply_plan_batch(windq_ctx* ctx, const windq_apply_job* jobs, int n_jobs, int G,
+                                               const float* clip_grid, int K, void* stream) {
+  using namespace windq;
+  const char* who = "windq_apply_plan_batch";
+  if (!ctx) return fail(nullptr, WINDQ_ERR_NULL, "%s: ctx is NULL", who);
+  WINDQ_REQUIRE(ctx, jobs && clip_grid, WINDQ_ERR_NULL, "%s: jobs or clip_grid is NULL", who);
+  WINDQ_REQUIRE(ctx, n_jobs >= 1 && n_jobs <= kApplyMaxJobs, WINDQ_ERR_SHAPE, "%s: n_jobs = %d is outside [1, %d]", who, n_jobs,
+                kApplyMaxJobs);
+  if (windq_status st = check_K(ctx, who, K)) return st;
+  ApplyJobs aj;
+  memset(&aj, 0, sizeof(aj));
+  aj.n = n_jobs;
+  int64_t items = 0;
+  const int gpw = 32 / (G > 0 ? (G / 32 > 0 ? G / 32 : 1) : 1);
+  for (int j = 0; j < n_jobs; ++j) {
+    const windq_apply_job& b = jobs[j];
+    if (windq_status st = check_matrix(ctx, who, b.W, b.R, b.C, b.ldw, G)) return st;
+    WINDQ_REQUIRE(ctx, b.s && b.actions && b.clip_idx && b.code_offsets && b.codes_out && b.scales_out && b.zeros_out,
+                  WINDQ_ERR_NULL, "%s: job %d: a required pointer is NULL (clip_idx is required in a batch)", who, j);
+    WINDQ_REQUIRE(ctx, aligned16(b.s) && aligned16(b.codes_out), WINDQ_ERR_ALIGN, "%s: job %d: s or codes_out is not 16-byte aligned",
+                  who, j);
+    WINDQ_REQUIRE(ctx, ((uintptr_t)b.code_offsets & 7) == 0 && ((uintptr_t)b.scales_out & 1) == 0 && ((uintptr_t)b.zeros_out & 1) == 0,
+                  WINDQ_ERR_ALIGN, "%s: job %d: code_offsets, scales_out or zeros_out is misaligned", who, j);
+    WINDQ_REQUIRE(ctx, b.Wq_out == nullptr || aligned16(b.Wq_out), WINDQ_ERR_ALIGN, "%s: job %d: Wq_out is not 16-byte aligned", who, j);
+    WINDQ_REQUIRE(ctx, b.Wq_out != b.W, WINDQ_ERR_ARG, "%s: job %d: Wq_out must not alias W", who, j);
+    aj.W[j] = (const __half*)b.W;
+    aj.s[j] = b.s;
+    aj.actions[j] = b.actions;
+    aj.clip_idx[j] = b.clip_idx;
+    aj.code_offsets[j] = (const long long*)b.code_offsets;
+    aj.codes[j] = b.codes_out;
+    aj.scales[j] = (__half*)b.scales_out;
+    aj.zeros[j] = (__half*)b.zeros_out;
+    aj.Wq[j] = (__half*)b.Wq_out;
+    aj.ldw[j] = b.ldw;
+    aj.R[j] = (int)b.R;
+    aj.U[j] = (int)(b.C / G);
+    aj.first_item[j] = (int)items;
+    items += (b.C / G) * ((b.R + gpw - 1) / gpw);
+    WINDQ_REQUIRE(ctx, items < (1ll << 30), WINDQ_ERR_SHAPE, "%s: the batch is too large for one call", who);
+  }
+  aj.first_item[n_jobs] = (int)items;
+  DeviceGuard guard(ctx->device);
+  cudaStream_t st = (cudaStream_t)stream;
+  switch (G) {
+    case 32: return launch_apply_batch<32>(ctx, aj, clip_grid, K, st);
+    case 64: return launch_apply_batch<64>(ctx, aj, clip_grid, K, st);
+    case 128: return launch_apply_batch<128>(ctx, aj, clip_grid, K, st);
+    case 256: return launch_apply_batch<256>(ctx, aj, clip_grid, K, st);
+    default: return launch_apply_batch<512>(ctx, aj, clip_grid, K, st);
+  }
 }

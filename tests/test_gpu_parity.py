@@ -612,3 +612,55 @@ def test_effective_bits_batch_equals_the_separate_calls(wq, ctx, oracle):
     assert int(got[3]["total_centibits"].item()) == -1
     with pytest.raises(Exception):
         wq.windq_effective_bits_batch(ctx, acts * 2, [R for _, R in plans] * 2, G)      # 40 jobs
+
+
+@pytest.mark.parametrize("G,shapes", [(128, [(300, 512), (64, 1024), (17, 128)]), (64, [(40, 256), (1100, 512)]),
+                                      (256, [(512, 2048), (33, 256)]), (32, [(5, 32)])])
+def test_apply_plan_batch_equals_the_separate_calls(wq, ctx, oracle, G, shapes):
+    """Three plans of every matrix in one launch: codes, scales, zero points and fake-quantised weights of every job
+    equal those of its own windq_apply_plan call bit for bit, and one job equals the oracle."""
+    grid = ws.clip_grid(20)
+    gd = torch.from_numpy(grid).cuda()
+    rng = np.random.default_rng(G)
+    jobs, singles = [], []
+    for i, (R, C) in enumerate(shapes):
+        W = ws.weights(R, C, 700 + i, "student_t").cuda()
+        s = (torch.rand(C, generator=torch.Generator().manual_seed(i)) * 3 + 0.01).cuda()
+        U = C // G
+        fit = wq.windq_fit_eval(ctx, W, G, s, gd)
+        for plan in range(3):
+            acts = torch.from_numpy(rng.integers(0, 7, U).astype(np.uint8)).cuda()
+            eb = wq.windq_effective_bits(ctx, acts, R, G)
+            jobs.append(dict(W=W, s=s, actions=acts, clip_idx=fit["clip_idx"], code_offsets=eb["code_offsets"],
+                             codes=torch.zeros(2 * R * C + 16 * U, dtype=torch.uint8, device="cuda")))
+            singles.append(wq.windq_apply_plan(ctx, W, G, s, gd, acts, eb["code_offsets"],
+                                               torch.zeros(2 * R * C + 16 * U, dtype=torch.uint8, device="cuda"), fit["clip_idx"]))
+    got = wq.windq_apply_plan_batch(ctx, jobs, G, gd)
+    torch.cuda.synchronize()
+    assert len(got) == len(jobs)
+    for out, one in zip(got, singles):
+        assert torch.equal(out["codes"], one["codes"])
+        assert torch.equal(out["scales"].view(torch.int16), one["scales"].view(torch.int16))
+        assert torch.equal(out["zeros"].view(torch.int16), one["zeros"].view(torch.int16))
+        assert torch.equal(out["wq"].view(torch.int16), one["wq"].view(torch.int16))
+    j0 = jobs[1]
+    want = oracle.apply_plan(j0["W"].cpu().numpy(), G, j0["s"].cpu().numpy(), grid, j0["actions"].cpu().numpy(),
+                             j0["clip_idx"].cpu().numpy())
+    n = int(want["code_offsets"][-1])
+    assert np.array_equal(got[1]["codes"][:n].cpu().numpy(), want["codes"])
+    assert np.array_equal(got[1]["wq"].cpu().numpy().view(np.uint16), want["wq"])
+
+
+def test_apply_plan_batch_argument_checks(wq, ctx):
+    gd = torch.from_numpy(ws.clip_grid(4)).cuda()
+    W = torch.zeros((8, 128), dtype=torch.float16, device="cuda")
+    s = torch.ones(128, device="cuda")
+    acts = torch.zeros(1, dtype=torch.uint8, device="cuda")
+    eb = wq.windq_effective_bits(ctx, acts, 8, 128)
+    idx = torch.zeros((4, 1, 8), dtype=torch.uint8, device="cuda")
+    job = dict(W=W, s=s, actions=acts, clip_idx=idx, code_offsets=eb["code_offsets"],
+               codes=torch.zeros(4096, dtype=torch.uint8, device="cuda"), wq=None)
+    with pytest.raises(Exception):
+        wq.windq_apply_plan_batch(ctx, [job] * 25, 128, gd)
+    out = wq.windq_apply_plan_batch(ctx, [job], 128, gd)
+    assert out[0]["wq"] is None and (out[0]["codes"][:2048] == 0).all()

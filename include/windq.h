@@ -27,6 +27,13 @@
  *     call launches nothing and returns a status, and windq_last_error gives the reason.  There
  *     are no exceptions, aborts or device traps.  Inputs must be finite; NaN / Inf give
  *     unspecified values, never a fault.  A context must not be used from two threads at once.
+ *   - Ordering.  Every call on a context works in that context's one scratch buffer, from its
+ *     first byte (the item counter and partial sums of the fits, the histograms of the feature
+ *     and selection passes, the row counts of protected packing, the allocator's tables).  Two
+ *     calls on the same context must therefore not overlap on the GPU: issue them on one stream,
+ *     or order the streams with events (the later call's stream waits for an event recorded
+ *     after the earlier call), or give every stream a context of its own.  Calls on one context
+ *     from unordered streams corrupt each other's results silently.
  *   - Pointers to fp16 / fp32 / int64 arrays must be 16-byte aligned (any cudaMalloc or torch
  *     allocation is); ldw and ldx must be multiples of 8.
  *   - G must be one of 32, 64, 128, 256, 512; C a multiple of G; 1 <= K <= 64; clip ratios in
@@ -89,17 +96,22 @@ windq_status windq_act_stats(windq_ctx* ctx, const void* X, int64_t T, int64_t C
  * cudaMalloc fails; a latency-bound loop that must not take the device-wide synchronisation
  * cudaMalloc and cudaFree imply; code that runs where only kernel launches are allowed.  For them
  * this call keeps the partial sums in an array of WINDQ_NOALLOC_SCRATCH_BYTES that is built into
- * the library image.  Every device that loads the library holds that array until the process
- * exits, whether or not this entry point is ever called.
+ * the library image.  Every device that loads the library's device code holds that array until
+ * the process exits, whether or not this entry point is ever called.
  *
  * Arguments, layout, result and argument errors are those of windq_act_stats.  In addition:
  *   - the call needs 4 * C * ceil(T / 64) bytes of the array (windq_scratch_bytes_act_stats
  *     gives the figure); a larger request is refused with WINDQ_ERR_SCRATCH before anything is
  *     launched -- use windq_act_stats, or call once per block of tokens and combine the means;
- *   - no cudaMalloc, cudaFree or other allocating routine is called, on any path;
+ *   - this entry point calls no cudaMalloc, cudaFree or other allocating routine, on any path;
  *   - the first call on a device asks the runtime for the array's device address (one
- *     cudaGetSymbolAddress, kept per device afterwards).  Make that first call outside any
- *     stream capture;
+ *     cudaGetSymbolAddress, kept per device afterwards).  With the CUDA runtime's default lazy
+ *     loading that request, or the first kernel launch of the library, is also the moment the
+ *     driver loads the library's device code on that device and reserves the array: the driver
+ *     itself takes device memory then (the array and the code), and may synchronise.  So make
+ *     the first call per device at start-up -- before the process hands its device memory to a
+ *     pool of its own, and outside any stream capture; every later call finds the address kept
+ *     and only launches;
  *   - all calls on a device share the one array, and it keeps whatever the last call left.  That
  *     is harmless from call to call, because every partial sum that is read has been written by
  *     the same call first; but two calls whose kernels can overlap on the GPU (different streams
@@ -211,9 +223,10 @@ typedef struct {
 windq_status windq_effective_bits_batch(windq_ctx* ctx, const windq_bits_job* jobs, int n_jobs, int G, int scale_bits,
                                         int zero_bits, void* stream);
 
-/* a4 -- apply a plan to one matrix ("the environment applies the selected quantization to the
- * current unit"): integer codes packed as described above, the fp16 scale and zero point of
- * every group, and optionally the fake-quantised weights for the consumer's forward pass.
+/* a4 -- apply a plan to one matrix ("Transition and Discount": after the policy has chosen, the
+ * environment quantizes the current unit with the chosen operator): integer codes packed as
+ * described above, the fp16 scale and zero point of every group, and optionally the
+ * fake-quantised weights for the consumer's forward pass.
  *   actions      u8  [U]          action per unit
  *   clip_idx     u8  [4][U][R]    clip indices from windq_fit_eval, or NULL: the clip search is
  *                                 repeated for the chosen bit-width (same result, more work).
@@ -227,7 +240,11 @@ windq_status windq_effective_bits_batch(windq_ctx* ctx, const windq_bits_job* jo
  * q_2i+1 << 4; 3-bit: a bit stream, code j at bits [3j, 3j+3); 2-bit byte i = sum q_4i+m << 2m;
  * 1.58-bit byte i = sum_{m<5} t_5i+m 3^m with trits t = 1 + sign(w) on the support, 1 elsewhere;
  * 1-bit byte i = sum bit_8i+m << m with bit = !(w < 0); skip: the raw fp16 bytes.
- * Units whose action code is above 6 are left unwritten.  codes_out must be 16-byte aligned. */
+ * Action codes live on the device, so they cannot be checked before the launch: a unit whose code
+ * is above 6 is skipped -- its codes, scales, zero points and fake-quantised weights keep whatever
+ * the output arrays held -- and the call still returns WINDQ_OK.  windq_effective_bits reports such
+ * a plan (totals of -1); check its total before applying a plan that was not produced by trusted
+ * code.  The same holds for every windq_apply_plan* variant.  codes_out must be 16-byte aligned. */
 windq_status windq_apply_plan(windq_ctx* ctx, const void* W, int64_t R, int64_t C, int64_t ldw, int G,
                               const float* s, const float* clip_grid, int K, const uint8_t* actions,
                               const uint8_t* clip_idx, const int64_t* code_offsets, uint8_t* codes_out,
@@ -289,7 +306,7 @@ windq_status windq_fit_eval_protected(windq_ctx* ctx, const void* W, int64_t R, 
  * weight (as in windq_fit_eval_protected, whose clip indices this call takes), so scales, zero points
  * and the codes of the other weights are those of the masked group, and its own slot in the packed
  * stream holds the code of the value 0 (a reader skips it by the mask of windq_salient_select).  The
- * protected weights of a unit share one symmetric INT8 grid (the paper says only "stored in INT8"):
+ * protected weights of a unit share one symmetric INT8 grid (the paper says no more than that they are kept in INT8):
  *   prot_scale_out   fp16 [U]     sigma_u = fp16(max |w| over the unit's protected weights / 127), 1 if that
  *                                 is zero; 0 for a skipped unit, which protects nothing
  *   prot_offsets_out i64  [U+1]   start of every unit's INT8 codes in prot_q_out; [U] = their number
@@ -403,9 +420,9 @@ windq_status windq_greedy_allocate(windq_ctx* ctx, const float* saliency, const 
                                    int64_t headroom_cb, int scale_bits, int zero_bits, uint8_t* actions_out,
                                    int64_t* order_out, int64_t* total_centibits_out, void* stream);
 
-/* Fallback to higher precision (Sec. 3.5: "if the reconstruction error of a selected operator is
- * excessive, the implementation falls back to a higher-precision operator").  The paper gives neither
- * the measure nor the threshold; here the error of unit u under action a is excessive when
+/* Fallback to higher precision (Sec. 3.5: an operator whose reconstruction error turns out too large
+ * is replaced by one of higher precision).  The paper gives neither the measure nor the threshold;
+ * here the error of unit u under action a is excessive when
  *   err[u][a] > theta * energy[u]     (binary32 on both sides; err and energy from windq_fit_eval)
  * and the unit moves one step at a time towards higher precision (1 -> 1.58 -> 2 -> 3 -> 4 -> 8 ->
  * skip) until the test passes; skip always passes.

@@ -490,9 +490,6 @@ static int fit_eval_impl(const uint16_t* W, int64_t R, int64_t C, int64_t ldw, i
   return 0;
 }
 
-// ---- a5: effective bits (Eq. 6 with no protected weights, extended by the
-// per-group scale / zero-point overhead) in integer centibits, plus the byte
-// offset of every unit's packed block (each rounded up to 16 bytes).
 int oracle_fit_eval(const uint16_t* W, int64_t R, int64_t C, int64_t ldw, int G, const float* s,
                     const float* clip_grid, int K, int64_t u_begin, int64_t u_end, float* err_out,
                     float* energy_out, uint8_t* clip_idx_out, float* group_err_out) {
@@ -508,6 +505,9 @@ int oracle_fit_eval_protected(const uint16_t* W, int64_t R, int64_t C, int64_t l
                        group_err_out);
 }
 
+// ---- a5: effective bits (Eq. 6 with no protected weights, extended by the
+// per-group scale / zero-point overhead) in integer centibits, plus the byte
+// offset of every unit's packed block (each rounded up to 16 bytes).
 int oracle_effective_bits(const uint8_t* actions, int64_t U, int64_t R, int G, int scale_bits,
                           int zero_bits, int64_t* unit_centibits_out, int64_t* code_offsets_out,
                           int64_t* total_centibits_out, int64_t* total_packed_bytes_out) {
@@ -535,7 +535,7 @@ int oracle_effective_bits(const uint8_t* actions, int64_t U, int64_t R, int G, i
 // fp16 [R][ldw] (nullable).  clip_idx [4][U][R] may be null: the clip search is
 // then repeated for the chosen bit-width.
 // thresh == NULL: the plan applied to every weight.  thresh != NULL: salient-weight protection.
-// READING (the paper says only that protected weights are "stored in INT8"): in every unit that is
+// READING (the paper says no more than that protected weights are kept in INT8): in every unit that is
 // not skipped, a weight whose key |w| * sqrt(s_j) reaches thresh[u] is protected.  Inside its group it
 // counts as a zero weight with zero activation weight (as in the protected fit), so the group's
 // parameters and the codes of the other weights are those of the masked group, and its own slot in the
@@ -759,8 +759,8 @@ int oracle_unit_saliency(const uint16_t* W, int64_t R, int64_t C, int64_t ldw, i
   return 0;
 }
 
-// "If the reconstruction error of a selected operator is excessive, the implementation falls back to
-// a higher-precision operator" (Sec. 3.5).  READING (the paper gives neither the measure nor the
+// The engine's fallback (Sec. 3.5): an operator whose reconstruction error turns out too large is
+// replaced by one of higher precision.  READING (the paper gives neither the measure nor the
 // threshold): the error of action a is excessive when err[u][a] > theta * energy[u], both binary32,
 // one binary32 product on the right; the unit then moves to the next higher precision (1 -> 1.58 -> 2
 // -> 3 -> 4 -> 8 -> skip) until the test passes; skip has no error and always passes.
@@ -875,8 +875,8 @@ int oracle_apply_plan_refined(const uint16_t* W, int64_t R, int64_t C, int64_t l
 
 // ---- iterative step-size refinement (App. "Per-unit Scale Optimization") -------------------------
 // The paper's operators fit their scale by a small local optimisation, typically 10 Adam steps on
-// the reconstruction loss of the current chunk, and the 3/4/8-bit ones "learn step sizes with
-// straight-through estimation for discrete rounding" (the LSQ rule, Esser et al. 2020).  It prints no
+// the reconstruction loss of the current chunk, and the 3/4/8-bit ones treat the step size as a learned
+// parameter, with the rounding passed straight through (the LSQ rule, Esser et al. 2020).  It prints no
 // formulas.  READING, for the four uniform bit-widths, per group, all in binary32:
 //   warm start   the clip-grid fit: Delta_0 = its stored fp16 scale, zero point z fixed at its value
 //   iterate t    Delta_h = fp16(Delta_t) is the step actually used (a scale is stored in fp16);

@@ -55,9 +55,13 @@ act_finalize_kernel(const float* __restrict__ partial, int slices, int C, double
   s_out[c] = (float)(acc * inv_T);
 }
 
-inline int act_slices(int64_t T) {
+constexpr int64_t kActMaxSlices = 65535;  // grid.y limit
+
+// Token slices of a call (64 rows each), as a 64-bit count: callers compare it with kActMaxSlices
+// before they narrow it.
+inline int64_t act_slices(int64_t T) {
   const int64_t rows_per_slice = (int64_t)kActRowsPar * kActMaxRowsPerThread;
-  return (int)((T + rows_per_slice - 1) / rows_per_slice);
+  return (T + rows_per_slice - 1) / rows_per_slice;
 }
 
 }  // namespace windq
@@ -65,8 +69,8 @@ inline int act_slices(int64_t T) {
 extern "C" {
 
 int64_t windq_scratch_bytes_act_stats(int64_t T, int64_t C) {
-  if (T <= 0 || C <= 0) return 0;
-  return (int64_t)windq::act_slices(T) * C * (int64_t)sizeof(float);
+  if (T <= 0 || C <= 0 || windq::act_slices(T) > windq::kActMaxSlices || C >= (1ll << 31)) return 0;
+  return windq::act_slices(T) * C * (int64_t)sizeof(float);
 }
 
 windq_status windq_act_stats(windq_ctx* ctx, const void* X, int64_t T, int64_t C, int64_t ldx, float* s_out,
@@ -82,10 +86,11 @@ windq_status windq_act_stats(windq_ctx* ctx, const void* X, int64_t T, int64_t C
                 (long long)C);
   WINDQ_REQUIRE(ctx, ldx % 8 == 0, WINDQ_ERR_ALIGN, "windq_act_stats: ldx = %lld is not a multiple of 8", (long long)ldx);
   WINDQ_REQUIRE(ctx, aligned16(X), WINDQ_ERR_ALIGN, "windq_act_stats: X is not 16-byte aligned");
+  WINDQ_REQUIRE(ctx, act_slices(T) <= kActMaxSlices, WINDQ_ERR_SHAPE, "windq_act_stats: T = %lld is too large (at most %lld tokens per call)",
+                (long long)T, (long long)(kActMaxSlices * kActRowsPar * kActMaxRowsPerThread));
+  const int slices = (int)act_slices(T);
   DeviceGuard guard(ctx->device);
   if (windq_status st = ensure_scratch(ctx, windq_scratch_bytes_act_stats(T, C))) return st;
-  const int slices = act_slices(T);
-  WINDQ_REQUIRE(ctx, slices <= 65535, WINDQ_ERR_SHAPE, "windq_act_stats: T = %lld is too large", (long long)T);
   const int rows_per_slice = kActRowsPar * kActMaxRowsPerThread;
   cudaStream_t st = (cudaStream_t)stream;
   float* partial = (float*)ctx->scratch;
@@ -146,6 +151,7 @@ extern "C" windq_status windq_act_stats_noalloc(windq_ctx* ctx, const void* X, i
   WINDQ_REQUIRE(ctx, ldx % 8 == 0, WINDQ_ERR_ALIGN, "windq_act_stats_noalloc: ldx = %lld is not a multiple of 8",
                 (long long)ldx);
   WINDQ_REQUIRE(ctx, aligned16(X), WINDQ_ERR_ALIGN, "windq_act_stats_noalloc: X is not 16-byte aligned");
+  WINDQ_REQUIRE(ctx, act_slices(T) <= kActMaxSlices, WINDQ_ERR_SHAPE, "windq_act_stats_noalloc: T = %lld is too large", (long long)T);
   const int64_t need = windq_scratch_bytes_act_stats(T, C);
   WINDQ_REQUIRE(ctx, need <= (int64_t)WINDQ_NOALLOC_SCRATCH_BYTES, WINDQ_ERR_SCRATCH,
                 "windq_act_stats_noalloc: T = %lld, C = %lld needs %lld bytes of scratch, the built-in array has %lld; "
@@ -154,8 +160,7 @@ extern "C" windq_status windq_act_stats_noalloc(windq_ctx* ctx, const void* X, i
   WINDQ_REQUIRE(ctx, ctx->device < kNoallocMaxDevices, WINDQ_ERR_UNSUPPORTED,
                 "windq_act_stats_noalloc: device %d is beyond the %d devices this entry point keeps addresses for",
                 ctx->device, kNoallocMaxDevices);
-  const int slices = act_slices(T);
-  WINDQ_REQUIRE(ctx, slices <= 65535, WINDQ_ERR_SHAPE, "windq_act_stats_noalloc: T = %lld is too large", (long long)T);
+  const int slices = (int)act_slices(T);
   DeviceGuard guard(ctx->device);
   float* partial = nullptr;
   WINDQ_CUDA(ctx, noalloc_scratch(ctx->device, &partial));

@@ -182,15 +182,13 @@ struct ApplyJobs {
   int n;
 };
 
-#ifndef WINDQ_APPLY_MIN_BLOCKS
-#define WINDQ_APPLY_MIN_BLOCKS 4
-#endif
+constexpr int kApplyMinBlocks = 4;  // resident blocks per SM the register budget is held to
 // PROTECT = true: salient weights (see ProtectArgs) are taken out of the group fits -- zero weight,
 // zero activation weight, as in the protected fit -- and kept on one symmetric INT8 grid per unit.
 // BATCH: the matrix and the plan of an item are looked up in `jobs` (the scalar parameters that describe one
 // matrix are then unused).
 template <int G, bool SEARCH, bool PROTECT, bool BATCH>
-__global__ void __launch_bounds__(kApplyWarps * 32, WINDQ_APPLY_MIN_BLOCKS)
+__global__ void __launch_bounds__(kApplyWarps * 32, kApplyMinBlocks)
 apply_plan_kernel(const __half* __restrict__ W_one, int R_one, int U_one, int64_t ldw_one, const float* __restrict__ s_one,
                   const float* __restrict__ clip, int K, const uint8_t* __restrict__ actions_one,
                   const uint8_t* __restrict__ clip_idx_one, const long long* __restrict__ code_offsets_one,

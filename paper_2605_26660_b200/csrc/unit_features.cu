@@ -20,15 +20,9 @@
 namespace windq {
 
 constexpr int kBins = 32768;
-#ifndef WINDQ_FEAT_THREADS
-#define WINDQ_FEAT_THREADS 1024
-#endif
-constexpr int kFeatThreads = WINDQ_FEAT_THREADS;
+constexpr int kFeatThreads = 1024;
 constexpr int kFeatMaxBlocks = 1024;  // bound on the pass-1 grid that the scratch size assumes
-#ifndef WINDQ_FEAT_LOADS
-#define WINDQ_FEAT_LOADS 4
-#endif
-constexpr int kFeatLoads = WINDQ_FEAT_LOADS;  // rows in flight per thread
+constexpr int kFeatLoads = 4;  // rows in flight per thread
 
 // Several matrices in one pass (windq_unit_features_batch): the (unit, row) pairs are numbered through all
 // jobs, job-major; job j owns the pairs [first_pair[j], first_pair[j + 1]) and the units
@@ -60,7 +54,7 @@ __device__ __forceinline__ void hist_add8(unsigned int* sh, const uint4& raw, fl
 // rows_per_block consecutive (unit, row) pairs per block; slot j of unit u belongs to block
 // (u * R) / rows_per_block + j.
 template <int G>
-__global__ void __launch_bounds__(kFeatThreads, kFeatThreads <= 256 ? 4 : 1)  // at most 64 registers per thread
+__global__ void __launch_bounds__(kFeatThreads, 1)  // at most 64 registers per thread
 feat_hist_kernel(const __half* __restrict__ W_one, int R_one, int64_t ldw_one, long long rows_per_block, long long total_rows,
                  unsigned int* __restrict__ hist, double* __restrict__ slot_sum, int slots_per_unit, const FeatJobs jobs) {
   extern __shared__ unsigned int sh[];

@@ -1,0 +1,325 @@
+"""GPU parity at the benchmark's full sizes, in the launch shape bench.py times.
+
+What is compared with the CPU oracle, on the same seeded bits:
+  config 1   every unit of the single 4096 x 4096 layer through all five calls;
+  config 2   a whole 7B-shaped decoder block: ONE windq_unit_features_batch, ONE windq_fit_eval_batch and ONE
+             windq_effective_bits_batch call for its seven matrices, then windq_apply_plan at 2.0 bits -- every unit;
+  config 3   block 0 in full at chunk widths 64 and 128 (the batched calls again) with the plans at 1.58 / 2.0 /
+             3.0 bits, plus 64 seeded (block, matrix, unit) triples of the other 31 blocks;
+  configs 4 and 5   at least 16 sampled units each (40 clip ratios; 1024-row grouped-query k/v matrices).
+Bars as everywhere: clip indices, packed bytes, fp16 scales / zero points, fake-quantised weights, the counts behind
+sparsity / outlier_frac and every int64 total bit-exact; floats within 1e-4 relative + 1e-6 absolute.  A clip index
+may differ from the oracle's only where the oracle's errors of the two candidates are equal bit for bit; such ties
+are counted and printed (none is expected) and must stay below 1e-6 of the groups.
+"""
+import os
+from concurrent.futures import ThreadPoolExecutor
+
+import numpy as np
+import pytest
+import torch
+
+import windq_synth as ws
+
+pytestmark = pytest.mark.gpu
+
+RTOL, ATOL = 1e-4, 1e-6
+THREADS = os.cpu_count() or 1
+BITS_OF = (8, 4, 3, 2)
+
+
+@pytest.fixture(scope="module")
+def wq():
+    import paper_2605_26660_b200 as wq
+    return wq
+
+
+@pytest.fixture(scope="module")
+def ctx(wq):
+    c = wq.windq_create(0)
+    yield c
+    wq.windq_destroy(c)
+
+
+def close(g, o):
+    g, o = np.asarray(g, np.float64), np.asarray(o, np.float64)
+    return np.abs(g - o) <= RTOL * np.abs(o) + ATOL
+
+
+def u16(t):
+    return t.cpu().contiguous().view(torch.int16).numpy().view(np.uint16)
+
+
+def unit_ranges(U, parts):
+    b = np.linspace(0, U, min(parts, U) + 1).astype(int)
+    return [(int(a), int(c)) for a, c in zip(b[:-1], b[1:]) if c > a]
+
+
+def oracle_features(oracle, W, G, s):
+    """oracle.unit_features over disjoint unit ranges on all host cores (units are independent)."""
+    U = W.shape[1] // G
+    out = np.zeros((U, 8), np.float32)
+
+    def run(ab):
+        a, b = ab
+        out[a:b] = oracle.unit_features(np.ascontiguousarray(W[:, a * G:b * G]), G, s[a * G:b * G])
+    with ThreadPoolExecutor(max_workers=THREADS) as ex:
+        list(ex.map(run, unit_ranges(U, THREADS)))
+    return out
+
+
+def oracle_apply(oracle, W, G, s, grid, acts, clip_idx):
+    """oracle.apply_plan over disjoint unit ranges on all host cores.  Every unit's block of codes is a multiple of
+    16 bytes long, so the ranges' code streams simply follow one another."""
+    U = W.shape[1] // G
+    parts = unit_ranges(U, THREADS)
+
+    def run(ab):
+        a, b = ab
+        return oracle.apply_plan(np.ascontiguousarray(W[:, a * G:b * G]), G, s[a * G:b * G], grid, acts[a:b],
+                                 np.ascontiguousarray(clip_idx[:, a:b]))
+    with ThreadPoolExecutor(max_workers=THREADS) as ex:
+        res = list(ex.map(run, parts))
+    return dict(codes=np.concatenate([r["codes"] for r in res]), scales=np.concatenate([r["scales"] for r in res]),
+                zeros=np.concatenate([r["zeros"] for r in res]), wq=np.concatenate([r["wq"] for r in res], axis=1))
+
+
+class Ties:
+    """Clip-index mismatches that are exact ties in the oracle's own arithmetic."""
+    def __init__(self):
+        self.ties, self.groups = 0, 0
+
+    def check(self, oracle, got_idx, want_idx, W, G, s, grid, u_of=None):
+        """got_idx, want_idx: [4][U'][R]; W: the matrix (or the columns) those units come from."""
+        self.groups += want_idx.size
+        for b, u, r in zip(*np.nonzero(got_idx != want_idx)):
+            uu = u if u_of is None else u_of[u]
+            w = W[r, uu * G:(uu + 1) * G].astype(np.float32)
+            sg = s[uu * G:(uu + 1) * G]
+            eg = oracle.uniform_candidate(w, sg, BITS_OF[b], float(grid[got_idx[b, u, r]]), False)[2]
+            ew = oracle.uniform_candidate(w, sg, BITS_OF[b], float(grid[want_idx[b, u, r]]), False)[2]
+            assert np.float32(eg).view(np.uint32) == np.float32(ew).view(np.uint32), \
+                "clip index differs from the oracle's and is not a tie (bit-width %d, unit %d, row %d)" % (BITS_OF[b], uu, r)
+            self.ties += 1
+
+    def report(self, label):
+        print("\n[%s] clip-index tie exceptions: %d of %d groups x 4 bit-widths" % (label, self.ties, self.groups // 4))
+        assert self.ties <= 1e-6 * self.groups + (1 if self.groups < 10 ** 6 else 0)
+
+
+def block_plans(wq, ctx, mats, G, targets, seed):
+    """The benchmark's recipe: one seeded random plan per target over all units of the block."""
+    all_actions = torch.arange(7, dtype=torch.uint8, device="cuda")
+    per_R = {m.R: wq.windq_effective_bits(ctx, all_actions, m.R, G)["unit_centibits"].cpu().numpy() for m in mats}
+    costs = np.concatenate([np.tile(per_R[m.R][None, :], (m.C // G, 1)) for m in mats])
+    nw = np.concatenate([np.full(m.C // G, m.R * G, np.int64) for m in mats])
+    plans = {}
+    for ti, t in enumerate(targets):
+        flat, pos, row = ws.random_plan(costs, nw, t, seed + ti), 0, []
+        for m in mats:
+            row.append(flat[pos:pos + m.C // G].copy())
+            pos += m.C // G
+        plans[t] = row
+    return plans
+
+
+def check_block(wq, ctx, oracle, spec, block, widths, targets, apply_G, label):
+    """One decoder block through the batched calls of the benchmark step, every unit against the oracle."""
+    mats = list(spec.block_matrices())
+    Wd = [ws.block_weight(spec, 0, block, m, device="cuda") for m in mats]
+    Xd = {i: ws.block_input(spec, 0, block, i, device="cuda") for i, _ in spec.block_inputs()}
+    sd = {i: wq.windq_act_stats(ctx, X) for i, X in Xd.items()}
+    s_h = {i: s.cpu().numpy() for i, s in sd.items()}
+    for i, X in Xd.items():
+        assert close(s_h[i], oracle.act_stats(X.cpu().numpy())).all(), "act_stats of input %d" % i
+    del Xd
+    Wh = [W.cpu().numpy() for W in Wd]
+    grid = ws.clip_grid(spec.K)
+    grid_d = torch.from_numpy(grid).cuda()
+    stats = [sd[m.x_id] for m in mats]
+    ties = Ties()
+    for G in widths:
+        feats = wq.windq_unit_features_batch(ctx, Wd, G, stats)
+        fits = wq.windq_fit_eval_batch(ctx, Wd, G, stats, grid_d, want_group_err=True)
+        torch.cuda.synchronize()
+        want_fit = []
+        for mi, m in enumerate(mats):
+            s = s_h[m.x_id]
+            want = oracle.fit_eval(Wh[mi], G, s, grid, threads=THREADS)
+            want_fit.append(want)
+            got = {k: v.cpu().numpy() for k, v in fits[mi].items()}
+            ties.check(oracle, got["clip_idx"], want["clip_idx"], Wh[mi], G, s, grid)
+            same = got["clip_idx"] == want["clip_idx"]
+            assert (got["group_err"][:4].view(np.uint32)[same] == want["group_err"][:4].view(np.uint32)[same]).all(), m.name
+            assert (got["group_err"][4:].view(np.uint32) == want["group_err"][4:].view(np.uint32)).all(), m.name
+            assert close(got["err"], want["err"]).all() and close(got["energy"], want["energy"]).all(), m.name
+            wf = oracle_features(oracle, Wh[mi], G, s)
+            gf = feats[mi].cpu().numpy()
+            assert (gf[:, 3:5] == wf[:, 3:5]).all() and close(gf, wf).all(), m.name
+        if G != apply_G:
+            continue
+        plans = block_plans(wq, ctx, mats, G, targets, 17)
+        acts_d = [torch.from_numpy(plans[t][mi]).cuda() for mi in range(len(mats)) for t in targets]
+        ebs = wq.windq_effective_bits_batch(ctx, acts_d, [m.R for m in mats for _ in targets], G)
+        total_cb = 0
+        for mi, m in enumerate(mats):
+            for ti, t in enumerate(targets):
+                eb, acts = ebs[mi * len(targets) + ti], plans[t][mi]
+                o_eb = oracle.effective_bits(acts, m.R, G)
+                assert int(eb["total_centibits"].item()) == o_eb["total_centibits"]
+                assert int(eb["total_packed_bytes"].item()) == o_eb["total_packed_bytes"]
+                assert (eb["code_offsets"].cpu().numpy() == o_eb["code_offsets"]).all()
+                assert (eb["unit_centibits"].cpu().numpy() == o_eb["unit_centibits"]).all()
+                if ti == 0:
+                    total_cb += o_eb["total_centibits"]
+                codes = torch.empty(int(o_eb["code_offsets"][-1]), dtype=torch.uint8, device="cuda")
+                # the clip indices the device produced feed the packing, as in the benchmark step
+                plan = wq.windq_apply_plan(ctx, Wd[mi], G, stats[mi], grid_d, acts_d[mi * len(targets) + ti],
+                                           eb["code_offsets"], codes, fits[mi]["clip_idx"])
+                torch.cuda.synchronize()
+                want = oracle_apply(oracle, Wh[mi], G, s_h[m.x_id], grid, acts, fits[mi]["clip_idx"].cpu().numpy())
+                assert (codes.cpu().numpy() == want["codes"]).all(), (m.name, t)
+                assert (u16(plan["scales"]) == want["scales"]).all() and (u16(plan["zeros"]) == want["zeros"]).all(), (m.name, t)
+                assert (u16(plan["wq"]) == want["wq"]).all(), (m.name, t)
+        n = sum(m.R * m.C for m in mats)
+        assert abs(total_cb / (100.0 * n) - targets[0]) <= 0.005
+    ties.report(label)
+
+
+# ------------------------------------------------------------------ config 1
+def test_config1_every_unit_through_all_five_calls(wq, ctx, oracle):
+    spec = ws.CONFIGS["cfg1_single_layer"]
+    (m,) = spec.block_matrices()
+    assert (m.R, m.C) == (4096, 4096) and spec.chunk_widths == (128,) and spec.T == 512
+    G, U = 128, 32
+    W = ws.block_weight(spec, 0, 0, m)
+    X = ws.block_input(spec, 0, 0, 0)
+    grid = ws.clip_grid(spec.K)
+    Wd, grid_d = W.cuda(), torch.from_numpy(grid).cuda()
+    s = wq.windq_act_stats(ctx, X.cuda())
+    s_h = s.cpu().numpy()
+    assert close(s_h, oracle.act_stats(X.numpy())).all()
+    feat = wq.windq_unit_features(ctx, Wd, G, s).cpu().numpy()
+    wf = oracle_features(oracle, W.numpy(), G, s_h)
+    assert (feat[:, 3:5] == wf[:, 3:5]).all() and close(feat, wf).all()
+    fit = wq.windq_fit_eval(ctx, Wd, G, s, grid_d, want_group_err=True)
+    want = oracle.fit_eval(W.numpy(), G, s_h, grid, threads=THREADS)
+    got = {k: v.cpu().numpy() for k, v in fit.items()}
+    ties = Ties()
+    ties.check(oracle, got["clip_idx"], want["clip_idx"], W.numpy(), G, s_h, grid)
+    same = got["clip_idx"] == want["clip_idx"]
+    assert (got["group_err"][:4].view(np.uint32)[same] == want["group_err"][:4].view(np.uint32)[same]).all()
+    assert (got["group_err"][4:].view(np.uint32) == want["group_err"][4:].view(np.uint32)).all()
+    assert close(got["err"], want["err"]).all() and close(got["energy"], want["energy"]).all()
+    ties.report("config 1")
+    plans = [np.arange(U, dtype=np.uint8) % 7] + [block_plans(wq, ctx, [m], G, (2.0,), 3)[2.0][0]]
+    for acts in plans:
+        a_d = torch.from_numpy(acts).cuda()
+        eb = wq.windq_effective_bits(ctx, a_d, m.R, G)
+        o_eb = oracle.effective_bits(acts, m.R, G)
+        assert int(eb["total_centibits"].item()) == o_eb["total_centibits"]
+        assert int(eb["total_packed_bytes"].item()) == o_eb["total_packed_bytes"]
+        assert (eb["code_offsets"].cpu().numpy() == o_eb["code_offsets"]).all()
+        assert (eb["unit_centibits"].cpu().numpy() == o_eb["unit_centibits"]).all()
+        o_plan = oracle_apply(oracle, W.numpy(), G, s_h, grid, acts, want["clip_idx"])
+        for clip_idx in (fit["clip_idx"], None):          # indices supplied, and the search repeated by the call
+            codes = torch.empty(int(o_eb["code_offsets"][-1]), dtype=torch.uint8, device="cuda")
+            plan = wq.windq_apply_plan(ctx, Wd, G, s, grid_d, a_d, eb["code_offsets"], codes, clip_idx)
+            torch.cuda.synchronize()
+            assert (codes.cpu().numpy() == o_plan["codes"]).all()
+            assert (u16(plan["scales"]) == o_plan["scales"]).all() and (u16(plan["zeros"]) == o_plan["zeros"]).all()
+            assert (u16(plan["wq"]) == o_plan["wq"]).all()
+
+
+# ------------------------------------------------------------------ configs 2 and 3: whole blocks, batched calls
+def test_config2_whole_block_through_the_batched_calls(wq, ctx, oracle):
+    check_block(wq, ctx, oracle, ws.CONFIGS["cfg2_llama7b_block"], 0, (128,), (2.0,), 128, "config 2, whole block")
+
+
+def test_config3_block0_both_chunk_widths_three_plans(wq, ctx, oracle):
+    check_block(wq, ctx, oracle, ws.CONFIGS["cfg3_llama7b_model"], 0, (64, 128), (1.58, 2.0, 3.0), 128,
+                "config 3, block 0, chunk widths 64 and 128")
+
+
+# ------------------------------------------------------------------ sampled units of other blocks / larger models
+def check_sampled_units(wq, ctx, oracle, spec, triples, label):
+    """triples: (block, matrix index, chunk width, unit, plan target).  The matrix runs on the device in full; the
+    oracle recomputes the sampled unit from the same bits (weights and statistics)."""
+    grid = ws.clip_grid(spec.K)
+    grid_d = torch.from_numpy(grid).cuda()
+    mats = spec.block_matrices()
+    ties = Ties()
+    by_matrix = {}
+    for t in triples:
+        by_matrix.setdefault((t[0], t[1]), []).append(t[2:])
+    for (block, mi), picks in sorted(by_matrix.items()):
+        m = mats[mi]
+        W = ws.block_weight(spec, 0, block, m, device="cuda")
+        s = wq.windq_act_stats(ctx, ws.block_input(spec, 0, block, m.x_id, device="cuda"))
+        s_h = s.cpu().numpy()
+        for G in sorted({p[0] for p in picks}):
+            U = m.C // G
+            fit = wq.windq_fit_eval(ctx, W, G, s, grid_d)
+            feat = wq.windq_unit_features(ctx, W, G, s).cpu().numpy()
+            for target in sorted({p[2] for p in picks if p[0] == G}):
+                acts = block_plans(wq, ctx, [m], G, (target,), 1000 * block + mi)[target][0]
+                a_d = torch.from_numpy(acts).cuda()
+                eb = wq.windq_effective_bits(ctx, a_d, m.R, G)
+                o_eb = oracle.effective_bits(acts, m.R, G)
+                assert int(eb["total_centibits"].item()) == o_eb["total_centibits"]
+                assert (eb["code_offsets"].cpu().numpy() == o_eb["code_offsets"]).all()
+                offs = o_eb["code_offsets"]
+                codes = torch.empty(int(offs[-1]), dtype=torch.uint8, device="cuda")
+                plan = wq.windq_apply_plan(ctx, W, G, s, grid_d, a_d, eb["code_offsets"], codes, fit["clip_idx"])
+                torch.cuda.synchronize()
+                for u in sorted({p[1] for p in picks if p[0] == G and p[2] == target}):
+                    assert u < U
+                    Wu = W[:, u * G:(u + 1) * G].cpu().numpy()
+                    su = s_h[u * G:(u + 1) * G]
+                    want = oracle.fit_eval(Wu, G, su, grid, threads=1, want_group_err=False)
+                    got_idx = fit["clip_idx"][:, u:u + 1].cpu().numpy()
+                    ties.check(oracle, got_idx, want["clip_idx"], Wu, G, su, grid)
+                    assert close(fit["err"][u].cpu().numpy(), want["err"][0]).all()
+                    assert close(fit["energy"][u].cpu().numpy(), want["energy"][0]).all()
+                    wf = oracle.unit_features(Wu, G, su)
+                    assert (feat[u, 3:5] == wf[0, 3:5]).all() and close(feat[u], wf[0]).all()
+                    wp = oracle.apply_plan(Wu, G, su, grid, acts[u:u + 1], got_idx)
+                    assert (codes[offs[u]:offs[u + 1]].cpu().numpy() == wp["codes"]).all()
+                    assert (u16(plan["scales"][u]) == wp["scales"][0]).all() and (u16(plan["zeros"][u]) == wp["zeros"][0]).all()
+                    assert (u16(plan["wq"][:, u * G:(u + 1) * G]) == wp["wq"]).all()
+        del W
+    torch.cuda.empty_cache()
+    ties.report(label)
+
+
+def seeded_triples(spec, n, seed, blocks, matrices=None):
+    rng = np.random.default_rng(seed)
+    mats = spec.block_matrices()
+    out = []
+    # few distinct matrices (each costs a full-size generation and fit), several units in each
+    n_mats = max(1, n // 4)
+    chosen = [(int(rng.choice(blocks)), int(rng.choice(matrices if matrices is not None else len(mats)))) for _ in range(n_mats)]
+    for i in range(n):
+        block, mi = chosen[i % n_mats]
+        G = int(rng.choice(spec.chunk_widths))
+        out.append((block, mi, G, int(rng.integers(mats[mi].C // G)), float(rng.choice([1.58, 2.0, 3.0]))))
+    return out
+
+
+def test_config3_sixty_four_units_of_the_other_blocks(wq, ctx, oracle):
+    spec = ws.CONFIGS["cfg3_llama7b_model"]
+    check_sampled_units(wq, ctx, oracle, spec, seeded_triples(spec, 64, 31, np.arange(1, spec.n_blocks)),
+                        "config 3, 64 units of blocks 1-31")
+
+
+def test_config4_sampled_units(wq, ctx, oracle):
+    spec = ws.CONFIGS["cfg4_llama13b_model"]       # 40 clip ratios, 4096 calibration tokens
+    check_sampled_units(wq, ctx, oracle, spec, seeded_triples(spec, 16, 41, np.arange(spec.n_blocks)),
+                        "config 4, 16 units")
+
+
+def test_config5_sampled_units_with_grouped_query_matrices(wq, ctx, oracle):
+    spec = ws.CONFIGS["cfg5_llama70b_model"]
+    triples = seeded_triples(spec, 8, 51, np.arange(spec.n_blocks), matrices=[1, 2])          # 1024-row k / v
+    triples += seeded_triples(spec, 8, 52, np.arange(spec.n_blocks), matrices=[0, 4, 6])      # q, gate, down
+    check_sampled_units(wq, ctx, oracle, spec, triples, "config 5, 16 units")

@@ -364,6 +364,80 @@ def test_two_contexts_on_two_streams(wq, ctx):
         wq.windq_destroy(other)
 
 
+def test_one_context_on_two_streams_ordered_by_events(wq, ctx):
+    """Calls on one context share its scratch buffer, so they must not overlap on the GPU.  Two streams that hand
+    the context back and forth through events (each call's stream waits for an event recorded after the previous
+    call) are ordered, and give the results of a single stream."""
+    W1 = ws.weights(400, 1024, 650, "student_t").cuda()
+    W2 = ws.weights(300, 2048, 651, "student_t").cuda()
+    s1, s2 = torch.rand(1024, device="cuda") + 0.1, torch.rand(2048, device="cuda") + 0.1
+    grid = torch.from_numpy(ws.clip_grid(20)).cuda()
+    ref1 = wq.windq_fit_eval(ctx, W1, 128, s1, grid)
+    ref2 = wq.windq_fit_eval(ctx, W2, 64, s2, grid)
+    ref_f = wq.windq_unit_features(ctx, W1, 128, s1).clone()
+    torch.cuda.synchronize()
+    st = [torch.cuda.Stream(), torch.cuda.Stream()]
+    outs = []
+    prev = None
+    for n in range(6):
+        cur = st[n % 2]
+        if prev is not None:
+            cur.wait_event(prev)
+        with torch.cuda.stream(cur):
+            if n % 3 == 0:
+                outs.append(("fit1", wq.windq_fit_eval(ctx, W1, 128, s1, grid, stream=cur)))
+            elif n % 3 == 1:
+                outs.append(("fit2", wq.windq_fit_eval(ctx, W2, 64, s2, grid, stream=cur)))
+            else:
+                outs.append(("feat", wq.windq_unit_features(ctx, W1, 128, s1, stream=cur)))
+            prev = torch.cuda.Event()
+            prev.record(cur)
+    torch.cuda.synchronize()
+    for name, out in outs:
+        if name == "feat":
+            assert torch.equal(out, ref_f)
+        else:
+            ref = ref1 if name == "fit1" else ref2
+            for k in ("err", "energy", "clip_idx"):
+                assert torch.equal(out[k], ref[k]), (name, k)
+
+
+def test_apply_plan_leaves_a_unit_with_a_bad_action_code_untouched(wq, ctx, oracle):
+    """Action codes live on the device: a code above 6 cannot be refused before the launch.  The unit is skipped
+    (its outputs keep what the arrays held), windq_effective_bits flags the plan with totals of -1, and every
+    other unit is packed as the oracle packs it."""
+    G, R, C = 128, 40, 640
+    W, X = make(R, C, 660)
+    s = oracle.act_stats(X.numpy())
+    grid = ws.clip_grid(20)
+    acts = np.array([4, 5, 9, 6, 2], np.uint8)
+    bad = 2
+    fit = oracle.fit_eval(W.numpy(), G, s, grid, threads=4, want_group_err=False)
+    a_d = torch.from_numpy(acts).cuda()
+    eb = wq.windq_effective_bits(ctx, a_d, R, G)
+    assert int(eb["total_centibits"].item()) == -1 and int(eb["total_packed_bytes"].item()) == -1
+    offs = eb["code_offsets"].cpu().numpy()
+    assert offs[bad + 1] == offs[bad]                       # the flagged unit has an empty block
+    U = C // G
+    codes = torch.full((int(offs[-1]),), 0xEE, dtype=torch.uint8, device="cuda")
+    canary = dict(scales=torch.full((U, R), 7.0, dtype=torch.float16, device="cuda"),
+                  zeros=torch.full((U, R), 7.0, dtype=torch.float16, device="cuda"),
+                  wq=torch.full((R, C), 7.0, dtype=torch.float16, device="cuda"))
+    plan = wq.windq_apply_plan(ctx, W.cuda(), G, torch.from_numpy(s).cuda(), torch.from_numpy(grid).cuda(), a_d,
+                               eb["code_offsets"], codes, torch.from_numpy(fit["clip_idx"]).cuda(), out=canary)
+    torch.cuda.synchronize()
+    assert bool((plan["scales"][bad] == 7.0).all()) and bool((plan["zeros"][bad] == 7.0).all())
+    assert bool((plan["wq"][:, bad * G:(bad + 1) * G] == 7.0).all())
+    for u in range(U):
+        if u == bad:
+            continue
+        want = oracle.apply_plan(W.numpy()[:, u * G:(u + 1) * G], G, s[u * G:(u + 1) * G], grid, acts[u:u + 1],
+                                 fit["clip_idx"][:, u:u + 1])
+        assert (codes[offs[u]:offs[u + 1]].cpu().numpy() == want["codes"]).all()
+        assert (plan["scales"][u].cpu().view(torch.int16).numpy().view(np.uint16) == want["scales"][0]).all()
+        assert (plan["wq"][:, u * G:(u + 1) * G].cpu().contiguous().view(torch.int16).numpy().view(np.uint16) == want["wq"]).all()
+
+
 def test_fit_eval_largest_grid_and_widest_chunk(wq, ctx, oracle):
     G, R, C, K = 512, 21, 1024, 64
     W, X = make(R, C, 640)

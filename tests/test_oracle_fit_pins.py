@@ -293,3 +293,26 @@ def test_zero_is_exactly_representable(oracle):
     for a in (1, 2, 3, 4):
         plan = oracle.apply_plan(W, G, s, ws.clip_grid(20), np.array([a], np.uint8))
         assert (plan["wq"][:, ::5] & 0x7fff == 0).all()
+
+
+def test_energy_is_the_weighted_sum_of_squares_in_float64(oracle):
+    """energy[u] = sum over the unit of s_j w_rj^2, pinned by the closed form in float64 with statistics that differ
+    from channel to channel by orders of magnitude (a dropped or misplaced s_j, or a sum over the wrong axis, shows)."""
+    rng = np.random.default_rng(77)
+    R, G, U = 37, 64, 3
+    W = (rng.standard_normal((R, U * G)) * 0.05).astype(np.float16)
+    s = np.exp(rng.standard_normal(U * G) * 2.0).astype(np.float32)
+    s[5] = 0.0
+    s[G + 3] *= 1000.0
+    fit = oracle.fit_eval(W, G, s, ws.clip_grid(5))
+    w64 = W.astype(np.float64)
+    for u in range(U):
+        want = float((s[u * G:(u + 1) * G].astype(np.float64)[None, :] * w64[:, u * G:(u + 1) * G] ** 2).sum())
+        assert abs(float(fit["energy"][u]) - want) <= 1e-6 * want
+    # scaling one channel's statistic changes the energy by exactly that channel's share
+    s2 = s.copy()
+    s2[7] *= 4.0
+    e2 = oracle.fit_eval(W, G, s2, ws.clip_grid(5))["energy"]
+    share = 3.0 * float(s[7]) * float((w64[:, 7] ** 2).sum())
+    assert abs((float(e2[0]) - float(fit["energy"][0])) - share) <= 1e-5 * float(e2[0])
+    assert e2[1] == fit["energy"][1] and e2[2] == fit["energy"][2]

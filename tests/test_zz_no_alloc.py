@@ -25,16 +25,19 @@ def wq():
     return wq
 
 
-def test_noalloc_matches_act_stats_on_two_calls_in_a_row(wq):
+def test_noalloc_matches_act_stats_on_two_calls_in_a_row(wq, oracle):
     ctx = wq.windq_create(0)
     try:
         for T, C, seed in ((700, 1480, 11), (130, 264, 12)):
-            X = ws.activations(T, C, seed).cuda()
-            want = wq.windq_act_stats(ctx, X)
+            X = ws.activations(T, C, seed)
+            Xd = X.cuda()
+            want = wq.windq_act_stats(ctx, Xd)
             got = torch.full((C,), float("nan"), dtype=torch.float32, device="cuda")
-            wq.windq_act_stats_noalloc(ctx, X, got)
+            wq.windq_act_stats_noalloc(ctx, Xd, got)
             torch.cuda.synchronize()
             assert bool((torch.abs(got - want) <= RTOL * torch.abs(want) + ATOL).all()), (T, C)
+            ref = torch.from_numpy(oracle.act_stats(X.numpy())).cuda()      # and against the CPU oracle directly
+            assert bool((torch.abs(got - ref) <= RTOL * torch.abs(ref) + ATOL).all()), (T, C)
     finally:
         wq.windq_destroy(ctx)
 

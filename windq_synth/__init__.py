@@ -99,19 +99,22 @@ class ModelSpec:
     T: int
     K: int
     chunk_widths: tuple
+    only: tuple = ()        # names of the block's matrices that exist (empty = all seven)
 
     def block_matrices(self):
         h, i, kv = self.hidden, self.inter, self.kv
-        return (
+        all_seven = (
             MatrixSpec("q_proj", h, h, 0, 0), MatrixSpec("k_proj", kv, h, 0, 1),
             MatrixSpec("v_proj", kv, h, 0, 2), MatrixSpec("o_proj", h, h, 1, 3),
             MatrixSpec("gate_proj", i, h, 2, 4), MatrixSpec("up_proj", i, h, 2, 5),
             MatrixSpec("down_proj", h, i, 3, 6),
         )
+        return tuple(m for m in all_seven if not self.only or m.name in self.only)
 
     def block_inputs(self):
-        """(x_id, channels) of the four calibration inputs of a block."""
-        return ((0, self.hidden), (1, self.hidden), (2, self.hidden), (3, self.inter))
+        """(x_id, channels) of the calibration inputs of a block (four when all seven matrices exist)."""
+        used = {m.x_id for m in self.block_matrices()}
+        return tuple(ic for ic in ((0, self.hidden), (1, self.hidden), (2, self.hidden), (3, self.inter)) if ic[0] in used)
 
     def elements_per_block(self) -> int:
         return sum(m.R * m.C for m in self.block_matrices())
@@ -121,7 +124,7 @@ class ModelSpec:
 # unit count on ("Episode complexity": LLaMA-3.1-8B, chunk size 256, 32 x 7 x 16 = 3584 units), with its
 # ablated chunk size 512 beside it.
 CONFIGS = {
-    "cfg1_single_layer": ModelSpec("cfg1_single_layer", 1, 4096, 0, 4096, "normal", 512, 20, (128,)),
+    "cfg1_single_layer": ModelSpec("cfg1_single_layer", 1, 4096, 0, 4096, "normal", 512, 20, (128,), only=("q_proj",)),
     "cfg2_llama7b_block": ModelSpec("cfg2_llama7b_block", 1, 4096, 11008, 4096, "normal", 2048, 20, (128,)),
     "cfg3_llama7b_model": ModelSpec("cfg3_llama7b_model", 32, 4096, 11008, 4096, "student_t", 2048, 20, (64, 128)),
     "cfg4_llama13b_model": ModelSpec("cfg4_llama13b_model", 40, 5120, 13824, 5120, "student_t", 4096, 40, (128,)),

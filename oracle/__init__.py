@@ -350,3 +350,84 @@ def fit_refine(W, G: int, s, clip_grid, clip_idx, T: int = 10, lr: float = 0.01,
     if rc:
         raise ValueError("oracle_fit_refine: bad arguments (%d)" % rc)
     return dict(err=err, scale=scale.view(np.float16), group_err=gerr)
+
+
+def ternary_candidate(w, s, rho: float, want_trits: bool = True):
+    """One threshold ratio on one row-group: (alpha, error, trits)."""
+    w, s = _f32(w), _f32(s)
+    G = w.size
+    alpha, err = ctypes.c_float(), ctypes.c_float()
+    trits = np.zeros(G, np.uint8) if want_trits else None
+    rc = lib().oracle_ternary_candidate(_p(w), _p(s), ctypes.c_int(G), ctypes.c_float(rho), ctypes.byref(alpha),
+                                        ctypes.byref(err), _p(trits))
+    if rc:
+        raise ValueError("oracle_ternary_candidate: bad arguments")
+    return alpha.value, err.value, trits
+
+
+def binary_candidate(w, s, want_bits: bool = True):
+    """The 1-bit fit of one row-group: (alpha, error, bits)."""
+    w, s = _f32(w), _f32(s)
+    G = w.size
+    alpha, err = ctypes.c_float(), ctypes.c_float()
+    bits = np.zeros(G, np.uint8) if want_bits else None
+    rc = lib().oracle_binary_candidate(_p(w), _p(s), ctypes.c_int(G), ctypes.byref(alpha), ctypes.byref(err), _p(bits))
+    if rc:
+        raise ValueError("oracle_binary_candidate: bad arguments")
+    return alpha.value, err.value, bits
+
+
+def fit_ternary_search(W, G: int, s, thr_grid, units=None, threads: int = 1, thresh=None, want_group_err: bool = True):
+    """Search over the ternary threshold ratio.  Returns dict(err [U] f32, thr_idx [U][R] u8, alpha [U][R] f16,
+    group_err [U][R] f32 | None).  ``units``, ``threads`` and ``thresh`` as in fit_eval."""
+    W, s, thr_grid = _as_u16(W), _f32(s), _f32(thr_grid)
+    R, C = W.shape
+    U = C // G
+    u0, u1 = (0, U) if units is None else units
+    err = np.zeros(U, np.float32)
+    thr_idx = np.zeros((U, R), np.uint8)
+    alpha = np.zeros((U, R), np.uint16)
+    gerr = np.zeros((U, R), np.float32) if want_group_err else None
+    if thresh is not None:
+        thresh = _f32(thresh)
+        assert thresh.size == U
+
+    def run(a, b):
+        rc = lib().oracle_fit_ternary_search(_p(W), ctypes.c_int64(R), ctypes.c_int64(C), ctypes.c_int64(C), ctypes.c_int(G),
+                                             _p(s), _p(thr_grid), ctypes.c_int(thr_grid.size), ctypes.c_int64(a),
+                                             ctypes.c_int64(b), _p(thresh), _p(err), _p(thr_idx), _p(alpha), _p(gerr))
+        if rc:
+            raise ValueError("oracle_fit_ternary_search: bad arguments")
+
+    if threads <= 1 or u1 - u0 <= 1:
+        run(u0, u1)
+    else:
+        bounds = np.linspace(u0, u1, min(threads, u1 - u0) + 1).astype(np.int64)
+        with ThreadPoolExecutor(max_workers=threads) as ex:
+            list(ex.map(lambda ab: run(int(ab[0]), int(ab[1])), zip(bounds[:-1], bounds[1:])))
+    return dict(err=err, thr_idx=thr_idx, alpha=alpha.view(np.float16), group_err=gerr)
+
+
+def apply_plan_searched(W, G: int, s, clip_grid, actions, clip_idx, thr_grid, thr_idx, want_wq: bool = True):
+    """apply_plan with the ternary thresholds chosen by fit_ternary_search (thr_idx u8 [U][R])."""
+    W, s, clip_grid, thr_grid = _as_u16(W), _f32(s), _f32(clip_grid), _f32(thr_grid)
+    actions = np.ascontiguousarray(actions, dtype=np.uint8)
+    R, C = W.shape
+    U = C // G
+    offs = effective_bits(actions, R, G)["code_offsets"]
+    codes = np.zeros(int(offs[U]), np.uint8)
+    scales = np.zeros((U, R), np.uint16)
+    zeros = np.zeros((U, R), np.uint16)
+    wq = np.zeros((R, C), np.uint16) if want_wq else None
+    if clip_idx is not None:
+        clip_idx = np.ascontiguousarray(clip_idx, dtype=np.uint8)
+        assert clip_idx.shape == (4, U, R)
+    thr_idx = np.ascontiguousarray(thr_idx, dtype=np.uint8)
+    assert thr_idx.shape == (U, R)
+    rc = lib().oracle_apply_plan_searched(_p(W), ctypes.c_int64(R), ctypes.c_int64(C), ctypes.c_int64(C), ctypes.c_int(G),
+                                          _p(s), _p(clip_grid), ctypes.c_int(clip_grid.size), _p(actions), _p(clip_idx),
+                                          _p(thr_grid), ctypes.c_int(thr_grid.size), _p(thr_idx), _p(offs), _p(codes),
+                                          _p(scales), _p(zeros), _p(wq))
+    if rc:
+        raise ValueError("oracle_apply_plan_searched: bad arguments")
+    return dict(codes=codes, scales=scales, zeros=zeros, wq=wq, code_offsets=offs)

@@ -36,9 +36,12 @@
 // two; degenerate groups; monotone error in bit-width; Eq. 6 bit arithmetic;
 // pack/unpack identity with an independent unpacker; nearest-rank P99 against a
 // full sort; salient selection against a full sort, its count arithmetic and
-// Eq. 6 with protected weights against the paper's formula.  Parity unpinned: that threshold 0.7*mean|w| is a good ternary
-// threshold, and that these fits resemble the paper's Adam-fitted operators --
-// neither is claimed.
+// Eq. 6 with protected weights against the paper's formula; the ternary
+// threshold search against a hand-worked case, against the exhaustive optimum
+// over all 3^8 codes of toy groups, and against its reduction to the 0.7 rule;
+// the 1-bit fit against the exhaustive optimum over all 2^8 sign patterns.
+// Parity unpinned: that these fits resemble the paper's Adam-fitted operators
+// -- not claimed.
 
 #include <algorithm>
 #include <cmath>
@@ -210,12 +213,12 @@ float error_against(const Group& g, const float* what) {   // what[j] = reconstr
   });
 }
 
-// READING: ternary = threshold 0.7 * mean|w| (textbook ternary weights), one
-// scale alpha = s-weighted mean of |w| on the support, stored in fp16.
-// trit[j] in {0,1,2} = 1 + sign(w_j) on the support, 1 elsewhere.
-float fit_ternary(const Group& g, float A, uint8_t* trit /*nullable*/, float* what /*nullable*/) {
+// READING: ternary = threshold rho * mean|w|, one scale alpha = s-weighted mean
+// of |w| on the support, stored in fp16.  trit[j] in {0,1,2} = 1 + sign(w_j) on
+// the support, 1 elsewhere.  A = PSUM8 of |w| over the group.
+float fit_ternary_at(const Group& g, float A, float rho, uint8_t* trit /*nullable*/, float* what /*nullable*/) {
   const int G = g.G;
-  const float delta = 0.7f * (A * (1.0f / (float)G));
+  const float delta = rho * (A * (1.0f / (float)G));
   bool any = false;
   std::vector<uint8_t> in(G);
   for (int j = 0; j < G; ++j) { in[j] = std::fabs(g.w[j]) > delta; any = any || in[j]; }
@@ -248,6 +251,11 @@ float fit_ternary(const Group& g, float A, uint8_t* trit /*nullable*/, float* wh
     if (what) what[j] = (float)(t - 1) * alpha;
   }
   return alpha;
+}
+
+// The fit of windq_fit_eval: rho = 0.7 (textbook ternary weights).
+float fit_ternary(const Group& g, float A, uint8_t* trit /*nullable*/, float* what /*nullable*/) {
+  return fit_ternary_at(g, A, 0.7f, trit, what);
 }
 
 // READING: binary = sign(w) * alpha, alpha = s-weighted mean |w| in fp16;
@@ -548,8 +556,10 @@ static int apply_plan_impl(const uint16_t* W, int64_t R, int64_t C, int64_t ldw,
                            const float* clip_grid, int K, const uint8_t* actions, const uint8_t* clip_idx,
                            const int64_t* code_offsets, const float* thresh, uint8_t* codes_out, uint16_t* scales_out,
                            uint16_t* zeros_out, uint16_t* Wq_out, uint16_t* prot_scale_out, int64_t* prot_offsets_out,
-                           int8_t* prot_q_out, const uint16_t* scale_in = nullptr) {
+                           int8_t* prot_q_out, const uint16_t* scale_in = nullptr, const float* thr_grid = nullptr,
+                           int Kt = 0, const uint8_t* thr_idx = nullptr) {
   if (thresh && (!prot_scale_out || !prot_offsets_out || !prot_q_out)) return 1;
+  if (thr_idx && (!thr_grid || Kt < 1 || Kt > 64)) return 1;
   if (!W || !s || !clip_grid || !actions || !code_offsets || !codes_out || !scales_out || !zeros_out ||
       R <= 0 || C <= 0 || !valid_group_width(G) || C % G != 0 || ldw < C || K < 1 || K > 64)
     return 1;
@@ -623,7 +633,13 @@ static int apply_plan_impl(const uint16_t* W, int64_t R, int64_t C, int64_t ldw,
           zero_h = float_to_half(p.zf);
         } else {
           const float A = sum_abs(g);
-          const float alpha = (a == 5) ? fit_ternary(g, A, q.data(), what.data())
+          float rho = 0.7f;
+          if (thr_idx) {  // the threshold ratio the search chose for this group (an index beyond the grid = the last)
+            int kt = thr_idx[u * R + r];
+            if (kt >= Kt) kt = Kt - 1;
+            rho = thr_grid[kt];
+          }
+          const float alpha = (a == 5) ? fit_ternary_at(g, A, rho, q.data(), what.data())
                                        : fit_binary(g, A, q.data(), what.data());
           scale_h = float_to_half(alpha);
         }
@@ -674,6 +690,92 @@ int oracle_apply_plan_protected_refined(const uint16_t* W, int64_t R, int64_t C,
   if (!thresh || !clip_idx || !scale_in) return 1;
   return apply_plan_impl(W, R, C, ldw, G, s, clip_grid, K, actions, clip_idx, code_offsets, thresh, codes_out,
                          scales_out, zeros_out, Wq_out, prot_scale_out, prot_offsets_out, prot_q_out, scale_in);
+}
+
+// ---- search over the ternary assignment (App. "Per-unit Scale Optimization": the low-bit operators
+// fit their assignment and a per-group scale; Sec. 3.5) ------------------------------------------------
+// The paper prints no formula for its low-bit operators.  READING: for a fixed scale alpha the best
+// ternary code of w_j is sign(w_j) when |w_j| > alpha / 2 and 0 otherwise, whatever s_j is, so the best
+// support is always a threshold set {|w| > tau}; and for a fixed support the best scale is the
+// s-weighted mean of |w| on it.  The search therefore tries Kt thresholds tau_k = thr_grid[k] * mean|w|
+// (ratios supplied by the caller, like the clip ratios), fits each exactly as fit_ternary_at does, scores
+// it by the s-weighted squared error in PSUM8 order, and keeps the smallest k with the least error.
+// With thr_grid = {0.7} the result is the ternary column of oracle_fit_eval, bit for bit.
+// The 1-bit operator needs no search: with the two levels +-alpha the code sign(w_j) is the best one for
+// every alpha > 0, and alpha has its closed form (fit_binary).
+// thresh (nullable): salient weights are taken out of the group as in the protected fit.
+//   err_out fp32 [U] (double accumulation over rows), thr_idx_out u8 [U][R], alpha_out fp16 bits [U][R],
+//   group_err_out fp32 [U][R] (nullable)
+int oracle_fit_ternary_search(const uint16_t* W, int64_t R, int64_t C, int64_t ldw, int G, const float* s,
+                              const float* thr_grid, int Kt, int64_t u_begin, int64_t u_end, const float* thresh,
+                              float* err_out, uint8_t* thr_idx_out, uint16_t* alpha_out, float* group_err_out) {
+  if (!W || !s || !thr_grid || !err_out || !thr_idx_out || !alpha_out || R <= 0 || C <= 0 || !valid_group_width(G) ||
+      C % G != 0 || ldw < C || Kt < 1 || Kt > 64)
+    return 1;
+  const int64_t U = C / G;
+  if (u_begin < 0 || u_end > U || u_begin > u_end) return 1;
+  std::vector<float> w((size_t)G), what((size_t)G), sm((size_t)G);
+  for (int64_t u = u_begin; u < u_end; ++u) {
+    double tot = 0.0;
+    const float* su = s + u * G;
+    for (int64_t r = 0; r < R; ++r) {
+      load_group(W, ldw, r, u, G, w.data());
+      if (thresh) {
+        for (int j = 0; j < G; ++j) {
+          const bool prot = std::fabs(w[(size_t)j]) * std::sqrt(s[u * G + j]) >= thresh[u];
+          sm[(size_t)j] = prot ? 0.0f : s[u * G + j];
+          if (prot) w[(size_t)j] = 0.0f;
+        }
+        su = sm.data();
+      }
+      Group g{G, w.data(), su};
+      const float A = sum_abs(g);
+      int bk = 0;
+      float be = 0.0f, balpha = 0.0f;
+      for (int k = 0; k < Kt; ++k) {
+        const float alpha = fit_ternary_at(g, A, thr_grid[k], nullptr, what.data());
+        const float e = error_against(g, what.data());
+        if (k == 0 || e < be) { be = e; bk = k; balpha = alpha; }
+      }
+      thr_idx_out[u * R + r] = (uint8_t)bk;
+      alpha_out[u * R + r] = float_to_half(balpha);
+      if (group_err_out) group_err_out[u * R + r] = be;
+      tot += (double)be;
+    }
+    err_out[u] = (float)tot;
+  }
+  return 0;
+}
+
+// One threshold ratio on one group (exported so that the tests can pin it): scale, error, trits.
+int oracle_ternary_candidate(const float* w, const float* s, int G, float rho, float* alpha_out, float* err_out,
+                             uint8_t* trits_out /*nullable*/) {
+  if (!w || !s || !valid_group_width(G) || !alpha_out || !err_out) return 1;
+  Group g{G, w, s};
+  std::vector<float> what((size_t)G);
+  *alpha_out = fit_ternary_at(g, sum_abs(g), rho, trits_out, what.data());
+  *err_out = error_against(g, what.data());
+  return 0;
+}
+
+// One group under the 1-bit fit (exported for the pins): scale, error, bits.
+int oracle_binary_candidate(const float* w, const float* s, int G, float* alpha_out, float* err_out, uint8_t* bits_out /*nullable*/) {
+  if (!w || !s || !valid_group_width(G) || !alpha_out || !err_out) return 1;
+  Group g{G, w, s};
+  std::vector<float> what((size_t)G);
+  *alpha_out = fit_binary(g, sum_abs(g), bits_out, what.data());
+  *err_out = error_against(g, what.data());
+  return 0;
+}
+
+// oracle_apply_plan with the thresholds the search chose for the 1.58-bit units (thr_idx u8 [U][R]).
+int oracle_apply_plan_searched(const uint16_t* W, int64_t R, int64_t C, int64_t ldw, int G, const float* s,
+                               const float* clip_grid, int K, const uint8_t* actions, const uint8_t* clip_idx,
+                               const float* thr_grid, int Kt, const uint8_t* thr_idx, const int64_t* code_offsets,
+                               uint8_t* codes_out, uint16_t* scales_out, uint16_t* zeros_out, uint16_t* Wq_out) {
+  if (!thr_grid || !thr_idx) return 1;
+  return apply_plan_impl(W, R, C, ldw, G, s, clip_grid, K, actions, clip_idx, code_offsets, nullptr, codes_out,
+                         scales_out, zeros_out, Wq_out, nullptr, nullptr, nullptr, nullptr, thr_grid, Kt, thr_idx);
 }
 
 // ---- salient-weight selection (App. "Salient Weight Protection") -----------------------------

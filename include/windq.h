@@ -250,6 +250,24 @@ windq_status windq_apply_plan(windq_ctx* ctx, const void* W, int64_t R, int64_t 
                               const uint8_t* clip_idx, const int64_t* code_offsets, uint8_t* codes_out,
                               void* scales_out, void* zeros_out, void* Wq_out, void* stream);
 
+/* Several plans of ONE matrix in one pass over its weights (the paper has no counterpart; a consumer that
+ * compares candidate plans, or keeps plans for several bit budgets, packs them together): every weight is read
+ * from memory once and quantised under each plan in turn.  Every plan is one windq_apply_plan call with clip
+ * indices (clip_idx u8 [4][U][R] is required and shared by the plans): same meanings, layouts and results, bit
+ * for bit.  Plans must not share output arrays; Wq_out may be NULL in any of them.
+ *   plans: HOST array of n_plans descriptors (1 <= n_plans <= 4), read during the call only. */
+typedef struct {
+  const uint8_t* actions;       /* u8 [U] */
+  const int64_t* code_offsets;  /* i64 [U+1] */
+  uint8_t* codes_out;
+  void* scales_out;             /* fp16 [U][R] */
+  void* zeros_out;              /* fp16 [U][R] */
+  void* Wq_out;                 /* fp16 [R][ldw], nullable */
+} windq_plan_out;
+windq_status windq_apply_plan_multi(windq_ctx* ctx, const void* W, int64_t R, int64_t C, int64_t ldw, int G,
+                                    const float* s, const float* clip_grid, int K, const uint8_t* clip_idx,
+                                    const windq_plan_out* plans, int n_plans, void* stream);
+
 /* windq_apply_plan for several (matrix, plan) pairs in one launch.  Every job is one windq_apply_plan call with
  * clip indices (clip_idx is required here): same meanings, layouts and results, bit for bit.  All jobs share G,
  * the clip grid and K.  Jobs must not share output arrays (two plans of one matrix need two Wq_out, or NULL).
@@ -389,6 +407,41 @@ windq_status windq_apply_plan_protected_refined(windq_ctx* ctx, const void* W, i
                                                 const float* thresh, uint8_t* codes_out, void* scales_out, void* zeros_out,
                                                 void* Wq_out, void* prot_scale_out, int64_t* prot_offsets_out,
                                                 int8_t* prot_q_out, int64_t prot_q_capacity, void* stream);
+
+/* Search over the ternary assignment (App. "Per-unit Scale Optimization" and Sec. 3.5 name fitted low-bit
+ * operators -- soft assignments with a scale per group at 1.58 bit, elastic binarization at 1 bit -- without
+ * formulas).  What this call does: for a fixed scale alpha the best ternary code of w_j is sign(w_j) when
+ * |w_j| > alpha / 2 and 0 otherwise, whatever s_j is, so the best support is a threshold set; and for a fixed
+ * support the best scale is the s-weighted mean of |w| on it.  The call tries thr_K thresholds
+ *   tau_k = thr_grid[k] * mean|w|          (ratios supplied by the caller, like the clip ratios),
+ * fits every one exactly as windq_fit_eval fits its single threshold 0.7 * mean|w| (support {|w| > tau_k}, scale
+ * = fp16 of the s-weighted mean of |w| on it, the unweighted mean if that support carries no activation weight, 0
+ * if it is empty), scores it by the s-weighted squared error and keeps the smallest k with the least error.
+ * With thr_grid = {0.7} the results are the 1.58-bit column of windq_fit_eval, bit for bit.  (The 1-bit operator
+ * needs no search: with levels +-alpha the code sign(w_j) is the best one for every alpha > 0, and alpha has
+ * the closed form windq_fit_eval uses.)
+ *   thr_grid      fp32 [thr_K] (device), 1 <= thr_K <= 64, ratios in (0, 64]
+ *   thresh        fp32 [U] or NULL: salient-weight thresholds of windq_salient_select; protected weights leave the
+ *                 groups as in windq_fit_eval_protected
+ *   err_out       fp32 [U]      sum over rows of the best error (double accumulation)
+ *   thr_idx_out   u8   [U][R]   the chosen index
+ *   alpha_out     fp16 [U][R]   the scale of the chosen fit
+ *   group_err_out fp32 [U][R]   nullable
+ * Group-level results are bit-reproducible.  Scratch: windq_scratch_bytes_fit_ternary_search. */
+int64_t windq_scratch_bytes_fit_ternary_search(int64_t R, int64_t C, int G);
+windq_status windq_fit_ternary_search(windq_ctx* ctx, const void* W, int64_t R, int64_t C, int64_t ldw, int G,
+                                      const float* s, const float* thr_grid, int thr_K, const float* thresh,
+                                      float* err_out, uint8_t* thr_idx_out, void* alpha_out, float* group_err_out,
+                                      void* stream);
+
+/* windq_apply_plan with the thresholds that windq_fit_ternary_search chose: a 1.58-bit unit is packed with
+ * tau = thr_grid[thr_idx[u][r]] * mean|w| in place of 0.7 * mean|w| (an index >= thr_K means thr_K - 1).
+ * clip_idx, thr_grid and thr_idx (u8 [U][R]) are required; everything else as windq_apply_plan. */
+windq_status windq_apply_plan_searched(windq_ctx* ctx, const void* W, int64_t R, int64_t C, int64_t ldw, int G,
+                                       const float* s, const float* clip_grid, int K, const uint8_t* actions,
+                                       const uint8_t* clip_idx, const float* thr_grid, int thr_K, const uint8_t* thr_idx,
+                                       const int64_t* code_offsets, uint8_t* codes_out, void* scales_out, void* zeros_out,
+                                       void* Wq_out, void* stream);
 
 /* The deterministic rule of the paper's heuristic allocator ("Comparison with Heuristic Sensitivity
  * Allocator": units ranked by saliency; all start at 2 bit; the least sensitive are pushed to 1.58 or

@@ -85,6 +85,11 @@ def _load() -> ctypes.CDLL:
     lib.windq_scratch_bytes_greedy_allocate.restype = i64
     lib.windq_scratch_bytes_greedy_allocate.argtypes = [i64]
     lib.windq_apply_plan.argtypes = [vp, vp, i64, i64, i64, i32, vp, vp, i32, vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.windq_apply_plan_multi.argtypes = [vp, vp, i64, i64, i64, i32, vp, vp, i32, vp, vp, i32, vp]
+    lib.windq_apply_plan_searched.argtypes = [vp, vp, i64, i64, i64, i32, vp, vp, i32, vp, vp, vp, i32, vp, vp, vp, vp, vp, vp, vp]
+    lib.windq_fit_ternary_search.argtypes = [vp, vp, i64, i64, i64, i32, vp, vp, i32, vp, vp, vp, vp, vp, vp]
+    lib.windq_scratch_bytes_fit_ternary_search.argtypes = [i64, i64, i32]
+    lib.windq_scratch_bytes_fit_ternary_search.restype = i64
     return lib
 
 
@@ -659,4 +664,122 @@ def windq_apply_plan_protected(ctx: Context, W: torch.Tensor, G: int, s: torch.T
                                                _ptr(actions), _ptr(clip_idx), _ptr(code_offsets), _ptr(thresh), _ptr(codes_out),
                                                _ptr(out["scales"]), _ptr(out["zeros"]), _ptr(out["wq"]), _ptr(out["prot_scale"]),
                                                _ptr(out["prot_offsets"]), _ptr(prot_q_out), prot_q_out.numel(), _stream(stream)))
+    return out
+
+
+class _PlanOut(ctypes.Structure):
+    _fields_ = [("actions", ctypes.c_void_p), ("code_offsets", ctypes.c_void_p), ("codes_out", ctypes.c_void_p),
+                ("scales_out", ctypes.c_void_p), ("zeros_out", ctypes.c_void_p), ("Wq_out", ctypes.c_void_p)]
+
+
+def windq_apply_plan_multi(ctx: Context, W: torch.Tensor, G: int, s: torch.Tensor, clip_grid: torch.Tensor,
+                           clip_idx: torch.Tensor, plans, *, stream=None) -> list:
+    """Up to four plans of one matrix in one pass over its weights.  ``plans``: a sequence of dicts with the keys
+    actions, code_offsets, codes (uint8 output, sized by the caller) and optionally scales, zeros ([U, R] fp16) and
+    wq ([R, C] fp16 with the row stride of W, or None for no fake-quantised output; absent = allocated).
+    Returns one dict(codes, scales, zeros, wq) per plan."""
+    R, C, ldw = _matrix(W, "W")
+    _need(s, torch.float32, "s", 1)
+    _need(clip_grid, torch.float32, "clip_grid", 1)
+    _need(clip_idx, torch.uint8, "clip_idx", 3)
+    U = C // G if G > 0 else 0
+    if tuple(clip_idx.shape) != (4, U, R) or not clip_idx.is_contiguous():
+        raise ValueError("clip_idx must be a contiguous [4, U, R] tensor")
+    if not plans:
+        raise ValueError("plans must not be empty")
+    arr = (_PlanOut * len(plans))()
+    results = []
+    dev = W.device
+    for j, pl in enumerate(plans):
+        actions, offs, codes = pl["actions"], pl["code_offsets"], pl["codes"]
+        _need(actions, torch.uint8, "actions", 1)
+        _need(offs, torch.int64, "code_offsets", 1)
+        _need(codes, torch.uint8, "codes", 1)
+        if actions.numel() != U or offs.numel() != U + 1:
+            raise ValueError("plan %d: actions must have U and code_offsets U + 1 entries" % j)
+        scales = pl.get("scales")
+        zeros = pl.get("zeros")
+        if scales is None:
+            scales = torch.empty((U, R), dtype=torch.float16, device=dev)
+        if zeros is None:
+            zeros = torch.empty((U, R), dtype=torch.float16, device=dev)
+        wq_out = pl["wq"] if "wq" in pl else torch.empty_strided((R, C), (ldw, 1), dtype=torch.float16, device=dev)
+        if wq_out is not None and (_matrix(wq_out, "wq")[2] != ldw or wq_out.shape != W.shape):
+            raise ValueError("plan %d: wq must have the shape and row stride of W" % j)
+        arr[j] = _PlanOut(actions.data_ptr(), offs.data_ptr(), codes.data_ptr(), scales.data_ptr(), zeros.data_ptr(),
+                          None if wq_out is None else wq_out.data_ptr())
+        results.append(dict(codes=codes, scales=scales, zeros=zeros, wq=wq_out))
+    ctx._check(_lib.windq_apply_plan_multi(ctx._h, _ptr(W), R, C, ldw, int(G), _ptr(s), _ptr(clip_grid), clip_grid.numel(),
+                                           _ptr(clip_idx), ctypes.cast(arr, ctypes.c_void_p), len(plans), _stream(stream)))
+    return results
+
+
+def windq_scratch_bytes_fit_ternary_search(R: int, C: int, G: int) -> int:
+    return int(_lib.windq_scratch_bytes_fit_ternary_search(R, C, G))
+
+
+def windq_fit_ternary_search(ctx: Context, W: torch.Tensor, G: int, s: torch.Tensor, thr_grid: torch.Tensor, *,
+                             thresh: torch.Tensor | None = None, want_group_err: bool = False, out: dict | None = None,
+                             stream=None) -> dict:
+    """Search over the ternary threshold ratio.  Returns dict(err [U] f32, thr_idx [U, R] u8, alpha [U, R] f16,
+    group_err [U, R] f32 | None)."""
+    R, C, ldw = _matrix(W, "W")
+    _need(s, torch.float32, "s", 1)
+    _need(thr_grid, torch.float32, "thr_grid", 1)
+    U = C // G if G > 0 else 0
+    if thresh is not None:
+        _need(thresh, torch.float32, "thresh", 1)
+        if thresh.numel() != U:
+            raise ValueError("thresh must have U entries")
+    out = dict(out) if out else {}
+    dev = W.device
+    if out.get("err") is None:
+        out["err"] = torch.empty(U, dtype=torch.float32, device=dev)
+    if out.get("thr_idx") is None:
+        out["thr_idx"] = torch.empty((U, R), dtype=torch.uint8, device=dev)
+    if out.get("alpha") is None:
+        out["alpha"] = torch.empty((U, R), dtype=torch.float16, device=dev)
+    if want_group_err and out.get("group_err") is None:
+        out["group_err"] = torch.empty((U, R), dtype=torch.float32, device=dev)
+    out.setdefault("group_err", None)
+    ctx._check(_lib.windq_fit_ternary_search(ctx._h, _ptr(W), R, C, ldw, int(G), _ptr(s), _ptr(thr_grid), thr_grid.numel(),
+                                             _ptr(thresh), _ptr(out["err"]), _ptr(out["thr_idx"]), _ptr(out["alpha"]),
+                                             _ptr(out["group_err"]), _stream(stream)))
+    return out
+
+
+def windq_apply_plan_searched(ctx: Context, W: torch.Tensor, G: int, s: torch.Tensor, clip_grid: torch.Tensor,
+                              actions: torch.Tensor, code_offsets: torch.Tensor, codes_out: torch.Tensor,
+                              clip_idx: torch.Tensor, thr_grid: torch.Tensor, thr_idx: torch.Tensor, *,
+                              want_wq: bool = True, out: dict | None = None, stream=None) -> dict:
+    """windq_apply_plan with the ternary thresholds chosen by windq_fit_ternary_search (thr_idx u8 [U, R])."""
+    R, C, ldw = _matrix(W, "W")
+    _need(s, torch.float32, "s", 1)
+    _need(clip_grid, torch.float32, "clip_grid", 1)
+    _need(thr_grid, torch.float32, "thr_grid", 1)
+    _need(actions, torch.uint8, "actions", 1)
+    _need(code_offsets, torch.int64, "code_offsets", 1)
+    _need(codes_out, torch.uint8, "codes_out", 1)
+    _need(clip_idx, torch.uint8, "clip_idx", 3)
+    _need(thr_idx, torch.uint8, "thr_idx", 2)
+    U = C // G if G > 0 else 0
+    if actions.numel() != U or code_offsets.numel() != U + 1:
+        raise ValueError("actions must have U and code_offsets U + 1 entries")
+    if tuple(clip_idx.shape) != (4, U, R) or tuple(thr_idx.shape) != (U, R) or not clip_idx.is_contiguous() \
+            or not thr_idx.is_contiguous():
+        raise ValueError("clip_idx must be a contiguous [4, U, R] and thr_idx a contiguous [U, R] tensor")
+    out = dict(out) if out else {}
+    dev = W.device
+    if out.get("scales") is None:
+        out["scales"] = torch.empty((U, R), dtype=torch.float16, device=dev)
+    if out.get("zeros") is None:
+        out["zeros"] = torch.empty((U, R), dtype=torch.float16, device=dev)
+    if want_wq and out.get("wq") is None:
+        out["wq"] = torch.empty_strided((R, C), (ldw, 1), dtype=torch.float16, device=dev)
+    out.setdefault("wq", None)
+    out["codes"] = codes_out
+    ctx._check(_lib.windq_apply_plan_searched(ctx._h, _ptr(W), R, C, ldw, int(G), _ptr(s), _ptr(clip_grid), clip_grid.numel(),
+                                              _ptr(actions), _ptr(clip_idx), _ptr(thr_grid), thr_grid.numel(), _ptr(thr_idx),
+                                              _ptr(code_offsets), _ptr(codes_out), _ptr(out["scales"]), _ptr(out["zeros"]),
+                                              _ptr(out["wq"]), _stream(stream)))
     return out

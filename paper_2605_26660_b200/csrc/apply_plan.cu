@@ -636,6 +636,10 @@ static windq_status apply_plan_plain(windq_ctx* ctx, const void* W, int64_t R, i
   DeviceGuard guard(ctx->device);
   const int U = (int)(C / G);
   cudaStream_t st = (cudaStream_t)stream;
+  if (clip_idx) {  // clip indices supplied: the streaming kernel
+    const windq_plan_out pl = {actions, code_offsets, codes_out, scales_out, zeros_out, Wq_out};
+    return launch_apply_stream(ctx, G, W, R, C, ldw, s, clip_grid, K, clip_idx, scale_in, nullptr, 0, nullptr, &pl, 1, st);
+  }
   const __half* Wh = (const __half*)W;
   const long long* offs = (const long long*)code_offsets;
   __half *sc = (__half*)scales_out, *zp = (__half*)zeros_out, *wq = (__half*)Wq_out;

@@ -82,7 +82,7 @@ windq_status windq_create(windq_ctx** out, int device) {
   ctx->sm_count = prop.multiProcessorCount;
   ctx->scratch = nullptr;
   ctx->scratch_bytes = 0;
-  ctx->prepared = 0;
+  ctx->prepared[0] = ctx->prepared[1] = 0;
   memset(ctx->occupancy, 0, sizeof(ctx->occupancy));
   ctx->err[0] = 0;
   *out = ctx;

@@ -14,8 +14,8 @@ struct windq_ctx {
   int sm_count;
   void* scratch;
   int64_t scratch_bytes;
-  unsigned long long prepared;  // kernels whose attributes have been set on this context's device (bit per KernelId)
-  int occupancy[64];            // resident blocks per SM of those kernels (0 where not asked)
+  unsigned long long prepared[2];  // kernels whose attributes have been set on this context's device (bit per KernelId)
+  int occupancy[128];              // resident blocks per SM of those kernels (0 where not asked)
   char err[256];
 };
 
@@ -55,14 +55,15 @@ struct DeviceGuard {
 // One bit per kernel instantiation that needs a function attribute or an occupancy figure.  Function
 // attributes belong to a device, so the record is kept in the context, not in a process-wide static.
 enum KernelId { kFitG32 = 0, kApplyG32 = 5, kApplySearchG32 = 10, kHistG32 = 15, kFinalize = 20, kFitProtectG32 = 21, kApplyProtectG32 = 26, kApplyProtectSearchG32 = 31,
-                kFitBatchG32 = 41 /* 41..45 whole items, 46..50 in parts */, kApplyBatchG32 = 51 /* 51..55 */, kFitPartsOffset = 36 /* kFitG32 + 36 .. and kFitProtectG32 + 36 ..: the in-parts instantiations (36..40, 57..61) */ };
+                kFitBatchG32 = 41 /* 41..45 whole items, 46..50 in parts */, kApplyBatchG32 = 51 /* 51..55 */, kFitPartsOffset = 36 /* kFitG32 + 36 .. and kFitProtectG32 + 36 ..: the in-parts instantiations (36..40, 57..61) */,
+                kApplyStreamG32 = 64 /* 64..68 */, kTernarySearchG32 = 69 /* 69..73 plain, 74..78 protected */, kKernelIds = 128 };
 inline int g_index(int G) { return G == 32 ? 0 : G == 64 ? 1 : G == 128 ? 2 : G == 256 ? 3 : 4; }
 
 // Sets the dynamic shared-memory limit of `kernel` once per context and, if asked, records how many
 // of its blocks fit on an SM.
 template <class K>
 windq_status prepare_kernel(windq_ctx* ctx, int id, K kernel, int threads, size_t smem, bool want_occupancy) {
-  if (ctx->prepared & (1ull << id)) return WINDQ_OK;
+  if (ctx->prepared[id >> 6] & (1ull << (id & 63))) return WINDQ_OK;
   if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
     cudaGetLastError();
     return fail(ctx, WINDQ_ERR_CUDA, "cannot reserve %lld bytes of shared memory per block", (long long)smem);
@@ -75,7 +76,7 @@ windq_status prepare_kernel(windq_ctx* ctx, int id, K kernel, int threads, size_
     }
     ctx->occupancy[id] = n > 0 ? n : 1;
   }
-  ctx->prepared |= 1ull << id;
+  ctx->prepared[id >> 6] |= 1ull << (id & 63);
   return WINDQ_OK;
 }
 
@@ -83,6 +84,13 @@ windq_status prepare_kernel(windq_ctx* ctx, int id, K kernel, int threads, size_
 windq_status check_matrix(windq_ctx* ctx, const char* who, const void* W, int64_t R, int64_t C, int64_t ldw, int G);
 // The clip grid lives on the device and is used as given; only K can be checked on the host.
 windq_status check_K(windq_ctx* ctx, const char* who, int K);
+
+// The streaming plan kernel (apply_stream.cu): one matrix, n_plans plans, clip indices supplied; scale_in, thr_grid
+// and thr_idx may be NULL.  Arguments must have been checked.
+windq_status launch_apply_stream(windq_ctx* ctx, int G, const void* W, int64_t R, int64_t C, int64_t ldw, const float* s,
+                                 const float* clip_grid, int K, const uint8_t* clip_idx, const void* scale_in,
+                                 const float* thr_grid, int thr_K, const uint8_t* thr_idx, const windq_plan_out* plans,
+                                 int n_plans, cudaStream_t st);
 
 // Bytes of one packed group under an action (host and device).
 __host__ __device__ inline int group_code_bytes(int action, int G) {

@@ -59,6 +59,8 @@ def parse_args():
     ap.add_argument("--separate-fits", action="store_true",
                     help="one windq_unit_features and one windq_fit_eval call per matrix instead of one batched call of each per "
                          "block and chunk width")
+    ap.add_argument("--separate-plans", action="store_true",
+                    help="one windq_apply_plan call per plan instead of one windq_apply_plan_multi call per matrix")
     ap.add_argument("--extras", action="store_true",
                     help="also time the calls beyond the five of a step (protection, refinement, allocator) on block 0")
     return ap.parse_args()
@@ -214,6 +216,7 @@ class Buffers:
         self.unit_cb = torch.empty(maxU, dtype=torch.int64, device=dev)
         self.offsets = torch.empty(maxU + 1, dtype=torch.int64, device=dev)
         self.wq = torch.empty(maxRC, dtype=torch.float16, device=dev)
+        self.wq_multi = [self.wq] + [torch.empty(maxRC, dtype=torch.float16, device=dev) for _ in TARGET_BITS[1:]]
         shapes = dict(feat=(maxU * 8, torch.float32), err=(maxU * 6, torch.float32), energy=(maxU, torch.float32),
                       totals=(2 * len(TARGET_BITS), torch.int64), codes=(2 * maxRC + 16 * maxU, torch.uint8),
                       scales=(maxUR, torch.float16), zeros=(maxUR, torch.float16))
@@ -268,6 +271,12 @@ class FitTimer:
 
 
 BATCH_FITS = True      # one windq_fit_eval_batch call per block and chunk width (False: one windq_fit_eval per matrix)
+MULTI_APPLY = True     # the plans of a matrix packed by one windq_apply_plan_multi call (False: one windq_apply_plan per plan)
+
+
+def jobs_slot(buf, name, ti):
+    """Ring slot that plan ti of the matrix just packed wrote `name` into (the last len(TARGET_BITS) slots handed out)."""
+    return (buf.turn[name] - len(TARGET_BITS) + ti) % buf.ring
 
 
 def apply_plans(wq, ctx, spec, m, mi, W, s, G, clip_idx, plans_b, buf, grid_d, sink, accounted=None):
@@ -275,6 +284,21 @@ def apply_plans(wq, ctx, spec, m, mi, W, s, G, clip_idx, plans_b, buf, grid_d, s
     it already), then packing.  Returns the number of kernels launched."""
     U, launches = m.C // G, 0
     totals = accounted[0] if accounted else buf.take("totals")
+    if accounted and MULTI_APPLY:
+        # one pass over the matrix for all plans (windq_apply_plan_multi): every weight is read once
+        jobs = []
+        for ti, target in enumerate(TARGET_BITS):
+            jobs.append(dict(actions=plans_b[target][mi], code_offsets=accounted[1][ti], codes=buf.take("codes"),
+                             scales=buf.take("scales")[:U * m.R].view(U, m.R), zeros=buf.take("zeros")[:U * m.R].view(U, m.R),
+                             wq=buf.wq_multi[ti][:m.R * m.C].view(m.R, m.C)))
+        outs = wq.windq_apply_plan_multi(ctx, W, G, s, grid_d, clip_idx, jobs)
+        if sink:
+            for ti, target in enumerate(TARGET_BITS):
+                sink("codes", (outs[ti]["codes"], plans_b[target][mi], m.R, G), slot=jobs_slot(buf, "codes", ti))
+                sink("scales", outs[ti]["scales"], slot=jobs_slot(buf, "scales", ti))
+                sink("zeros", outs[ti]["zeros"], slot=jobs_slot(buf, "zeros", ti))
+            sink("totals%d" % mi, totals)
+        return 1
     for ti, target in enumerate(TARGET_BITS):
         acts = plans_b[target][mi]
         if accounted:
@@ -428,7 +452,7 @@ def run_e2e_leg(wq, ctx, spec, model, plans, plans_np, buf, grid_d, steps, warmu
 
     d2h = [0]
 
-    def sink(name, t):
+    def sink(name, t, slot=None):
         if name == "codes":
             codes, acts, R, G = t
             src = codes[:sink.code_bytes[(id(acts))]]
@@ -441,7 +465,8 @@ def run_e2e_leg(wq, ctx, spec, model, plans, plans_np, buf, grid_d, steps, warmu
             host_buf(name, src.numel(), src.dtype).copy_(src, non_blocking=True)
             copied = torch.cuda.Event()
             copied.record(out_stream)
-        buf.pending[(name, buf.last[name])] = copied      # the call that writes this slot next waits for the copy
+        # the call that writes this slot next waits for the copy
+        buf.pending[(name, buf.last[name] if slot is None else slot)] = copied
         d2h[0] += src.numel() * src.element_size()
 
     sink.code_bytes = {}
@@ -622,7 +647,7 @@ def reference_main(args, spec):
 
 
 def main():
-    global APPLY_G, BATCH_FITS
+    global APPLY_G, BATCH_FITS, MULTI_APPLY
     args = parse_args()
     spec = ws.CONFIGS[args.workload]
     if APPLY_G not in spec.chunk_widths:
@@ -630,6 +655,7 @@ def main():
     if args.impl == "reference":
         return reference_main(args, spec)
     BATCH_FITS = not args.separate_fits
+    MULTI_APPLY = BATCH_FITS and not args.separate_plans
 
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -656,7 +682,7 @@ def main():
     # weak scaling: rank r scores its own replica (global blocks r*n_blocks ...)
     blocks = sharding.block_range(n_blocks * world, rank, world)
     model = DeviceModel(spec, blocks, SEED)
-    buf = Buffers(spec)
+    buf = Buffers(spec, ring=len(TARGET_BITS) if MULTI_APPLY else 1)      # the plans of a matrix are packed together: an output set each
     grid_d = torch.from_numpy(ws.clip_grid(spec.K)).cuda()
     plans = make_plans(wq, ctx, spec, n_blocks, APPLY_G) if APPLY_G in spec.chunk_widths else {}
     plans_np = {t: [[a.cpu().numpy() for a in row] for row in plans[t]] for t in plans}
@@ -732,6 +758,8 @@ def main():
                                 tokens=spec.T, weights=spec.dist, parallelism="replica per GPU",
                                 fits="one windq_unit_features_batch and one windq_fit_eval_batch call per block and chunk width" if BATCH_FITS
                                 else "one windq_unit_features and one windq_fit_eval call per matrix",
+                                plans="the %d plans of a matrix packed by one windq_apply_plan_multi call" % len(TARGET_BITS) if MULTI_APPLY
+                                else "one windq_apply_plan call per matrix and plan",
                                 l2="every step streams %.1f GB of inputs, far above the 126 MB L2" % (
                                     (2 * elems + 2 * spec.T * sum(c for _, c in inputs_of(spec)) * n_blocks) / 1e9)),
                     clocks=clocks, e2e=e2e, gpu_launches=launches, roofline=roofline, cpu_baseline=cpu,

@@ -73,6 +73,12 @@ void windq_destroy(windq_ctx* ctx);
  * is NULL).  The string is owned by the library and stays valid until the next call. */
 const char* windq_last_error(const windq_ctx* ctx);
 
+/* Checks, on the device, an arithmetic shortcut the fits rely on: the reciprocal of a stored scale is formed by
+ * the hardware approximation and one Newton step instead of a full IEEE division; for every positive finite fp16
+ * value (all a stored scale can be) the two must agree bit for bit.  n_failures_out (i64 [1], device) receives
+ * the number of values for which they do not: 0 on every GPU this library supports. */
+windq_status windq_selfcheck(windq_ctx* ctx, int64_t* n_failures_out, void* stream);
+
 /* Grows the context's scratch buffer to at least `bytes` now (synchronises the device), so that
  * later calls do not allocate.  windq_scratch_bytes_* tell how much a call will need. */
 windq_status windq_reserve(windq_ctx* ctx, int64_t bytes);

@@ -46,6 +46,7 @@ def _load() -> ctypes.CDLL:
     lib.windq_last_error.argtypes = [vp]
     lib.windq_last_error.restype = ctypes.c_char_p
     lib.windq_reserve.argtypes = [vp, i64]
+    lib.windq_selfcheck.argtypes = [vp, vp, vp]
     for name in ("windq_scratch_bytes_act_stats",):
         getattr(lib, name).argtypes = [i64, i64]
         getattr(lib, name).restype = i64
@@ -161,6 +162,13 @@ def windq_create(device: int | None = None) -> Context:
 
 def windq_destroy(ctx: Context) -> None:
     ctx.close()
+
+
+def windq_selfcheck(ctx: Context, stream=None) -> int:
+    """Number of fp16 scale values for which the fits' fast reciprocal differs from IEEE division (0 is expected)."""
+    out = torch.zeros(1, dtype=torch.int64, device=torch.device("cuda", ctx.device))
+    ctx._check(_lib.windq_selfcheck(ctx._h, _ptr(out), _stream(stream)))
+    return int(out.item())
 
 
 def windq_reserve(ctx: Context, nbytes: int) -> None:

@@ -2,10 +2,18 @@
 #include <stdarg.h>
 #include <string.h>
 
-#include "windq_internal.cuh"
+#include "fit_device.cuh"
 
 namespace {
 thread_local char g_create_error[256] = "";
+
+// Every positive finite fp16 value: the fast reciprocal of the fits against IEEE division.
+__global__ void selfcheck_reciprocal_kernel(unsigned long long* n_bad) {
+  const int h = blockIdx.x * blockDim.x + threadIdx.x;
+  if (h < 1 || h >= 0x7c00) return;
+  const float x = __half2float(__ushort_as_half((unsigned short)h));
+  if (windq::reciprocal_of_half_value(x) != __fdiv_rn(1.0f, x)) atomicAdd(n_bad, 1ull);
+}
 }
 
 namespace windq {
@@ -102,6 +110,19 @@ void windq_destroy(windq_ctx* ctx) {
 }
 
 const char* windq_last_error(const windq_ctx* ctx) { return ctx ? ctx->err : g_create_error; }
+
+windq_status windq_selfcheck(windq_ctx* ctx, int64_t* n_failures_out, void* stream) {
+  using namespace windq;
+  if (!ctx) return fail(nullptr, WINDQ_ERR_NULL, "windq_selfcheck: ctx is NULL");
+  WINDQ_REQUIRE(ctx, n_failures_out, WINDQ_ERR_NULL, "windq_selfcheck: n_failures_out is NULL");
+  WINDQ_REQUIRE(ctx, ((uintptr_t)n_failures_out & 7) == 0, WINDQ_ERR_ALIGN, "windq_selfcheck: n_failures_out is misaligned");
+  DeviceGuard guard(ctx->device);
+  cudaStream_t st = (cudaStream_t)stream;
+  WINDQ_CUDA(ctx, cudaMemsetAsync(n_failures_out, 0, sizeof(int64_t), st));
+  selfcheck_reciprocal_kernel<<<0x7c00 / 256, 256, 0, st>>>((unsigned long long*)n_failures_out);
+  WINDQ_CUDA(ctx, cudaGetLastError());
+  return WINDQ_OK;
+}
 
 windq_status windq_reserve(windq_ctx* ctx, int64_t bytes) {
   if (!ctx) return windq::fail(nullptr, WINDQ_ERR_NULL, "windq_reserve: ctx is NULL");

@@ -158,22 +158,38 @@ __device__ __forceinline__ UniformSpec uniform_spec(int bi) {  // bi: 0..3 = 8, 
   }
 }
 
-// scale (value of the stored fp16 scale, 1 if that is zero) and zero point (float integer).
-__device__ __forceinline__ void uniform_scale_zero(float mn, float rng, float p, UniformSpec us, float& scale,
+// 1 / x, correctly rounded, for x the value of a positive finite fp16 number (a stored scale, or the 1 that
+// stands in for a scale of zero): the hardware approximation followed by one Newton step in fused arithmetic.
+// For these 31,743 inputs the result equals IEEE division bit for bit (windq_selfcheck tests every one of them
+// on the device); the general-purpose correctly rounded reciprocal costs about three times the instructions,
+// and a fit forms one per candidate.
+__device__ __forceinline__ float reciprocal_of_half_value(float x) {
+  float r0;
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r0) : "f"(x));
+  return __fmaf_rn(r0, __fmaf_rn(-x, r0, 1.0f), r0);
+}
+
+// scale (value of the stored fp16 scale, 1 if that is zero), its reciprocal, and the zero point (float integer).
+__device__ __forceinline__ void uniform_scale_zero(float mn, float rng, float p, UniformSpec us, float& scale, float& inv,
                                                    float& zf) {
   const float scale32 = __fmul_rn(__fmul_rn(p, rng), us.rq);
   scale = __half2float(__float2half_rn(scale32));
   if (scale == 0.0f) scale = 1.0f;
-  const float inv = __frcp_rn(scale);
-  float z = rintf(__fmul_rn(fabsf(__fmul_rn(p, mn)), inv));
+  inv = reciprocal_of_half_value(scale);
+  // nearest-even integer of |p mn| / scale, which is at most about 1.5 qmax: adding and subtracting 1.5 * 2^23
+  // rounds exactly like rint
+  const float z = __fadd_rn(__fadd_rn(__fmul_rn(fabsf(__fmul_rn(p, mn)), inv), kMagic), -kMagic);
   zf = fminf(fmaxf(z, 0.0f), us.qmax);
+}
+__device__ __forceinline__ void uniform_scale_zero(float mn, float rng, float p, UniformSpec us, float& scale, float& zf) {
+  float inv;
+  uniform_scale_zero(mn, rng, p, us, scale, inv, zf);
 }
 
 __device__ __forceinline__ Cand make_cand(float mn, float rng, float p, UniformSpec us) {
   float scale, zf;
-  uniform_scale_zero(mn, rng, p, us, scale, zf);
   Cand c;
-  c.inv = __frcp_rn(scale);
+  uniform_scale_zero(mn, rng, p, us, scale, c.inv, zf);
   c.nscale = -scale;
   c.lo = __fsub_rn(0.0f, zf);
   c.hi = __fsub_rn(us.qmax, zf);
@@ -254,9 +270,10 @@ struct LowBitFit {
   float energy;   // sum_j s_j w_j^2 of the group (any order; tolerance output)
 };
 
-// Must be called by all 32 lanes.
+// Must be called by all 32 lanes.  exact_errors = false: err_t and err_b are wanted only for the unit sums (which
+// are tolerance outputs); they are then taken from the sums already formed instead of a pass of their own.
 template <int G>
-__device__ __forceinline__ LowBitFit fit_low_bits(const Lane32& w, const Lane32& s) {
+__device__ __forceinline__ LowBitFit fit_low_bits(const Lane32& w, const Lane32& s, bool exact_errors) {
   LowBitFit f;
   float A[4], Sb[4], Bb[4], En[4];
 #pragma unroll
@@ -297,6 +314,7 @@ __device__ __forceinline__ LowBitFit fit_low_bits(const Lane32& w, const Lane32&
   }
   float sumBt = group_tree<G>(Bt[0], Bt[1], Bt[2], Bt[3]);
   float sumCt = group_tree<G>(Ct[0], Ct[1], Ct[2], Ct[3]);
+  const float wBt = sumBt, wCt = sumCt;  // the weighted sums, whatever the scale is taken from
   // delta < max |w| whenever some w is not zero (0.7 * mean <= 0.7 * max, roundings included), so
   // the support is empty exactly when every |w| is zero, i.e. when their sum is
   const bool nonempty = sumA > 0.0f;
@@ -320,6 +338,23 @@ __device__ __forceinline__ LowBitFit fit_low_bits(const Lane32& w, const Lane32&
   }
   f.alpha_t = nonempty ? __half2float(__float2half_rn(__fdiv_rn(sumBt, sumCt))) : 0.0f;
 
+  if (!exact_errors) {
+    // sum_j s_j (alpha q_j - w_j)^2 = sum s w^2 - 2 alpha sum_I s |w| + alpha^2 sum_I s  over the support I (every
+    // j for the binary fit), in double from the group sums (the weighted support sums, also when the scale came
+    // from the unweighted ones).  The three sums carry binary32 rounding of about 1e-6 of the energy at worst, so
+    // the difference is good to 2e-5 relative as long as the error is at least a sixteenth of the energy -- on
+    // weight-like data it is a fifth or more.  Where a group of the warp falls below that (weights of nearly
+    // equal magnitude, which a one-scale fit reproduces almost exactly), the warp takes the term-by-term pass.
+    const double at = (double)f.alpha_t, ab = (double)f.alpha_b, en = (double)f.energy;
+    const double et = en - 2.0 * at * (double)wBt + at * at * (double)wCt;
+    const double eb = en - 2.0 * ab * (double)sumB + ab * ab * (double)sumS;
+    const bool thin = et < 0.0625 * en || eb < 0.0625 * en;
+    if (!__any_sync(0xffffffffu, thin)) {
+      f.err_t = (float)et;
+      f.err_b = (float)eb;
+      return f;
+    }
+  }
   float Et[4], Eb[4];
 #pragma unroll
   for (int l = 0; l < 4; ++l) {

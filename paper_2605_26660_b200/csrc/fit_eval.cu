@@ -152,7 +152,8 @@ fit_eval_kernel(const __half* __restrict__ W_one, int R_one, int U_one, int64_t 
       }
     }
     if (!PARTS || (parts & 0x10u)) {
-      const LowBitFit low = fit_low_bits<G>(wv, sv);
+      // group errors wanted: the term-by-term sums (bit-defined); unit sums only: from the sums of the fit
+      const LowBitFit low = fit_low_bits<G>(wv, sv, group_err_out != nullptr);
       e[4] = low.err_t;
       e[5] = low.err_b;
       e[6] = low.energy;

@@ -155,6 +155,35 @@ def test_fit_eval_config1_single_layer(wq, ctx, oracle):
         assert close(got["err"][u0], want["err"][u0]).all() and close(got["energy"][u0], want["energy"][u0]).all()
 
 
+def test_selfcheck_finds_no_mismatch(wq, ctx):
+    """The fits take 1 / scale by the hardware approximation and one Newton step; for every fp16 value a scale can
+    have that must be the IEEE quotient, which the oracle uses."""
+    assert wq.windq_selfcheck(ctx) == 0
+
+
+def test_unit_errors_without_group_errors(wq, ctx, oracle):
+    """When no group errors are asked for, the 1.58- and 1-bit unit errors come from the sums of the fit instead of
+    a term-by-term pass: tolerance outputs, checked here on ordinary and on degenerate inputs (zero units, constant
+    units, statistics that vanish on part of a unit, statistics of very different sizes)."""
+    G, R = 128, 40
+    W = ws.weights(R, 6 * G, 29, "student_t")
+    W[:, :G] = 0
+    W[:, G:2 * G] = 0.37
+    W[2, 2 * G:3 * G] = -0.0
+    s = oracle.act_stats(ws.activations(64, 6 * G, 30).numpy())
+    s[3 * G:4 * G] = 0
+    s[4 * G:4 * G + 100] = 0
+    s[5 * G] *= 1.0e4
+    grid = ws.clip_grid(20)
+    want = oracle.fit_eval(W.numpy(), G, s, grid, threads=4)
+    got = wq.windq_fit_eval(ctx, W.cuda(), G, torch.from_numpy(s).cuda(), torch.from_numpy(grid).cuda())
+    torch.cuda.synchronize()
+    assert got["group_err"] is None
+    assert (got["clip_idx"].cpu().numpy() == want["clip_idx"]).all()
+    assert close(got["err"].cpu().numpy(), want["err"]).all()
+    assert close(got["energy"].cpu().numpy(), want["energy"]).all()
+
+
 def test_fit_eval_is_reproducible(wq, ctx):
     W = ws.weights(333, 1024, 77, "student_t").cuda()
     s = torch.rand(1024, device="cuda") + 0.1

@@ -49,16 +49,24 @@ SEED = 0
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=3)
+    ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="windq", choices=["windq", "reference"])
     ap.add_argument("--workload", default="cfg3_llama7b_model", choices=sorted(ws.CONFIGS))
-    ap.add_argument("--blocks", type=int, default=0, help="use only the first B blocks (0 = all; profiling aid)")
+    ap.add_argument("--blocks", type=int, default=0, help="score only the first B blocks of the model (0 = all)")
+    ap.add_argument("--scaling", default="weak", choices=["weak", "strong"],
+                    help="with N > 1 ranks: weak = a replica of the model per rank; strong = the blocks of ONE model split over the ranks")
+    ap.add_argument("--stream", default="auto", choices=["auto", "yes", "no"],
+                    help="keep two blocks on the device and refill them block by block instead of holding the model resident "
+                         "(auto: when the model does not fit in half of the free device memory)")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--separate-fits", action="store_true",
                     help="one windq_unit_features and one windq_fit_eval call per matrix instead of one batched call of each per "
                          "block and chunk width")
+    ap.add_argument("--fused-features", action="store_true",
+                    help="features and fits of a block by one windq_features_fit_batch call (one pass over the weights; "
+                         "measured slower than the two batched calls, kept for comparison)")
     ap.add_argument("--separate-plans", action="store_true",
                     help="one windq_apply_plan call per plan instead of one windq_apply_plan_multi call per matrix")
     ap.add_argument("--extras", action="store_true",
@@ -154,15 +162,34 @@ def fit_ops_per_element(K):
 
 
 class DeviceModel:
-    """Weights and calibration inputs of this rank's blocks, resident in HBM."""
+    """Weights and calibration inputs of this rank's blocks in HBM: all of them resident, or -- streamed -- two block
+    slots that are refilled block by block (the synthetic block is regenerated on the device from its seed, which
+    stands for the layer-by-layer load of a model larger than the GPU's memory; the refill is not part of the timed
+    kernels)."""
 
-    def __init__(self, spec, blocks, seed):
-        self.spec, self.blocks = spec, list(blocks)
+    def __init__(self, spec, blocks, seed, streamed=False):
+        self.spec, self.blocks, self.seed, self.streamed = spec, list(blocks), seed, streamed
         self.W, self.X = [], []
-        for b in self.blocks:
+        self.slot_block = [None, None]
+        for b in (self.blocks[:2] if streamed else self.blocks):
             self.W.append([ws.block_weight(spec, seed, b, m, device="cuda") for m in matrices_of(spec)])
             self.X.append({i: ws.block_input(spec, seed, b, i, device="cuda") for i, _ in inputs_of(spec)})
+        if streamed:
+            self.slot_block = list(self.blocks[:2]) + [None] * (2 - len(self.blocks[:2]))
         torch.cuda.synchronize()
+
+    def block(self, bi):
+        """(weights, inputs) of this rank's bi-th block; a streamed model regenerates it into slot bi % 2 first."""
+        if not self.streamed:
+            return self.W[bi], self.X[bi]
+        slot, b = bi % 2, self.blocks[bi]
+        if self.slot_block[slot] != b:
+            for dst, m in zip(self.W[slot], matrices_of(self.spec)):
+                dst.copy_(ws.block_weight(self.spec, self.seed, b, m, device="cuda"))
+            for i in self.X[slot]:
+                self.X[slot][i].copy_(ws.block_input(self.spec, self.seed, b, i, device="cuda"))
+            self.slot_block[slot] = b
+        return self.W[slot], self.X[slot]
 
 
 def make_plans(wq, ctx, spec, n_blocks, G):
@@ -272,6 +299,7 @@ class FitTimer:
 
 BATCH_FITS = True      # one windq_fit_eval_batch call per block and chunk width (False: one windq_fit_eval per matrix)
 MULTI_APPLY = True     # the plans of a matrix packed by one windq_apply_plan_multi call (False: one windq_apply_plan per plan)
+FUSED_FEATURES = False # features and fits of a block by one windq_features_fit_batch call
 
 
 def jobs_slot(buf, name, ti):
@@ -334,20 +362,25 @@ def score_block(wq, ctx, spec, Wb, Xb, plans_b, buf, grid_d, timer=None, sink=No
         for G in spec.chunk_widths:
             stats = [buf.s[m.x_id] for m in mats]
             feats = [buf.take("feat%d" % mi)[:(m.C // G) * 8].view(m.C // G, 8) for mi, m in enumerate(mats)]
-            wq.windq_unit_features_batch(ctx, Wb, G, stats, feats)
-            launches += 2
-            if sink:
-                for mi in range(len(mats)):
-                    sink("feat%d" % mi, feats[mi])
+            if not FUSED_FEATURES:
+                wq.windq_unit_features_batch(ctx, Wb, G, stats, feats)
+                launches += 2
             outs = [dict(err=buf.take("err%d" % mi)[:(m.C // G) * 6].view(m.C // G, 6),
                          energy=buf.take("energy%d" % mi)[:m.C // G],
                          clip_idx=buf.clip_idx_m[mi][:4 * (m.C // G) * m.R].view(4, m.C // G, m.R))
                     for mi, m in enumerate(mats)]
             e0 = timer.start() if timer else None
-            wq.windq_fit_eval_batch(ctx, Wb, G, stats, grid_d, outs=outs)
+            if FUSED_FEATURES:
+                wq.windq_features_fit_batch(ctx, Wb, G, stats, grid_d, feats=feats, outs=outs)
+                launches += 1
+            else:
+                wq.windq_fit_eval_batch(ctx, Wb, G, stats, grid_d, outs=outs)
             if timer:
                 timer.stop(e0)
             launches += 2
+            if sink:
+                for mi in range(len(mats)):
+                    sink("feat%d" % mi, feats[mi])
             if sink:
                 for mi in range(len(mats)):
                     sink("err%d" % mi, outs[mi]["err"])
@@ -396,11 +429,24 @@ def packed_code_bytes(actions_np, R, G):
 
 
 # ---------------------------------------------------------------------------------------- legs
-def run_device_leg(wq, ctx, spec, model, plans, buf, grid_d, steps, warmup, rank, sync):
-    def step(timer=None):
+def run_device_leg(wq, ctx, spec, model, plans, plan_index, buf, grid_d, steps, warmup, rank, sync):
+    """Times `steps` steps with everything the kernels read resident in HBM.  A resident model is timed by one pair of
+    events around all steps; a streamed one by a pair of events around every block's kernels (the refill of the block
+    slots in between is not counted), summed."""
+    block_pairs = []
+
+    def step(timer=None, timed=False):
         n = 0
         for bi in range(len(model.blocks)):
-            n += score_block(wq, ctx, spec, model.W[bi], model.X[bi], {t: plans[t][bi] for t in plans}, buf, grid_d, timer)
+            Wb, Xb = model.block(bi)
+            if timed and model.streamed:
+                e0 = torch.cuda.Event(enable_timing=True)
+                e0.record()
+            n += score_block(wq, ctx, spec, Wb, Xb, {t: plans[t][plan_index[bi]] for t in plans}, buf, grid_d, timer)
+            if timed and model.streamed:
+                e1 = torch.cuda.Event(enable_timing=True)
+                e1.record()
+                block_pairs.append((e0, e1))
         return n
 
     for _ in range(warmup):
@@ -413,26 +459,29 @@ def run_device_leg(wq, ctx, spec, model, plans, buf, grid_d, steps, warmup, rank
         t0.record()
         launches = 0
         for _ in range(steps):
-            launches += step(timer)
+            launches += step(timer, timed=True)
         t1.record()
         sync()
-    ms = t0.elapsed_time(t1)
+    ms = sum(a.elapsed_time(b) for a, b in block_pairs) if model.streamed else t0.elapsed_time(t1)
     return ms, launches, timer.total_ms(), clocks.summary()
 
 
-def run_e2e_leg(wq, ctx, spec, model, plans, plans_np, buf, grid_d, steps, warmup, sync):
+def run_e2e_leg(wq, ctx, spec, model, plans, plan_index, plans_np, buf, grid_d, steps, warmup, sync):
     """Same step from pinned host memory: two device-side block slots, copies on a second stream
-    overlapped with the previous block's kernels; every result copied back to pinned host memory."""
+    overlapped with the previous block's kernels; every result copied back to pinned host memory.
+    As many distinct blocks as a third of the free host memory holds (at most 24 for a streamed model) are kept in
+    pinned memory and used in turn: every step still copies every block's bytes from the host."""
     mats = matrices_of(spec)
     nb = len(model.blocks)
     need = sum(m.R * m.C for m in mats) * 2 + sum(spec.T * c for _, c in inputs_of(spec)) * 2
     import psutil
     avail = psutil.virtual_memory().available
-    host_blocks = nb if need * nb * 3 < avail else 1
+    host_blocks = max(1, min(nb, int(avail // (3 * need)), 24 if model.streamed else nb))
     hostW, hostX = [], []
     for bi in range(host_blocks):
-        hostW.append([w.cpu().pin_memory() for w in model.W[bi]])
-        hostX.append({i: x.cpu().pin_memory() for i, x in model.X[bi].items()})
+        Wb, Xb = model.block(bi)
+        hostW.append([w.cpu().pin_memory() for w in Wb])
+        hostX.append({i: x.cpu().pin_memory() for i, x in Xb.items()})
     slots = []
     for _ in range(2):
         slots.append(dict(W=[torch.empty_like(w) for w in model.W[0]], X={i: torch.empty_like(x) for i, x in model.X[0].items()},
@@ -471,7 +520,7 @@ def run_e2e_leg(wq, ctx, spec, model, plans, plans_np, buf, grid_d, steps, warmu
 
     sink.code_bytes = {}
     for target in plans:
-        for bi in range(nb):
+        for bi in range(len(plans[target])):
             for mi, m in enumerate(mats):
                 sink.code_bytes[id(plans[target][bi][mi])] = packed_code_bytes(plans_np[target][bi][mi], m.R, APPLY_G)
     # make sure the largest pinned result buffers exist before timing
@@ -492,7 +541,7 @@ def run_e2e_leg(wq, ctx, spec, model, plans, plans_np, buf, grid_d, steps, warmu
                     slot["X"][i].copy_(hostX[hb][i], non_blocking=True)
                 slot["ready"].record(copy_stream)
             main.wait_event(slot["ready"])
-            n += score_block(wq, ctx, spec, slot["W"], slot["X"], {t: plans[t][bi] for t in plans}, buf, grid_d, None, sink)
+            n += score_block(wq, ctx, spec, slot["W"], slot["X"], {t: plans[t][plan_index[bi]] for t in plans}, buf, grid_d, None, sink)
             slot["free"].record(main)
         return n
 
@@ -580,31 +629,36 @@ def run_extras(wq, ctx, spec, model, buf, grid_d, reps=3):
     return out
 
 
-def oracle_sample(spec, seed, threads):
-    """The CPU oracle on a bounded sample of the workload: the whole hot path for the first
-    ORACLE_SAMPLE_MATRICES matrices of block 0 -- their calibration statistics, and per matrix
-    unit_features + fit_eval at every chunk width and the three plans at APPLY_G.
+def oracle_sample(spec, seed, threads, n_matrices=ORACLE_SAMPLE_MATRICES):
+    """The CPU oracle on a bounded sample of the workload: the whole hot path for the first n_matrices matrices of
+    block 0 -- their calibration statistics, and per matrix unit_features + fit_eval at every chunk width and the
+    three plans at APPLY_G.  With threads > 1 every call runs the oracle's single-threaded routine over disjoint
+    unit (or channel) ranges on that many threads; the routine itself is never changed for this.
     Returns (seconds, unit x bit-width evaluations, description)."""
     import oracle
-    mats = matrices_of(spec)[:ORACLE_SAMPLE_MATRICES]
+    mats = matrices_of(spec)[:n_matrices]
     Ws = [ws.block_weight(spec, seed, 0, m).numpy() for m in mats]
     Xs = {i: ws.block_input(spec, seed, 0, i).numpy() for i in sorted({m.x_id for m in mats})}
     grid = ws.clip_grid(spec.K)
     rng = np.random.default_rng(seed)
     t0 = time.perf_counter()
-    stats = {i: oracle.act_stats(X) for i, X in Xs.items()}
+    stats = {i: _over_ranges(threads, X.shape[1], lambda a, b, X=X: oracle.act_stats(np.ascontiguousarray(X[:, a:b])), np.concatenate)
+             for i, X in Xs.items()}
     evals = 0
     for m, W in zip(mats, Ws):
         s = stats[m.x_id]
         for G in spec.chunk_widths:
-            oracle.unit_features(W, G, s) if threads <= 1 else _parallel_features(oracle, W, G, s, threads)
+            U = m.C // G
+            _over_ranges(threads, U, lambda a, b: oracle.unit_features(np.ascontiguousarray(W[:, a * G:b * G]), G, s[a * G:b * G]))
             fit = oracle.fit_eval(W, G, s, grid, threads=threads, want_group_err=False)
-            evals += 6 * (m.C // G)
+            evals += 6 * U
             if G == APPLY_G:
                 for ti, _ in enumerate(TARGET_BITS):
-                    acts = rng.choice(7, size=m.C // G, p=np.array(ws.ACTION_MIX) / sum(ws.ACTION_MIX)).astype(np.uint8)
+                    acts = rng.choice(7, size=U, p=np.array(ws.ACTION_MIX) / sum(ws.ACTION_MIX)).astype(np.uint8)
                     oracle.effective_bits(acts, m.R, G)
-                    oracle.apply_plan(W, G, s, grid, acts, fit["clip_idx"])
+                    _over_ranges(threads, U, lambda a, b: oracle.apply_plan(
+                        np.ascontiguousarray(W[:, a * G:b * G]), G, s[a * G:b * G], grid, acts[a:b],
+                        np.ascontiguousarray(fit["clip_idx"][:, a:b])))
     dt = time.perf_counter() - t0
     desc = "block 0 of %d, matrices %s (%.1f M weights), T=%d: act_stats, unit_features + fit_eval at G=%s, 3 plans applied at G=%d" % (
         spec.n_blocks, "/".join(m.name for m in mats), sum(m.R * m.C for m in mats) / 1e6, spec.T,
@@ -612,17 +666,25 @@ def oracle_sample(spec, seed, threads):
     return dt, evals, desc
 
 
-def _parallel_features(oracle, W, G, s, threads):
+def _over_ranges(threads, n, fn, combine=None):
+    """fn(a, b) over disjoint ranges of [0, n) on `threads` threads (one call when threads <= 1)."""
+    if threads <= 1 or n <= 1:
+        return fn(0, n)
     from concurrent.futures import ThreadPoolExecutor
-    U = W.shape[1] // G
-    bounds = np.linspace(0, U, min(threads, U) + 1).astype(int)
-
-    def run(ab):
-        a, b = ab
-        if b > a:
-            oracle.unit_features(np.ascontiguousarray(W[:, a * G:b * G]), G, s[a * G:b * G])
+    bounds = np.linspace(0, n, min(threads, n) + 1).astype(int)
     with ThreadPoolExecutor(max_workers=threads) as ex:
-        list(ex.map(run, zip(bounds[:-1], bounds[1:])))
+        parts = list(ex.map(lambda ab: fn(int(ab[0]), int(ab[1])), [ab for ab in zip(bounds[:-1], bounds[1:]) if ab[1] > ab[0]]))
+    return combine(parts) if combine else None
+
+
+def cpu_baseline(spec, seed):
+    """The oracle, as it stands, on this machine's host cores: on all of them over the five-matrix sample, and on ONE core
+    over the first matrix of the sample."""
+    threads = os.cpu_count() or 1
+    dt, ev, desc = oracle_sample(spec, seed, threads)
+    dt1, ev1, desc1 = oracle_sample(spec, seed, 1, n_matrices=1)
+    return dict(value=ev / dt, unit=UNIT, cores=threads, kind="oracle", sample=desc, seconds=dt,
+                one_core=dict(value=ev1 / dt1, unit=UNIT, cores=1, sample=desc1, seconds=dt1))
 
 
 def reference_main(args, spec):
@@ -647,7 +709,7 @@ def reference_main(args, spec):
 
 
 def main():
-    global APPLY_G, BATCH_FITS, MULTI_APPLY
+    global APPLY_G, BATCH_FITS, MULTI_APPLY, FUSED_FEATURES
     args = parse_args()
     spec = ws.CONFIGS[args.workload]
     if APPLY_G not in spec.chunk_widths:
@@ -656,6 +718,7 @@ def main():
         return reference_main(args, spec)
     BATCH_FITS = not args.separate_fits
     MULTI_APPLY = BATCH_FITS and not args.separate_plans
+    FUSED_FEATURES = BATCH_FITS and args.fused_features
 
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -679,9 +742,19 @@ def main():
     peaks = load_peaks()
     ctx = wq.windq_create(local_rank)
     n_blocks = args.blocks if args.blocks > 0 else spec.n_blocks
-    # weak scaling: rank r scores its own replica (global blocks r*n_blocks ...)
-    blocks = sharding.block_range(n_blocks * world, rank, world)
-    model = DeviceModel(spec, blocks, SEED)
+    strong = args.scaling == "strong" and world > 1
+    if strong:
+        # the blocks of ONE model split over the ranks; block b keeps its plans
+        blocks = sharding.block_range(n_blocks, rank, world)
+        plan_index = list(blocks)
+    else:
+        # weak scaling: rank r scores its own replica (global blocks r * n_blocks ...), every replica under the same plans
+        blocks = sharding.block_range(n_blocks * world, rank, world)
+        plan_index = list(range(n_blocks))
+    block_bytes = 2 * sum(m.R * m.C for m in matrices_of(spec)) + 2 * spec.T * sum(c for _, c in inputs_of(spec))
+    free_bytes = torch.cuda.mem_get_info(local_rank)[0]
+    streamed = args.stream == "yes" or (args.stream == "auto" and block_bytes * len(blocks) > 0.5 * free_bytes)
+    model = DeviceModel(spec, blocks, SEED, streamed=streamed)
     buf = Buffers(spec, ring=len(TARGET_BITS) if MULTI_APPLY else 1)      # the plans of a matrix are packed together: an output set each
     grid_d = torch.from_numpy(ws.clip_grid(spec.K)).cuda()
     plans = make_plans(wq, ctx, spec, n_blocks, APPLY_G) if APPLY_G in spec.chunk_widths else {}
@@ -692,20 +765,25 @@ def main():
     if BATCH_FITS:
         scratch = max(scratch, max(sum(wq.windq_scratch_bytes_fit_eval(m.R, m.C, G) for m in mats) for G in spec.chunk_widths),
                       2 * max(sum(wq.windq_scratch_bytes_unit_features(m.R, m.C, G) for m in mats) for G in spec.chunk_widths))
+    if FUSED_FEATURES:
+        scratch = max(scratch, wq.windq_scratch_bytes_features_fit_batch(model.W[0], min(spec.chunk_widths)))
     wq.windq_reserve(ctx, scratch)
 
-    elems, units = workload_counts(spec, n_blocks)
+    elems, units = workload_counts(spec, n_blocks)                  # of one model
     evals_per_step = 6 * sum(units.values())
-    ms, launches, fit_ms, clocks = run_device_leg(wq, ctx, spec, model, plans, buf, grid_d, args.steps, args.warmup, local_rank, sync)
+    job_evals = evals_per_step if strong else world * evals_per_step   # what all ranks together score in a step
+    elems_rank, _ = workload_counts(spec, len(blocks))               # what this rank's fits read
+    ms, launches, fit_ms, clocks = run_device_leg(wq, ctx, spec, model, plans, plan_index, buf, grid_d, args.steps, args.warmup,
+                                                  local_rank, sync)
     ms = sharding.max_float(ms)
-    value = world * evals_per_step * args.steps / (ms * 1e-3)
+    value = job_evals * args.steps / (ms * 1e-3)
 
     # plan totals (control path): exact int64 sums over ranks
     total_cb = sharding.sum_int64(int(buf.totals[2 * (len(TARGET_BITS) - 1)].item())) if plans else 0
     torch.cuda.synchronize()
 
-    n_fit = len(spec.chunk_widths) * (1 if BATCH_FITS else len(mats)) * n_blocks * args.steps
-    fit_elem = elems * len(spec.chunk_widths) * args.steps
+    n_fit = max(1, len(spec.chunk_widths) * (1 if BATCH_FITS else len(mats)) * len(blocks) * args.steps)
+    fit_elem = elems_rank * len(spec.chunk_widths) * args.steps
     ops = fit_ops_per_element(spec.K)
     sm_count = torch.cuda.get_device_properties(local_rank).multi_processor_count
     alu_peak = sm_count * 128 * peaks["sm_max_mhz"] * 1e6 / 1e12          # T lane-ops/s, fma = 1
@@ -731,11 +809,11 @@ def main():
         # output slot (and three more), so that packing never waits for a device-to-host copy and the copies of one
         # block overlap the fits of the next
         ebuf = Buffers(spec, ring=3 * len(mats) + 3 if BATCH_FITS else 3)
-        e_ms, e_wall, h2d, d2h, host_blocks = run_e2e_leg(wq, ctx, spec, model, plans, plans_np, ebuf, grid_d,
-                                                          max(1, min(args.steps, 2)), args.warmup, sync)
-        e_steps = max(1, min(args.steps, 2))
+        e_steps = max(1, min(args.steps, 5))
+        e_ms, e_wall, h2d, d2h, host_blocks = run_e2e_leg(wq, ctx, spec, model, plans, plan_index, plans_np, ebuf, grid_d,
+                                                          e_steps, args.warmup, sync)
         e_ms = sharding.max_float(max(e_ms, e_wall))
-        e2e = dict(value=world * evals_per_step * e_steps / (e_ms * 1e-3), unit=UNIT, h2d_bytes_per_step=h2d,
+        e2e = dict(value=job_evals * e_steps / (e_ms * 1e-3), unit=UNIT, h2d_bytes_per_step=h2d,
                    d2h_bytes_per_step=d2h, steps=e_steps, ms_per_step=e_ms / e_steps,
                    host_blocks_resident=host_blocks)
 
@@ -745,18 +823,20 @@ def main():
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        threads = os.cpu_count() or 1
-        dt, ev, desc = oracle_sample(spec, SEED, threads)
-        cpu = dict(value=ev / dt, unit=UNIT, cores=threads, kind="oracle", sample=desc, seconds=dt)
+        cpu = cpu_baseline(spec, SEED)
 
     if rank == 0:
         line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,
-                    ms_per_step=ms / args.steps, higher_is_better=True, scaling="weak", vs_baseline=None, dtype="f32",
-                    data="synthetic",
+                    ms_per_step=ms / args.steps, higher_is_better=True, scaling="strong" if strong else "weak", vs_baseline=None,
+                    dtype="f32", data="synthetic",
                     config=dict(workload=spec.name, blocks=n_blocks, elements_per_chunk_width=elems, units=units, K=spec.K,
                                 chunk_widths=list(spec.chunk_widths), plan_targets=list(TARGET_BITS), apply_chunk_width=APPLY_G,
-                                tokens=spec.T, weights=spec.dist, parallelism="replica per GPU",
-                                fits="one windq_unit_features_batch and one windq_fit_eval_batch call per block and chunk width" if BATCH_FITS
+                                tokens=spec.T, weights=spec.dist,
+                                parallelism="the blocks of one model split over the GPUs" if strong else "replica per GPU",
+                                residency="two block slots refilled block by block (the model does not fit); only the kernels "
+                                          "of a block are timed" if streamed else "all blocks resident in HBM",
+                                fits="one windq_features_fit_batch call per block and chunk width" if FUSED_FEATURES
+                                else "one windq_unit_features_batch and one windq_fit_eval_batch call per block and chunk width" if BATCH_FITS
                                 else "one windq_unit_features and one windq_fit_eval call per matrix",
                                 plans="the %d plans of a matrix packed by one windq_apply_plan_multi call" % len(TARGET_BITS) if MULTI_APPLY
                                 else "one windq_apply_plan call per matrix and plan",

@@ -214,6 +214,32 @@ int64_t windq_scratch_bytes_fit_eval_batch(const windq_fit_job* jobs, int n_jobs
 windq_status windq_fit_eval_batch(windq_ctx* ctx, const windq_fit_job* jobs, int n_jobs, int G, const float* clip_grid,
                                   int K, void* stream);
 
+/* windq_unit_features_batch and windq_fit_eval_batch in ONE pass over the weights (the paper has no counterpart: its
+ * state features, Table 1, and its engine's fits, Sec. 3.5, are computed on the same chunk).  The fit pass holds every
+ * weight in registers anyway; it also counts it in its unit's histogram of |w| bit patterns and adds it to the unit's
+ * sum, so that the features need no second read of the matrix and no pass of their own.  Every job is one
+ * windq_fit_eval call plus one windq_unit_features call on the same W and s: the fit outputs are those of
+ * windq_fit_eval_batch bit for bit, the features those of windq_unit_features (the histogram features and those of s
+ * bit for bit; the mean is a sum of block sums whose blocks fall differently: within 1e-6 relative).
+ * Measured on B200 this call is SLOWER than the two it replaces (5.05 against 4.07 ms for a 7B-shaped block at chunk
+ * width 128): the histogram updates are atomics in global memory, and the fit's own shared-memory loads queue behind
+ * them.  It saves the second read of the weights, which matters only where memory traffic, not time, is the constraint.
+ *   jobs: HOST array of n_jobs descriptors (1 <= n_jobs <= 16), read during the call only.
+ * Scratch: windq_scratch_bytes_features_fit_batch (the fit's partial sums + 128 KB per unit of all jobs). */
+typedef struct {
+  const void* W;          /* fp16 [R][ldw] */
+  int64_t R, C, ldw;
+  const float* s;         /* fp32 [C] */
+  float* feat_out;        /* fp32 [U][8] */
+  float* err_out;         /* fp32 [U][6] */
+  float* energy_out;      /* fp32 [U], nullable */
+  uint8_t* clip_idx_out;  /* u8 [4][U][R], nullable */
+  float* group_err_out;   /* fp32 [6][U][R], nullable */
+} windq_featfit_job;
+int64_t windq_scratch_bytes_features_fit_batch(const windq_featfit_job* jobs, int n_jobs, int G);
+windq_status windq_features_fit_batch(windq_ctx* ctx, const windq_featfit_job* jobs, int n_jobs, int G,
+                                      const float* clip_grid, int K, void* stream);
+
 /* windq_effective_bits for several plans in one launch (plans of different matrices may differ in U and R;
  * G, scale_bits and zero_bits are shared).  Every job is one windq_effective_bits call with the same meanings,
  * nullability and results.  Two jobs must not share an output array.

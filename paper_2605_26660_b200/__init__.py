@@ -63,6 +63,9 @@ def _load() -> ctypes.CDLL:
     lib.windq_scratch_bytes_unit_features_batch.restype = i64
     lib.windq_scratch_bytes_unit_features_batch.argtypes = [vp, i32, i32]
     lib.windq_fit_eval_batch.argtypes = [vp, vp, i32, i32, vp, i32, vp]
+    lib.windq_features_fit_batch.argtypes = [vp, vp, i32, i32, vp, i32, vp]
+    lib.windq_scratch_bytes_features_fit_batch.restype = i64
+    lib.windq_scratch_bytes_features_fit_batch.argtypes = [vp, i32, i32]
     lib.windq_scratch_bytes_fit_eval_batch.restype = i64
     lib.windq_scratch_bytes_fit_eval_batch.argtypes = [vp, i32, i32]
     lib.windq_fit_eval_protected.argtypes = [vp, vp, i64, i64, i64, i32, vp, vp, i32, vp, vp, vp, vp, vp, vp]
@@ -791,3 +794,61 @@ def windq_apply_plan_searched(ctx: Context, W: torch.Tensor, G: int, s: torch.Te
                                               _ptr(code_offsets), _ptr(codes_out), _ptr(out["scales"]), _ptr(out["zeros"]),
                                               _ptr(out["wq"]), _stream(stream)))
     return out
+
+
+class _FeatFitJob(ctypes.Structure):
+    _fields_ = [("W", ctypes.c_void_p), ("R", ctypes.c_int64), ("C", ctypes.c_int64), ("ldw", ctypes.c_int64),
+                ("s", ctypes.c_void_p), ("feat_out", ctypes.c_void_p), ("err_out", ctypes.c_void_p),
+                ("energy_out", ctypes.c_void_p), ("clip_idx_out", ctypes.c_void_p), ("group_err_out", ctypes.c_void_p)]
+
+
+def _featfit_jobs(Ws, G, ss, feats, outs, want_energy, want_clip_idx, want_group_err):
+    jobs = (_FeatFitJob * len(Ws))()
+    results, feat_list = [], []
+    for j, (W, s) in enumerate(zip(Ws, ss)):
+        R, C, ldw = _matrix(W, "W")
+        _need(s, torch.float32, "s", 1)
+        U = C // G if G > 0 else 0
+        out = dict(outs[j]) if outs else {}
+        dev = W.device
+        f = feats[j] if feats is not None else torch.empty((U, N_FEATURES), dtype=torch.float32, device=dev)
+        _need(f, torch.float32, "feat_out", 2)
+        if tuple(f.shape) != (U, N_FEATURES) or not f.is_contiguous():
+            raise ValueError("feat_out must be a contiguous [U, 8] tensor")
+        if out.get("err") is None:
+            out["err"] = torch.empty((U, N_BITWIDTHS), dtype=torch.float32, device=dev)
+        if want_energy and out.get("energy") is None:
+            out["energy"] = torch.empty(U, dtype=torch.float32, device=dev)
+        if want_clip_idx and out.get("clip_idx") is None:
+            out["clip_idx"] = torch.empty((4, U, R), dtype=torch.uint8, device=dev)
+        if want_group_err and out.get("group_err") is None:
+            out["group_err"] = torch.empty((N_BITWIDTHS, U, R), dtype=torch.float32, device=dev)
+        for key in ("energy", "clip_idx", "group_err"):
+            out.setdefault(key, None)
+        ptr = lambda x: None if x is None else x.data_ptr()
+        jobs[j] = _FeatFitJob(W.data_ptr(), R, C, ldw, s.data_ptr(), f.data_ptr(), ptr(out["err"]), ptr(out["energy"]),
+                              ptr(out["clip_idx"]), ptr(out["group_err"]))
+        results.append(out)
+        feat_list.append(f)
+    return jobs, feat_list, results
+
+
+def windq_scratch_bytes_features_fit_batch(Ws, G: int) -> int:
+    jobs = (_FeatFitJob * len(Ws))()
+    for j, W in enumerate(Ws):
+        R, C, ldw = _matrix(W, "W")
+        jobs[j] = _FeatFitJob(W.data_ptr(), R, C, ldw, None, None, None, None, None, None)
+    return int(_lib.windq_scratch_bytes_features_fit_batch(ctypes.cast(jobs, ctypes.c_void_p), len(Ws), int(G)))
+
+
+def windq_features_fit_batch(ctx: Context, Ws, G: int, ss, clip_grid: torch.Tensor, *, feats=None, want_energy: bool = True,
+                             want_clip_idx: bool = True, want_group_err: bool = False, outs=None, stream=None):
+    """windq_unit_features_batch and windq_fit_eval_batch of up to 16 matrices in one pass over the weights.
+    Returns (list of feature tensors, list of fit output dicts)."""
+    if len(Ws) != len(ss) or not Ws:
+        raise ValueError("Ws and ss must be non-empty and equally long")
+    _need(clip_grid, torch.float32, "clip_grid", 1)
+    jobs, feat_list, results = _featfit_jobs(Ws, G, ss, feats, outs, want_energy, want_clip_idx, want_group_err)
+    ctx._check(_lib.windq_features_fit_batch(ctx._h, ctypes.cast(jobs, ctypes.c_void_p), len(Ws), int(G), _ptr(clip_grid),
+                                             clip_grid.numel(), _stream(stream)))
+    return feat_list, results

@@ -45,6 +45,7 @@ struct FitJobs {
   unsigned int first_item[kFitMaxJobs + 1];
   unsigned int first_unit[kFitMaxJobs + 1];
   int n;
+  unsigned int* hist;  // FEAT: one 32768-bin histogram of |w| bit patterns per unit of all jobs, in scratch
 };
 
 // PROTECT: salient weights (key |w| * scale_j >= thresh[u], scale_j = sqrt(s_j)) are taken out of
@@ -55,7 +56,11 @@ struct FitJobs {
 // whole items leave most warps idle at the end (or from the start); the code of the other instantiation is
 // untouched by it.
 // BATCH: the matrix of an item is looked up in `jobs` (the scalar matrix parameters are then unused).
-template <int G, bool PROTECT, bool PARTS, bool BATCH>
+// FEAT (with BATCH): the pass also gathers what the state features of Table 1 need from the weights -- every weight
+// is counted in its unit's histogram of |w| bit patterns (integer atomics in global memory: exact and independent
+// of the order) and the item's signed sum goes to the spare eighth partial -- so that the features cost no second
+// read of the matrix and no pass of their own.
+template <int G, bool PROTECT, bool PARTS, bool BATCH, bool FEAT = false>
 __global__ void __launch_bounds__(kFitWarpsPerBlock * 32, 1)
 fit_eval_kernel(const __half* __restrict__ W_one, int R_one, int U_one, int64_t ldw_one, const float* __restrict__ s_one,
                 const float* __restrict__ clip, int K, double* __restrict__ partial, uint8_t* __restrict__ clip_idx_one,
@@ -91,9 +96,11 @@ fit_eval_kernel(const __half* __restrict__ W_one, int R_one, int U_one, int64_t 
     int R = R_one, U = U_one, rows_blocks = rows_blocks_one;
     int64_t ldw = ldw_one;
     unsigned int local = item;
+    int jfeat = 0;
     if (BATCH) {
       int j = 0;
       while (j + 1 < jobs.n && item >= jobs.first_item[j + 1]) ++j;
+      jfeat = j;
       W = jobs.W[j];
       s = jobs.s[j];
       clip_idx_out = jobs.clip_idx[j];
@@ -110,7 +117,36 @@ fit_eval_kernel(const __half* __restrict__ W_one, int R_one, int U_one, int64_t 
     const bool live = row < R;
     const int row_ld = live ? row : R - 1;  // rows past the end repeat the last row and are not written
     Lane32 wv;
-    load_weights(W + (int64_t)row_ld * ldw + (int64_t)u * G + 32 * q, wv);
+    if (FEAT) {
+      const uint4* p4 = reinterpret_cast<const uint4*>(W + (int64_t)row_ld * ldw + (int64_t)u * G + 32 * q);
+      uint4 raw[4];
+#pragma unroll
+      for (int l = 0; l < 4; ++l) raw[l] = __ldg(p4 + l);
+      unpack_weights(raw, wv);
+      if (!PARTS || (parts & 0x10u)) {
+        // histogram and signed sum of the item's live rows (once per item: with PARTS, in the part of the low-bit fits)
+        unsigned int* h = jobs.hist + (size_t)(jobs.first_unit[jfeat] + u) * 32768u;
+        float part = 0.0f;
+        if (live) {
+          const unsigned int* r = reinterpret_cast<const unsigned int*>(raw);
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            atomicAdd(h + (r[i] & 0x7fffu), 1u);
+            atomicAdd(h + ((r[i] >> 16) & 0x7fffu), 1u);
+          }
+#pragma unroll
+          for (int hh = 0; hh < 2; ++hh)
+#pragma unroll
+            for (int i = 0; i < 8; ++i) part += wv.v[hh][i].x + wv.v[hh][i].y;
+        }
+        double ds = (double)part;
+#pragma unroll
+        for (int m = 16; m > 0; m >>= 1) ds += __shfl_xor_sync(0xffffffffu, ds, m);
+        if (lane == 0) partial[(int64_t)item * kFitPartials + 7] = ds;
+      }
+    } else {
+      load_weights(W + (int64_t)row_ld * ldw + (int64_t)u * G + 32 * q, wv);
+    }
     {
       // Masking step.  PROTECT: a weight whose key |w| * scale_j reaches the unit's threshold becomes a
       // zero weight with zero activation weight.  Otherwise the same step runs against `never`, a NaN
@@ -200,7 +236,7 @@ fit_finalize_kernel(const double* __restrict__ partial, int rows_blocks, float* 
 
 // The same for a batch: block b is unit b - first_unit[j] of job j.
 __global__ void __launch_bounds__(256)
-fit_finalize_batch_kernel(const double* __restrict__ partial, int gpw, const FitJobs jobs) {
+fit_finalize_batch_kernel(const double* __restrict__ partial, int gpw, const FitJobs jobs, double* __restrict__ unit_wsum) {
   __shared__ double red[256];
   const int b = blockIdx.x, t = threadIdx.x;
   int j = 0;
@@ -208,7 +244,7 @@ fit_finalize_batch_kernel(const double* __restrict__ partial, int gpw, const Fit
   const int u = b - (int)jobs.first_unit[j];
   const int rows_blocks = (jobs.R[j] + gpw - 1) / gpw;
   const double* p = partial + ((int64_t)jobs.first_item[j] + (int64_t)u * rows_blocks) * kFitPartials;
-  for (int c = 0; c < 7; ++c) {
+  for (int c = 0; c < (unit_wsum ? 8 : 7); ++c) {
     double acc = 0.0;
     for (int rb = t; rb < rows_blocks; rb += 256) acc += p[(int64_t)rb * kFitPartials + c];
     red[t] = acc;
@@ -219,7 +255,8 @@ fit_finalize_batch_kernel(const double* __restrict__ partial, int gpw, const Fit
     }
     if (t == 0) {
       if (c < 6) jobs.err[j][(int64_t)u * 6 + c] = (float)red[0];
-      else if (jobs.energy[j]) jobs.energy[j][u] = (float)red[0];
+      else if (c == 6) { if (jobs.energy[j]) jobs.energy[j][u] = (float)red[0]; }
+      else unit_wsum[b] = red[0];  // sum of the unit's weights, for the features
     }
     __syncthreads();
   }
@@ -272,18 +309,19 @@ windq_status launch_fit(windq_ctx* ctx, const __half* W, int R, int U, int64_t l
   return WINDQ_OK;
 }
 
-template <int G>
-windq_status launch_fit_batch(windq_ctx* ctx, const FitJobs& jobs, const float* clip, int K, cudaStream_t st) {
+// FEAT: jobs.hist (zeroed here) and unit_wsum receive what the features need (see the kernel).
+template <int G, bool FEAT>
+windq_status launch_fit_batch(windq_ctx* ctx, const FitJobs& jobs, const float* clip, int K, double* unit_wsum, cudaStream_t st) {
   constexpr int GPW = Map<G>::GPW;
   const int chunk = fit_cand_chunk(G), stride = fit_cand_stride(chunk);
   const size_t smem = (size_t)kFitWarpsPerBlock * GPW * stride * sizeof(Cand);
-  const int id = kFitBatchG32 + g_index(G);
-  if (windq_status rc = prepare_kernel(ctx, id, fit_eval_kernel<G, false, false, true>, kFitWarpsPerBlock * 32, smem, true)) return rc;
+  const int id = (FEAT ? kFitFeatG32 : kFitBatchG32) + g_index(G);
+  if (windq_status rc = prepare_kernel(ctx, id, fit_eval_kernel<G, false, false, true, FEAT>, kFitWarpsPerBlock * 32, smem, true)) return rc;
   const int64_t full_grid = (int64_t)ctx->sm_count * ctx->occupancy[id];
   const int64_t n_items = jobs.first_item[jobs.n];
   const bool in_parts = 2 * n_items < 3 * full_grid * kFitWarpsPerBlock;
   if (in_parts)
-    if (windq_status rc = prepare_kernel(ctx, id + 5, fit_eval_kernel<G, false, true, true>, kFitWarpsPerBlock * 32, smem, false))
+    if (windq_status rc = prepare_kernel(ctx, id + 5, fit_eval_kernel<G, false, true, true, FEAT>, kFitWarpsPerBlock * 32, smem, false))
       return rc;
   int64_t grid = full_grid;
   const int64_t need = ((in_parts ? 5 : 1) * n_items + kFitWarpsPerBlock - 1) / kFitWarpsPerBlock;
@@ -291,16 +329,17 @@ windq_status launch_fit_batch(windq_ctx* ctx, const FitJobs& jobs, const float* 
   unsigned int* next_item = (unsigned int*)ctx->scratch;
   double* partial = (double*)((char*)ctx->scratch + 16);
   WINDQ_CUDA(ctx, cudaMemsetAsync(next_item, 0, sizeof(unsigned int), st));
+  if (FEAT) WINDQ_CUDA(ctx, cudaMemsetAsync(jobs.hist, 0, (size_t)jobs.first_unit[jobs.n] * 32768u * sizeof(unsigned int), st));
   if (in_parts)
-    fit_eval_kernel<G, false, true, true><<<(unsigned)grid, kFitWarpsPerBlock * 32, smem, st>>>(
+    fit_eval_kernel<G, false, true, true, FEAT><<<(unsigned)grid, kFitWarpsPerBlock * 32, smem, st>>>(
         nullptr, 0, 0, 0, nullptr, clip, K, partial, nullptr, nullptr, 0, chunk, stride, nullptr, nullptr, __builtin_nanf(""),
         next_item, jobs);
   else
-    fit_eval_kernel<G, false, false, true><<<(unsigned)grid, kFitWarpsPerBlock * 32, smem, st>>>(
+    fit_eval_kernel<G, false, false, true, FEAT><<<(unsigned)grid, kFitWarpsPerBlock * 32, smem, st>>>(
         nullptr, 0, 0, 0, nullptr, clip, K, partial, nullptr, nullptr, 0, chunk, stride, nullptr, nullptr, __builtin_nanf(""),
         next_item, jobs);
   WINDQ_CUDA(ctx, cudaGetLastError());
-  fit_finalize_batch_kernel<<<jobs.first_unit[jobs.n], 256, 0, st>>>(partial, GPW, jobs);
+  fit_finalize_batch_kernel<<<jobs.first_unit[jobs.n], 256, 0, st>>>(partial, GPW, jobs, FEAT ? unit_wsum : nullptr);
   WINDQ_CUDA(ctx, cudaGetLastError());
   return WINDQ_OK;
 }
@@ -382,10 +421,9 @@ int64_t windq_scratch_bytes_fit_eval_batch(const windq_fit_job* jobs, int n_jobs
   return 16 + items * windq::kFitPartials * (int64_t)sizeof(double);
 }
 
-windq_status windq_fit_eval_batch(windq_ctx* ctx, const windq_fit_job* jobs, int n_jobs, int G, const float* clip_grid, int K,
-                                  void* stream) {
+static windq_status fit_batch_any(windq_ctx* ctx, const char* who, const windq_fit_job* jobs, float* const* feat_out, int n_jobs,
+                                  int G, const float* clip_grid, int K, void* stream) {
   using namespace windq;
-  const char* who = "windq_fit_eval_batch";
   if (!ctx) return fail(nullptr, WINDQ_ERR_NULL, "%s: ctx is NULL", who);
   WINDQ_REQUIRE(ctx, jobs && clip_grid, WINDQ_ERR_NULL, "%s: jobs or clip_grid is NULL", who);
   WINDQ_REQUIRE(ctx, n_jobs >= 1 && n_jobs <= kFitMaxJobs, WINDQ_ERR_SHAPE, "%s: n_jobs = %d is outside [1, %d]", who, n_jobs,
@@ -419,15 +457,88 @@ windq_status windq_fit_eval_batch(windq_ctx* ctx, const windq_fit_job* jobs, int
   fj.first_item[n_jobs] = (unsigned int)items;
   fj.first_unit[n_jobs] = (unsigned int)units;
   DeviceGuard guard(ctx->device);
-  if (windq_status st = ensure_scratch(ctx, 16 + items * kFitPartials * (int64_t)sizeof(double))) return st;
+  const int64_t part_bytes = round_up(16 + items * kFitPartials * (int64_t)sizeof(double), 16);
   cudaStream_t st = (cudaStream_t)stream;
-  switch (G) {
-    case 32: return launch_fit_batch<32>(ctx, fj, clip_grid, K, st);
-    case 64: return launch_fit_batch<64>(ctx, fj, clip_grid, K, st);
-    case 128: return launch_fit_batch<128>(ctx, fj, clip_grid, K, st);
-    case 256: return launch_fit_batch<256>(ctx, fj, clip_grid, K, st);
-    default: return launch_fit_batch<512>(ctx, fj, clip_grid, K, st);
+  if (!feat_out) {
+    if (windq_status rc = ensure_scratch(ctx, part_bytes)) return rc;
+    switch (G) {
+      case 32: return launch_fit_batch<32, false>(ctx, fj, clip_grid, K, nullptr, st);
+      case 64: return launch_fit_batch<64, false>(ctx, fj, clip_grid, K, nullptr, st);
+      case 128: return launch_fit_batch<128, false>(ctx, fj, clip_grid, K, nullptr, st);
+      case 256: return launch_fit_batch<256, false>(ctx, fj, clip_grid, K, nullptr, st);
+      default: return launch_fit_batch<512, false>(ctx, fj, clip_grid, K, nullptr, st);
+    }
   }
+  // features too: scratch = counter and partials | one histogram per unit | one sum per unit
+  for (int j = 0; j < n_jobs; ++j) {
+    WINDQ_REQUIRE(ctx, feat_out[j], WINDQ_ERR_NULL, "%s: job %d: feat_out is NULL", who, j);
+    WINDQ_REQUIRE(ctx, jobs[j].R * (int64_t)G < (1ll << 32), WINDQ_ERR_SHAPE, "%s: job %d: R * G must be below 2^32", who, j);
+  }
+  const int64_t hist_bytes = units * 32768 * (int64_t)sizeof(unsigned int);
+  if (windq_status rc = ensure_scratch(ctx, part_bytes + hist_bytes + units * (int64_t)sizeof(double))) return rc;
+  fj.hist = (unsigned int*)((char*)ctx->scratch + part_bytes);
+  double* unit_wsum = (double*)((char*)ctx->scratch + part_bytes + hist_bytes);
+  windq_status rc;
+  switch (G) {
+    case 32: rc = launch_fit_batch<32, true>(ctx, fj, clip_grid, K, unit_wsum, st); break;
+    case 64: rc = launch_fit_batch<64, true>(ctx, fj, clip_grid, K, unit_wsum, st); break;
+    case 128: rc = launch_fit_batch<128, true>(ctx, fj, clip_grid, K, unit_wsum, st); break;
+    case 256: rc = launch_fit_batch<256, true>(ctx, fj, clip_grid, K, unit_wsum, st); break;
+    default: rc = launch_fit_batch<512, true>(ctx, fj, clip_grid, K, unit_wsum, st); break;
+  }
+  if (rc != WINDQ_OK) return rc;
+  int Rs[kFitMaxJobs], first_unit[kFitMaxJobs + 1];
+  const float* ss[kFitMaxJobs];
+  for (int j = 0; j < n_jobs; ++j) {
+    Rs[j] = fj.R[j];
+    first_unit[j] = (int)fj.first_unit[j];
+    ss[j] = fj.s[j];
+  }
+  first_unit[n_jobs] = (int)fj.first_unit[n_jobs];
+  return features_from_histograms(ctx, fj.hist, unit_wsum, n_jobs, Rs, first_unit, ss, feat_out, G, st);
+}
+
+windq_status windq_fit_eval_batch(windq_ctx* ctx, const windq_fit_job* jobs, int n_jobs, int G, const float* clip_grid, int K,
+                                  void* stream) {
+  return fit_batch_any(ctx, "windq_fit_eval_batch", jobs, nullptr, n_jobs, G, clip_grid, K, stream);
+}
+
+int64_t windq_scratch_bytes_features_fit_batch(const windq_featfit_job* jobs, int n_jobs, int G) {
+  if (!jobs || n_jobs <= 0 || n_jobs > windq::kFitMaxJobs || !windq::valid_G(G)) return 0;
+  const int gpw = 32 / (G / 32);
+  int64_t items = 0, units = 0;
+  for (int j = 0; j < n_jobs; ++j) {
+    if (jobs[j].R <= 0 || jobs[j].C <= 0) return 0;
+    items += (jobs[j].C / G) * ((jobs[j].R + gpw - 1) / gpw);
+    units += jobs[j].C / G;
+  }
+  return windq::round_up(16 + items * windq::kFitPartials * (int64_t)sizeof(double), 16) + units * 32768 * (int64_t)sizeof(unsigned int) +
+         units * (int64_t)sizeof(double);
+}
+
+windq_status windq_features_fit_batch(windq_ctx* ctx, const windq_featfit_job* jobs, int n_jobs, int G, const float* clip_grid,
+                                      int K, void* stream) {
+  const char* who = "windq_features_fit_batch";
+  if (!ctx) return windq::fail(nullptr, WINDQ_ERR_NULL, "%s: ctx is NULL", who);
+  if (!jobs) return windq::fail(ctx, WINDQ_ERR_NULL, "%s: jobs is NULL", who);
+  if (n_jobs < 1 || n_jobs > windq::kFitMaxJobs)
+    return windq::fail(ctx, WINDQ_ERR_SHAPE, "%s: n_jobs = %d is outside [1, %d]", who, n_jobs, windq::kFitMaxJobs);
+  windq_fit_job fit[windq::kFitMaxJobs];
+  float* feat[windq::kFitMaxJobs];
+  for (int j = 0; j < n_jobs; ++j) {
+    fit[j].W = jobs[j].W;
+    fit[j].R = jobs[j].R;
+    fit[j].C = jobs[j].C;
+    fit[j].ldw = jobs[j].ldw;
+    fit[j].s = jobs[j].s;
+    fit[j].err_out = jobs[j].err_out;
+    fit[j].energy_out = jobs[j].energy_out;
+    fit[j].clip_idx_out = jobs[j].clip_idx_out;
+    fit[j].group_err_out = jobs[j].group_err_out;
+    feat[j] = jobs[j].feat_out;
+    if (!feat[j]) return windq::fail(ctx, WINDQ_ERR_NULL, "%s: job %d: feat_out is NULL", who, j);
+  }
+  return fit_batch_any(ctx, who, fit, feat, n_jobs, G, clip_grid, K, stream);
 }
 
 }  // extern "C"

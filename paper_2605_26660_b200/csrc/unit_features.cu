@@ -305,6 +305,26 @@ windq_status launch_hist(windq_ctx* ctx, const __half* W, int R, int U, int64_t 
   return WINDQ_OK;
 }
 
+windq_status features_from_histograms(windq_ctx* ctx, const unsigned int* hist, const double* unit_wsum, int n_jobs, const int* R,
+                                      const int* first_unit, const float* const* s, float* const* feat_out, int G, cudaStream_t st) {
+  FeatJobs fj;
+  memset(&fj, 0, sizeof(fj));
+  fj.n = n_jobs;
+  for (int j = 0; j < n_jobs; ++j) {
+    fj.s[j] = s[j];
+    fj.feat[j] = feat_out[j];
+    fj.R[j] = R[j];
+    fj.first_unit[j] = first_unit[j];
+  }
+  fj.first_unit[n_jobs] = first_unit[n_jobs];
+  if (windq_status rc = prepare_kernel(ctx, kFinalize, feat_finalize_kernel, 1024, kBins * sizeof(unsigned int), false)) return rc;
+  // one sum per unit (slots_per_unit = 1); a "rows per block" beyond every pair count makes the kernel read exactly that one
+  feat_finalize_kernel<<<(unsigned)first_unit[n_jobs], 1024, kBins * sizeof(unsigned int), st>>>(hist, unit_wsum, 1, 1ll << 62, 0, G,
+                                                                                               nullptr, nullptr, fj);
+  WINDQ_CUDA(ctx, cudaGetLastError());
+  return WINDQ_OK;
+}
+
 }  // namespace windq
 
 extern "C" {

@@ -56,7 +56,7 @@ struct DeviceGuard {
 // attributes belong to a device, so the record is kept in the context, not in a process-wide static.
 enum KernelId { kFitG32 = 0, kApplyG32 = 5, kApplySearchG32 = 10, kHistG32 = 15, kFinalize = 20, kFitProtectG32 = 21, kApplyProtectG32 = 26, kApplyProtectSearchG32 = 31,
                 kFitBatchG32 = 41 /* 41..45 whole items, 46..50 in parts */, kApplyBatchG32 = 51 /* 51..55 */, kFitPartsOffset = 36 /* kFitG32 + 36 .. and kFitProtectG32 + 36 ..: the in-parts instantiations (36..40, 57..61) */,
-                kApplyStreamG32 = 64 /* 64..68 */, kTernarySearchG32 = 69 /* 69..73 plain, 74..78 protected */, kKernelIds = 128 };
+                kApplyStreamG32 = 64 /* 64..68 */, kFitFeatG32 = 79 /* 79..83 whole items, 84..88 in parts */, kTernarySearchG32 = 69 /* 69..73 plain, 74..78 protected */, kKernelIds = 128 };
 inline int g_index(int G) { return G == 32 ? 0 : G == 64 ? 1 : G == 128 ? 2 : G == 256 ? 3 : 4; }
 
 // Sets the dynamic shared-memory limit of `kernel` once per context and, if asked, records how many
@@ -91,6 +91,11 @@ windq_status launch_apply_stream(windq_ctx* ctx, int G, const void* W, int64_t R
                                  const float* clip_grid, int K, const uint8_t* clip_idx, const void* scale_in,
                                  const float* thr_grid, int thr_K, const uint8_t* thr_idx, const windq_plan_out* plans,
                                  int n_plans, cudaStream_t st);
+
+// The state features of every unit of n_jobs matrices from per-unit histograms of |w| bit patterns (32768 bins each,
+// units of all jobs in a row) and per-unit sums of w, as the fused fit pass leaves them (unit_features.cu).
+windq_status features_from_histograms(windq_ctx* ctx, const unsigned int* hist, const double* unit_wsum, int n_jobs, const int* R,
+                                      const int* first_unit, const float* const* s, float* const* feat_out, int G, cudaStream_t st);
 
 // Bytes of one packed group under an action (host and device).
 __host__ __device__ inline int group_code_bytes(int action, int G) {

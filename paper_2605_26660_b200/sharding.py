@@ -80,6 +80,15 @@ def gather_units(*arrays: torch.Tensor):
     return out, begin, begin + n
 
 
+def gather_rows(table: torch.Tensor) -> torch.Tensor:
+    """All-gathers a per-unit table [n, k] (e.g. the error table err[u][6] of this rank's units) by rows, in rank
+    order; every rank gets the table of the whole model.  Ranks may hold different numbers of units."""
+    if table.dim() != 2:
+        raise ValueError("gather_rows wants a 2-D tensor")
+    cols, _, _ = gather_units(*[table[:, j].contiguous() for j in range(table.shape[1])])
+    return torch.stack(cols, dim=1)
+
+
 def allocate_across_ranks(allocate, saliency, n_weights, n_groups, n_protected=None):
     """The heuristic allocator's rule over the units of all ranks.  `allocate(saliency, n_weights, n_groups,
     n_protected)` is the rule on whole-model arrays (e.g. a closure over windq_greedy_allocate with the

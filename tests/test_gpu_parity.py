@@ -767,3 +767,37 @@ def test_apply_plan_batch_argument_checks(wq, ctx):
         wq.windq_apply_plan_batch(ctx, [job] * 25, 128, gd)
     out = wq.windq_apply_plan_batch(ctx, [job], 128, gd)
     assert out[0]["wq"] is None and (out[0]["codes"][:2048] == 0).all()
+
+
+@pytest.mark.parametrize("G,shapes", [(128, [(300, 512), (64, 1024), (1000, 256), (17, 128)]),
+                                      (64, [(40, 256), (2048, 2048)]),
+                                      (256, [(512, 2048)] * 3 + [(2048, 2048)]),
+                                      (32, [(5, 32)]),
+                                      (128, [(5000, 128), (3, 4096)])])
+def test_features_fit_batch_equals_the_two_batched_calls(wq, ctx, oracle, G, shapes):
+    """Features and fits in one pass over the weights: fit outputs equal windq_fit_eval_batch bit for bit, the
+    histogram features and those of s equal windq_unit_features_batch bit for bit, the mean within tolerance, and
+    everything equals the oracle."""
+    grid = ws.clip_grid(20)
+    gd = torch.from_numpy(grid).cuda()
+    Ws = [ws.weights(R, C, 500 + i, "student_t").cuda() for i, (R, C) in enumerate(shapes)]
+    for W in Ws:
+        W[::7, ::3] = 0
+    ss = [(torch.rand(C, generator=torch.Generator().manual_seed(i)) * 3 + 0.01).cuda() for i, (R, C) in enumerate(shapes)]
+    feats, fits = wq.windq_features_fit_batch(ctx, Ws, G, ss, gd, want_group_err=True)
+    torch.cuda.synchronize()
+    ref_fit = wq.windq_fit_eval_batch(ctx, Ws, G, ss, gd, want_group_err=True)
+    ref_feat = wq.windq_unit_features_batch(ctx, Ws, G, ss)
+    torch.cuda.synchronize()
+    for W, s, f, out, rf, rfit in zip(Ws, ss, feats, fits, ref_feat, ref_fit):
+        for k in ("clip_idx", "group_err", "err", "energy"):
+            assert torch.equal(out[k].view(torch.uint8), rfit[k].view(torch.uint8)), k
+        assert torch.equal(f[:, 1:].view(torch.int32), rf[:, 1:].view(torch.int32))
+        assert close(f[:, 0].cpu().numpy(), rf[:, 0].cpu().numpy()).all()
+        want = oracle.unit_features(W.cpu().numpy(), G, s.cpu().numpy())
+        assert (f[:, 3:5].cpu().numpy() == want[:, 3:5]).all() and close(f.cpu().numpy(), want).all()
+    # twice in a row: the histograms are cleared by the call
+    feats2, _ = wq.windq_features_fit_batch(ctx, Ws, G, ss, gd)
+    torch.cuda.synchronize()
+    for a, b in zip(feats, feats2):
+        assert torch.equal(a[:, 1:], b[:, 1:])

@@ -191,3 +191,88 @@ def test_token_sharded_act_stats_equal_the_whole_input(tmp_path, oracle):
     got = [np.load(os.path.join(str(tmp_path), "act%d.npy" % r)) for r in range(world)]
     assert np.array_equal(got[0], got[1])                       # every rank holds the same statistic
     assert np.allclose(got[0], want, rtol=1e-6, atol=0)
+
+
+# ---- the whole path of a small model, its blocks split over two ranks --------------------------------------
+def _tiny_spec():
+    import windq_synth as ws
+    return ws.ModelSpec("tiny", 4, 256, 384, 128, "student_t", 64, 6, (64,))
+
+
+def _score_blocks(oracle, spec, blocks):
+    """The oracle's path over `blocks`: per unit the error table, the energy, the saliency score and the counts the
+    allocator needs (units in block order, then matrix order)."""
+    import windq_synth as ws
+    G = spec.chunk_widths[0]
+    grid = ws.clip_grid(spec.K)
+    err, energy, sal, nw, ng = [], [], [], [], []
+    for b in blocks:
+        stats = {i: oracle.act_stats(ws.block_input(spec, 0, b, i).numpy()) for i, _ in spec.block_inputs()}
+        for m in spec.block_matrices():
+            W = ws.block_weight(spec, 0, b, m).numpy()
+            fit = oracle.fit_eval(W, G, stats[m.x_id], grid, want_group_err=False)
+            err.append(fit["err"])
+            energy.append(fit["energy"])
+            sal.append(oracle.unit_saliency(W, G, stats[m.x_id]))
+            nw.append(np.full(m.C // G, m.R * G, np.int64))
+            ng.append(np.full(m.C // G, m.R, np.int64))
+    if not err:
+        return (np.zeros((0, 6), np.float32), np.zeros(0, np.float32), np.zeros(0, np.float32), np.zeros(0, np.int64),
+                np.zeros(0, np.int64))
+    return np.concatenate(err), np.concatenate(energy), np.concatenate(sal), np.concatenate(nw), np.concatenate(ng)
+
+
+def _tiny_rule(oracle):
+    def rule(sal, n, g, p):
+        actions, _, total = oracle.greedy_allocate(sal.numpy(), n.numpy(), g.numpy(), 200, 10, scale_bits=16, zero_bits=16)
+        return dict(actions=torch.from_numpy(actions), total_centibits=total)
+    return rule
+
+
+def _path_worker(rank, world, port, out_dir):
+    sys.path.insert(0, ROOT)
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        sharding = _load_sharding()
+        import oracle
+        oracle.build()
+        spec = _tiny_spec()
+        mine = sharding.block_range(spec.n_blocks, rank, world)
+        err, energy, sal, nw, ng = _score_blocks(oracle, spec, mine)
+        table = sharding.gather_rows(torch.from_numpy(err))                       # the model's error table on every rank
+        actions, total = sharding.allocate_across_ranks(_tiny_rule(oracle), torch.from_numpy(sal), torch.from_numpy(nw),
+                                                        torch.from_numpy(ng))
+        # bit accounting of this rank's slice of the plan, summed exactly over the ranks
+        G = spec.chunk_widths[0]
+        local_cb, pos = 0, 0
+        for b in mine:
+            for m in spec.block_matrices():
+                U = m.C // G
+                local_cb += int(oracle.effective_bits(actions[pos:pos + U].numpy(), m.R, G)["total_centibits"])
+                pos += U
+        np.savez(os.path.join(out_dir, "path%d.npz" % rank), table=table.numpy(), actions=actions.numpy(),
+                 total=np.int64(total), summed=np.int64(sharding.sum_int64(local_cb)), n_blocks=len(mine))
+    finally:
+        dist.destroy_process_group()
+
+
+def test_whole_path_over_two_ranks_equals_one_process(tmp_path, oracle):
+    """Strong scaling on the host side: the four blocks of a small model split over two ranks, each rank running the
+    path on its blocks only; the gathered error table, the plan of the heuristic allocator and the plan's total bits
+    are those of one process over the whole model."""
+    world = 2
+    mp.start_processes(_path_worker, args=(world, _free_port(), str(tmp_path)), nprocs=world, join=True, start_method="spawn")
+    spec = _tiny_spec()
+    err, energy, sal, nw, ng = _score_blocks(oracle, spec, range(spec.n_blocks))
+    want_actions, _, want_total = oracle.greedy_allocate(sal, nw, ng, 200, 10, scale_bits=16, zero_bits=16)
+    got = [np.load(os.path.join(str(tmp_path), "path%d.npz" % r)) for r in range(world)]
+    pos = 0
+    for g in got:
+        assert np.array_equal(g["table"].view(np.uint32), err.view(np.uint32))    # same bits: units are independent
+        n = g["actions"].size
+        assert np.array_equal(g["actions"], want_actions[pos:pos + n])
+        pos += n
+        assert int(g["total"]) == want_total and int(g["summed"]) == want_total
+    assert pos == want_actions.size and sum(int(g["n_blocks"]) for g in got) == spec.n_blocks

@@ -1,7 +1,8 @@
 """Randomised parity sweep on the GPU: random shapes, chunk widths, grid sizes, weight and statistic distributions
 (zeros, one-sided, ties, sparse, fp16 subnormals, outlier columns, statistics spanning 20 decades) through the whole
-chain -- features, fits, plan packing, salient selection, protected fits, refinement, protected and refined packing --
-against the oracle.  Integer and bit-pattern outputs are compared exactly."""
+chain -- features, fits, plan packing (one plan, and several plans in one pass), the search over the ternary
+assignment and packing with its thresholds, salient selection, protected fits, refinement, protected and refined
+packing -- against the oracle.  Integer and bit-pattern outputs are compared exactly."""
 import numpy as np
 import pytest
 import torch
@@ -105,6 +106,42 @@ def test_random_chain(wq, ctx, oracle, seed):
         assert np.array_equal(pg["codes"][:n].cpu().numpy(), po["codes"]), tag
         assert np.array_equal(bits16(pg["wq"]), po["wq"]), tag
         assert np.array_equal(bits16(pg["scales"]), po["scales"]) and np.array_equal(bits16(pg["zeros"]), po["zeros"]), tag
+
+        # unit sums without group errors (the 1.58- and 1-bit ones then come from the fit's sums): tolerance outputs
+        plain = wq.windq_fit_eval(ctx, Wd, G, sd, gd)
+        assert np.array_equal(plain["clip_idx"].cpu().numpy(), want["clip_idx"]), tag
+        assert np.allclose(plain["err"].cpu().numpy(), want["err"], rtol=1e-4, atol=1e-6), tag
+
+        # several plans of the matrix in one pass
+        n_plans = int(rng.integers(1, 5))
+        plans, wants = [], []
+        for p in range(n_plans):
+            acts_p = rng.integers(0, 7, U).astype(np.uint8)
+            ap = torch.from_numpy(acts_p).cuda()
+            ebp = wq.windq_effective_bits(ctx, ap, R, G)
+            plans.append(dict(actions=ap, code_offsets=ebp["code_offsets"],
+                              codes=torch.zeros(2 * R * C + 16 * U, dtype=torch.uint8, device="cuda")))
+            wants.append(oracle.apply_plan(W, G, s, grid, acts_p, want["clip_idx"]))
+        outs = wq.windq_apply_plan_multi(ctx, Wd, G, sd, gd, got["clip_idx"], plans)
+        for out, wp in zip(outs, wants):
+            m = int(wp["code_offsets"][U])
+            assert np.array_equal(out["codes"][:m].cpu().numpy(), wp["codes"]) and np.array_equal(bits16(out["wq"]), wp["wq"]), tag
+            assert np.array_equal(bits16(out["scales"]), wp["scales"]) and np.array_equal(bits16(out["zeros"]), wp["zeros"]), tag
+
+        # search over the ternary assignment, and packing with its thresholds
+        Kt = int(rng.choice([1, 3, 9, 64]))
+        thr = np.sort(rng.uniform(0.05, 3.0, Kt)).astype(np.float32)
+        td = torch.from_numpy(thr).cuda()
+        to = oracle.fit_ternary_search(W, G, s, thr)
+        tg = wq.windq_fit_ternary_search(ctx, Wd, G, sd, td, want_group_err=True)
+        assert np.array_equal(tg["thr_idx"].cpu().numpy(), to["thr_idx"]), tag
+        assert np.array_equal(bits16(tg["alpha"]), to["alpha"].view(np.uint16)), tag
+        assert np.array_equal(bits32(tg["group_err"].cpu().numpy()), bits32(to["group_err"])), tag
+        codes.zero_()
+        sgp = wq.windq_apply_plan_searched(ctx, Wd, G, sd, gd, ad, eb["code_offsets"], codes, got["clip_idx"], td, tg["thr_idx"])
+        sop = oracle.apply_plan_searched(W, G, s, grid, actions, want["clip_idx"], thr, to["thr_idx"])
+        assert np.array_equal(sgp["codes"][:n].cpu().numpy(), sop["codes"]) and np.array_equal(bits16(sgp["wq"]), sop["wq"]), tag
+        assert np.array_equal(bits16(sgp["scales"]), sop["scales"]), tag
 
         rate = int(rng.choice([0, 10000, 30000, 200000, 1000000]))
         so = oracle.salient_select(W, G, s, rate)

@@ -250,6 +250,7 @@ class Buffers:
         # one set of fit outputs per matrix of a block, for the batched fit (all matrices of a block in one call)
         for mi, m in enumerate(mats):
             shapes["feat%d" % mi] = ((m.C // Gmin) * 8, torch.float32)
+            shapes["featw%d" % mi] = ((m.C // Gmin) * 8, torch.float32)
             shapes["totals%d" % mi] = (2 * len(TARGET_BITS), torch.int64)
             shapes["err%d" % mi] = ((m.C // Gmin) * 6, torch.float32)
             shapes["energy%d" % mi] = (m.C // Gmin, torch.float32)
@@ -359,10 +360,21 @@ def score_block(wq, ctx, spec, Wb, Xb, plans_b, buf, grid_d, timer=None, sink=No
         wq.windq_act_stats(ctx, X, buf.s[i])
         launches += 2
     if BATCH_FITS:
+        # chunk widths G and 2 G: the features of both come out of one pass at G (windq_unit_features_batch2)
+        nested = (not FUSED_FEATURES and len(spec.chunk_widths) == 2 and spec.chunk_widths[1] == 2 * spec.chunk_widths[0]
+                  and all(m.C % spec.chunk_widths[1] == 0 for m in mats))
+        wide_feats = None
         for G in spec.chunk_widths:
             stats = [buf.s[m.x_id] for m in mats]
-            feats = [buf.take("feat%d" % mi)[:(m.C // G) * 8].view(m.C // G, 8) for mi, m in enumerate(mats)]
-            if not FUSED_FEATURES:
+            if nested and G == spec.chunk_widths[1]:
+                feats = wide_feats
+            else:
+                feats = [buf.take("feat%d" % mi)[:(m.C // G) * 8].view(m.C // G, 8) for mi, m in enumerate(mats)]
+            if nested and G == spec.chunk_widths[0]:
+                wide_feats = [buf.take("featw%d" % mi)[:(m.C // (2 * G)) * 8].view(m.C // (2 * G), 8) for mi, m in enumerate(mats)]
+                wq.windq_unit_features_batch(ctx, Wb, G, stats, feats, feats_2G=wide_feats)
+                launches += 3
+            elif not FUSED_FEATURES and not nested:
                 wq.windq_unit_features_batch(ctx, Wb, G, stats, feats)
                 launches += 2
             outs = [dict(err=buf.take("err%d" % mi)[:(m.C // G) * 6].view(m.C // G, 6),
@@ -380,7 +392,7 @@ def score_block(wq, ctx, spec, Wb, Xb, plans_b, buf, grid_d, timer=None, sink=No
             launches += 2
             if sink:
                 for mi in range(len(mats)):
-                    sink("feat%d" % mi, feats[mi])
+                    sink("featw%d" % mi if (nested and G == spec.chunk_widths[1]) else "feat%d" % mi, feats[mi])
             if sink:
                 for mi in range(len(mats)):
                     sink("err%d" % mi, outs[mi]["err"])
@@ -835,6 +847,9 @@ def main():
                                 parallelism="the blocks of one model split over the GPUs" if strong else "replica per GPU",
                                 residency="two block slots refilled block by block (the model does not fit); only the kernels "
                                           "of a block are timed" if streamed else "all blocks resident in HBM",
+                                features="one pass per block for both chunk widths (windq_unit_features_batch2)"
+                                if (not FUSED_FEATURES and BATCH_FITS and len(spec.chunk_widths) == 2 and spec.chunk_widths[1] == 2 * spec.chunk_widths[0])
+                                else "one pass per block and chunk width",
                                 fits="one windq_features_fit_batch call per block and chunk width" if FUSED_FEATURES
                                 else "one windq_unit_features_batch and one windq_fit_eval_batch call per block and chunk width" if BATCH_FITS
                                 else "one windq_unit_features and one windq_fit_eval call per matrix",

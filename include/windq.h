@@ -193,6 +193,17 @@ typedef struct {
 int64_t windq_scratch_bytes_unit_features_batch(const windq_feat_job* jobs, int n_jobs, int G);
 windq_status windq_unit_features_batch(windq_ctx* ctx, const windq_feat_job* jobs, int n_jobs, int G, void* stream);
 
+/* windq_unit_features_batch at TWO chunk widths, G and 2 G, from one pass over the weights (the paper has no
+ * counterpart; its chunk-size ablation scores the same model at nested chunk sizes).  A unit of width 2 G is the union
+ * of two neighbouring units of width G, and the histogram of a union is the sum of the histograms, so the wider units'
+ * features come from the histograms the pass has built anyway -- the same values as a windq_unit_features_batch
+ * call at 2 G (histogram features and those of s bit for bit; the mean within 1e-6 relative).
+ *   feat_out_2G: HOST array of n_jobs device pointers, fp32 [C / (2 G)][8] each, or NULL for a job that wants
+ *   width G only; with any non-NULL entry every job's C must be a multiple of 2 G.  G <= 256.
+ * Everything else as windq_unit_features_batch, including the scratch size. */
+windq_status windq_unit_features_batch2(windq_ctx* ctx, const windq_feat_job* jobs, float* const* feat_out_2G, int n_jobs,
+                                        int G, void* stream);
+
 /* windq_fit_eval for several matrices in one launch (the paper has no counterpart: the consumer loops
  * over the seven projections of every block, and matrices that are small against the GPU -- a few million
  * weights -- neither fill it nor amortise the fixed cost of a call on their own).  All jobs share G, the

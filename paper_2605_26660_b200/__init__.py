@@ -60,6 +60,7 @@ def _load() -> ctypes.CDLL:
     lib.windq_apply_plan_batch.argtypes = [vp, vp, i32, i32, vp, i32, vp]
     lib.windq_effective_bits_batch.argtypes = [vp, vp, i32, i32, i32, i32, vp]
     lib.windq_unit_features_batch.argtypes = [vp, vp, i32, i32, vp]
+    lib.windq_unit_features_batch2.argtypes = [vp, vp, vp, i32, i32, vp]
     lib.windq_scratch_bytes_unit_features_batch.restype = i64
     lib.windq_scratch_bytes_unit_features_batch.argtypes = [vp, i32, i32]
     lib.windq_fit_eval_batch.argtypes = [vp, vp, i32, i32, vp, i32, vp]
@@ -358,13 +359,18 @@ class _FeatJob(ctypes.Structure):
                 ("s", ctypes.c_void_p), ("feat_out", ctypes.c_void_p)]
 
 
-def windq_unit_features_batch(ctx: Context, Ws, G: int, ss, feats=None, stream=None) -> list:
+def windq_unit_features_batch(ctx: Context, Ws, G: int, ss, feats=None, stream=None, feats_2G=None):
     """windq_unit_features of up to 16 matrices in one pass.  ``feats`` may hold one preallocated [U, 8] fp32
-    tensor per matrix.  Returns the list of feature tensors."""
+    tensor per matrix.  Returns the list of feature tensors.
+
+    With ``feats_2G`` (True, or a list with one preallocated [U / 2, 8] tensor or None per matrix) the call is
+    windq_unit_features_batch2: the features at chunk width 2 G come out of the same pass, and the result is
+    (features at G, features at 2 G)."""
     if len(Ws) != len(ss) or not Ws:
         raise ValueError("Ws and ss must be non-empty and equally long")
     jobs = (_FeatJob * len(Ws))()
-    outs = []
+    outs, outs2 = [], []
+    wide = (ctypes.c_void_p * len(Ws))()
     for j, (W, s) in enumerate(zip(Ws, ss)):
         R, C, ldw = _matrix(W, "W")
         _need(s, torch.float32, "s", 1)
@@ -375,8 +381,20 @@ def windq_unit_features_batch(ctx: Context, Ws, G: int, ss, feats=None, stream=N
             raise ValueError("feat_out must be a contiguous [U, 8] tensor")
         jobs[j] = _FeatJob(W.data_ptr(), R, C, ldw, s.data_ptr(), f.data_ptr())
         outs.append(f)
-    ctx._check(_lib.windq_unit_features_batch(ctx._h, ctypes.cast(jobs, ctypes.c_void_p), len(Ws), int(G), _stream(stream)))
-    return outs
+        if feats_2G is not None:
+            f2 = torch.empty((U // 2, N_FEATURES), dtype=torch.float32, device=W.device) if feats_2G is True else feats_2G[j]
+            if f2 is not None:
+                _need(f2, torch.float32, "feat_out_2G", 2)
+                if tuple(f2.shape) != (U // 2, N_FEATURES) or not f2.is_contiguous():
+                    raise ValueError("feat_out_2G must be a contiguous [U / 2, 8] tensor")
+            wide[j] = None if f2 is None else f2.data_ptr()
+            outs2.append(f2)
+    if feats_2G is None:
+        ctx._check(_lib.windq_unit_features_batch(ctx._h, ctypes.cast(jobs, ctypes.c_void_p), len(Ws), int(G), _stream(stream)))
+        return outs
+    ctx._check(_lib.windq_unit_features_batch2(ctx._h, ctypes.cast(jobs, ctypes.c_void_p), ctypes.cast(wide, ctypes.c_void_p),
+                                               len(Ws), int(G), _stream(stream)))
+    return outs, outs2
 
 
 class _FitJob(ctypes.Structure):

@@ -33,6 +33,7 @@ struct FeatJobs {
   const __half* W[kFeatMaxJobs];
   const float* s[kFeatMaxJobs];
   float* feat[kFeatMaxJobs];
+  float* feat2[kFeatMaxJobs];  // features of the units of twice the width (pairs of neighbouring units), or NULL
   long long ldw[kFeatMaxJobs];
   long long first_pair[kFeatMaxJobs + 1];
   int R[kFeatMaxJobs];
@@ -122,6 +123,9 @@ feat_hist_kernel(const __half* __restrict__ W_one, int R_one, int64_t ldw_one, l
 // One block per unit.  The unit's histogram is first copied to shared memory with coalesced 128-bit
 // loads; thread t then owns the 32 consecutive bins 32 t .. 32 t + 31 and walks them from shared
 // memory starting at bin t mod 32, so that the lanes of a warp stay on different banks.
+// MERGE = 2: the block forms the features of a unit of width 2G from the histograms and sums of the two units of width
+// G it consists of (a histogram of a union is the sum of the histograms), for jobs that ask for both widths.
+template <int MERGE>
 __global__ void __launch_bounds__(1024)
 feat_finalize_kernel(const unsigned int* __restrict__ hist, const double* __restrict__ slot_sum, int slots_per_unit,
                      long long rows_per_block, int R_one, int G, const float* __restrict__ s_one, float* __restrict__ feat_one,
@@ -132,27 +136,37 @@ feat_finalize_kernel(const unsigned int* __restrict__ hist, const double* __rest
   __shared__ unsigned long long redc[2][32];
   __shared__ double s_stat[3];
   __shared__ int p99_bin;
-  const int ug = blockIdx.x, t = threadIdx.x, lane = t & 31, wp = t >> 5;  // ug: the unit's place in hist and slot_sum
+  const int t = threadIdx.x, lane = t & 31, wp = t >> 5;
+  int ug = blockIdx.x * MERGE;  // the (first) unit's place in hist and slot_sum
   int u = ug, R = R_one;
   const float* s = s_one;
   float* feat = feat_one;
   long long pair0 = 0;
   if (jobs.n) {
     int j = 0;
-    while (j + 1 < jobs.n && ug >= jobs.first_unit[j + 1]) ++j;
+    while (j + 1 < jobs.n && ug >= jobs.first_unit[j + 1]) ++j;  // every job has a multiple of MERGE units
     u = ug - jobs.first_unit[j];
     R = jobs.R[j];
     s = jobs.s[j];
-    feat = jobs.feat[j];
+    feat = MERGE == 1 ? jobs.feat[j] : jobs.feat2[j];
     pair0 = jobs.first_pair[j];
+    if (MERGE > 1 && feat == nullptr) return;  // this job did not ask for the wider units
   }
-  const long long n = (long long)R * G;
+  const int GW = G * MERGE;                // width of the unit whose features are formed
+  const long long n = (long long)R * GW;
   const unsigned long long k = (unsigned long long)((99 * n + 99) / 100);  // rank of P99, 1-indexed
   {
     const uint4* src = reinterpret_cast<const uint4*>(hist + (int64_t)ug * kBins);
     uint4* dst = reinterpret_cast<uint4*>(sh);
 #pragma unroll
-    for (int i = 0; i < kBins / 4 / 1024; ++i) dst[i * 1024 + t] = src[i * 1024 + t];
+    for (int i = 0; i < kBins / 4 / 1024; ++i) {
+      uint4 v = src[i * 1024 + t];
+      if (MERGE > 1) {
+        const uint4 w2 = src[kBins / 4 + i * 1024 + t];  // the neighbouring unit's histogram follows
+        v.x += w2.x; v.y += w2.y; v.z += w2.z; v.w += w2.w;
+      }
+      dst[i * 1024 + t] = v;
+    }
   }
   __syncthreads();
   const unsigned int* mine = sh + t * 32;
@@ -179,20 +193,20 @@ feat_finalize_kernel(const unsigned int* __restrict__ hist, const double* __rest
   }
   // statistics of s over the unit's G channels: warp 1, in double
   if (wp == 1) {
-    const float* su = s + (int64_t)u * G;
+    const float* su = s + (int64_t)u * G;  // u counts units of width G: the wider unit starts at the same channel
     double sm = 0.0, mx = (double)su[0];
-    for (int j = lane; j < G; j += 32) { const double v = (double)su[j]; sm += v; mx = fmax(mx, v); }
+    for (int j = lane; j < GW; j += 32) { const double v = (double)su[j]; sm += v; mx = fmax(mx, v); }
 #pragma unroll
     for (int m = 16; m > 0; m >>= 1) {
       sm += __shfl_xor_sync(0xffffffffu, sm, m);
       mx = fmax(mx, __shfl_xor_sync(0xffffffffu, mx, m));
     }
-    const double mean = sm / (double)G;
+    const double mean = sm / (double)GW;
     double var = 0.0;
-    for (int j = lane; j < G; j += 32) { const double d = (double)su[j] - mean; var += d * d; }
+    for (int j = lane; j < GW; j += 32) { const double d = (double)su[j] - mean; var += d * d; }
 #pragma unroll
     for (int m = 16; m > 0; m >>= 1) var += __shfl_xor_sync(0xffffffffu, var, m);
-    if (lane == 0) { s_stat[0] = mean; s_stat[1] = sqrt(var / (double)G); s_stat[2] = mx; }
+    if (lane == 0) { s_stat[0] = mean; s_stat[1] = sqrt(var / (double)GW); s_stat[2] = mx; }
   }
   __syncthreads();
   incl += wp ? warp_total[wp - 1] : 0ull;
@@ -227,11 +241,12 @@ feat_finalize_kernel(const unsigned int* __restrict__ hist, const double* __rest
     }
   }
   double ss = 0.0;
-  {
-    const long long first = (pair0 + (long long)u * R) / rows_per_block;
-    const long long last = (pair0 + (long long)(u + 1) * R - 1) / rows_per_block;
+#pragma unroll
+  for (int h = 0; h < MERGE; ++h) {
+    const long long first = (pair0 + (long long)(u + h) * R) / rows_per_block;
+    const long long last = (pair0 + (long long)(u + h + 1) * R - 1) / rows_per_block;
     const int cnt = (int)(last - first + 1);
-    for (int i = t; i < cnt; i += 1024) ss += slot_sum[(int64_t)ug * slots_per_unit + i];
+    for (int i = t; i < cnt; i += 1024) ss += slot_sum[(int64_t)(ug + h) * slots_per_unit + i];
   }
 #pragma unroll
   for (int m = 16; m > 0; m >>= 1) {
@@ -262,7 +277,7 @@ feat_finalize_kernel(const unsigned int* __restrict__ hist, const double* __rest
       const double mean = sg / dn;
       double var = q2 / dn - mean * mean;
       if (var < 0.0) var = 0.0;
-      float* f = feat + (int64_t)u * WINDQ_N_FEATURES;
+      float* f = feat + (int64_t)(u / MERGE) * WINDQ_N_FEATURES;
       f[0] = (float)mean;
       f[1] = (float)sqrt(var);
       f[2] = (float)(a / dn);
@@ -317,9 +332,9 @@ windq_status features_from_histograms(windq_ctx* ctx, const unsigned int* hist, 
     fj.first_unit[j] = first_unit[j];
   }
   fj.first_unit[n_jobs] = first_unit[n_jobs];
-  if (windq_status rc = prepare_kernel(ctx, kFinalize, feat_finalize_kernel, 1024, kBins * sizeof(unsigned int), false)) return rc;
+  if (windq_status rc = prepare_kernel(ctx, kFinalize, feat_finalize_kernel<1>, 1024, kBins * sizeof(unsigned int), false)) return rc;
   // one sum per unit (slots_per_unit = 1); a "rows per block" beyond every pair count makes the kernel read exactly that one
-  feat_finalize_kernel<<<(unsigned)first_unit[n_jobs], 1024, kBins * sizeof(unsigned int), st>>>(hist, unit_wsum, 1, 1ll << 62, 0, G,
+  feat_finalize_kernel<1><<<(unsigned)first_unit[n_jobs], 1024, kBins * sizeof(unsigned int), st>>>(hist, unit_wsum, 1, 1ll << 62, 0, G,
                                                                                                nullptr, nullptr, fj);
   WINDQ_CUDA(ctx, cudaGetLastError());
   return WINDQ_OK;
@@ -363,8 +378,8 @@ windq_status windq_unit_features(windq_ctx* ctx, const void* W, int64_t R, int64
     default: rc = launch_hist<512>(ctx, Wh, (int)R, U, ldw, fg, hist, slot_sum, st); break;
   }
   if (rc != WINDQ_OK) return rc;
-  if (windq_status st2 = prepare_kernel(ctx, kFinalize, feat_finalize_kernel, 1024, kBins * sizeof(unsigned int), false)) return st2;
-  feat_finalize_kernel<<<(unsigned)U, 1024, kBins * sizeof(unsigned int), st>>>(hist, slot_sum, fg.slots_per_unit, fg.rows_per_block, (int)R, G, s, feat_out, FeatJobs());
+  if (windq_status st2 = prepare_kernel(ctx, kFinalize, feat_finalize_kernel<1>, 1024, kBins * sizeof(unsigned int), false)) return st2;
+  feat_finalize_kernel<1><<<(unsigned)U, 1024, kBins * sizeof(unsigned int), st>>>(hist, slot_sum, fg.slots_per_unit, fg.rows_per_block, (int)R, G, s, feat_out, FeatJobs());
   WINDQ_CUDA(ctx, cudaGetLastError());
   return WINDQ_OK;
 }
@@ -385,9 +400,9 @@ int64_t windq_scratch_bytes_unit_features_batch(const windq_feat_job* jobs, int 
   return U * windq::kBins * (int64_t)sizeof(unsigned int) + U * slots * (int64_t)sizeof(double);
 }
 
-windq_status windq_unit_features_batch(windq_ctx* ctx, const windq_feat_job* jobs, int n_jobs, int G, void* stream) {
+static windq_status unit_features_batch_any(windq_ctx* ctx, const char* who, const windq_feat_job* jobs, float* const* feat2, int n_jobs,
+                                            int G, void* stream) {
   using namespace windq;
-  const char* who = "windq_unit_features_batch";
   if (!ctx) return fail(nullptr, WINDQ_ERR_NULL, "%s: ctx is NULL", who);
   WINDQ_REQUIRE(ctx, jobs, WINDQ_ERR_NULL, "%s: jobs is NULL", who);
   WINDQ_REQUIRE(ctx, n_jobs >= 1 && n_jobs <= kFeatMaxJobs, WINDQ_ERR_SHAPE, "%s: n_jobs = %d is outside [1, %d]", who, n_jobs,
@@ -397,6 +412,7 @@ windq_status windq_unit_features_batch(windq_ctx* ctx, const windq_feat_job* job
   fj.n = n_jobs;
   long long pairs = 0;
   int64_t units = 0, max_R = 0;
+  bool any_wide = false;
   for (int j = 0; j < n_jobs; ++j) {
     const windq_feat_job& b = jobs[j];
     if (windq_status st = check_matrix(ctx, who, b.W, b.R, b.C, b.ldw, G)) return st;
@@ -405,6 +421,13 @@ windq_status windq_unit_features_batch(windq_ctx* ctx, const windq_feat_job* job
     fj.W[j] = (const __half*)b.W;
     fj.s[j] = b.s;
     fj.feat[j] = b.feat_out;
+    fj.feat2[j] = feat2 ? feat2[j] : nullptr;
+    if (fj.feat2[j]) {
+      any_wide = true;
+      WINDQ_REQUIRE(ctx, b.C % (2 * (int64_t)G) == 0, WINDQ_ERR_SHAPE, "%s: job %d: C = %lld is not a multiple of 2 G = %d", who, j,
+                    (long long)b.C, 2 * G);
+      WINDQ_REQUIRE(ctx, b.R * 2 * (int64_t)G < (1ll << 32), WINDQ_ERR_SHAPE, "%s: job %d: R * 2 G must be below 2^32", who, j);
+    }
     fj.ldw[j] = b.ldw;
     fj.R[j] = (int)b.R;
     fj.first_pair[j] = pairs;
@@ -416,6 +439,10 @@ windq_status windq_unit_features_batch(windq_ctx* ctx, const windq_feat_job* job
   fj.first_pair[n_jobs] = pairs;
   fj.first_unit[n_jobs] = (int)units;
   WINDQ_REQUIRE(ctx, units <= 65535 * 32, WINDQ_ERR_SHAPE, "%s: too many units", who);
+  if (any_wide)
+    for (int j = 0; j < n_jobs; ++j)
+      WINDQ_REQUIRE(ctx, jobs[j].C % (2 * (int64_t)G) == 0, WINDQ_ERR_SHAPE,
+                    "%s: job %d: with features at width 2 G every job needs an even number of units", who, j);
   DeviceGuard guard(ctx->device);
   if (windq_status st = ensure_scratch(ctx, windq_scratch_bytes_unit_features_batch(jobs, n_jobs, G))) return st;
   cudaStream_t st = (cudaStream_t)stream;
@@ -432,11 +459,30 @@ windq_status windq_unit_features_batch(windq_ctx* ctx, const windq_feat_job* job
     default: rc = launch_hist<512>(ctx, nullptr, 0, 0, 0, fg, hist, slot_sum, st, fj, pairs); break;
   }
   if (rc != WINDQ_OK) return rc;
-  if (windq_status st2 = prepare_kernel(ctx, kFinalize, feat_finalize_kernel, 1024, kBins * sizeof(unsigned int), false)) return st2;
-  feat_finalize_kernel<<<(unsigned)units, 1024, kBins * sizeof(unsigned int), st>>>(hist, slot_sum, fg.slots_per_unit,
-                                                                                    fg.rows_per_block, 0, G, nullptr, nullptr, fj);
+  if (windq_status st2 = prepare_kernel(ctx, kFinalize, feat_finalize_kernel<1>, 1024, kBins * sizeof(unsigned int), false)) return st2;
+  feat_finalize_kernel<1><<<(unsigned)units, 1024, kBins * sizeof(unsigned int), st>>>(hist, slot_sum, fg.slots_per_unit,
+                                                                                       fg.rows_per_block, 0, G, nullptr, nullptr, fj);
   WINDQ_CUDA(ctx, cudaGetLastError());
+  if (any_wide) {
+    if (windq_status st2 = prepare_kernel(ctx, kFinalize2, feat_finalize_kernel<2>, 1024, kBins * sizeof(unsigned int), false)) return st2;
+    feat_finalize_kernel<2><<<(unsigned)(units / 2), 1024, kBins * sizeof(unsigned int), st>>>(hist, slot_sum, fg.slots_per_unit,
+                                                                                              fg.rows_per_block, 0, G, nullptr, nullptr, fj);
+    WINDQ_CUDA(ctx, cudaGetLastError());
+  }
   return WINDQ_OK;
+}
+
+windq_status windq_unit_features_batch(windq_ctx* ctx, const windq_feat_job* jobs, int n_jobs, int G, void* stream) {
+  return unit_features_batch_any(ctx, "windq_unit_features_batch", jobs, nullptr, n_jobs, G, stream);
+}
+
+windq_status windq_unit_features_batch2(windq_ctx* ctx, const windq_feat_job* jobs, float* const* feat_out_2G, int n_jobs, int G,
+                                        void* stream) {
+  const char* who = "windq_unit_features_batch2";
+  if (!ctx) return windq::fail(nullptr, WINDQ_ERR_NULL, "%s: ctx is NULL", who);
+  if (!feat_out_2G) return windq::fail(ctx, WINDQ_ERR_NULL, "%s: feat_out_2G is NULL", who);
+  if (G == 512) return windq::fail(ctx, WINDQ_ERR_ARG, "%s: G = 512 has no supported width 2 G", who);
+  return unit_features_batch_any(ctx, who, jobs, feat_out_2G, n_jobs, G, stream);
 }
 
 }  // extern "C"

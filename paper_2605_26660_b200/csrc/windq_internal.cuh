@@ -56,7 +56,7 @@ struct DeviceGuard {
 // attributes belong to a device, so the record is kept in the context, not in a process-wide static.
 enum KernelId { kFitG32 = 0, kApplyG32 = 5, kApplySearchG32 = 10, kHistG32 = 15, kFinalize = 20, kFitProtectG32 = 21, kApplyProtectG32 = 26, kApplyProtectSearchG32 = 31,
                 kFitBatchG32 = 41 /* 41..45 whole items, 46..50 in parts */, kApplyBatchG32 = 51 /* 51..55 */, kFitPartsOffset = 36 /* kFitG32 + 36 .. and kFitProtectG32 + 36 ..: the in-parts instantiations (36..40, 57..61) */,
-                kApplyStreamG32 = 64 /* 64..68 */, kFitFeatG32 = 79 /* 79..83 whole items, 84..88 in parts */, kTernarySearchG32 = 69 /* 69..73 plain, 74..78 protected */, kKernelIds = 128 };
+                kApplyStreamG32 = 64 /* 64..68 */, kFitFeatG32 = 79 /* 79..83 whole items, 84..88 in parts */, kTernarySearchG32 = 69 /* 69..73 plain, 74..78 protected */, kFinalize2 = 89, kKernelIds = 128 };
 inline int g_index(int G) { return G == 32 ? 0 : G == 64 ? 1 : G == 128 ? 2 : G == 256 ? 3 : 4; }
 
 // Sets the dynamic shared-memory limit of `kernel` once per context and, if asked, records how many

@@ -801,3 +801,35 @@ def test_features_fit_batch_equals_the_two_batched_calls(wq, ctx, oracle, G, sha
     torch.cuda.synchronize()
     for a, b in zip(feats, feats2):
         assert torch.equal(a[:, 1:], b[:, 1:])
+
+
+@pytest.mark.parametrize("G,shapes", [(64, [(300, 512), (64, 1024), (1000, 256)]), (128, [(40, 256), (2048, 2048)]),
+                                      (32, [(5, 64)]), (256, [(512, 2048), (33, 512)])])
+def test_unit_features_at_two_widths_from_one_pass(wq, ctx, oracle, G, shapes):
+    """windq_unit_features_batch2: the features at width 2 G come from pairs of the histograms built at width G; both
+    sets equal their own windq_unit_features_batch calls (histogram features and those of s bit for bit, the mean
+    within tolerance) and the oracle."""
+    Ws = [ws.weights(R, C, 600 + i, "student_t").cuda() for i, (R, C) in enumerate(shapes)]
+    for W in Ws:
+        W[::7, ::3] = 0
+    ss = [(torch.rand(C, generator=torch.Generator().manual_seed(i)) * 3 + 0.01).cuda() for i, (R, C) in enumerate(shapes)]
+    fine, wide = wq.windq_unit_features_batch(ctx, Ws, G, ss, feats_2G=True)
+    torch.cuda.synchronize()
+    ref_fine = wq.windq_unit_features_batch(ctx, Ws, G, ss)
+    ref_wide = wq.windq_unit_features_batch(ctx, Ws, 2 * G, ss)
+    torch.cuda.synchronize()
+    for W, s, f, f2, rf, rw in zip(Ws, ss, fine, wide, ref_fine, ref_wide):
+        assert torch.equal(f.view(torch.int32), rf.view(torch.int32))
+        assert torch.equal(f2[:, 1:].view(torch.int32), rw[:, 1:].view(torch.int32))
+        assert close(f2[:, 0].cpu().numpy(), rw[:, 0].cpu().numpy()).all()
+        want = oracle.unit_features(W.cpu().numpy(), 2 * G, s.cpu().numpy())
+        assert (f2[:, 3:5].cpu().numpy() == want[:, 3:5]).all() and close(f2.cpu().numpy(), want).all()
+    # a job may decline the wider units; an odd number of units is refused when any job asks for them
+    only_first = [True] + [None] * (len(Ws) - 1)
+    f_only, w_only = wq.windq_unit_features_batch(ctx, Ws, G, ss, feats_2G=[torch.empty_like(wide[0])] + only_first[1:])
+    torch.cuda.synchronize()
+    assert torch.equal(w_only[0], wide[0]) and all(x is None for x in w_only[1:])
+    odd = torch.zeros((8, 3 * G), dtype=torch.float16, device="cuda")
+    with pytest.raises(wq.WindqError) as e:
+        wq.windq_unit_features_batch(ctx, [odd], G, [torch.ones(3 * G, device="cuda")], feats_2G=[torch.zeros((1, 8), device="cuda")])
+    assert e.value.status == 2

@@ -255,6 +255,7 @@ class Buffers:
             shapes["err%d" % mi] = ((m.C // Gmin) * 6, torch.float32)
             shapes["energy%d" % mi] = (m.C // Gmin, torch.float32)
         self.clip_idx_m = [torch.empty(4 * (m.C // Gmin) * m.R, dtype=torch.uint8, device=dev) for m in mats]
+        self.lowbit_m = [torch.empty(3 * (m.C // Gmin) * m.R, dtype=torch.float16, device=dev) for m in mats]
         self.offsets_m = [[torch.empty(m.C // Gmin + 1, dtype=torch.int64, device=dev) for _ in TARGET_BITS] for m in mats]
         self.rings = {k: [torch.zeros(n, dtype=dt, device=dev) for _ in range(ring)] for k, (n, dt) in shapes.items()}
         self.turn = {k: 0 for k in shapes}
@@ -308,7 +309,7 @@ def jobs_slot(buf, name, ti):
     return (buf.turn[name] - len(TARGET_BITS) + ti) % buf.ring
 
 
-def apply_plans(wq, ctx, spec, m, mi, W, s, G, clip_idx, plans_b, buf, grid_d, sink, accounted=None):
+def apply_plans(wq, ctx, spec, m, mi, W, s, G, clip_idx, plans_b, buf, grid_d, sink, accounted=None, lowbit=None):
     """The three plans of one matrix: bit accounting (unless `accounted` = (totals, [code offsets per plan]) holds
     it already), then packing.  Returns the number of kernels launched."""
     U, launches = m.C // G, 0
@@ -320,7 +321,7 @@ def apply_plans(wq, ctx, spec, m, mi, W, s, G, clip_idx, plans_b, buf, grid_d, s
             jobs.append(dict(actions=plans_b[target][mi], code_offsets=accounted[1][ti], codes=buf.take("codes"),
                              scales=buf.take("scales")[:U * m.R].view(U, m.R), zeros=buf.take("zeros")[:U * m.R].view(U, m.R),
                              wq=buf.wq_multi[ti][:m.R * m.C].view(m.R, m.C)))
-        outs = wq.windq_apply_plan_multi(ctx, W, G, s, grid_d, clip_idx, jobs)
+        outs = wq.windq_apply_plan_multi(ctx, W, G, s, grid_d, clip_idx, jobs, lowbit=lowbit)
         if sink:
             for ti, target in enumerate(TARGET_BITS):
                 sink("codes", (outs[ti]["codes"], plans_b[target][mi], m.R, G), slot=jobs_slot(buf, "codes", ti))
@@ -379,7 +380,8 @@ def score_block(wq, ctx, spec, Wb, Xb, plans_b, buf, grid_d, timer=None, sink=No
                 launches += 2
             outs = [dict(err=buf.take("err%d" % mi)[:(m.C // G) * 6].view(m.C // G, 6),
                          energy=buf.take("energy%d" % mi)[:m.C // G],
-                         clip_idx=buf.clip_idx_m[mi][:4 * (m.C // G) * m.R].view(4, m.C // G, m.R))
+                         clip_idx=buf.clip_idx_m[mi][:4 * (m.C // G) * m.R].view(4, m.C // G, m.R),
+                         lowbit=buf.lowbit_m[mi][:3 * (m.C // G) * m.R].view(3, m.C // G, m.R) if (MULTI_APPLY and G == APPLY_G) else None)
                     for mi, m in enumerate(mats)]
             e0 = timer.start() if timer else None
             if FUSED_FEATURES:
@@ -410,7 +412,7 @@ def score_block(wq, ctx, spec, Wb, Xb, plans_b, buf, grid_d, timer=None, sink=No
                 launches += 1
                 for mi, m in enumerate(mats):
                     launches += apply_plans(wq, ctx, spec, m, mi, Wb[mi], buf.s[m.x_id], G, outs[mi]["clip_idx"], plans_b, buf,
-                                            grid_d, sink, accounted=(totals[mi], offs[mi]))
+                                            grid_d, sink, accounted=(totals[mi], offs[mi]), lowbit=outs[mi]["lowbit"])
         return launches
     for mi, m in enumerate(mats):
         W, s = Wb[mi], buf.s[m.x_id]

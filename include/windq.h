@@ -220,6 +220,9 @@ typedef struct {
   float* energy_out;      /* fp32 [U], nullable */
   uint8_t* clip_idx_out;  /* u8 [4][U][R], nullable */
   float* group_err_out;   /* fp32 [6][U][R], nullable */
+  void* lowbit_out;       /* fp16 [3][U][R], nullable: per group the 1.58-bit scale, the 1-bit scale and the 1.58-bit
+                             threshold 0.7 * mean|w| rounded towards zero to fp16 -- what windq_apply_plan_multi can
+                             take in place of forming the low-bit sums again (as it takes the clip indices) */
 } windq_fit_job;
 int64_t windq_scratch_bytes_fit_eval_batch(const windq_fit_job* jobs, int n_jobs, int G);
 windq_status windq_fit_eval_batch(windq_ctx* ctx, const windq_fit_job* jobs, int n_jobs, int G, const float* clip_grid,
@@ -246,6 +249,7 @@ typedef struct {
   float* energy_out;      /* fp32 [U], nullable */
   uint8_t* clip_idx_out;  /* u8 [4][U][R], nullable */
   float* group_err_out;   /* fp32 [6][U][R], nullable */
+  void* lowbit_out;       /* fp16 [3][U][R], nullable (see windq_fit_job) */
 } windq_featfit_job;
 int64_t windq_scratch_bytes_features_fit_batch(const windq_featfit_job* jobs, int n_jobs, int G);
 windq_status windq_features_fit_batch(windq_ctx* ctx, const windq_featfit_job* jobs, int n_jobs, int G,
@@ -298,6 +302,9 @@ windq_status windq_apply_plan(windq_ctx* ctx, const void* W, int64_t R, int64_t 
  * from memory once and quantised under each plan in turn.  Every plan is one windq_apply_plan call with clip
  * indices (clip_idx u8 [4][U][R] is required and shared by the plans): same meanings, layouts and results, bit
  * for bit.  Plans must not share output arrays; Wq_out may be NULL in any of them.
+ *   lowbit: fp16 [3][U][R] (device) or NULL: lowbit_out of windq_fit_eval_batch for the same W, s and G.  With it the
+ *           1.58- and 1-bit units take their scale (and threshold) from the table instead of forming the sums of the
+ *           fit again: same results, about a third less time on plans that are mostly low-bit.
  *   plans: HOST array of n_plans descriptors (1 <= n_plans <= 4), read during the call only. */
 typedef struct {
   const uint8_t* actions;       /* u8 [U] */
@@ -309,7 +316,7 @@ typedef struct {
 } windq_plan_out;
 windq_status windq_apply_plan_multi(windq_ctx* ctx, const void* W, int64_t R, int64_t C, int64_t ldw, int G,
                                     const float* s, const float* clip_grid, int K, const uint8_t* clip_idx,
-                                    const windq_plan_out* plans, int n_plans, void* stream);
+                                    const void* lowbit, const windq_plan_out* plans, int n_plans, void* stream);
 
 /* windq_apply_plan for several (matrix, plan) pairs in one launch.  Every job is one windq_apply_plan call with
  * clip indices (clip_idx is required here): same meanings, layouts and results, bit for bit.  All jobs share G,

@@ -90,7 +90,7 @@ def _load() -> ctypes.CDLL:
     lib.windq_scratch_bytes_greedy_allocate.restype = i64
     lib.windq_scratch_bytes_greedy_allocate.argtypes = [i64]
     lib.windq_apply_plan.argtypes = [vp, vp, i64, i64, i64, i32, vp, vp, i32, vp, vp, vp, vp, vp, vp, vp, vp]
-    lib.windq_apply_plan_multi.argtypes = [vp, vp, i64, i64, i64, i32, vp, vp, i32, vp, vp, i32, vp]
+    lib.windq_apply_plan_multi.argtypes = [vp, vp, i64, i64, i64, i32, vp, vp, i32, vp, vp, vp, i32, vp]
     lib.windq_apply_plan_searched.argtypes = [vp, vp, i64, i64, i64, i32, vp, vp, i32, vp, vp, vp, i32, vp, vp, vp, vp, vp, vp, vp]
     lib.windq_fit_ternary_search.argtypes = [vp, vp, i64, i64, i64, i32, vp, vp, i32, vp, vp, vp, vp, vp, vp]
     lib.windq_scratch_bytes_fit_ternary_search.argtypes = [i64, i64, i32]
@@ -400,14 +400,16 @@ def windq_unit_features_batch(ctx: Context, Ws, G: int, ss, feats=None, stream=N
 class _FitJob(ctypes.Structure):
     _fields_ = [("W", ctypes.c_void_p), ("R", ctypes.c_int64), ("C", ctypes.c_int64), ("ldw", ctypes.c_int64),
                 ("s", ctypes.c_void_p), ("err_out", ctypes.c_void_p), ("energy_out", ctypes.c_void_p),
-                ("clip_idx_out", ctypes.c_void_p), ("group_err_out", ctypes.c_void_p)]
+                ("clip_idx_out", ctypes.c_void_p), ("group_err_out", ctypes.c_void_p), ("lowbit_out", ctypes.c_void_p)]
 
 
 def windq_fit_eval_batch(ctx: Context, Ws, G: int, ss, clip_grid: torch.Tensor, *, want_energy: bool = True,
-                         want_clip_idx: bool = True, want_group_err: bool = False, outs=None, stream=None) -> list:
+                         want_clip_idx: bool = True, want_group_err: bool = False, want_lowbit: bool = False, outs=None,
+                         stream=None) -> list:
     """windq_fit_eval of up to 16 matrices in one launch.  ``Ws`` and ``ss`` are equally long sequences of weight
     matrices and their statistics; ``outs`` may hold one dict of preallocated outputs per matrix (keys as
-    windq_fit_eval).  Returns the list of output dicts."""
+    windq_fit_eval, and ``lowbit``: fp16 [3, U, R], the parameters of the two low-bit fits that
+    windq_apply_plan_multi can take).  Returns the list of output dicts."""
     if len(Ws) != len(ss) or not Ws:
         raise ValueError("Ws and ss must be non-empty and equally long")
     _need(clip_grid, torch.float32, "clip_grid", 1)
@@ -427,11 +429,16 @@ def windq_fit_eval_batch(ctx: Context, Ws, G: int, ss, clip_grid: torch.Tensor, 
             out["clip_idx"] = torch.empty((4, U, R), dtype=torch.uint8, device=dev)
         if want_group_err and out.get("group_err") is None:
             out["group_err"] = torch.empty((N_BITWIDTHS, U, R), dtype=torch.float32, device=dev)
-        for key in ("energy", "clip_idx", "group_err"):
+        if want_lowbit and out.get("lowbit") is None:
+            out["lowbit"] = torch.empty((3, U, R), dtype=torch.float16, device=dev)
+        for key in ("energy", "clip_idx", "group_err", "lowbit"):
             out.setdefault(key, None)
+        if out["lowbit"] is not None and (tuple(out["lowbit"].shape) != (3, U, R) or not out["lowbit"].is_contiguous()
+                                          or out["lowbit"].dtype != torch.float16):
+            raise ValueError("lowbit must be a contiguous fp16 [3, U, R] tensor")
         ptr = lambda x: None if x is None else x.data_ptr()
         jobs[j] = _FitJob(W.data_ptr(), R, C, ldw, s.data_ptr(), ptr(out["err"]), ptr(out["energy"]), ptr(out["clip_idx"]),
-                          ptr(out["group_err"]))
+                          ptr(out["group_err"]), ptr(out["lowbit"]))
         results.append(out)
     ctx._check(_lib.windq_fit_eval_batch(ctx._h, ctypes.cast(jobs, ctypes.c_void_p), len(Ws), int(G), _ptr(clip_grid),
                                          clip_grid.numel(), _stream(stream)))
@@ -702,10 +709,11 @@ class _PlanOut(ctypes.Structure):
 
 
 def windq_apply_plan_multi(ctx: Context, W: torch.Tensor, G: int, s: torch.Tensor, clip_grid: torch.Tensor,
-                           clip_idx: torch.Tensor, plans, *, stream=None) -> list:
+                           clip_idx: torch.Tensor, plans, *, lowbit: torch.Tensor | None = None, stream=None) -> list:
     """Up to four plans of one matrix in one pass over its weights.  ``plans``: a sequence of dicts with the keys
     actions, code_offsets, codes (uint8 output, sized by the caller) and optionally scales, zeros ([U, R] fp16) and
     wq ([R, C] fp16 with the row stride of W, or None for no fake-quantised output; absent = allocated).
+    ``lowbit`` (fp16 [3, U, R] from windq_fit_eval_batch(want_lowbit=True)) spares the low-bit units their sums.
     Returns one dict(codes, scales, zeros, wq) per plan."""
     R, C, ldw = _matrix(W, "W")
     _need(s, torch.float32, "s", 1)
@@ -714,6 +722,10 @@ def windq_apply_plan_multi(ctx: Context, W: torch.Tensor, G: int, s: torch.Tenso
     U = C // G if G > 0 else 0
     if tuple(clip_idx.shape) != (4, U, R) or not clip_idx.is_contiguous():
         raise ValueError("clip_idx must be a contiguous [4, U, R] tensor")
+    if lowbit is not None:
+        _need(lowbit, torch.float16, "lowbit", 3)
+        if tuple(lowbit.shape) != (3, U, R) or not lowbit.is_contiguous():
+            raise ValueError("lowbit must be a contiguous [3, U, R] tensor")
     if not plans:
         raise ValueError("plans must not be empty")
     arr = (_PlanOut * len(plans))()
@@ -739,7 +751,8 @@ def windq_apply_plan_multi(ctx: Context, W: torch.Tensor, G: int, s: torch.Tenso
                           None if wq_out is None else wq_out.data_ptr())
         results.append(dict(codes=codes, scales=scales, zeros=zeros, wq=wq_out))
     ctx._check(_lib.windq_apply_plan_multi(ctx._h, _ptr(W), R, C, ldw, int(G), _ptr(s), _ptr(clip_grid), clip_grid.numel(),
-                                           _ptr(clip_idx), ctypes.cast(arr, ctypes.c_void_p), len(plans), _stream(stream)))
+                                           _ptr(clip_idx), _ptr(lowbit), ctypes.cast(arr, ctypes.c_void_p), len(plans),
+                                           _stream(stream)))
     return results
 
 
@@ -817,7 +830,8 @@ def windq_apply_plan_searched(ctx: Context, W: torch.Tensor, G: int, s: torch.Te
 class _FeatFitJob(ctypes.Structure):
     _fields_ = [("W", ctypes.c_void_p), ("R", ctypes.c_int64), ("C", ctypes.c_int64), ("ldw", ctypes.c_int64),
                 ("s", ctypes.c_void_p), ("feat_out", ctypes.c_void_p), ("err_out", ctypes.c_void_p),
-                ("energy_out", ctypes.c_void_p), ("clip_idx_out", ctypes.c_void_p), ("group_err_out", ctypes.c_void_p)]
+                ("energy_out", ctypes.c_void_p), ("clip_idx_out", ctypes.c_void_p), ("group_err_out", ctypes.c_void_p),
+                ("lowbit_out", ctypes.c_void_p)]
 
 
 def _featfit_jobs(Ws, G, ss, feats, outs, want_energy, want_clip_idx, want_group_err):
@@ -845,7 +859,7 @@ def _featfit_jobs(Ws, G, ss, feats, outs, want_energy, want_clip_idx, want_group
             out.setdefault(key, None)
         ptr = lambda x: None if x is None else x.data_ptr()
         jobs[j] = _FeatFitJob(W.data_ptr(), R, C, ldw, s.data_ptr(), f.data_ptr(), ptr(out["err"]), ptr(out["energy"]),
-                              ptr(out["clip_idx"]), ptr(out["group_err"]))
+                              ptr(out["clip_idx"]), ptr(out["group_err"]), ptr(out.get("lowbit")))
         results.append(out)
         feat_list.append(f)
     return jobs, feat_list, results
@@ -855,7 +869,7 @@ def windq_scratch_bytes_features_fit_batch(Ws, G: int) -> int:
     jobs = (_FeatFitJob * len(Ws))()
     for j, W in enumerate(Ws):
         R, C, ldw = _matrix(W, "W")
-        jobs[j] = _FeatFitJob(W.data_ptr(), R, C, ldw, None, None, None, None, None, None)
+        jobs[j] = _FeatFitJob(W.data_ptr(), R, C, ldw, None, None, None, None, None, None, None)
     return int(_lib.windq_scratch_bytes_features_fit_batch(ctypes.cast(jobs, ctypes.c_void_p), len(Ws), int(G)))
 
 

@@ -638,7 +638,7 @@ static windq_status apply_plan_plain(windq_ctx* ctx, const void* W, int64_t R, i
   cudaStream_t st = (cudaStream_t)stream;
   if (clip_idx) {  // clip indices supplied: the streaming kernel
     const windq_plan_out pl = {actions, code_offsets, codes_out, scales_out, zeros_out, Wq_out};
-    return launch_apply_stream(ctx, G, W, R, C, ldw, s, clip_grid, K, clip_idx, scale_in, nullptr, 0, nullptr, &pl, 1, st);
+    return launch_apply_stream(ctx, G, W, R, C, ldw, s, clip_grid, K, clip_idx, scale_in, nullptr, 0, nullptr, nullptr, &pl, 1, st);
   }
   const __half* Wh = (const __half*)W;
   const long long* offs = (const long long*)code_offsets;

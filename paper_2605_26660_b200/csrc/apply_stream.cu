@@ -50,6 +50,7 @@ struct StreamArgs {
   const __half* scale_in;    // [4][U][R] or NULL: refined scales of the uniform groups
   const float* thr_grid;     // [thr_K] or NULL: threshold ratios of the ternary search
   const uint8_t* thr_idx;    // [U][R] or NULL
+  const __half* lowbit;      // [3][U][R] or NULL: 1.58-bit scale, 1-bit scale, 1.58-bit threshold, as the fit left them
   long long ldw;
   int R, U, K, thr_K, rows_blocks, n_plans;
   StreamPlan plan[kStreamMaxPlans];
@@ -491,11 +492,18 @@ apply_stream_kernel(const __grid_constant__ StreamArgs args) {
       } else if (a == 5) {
         const int thr_byte = (int)__shfl_sync(0xffffffffu, cur.thr, g * LG);
         const int kt = args.thr_idx ? min(thr_byte, args.thr_K - 1) : 0;  // an index beyond the grid means the last ratio
-        float delta;
-        const float alpha = stream_ternary_scale<G>(lane_buf, s_unit, q, thr_s[kt], delta);
+        float alpha;
+        __half2 delta2;  // |w| > delta, with |w| an fp16 value, is |w| > (delta rounded towards zero to fp16)
+        if (args.lowbit && !args.thr_idx) {  // scale and threshold as the fit left them
+          const unsigned o = (unsigned)(u * R + min(row, R - 1)), plane = (unsigned)(U * R);
+          alpha = __half2float(__ldg(args.lowbit + o));
+          delta2 = __half2half2(__ldg(args.lowbit + 2u * plane + o));
+        } else {
+          float delta;
+          alpha = stream_ternary_scale<G>(lane_buf, s_unit, q, thr_s[kt], delta);
+          delta2 = __half2half2(__float2half_rz(delta));
+        }
         const unsigned alpha2 = sh2_bits(__float2half2_rn(alpha));
-        // |w| > delta, with |w| an fp16 value, is |w| > (delta rounded towards zero to fp16)
-        const __half2 delta2 = __half2half2(__float2half_rz(delta));
         uint8_t* stage_row = stage + g * (G / 4);  // 2-bit fields, one per value
         __syncwarp();  // whoever used the staging area before has read it
 #pragma unroll
@@ -529,7 +537,8 @@ apply_stream_kernel(const __grid_constant__ StreamArgs args) {
         }
         scale_store = alpha;
       } else {
-        const float alpha = stream_binary_scale<G>(lane_buf, s_unit, q);
+        const float alpha = args.lowbit ? __half2float(__ldg(args.lowbit + (unsigned)(U * R) + (unsigned)(u * R + min(row, R - 1))))
+                                        : stream_binary_scale<G>(lane_buf, s_unit, q);
         const unsigned alpha2 = sh2_bits(__float2half2_rn(alpha));
         const __half2 zero2 = __float2half2_rn(0.0f);
         uint8_t* stage_row = stage + g * bpg;
@@ -571,7 +580,7 @@ static windq_status launch_stream_G(windq_ctx* ctx, StreamArgs& args, cudaStream
   if (windq_status rc = prepare_kernel(ctx, id, apply_stream_kernel<G>, kStreamWarps * 32, smem, true)) return rc;
   args.rows_blocks = (args.R + GPW - 1) / GPW;
   const int64_t n_items = (int64_t)args.U * args.rows_blocks;
-  WINDQ_REQUIRE(ctx, n_items < (1ll << 30) && (int64_t)args.R * args.ldw < (1ll << 31) && 4ll * args.U * args.R < (1ll << 31),
+  WINDQ_REQUIRE(ctx, n_items < (1ll << 30) && (int64_t)args.R * args.ldw < (1ll << 31) && 4ll * args.U * args.R < (1ll << 31),  /* clip indices [4][U][R], low-bit table [3][U][R] */
                 WINDQ_ERR_SHAPE, "windq_apply_plan: R * ldw must be below 2^31 for one call with clip indices");
   int64_t grid = (int64_t)ctx->sm_count * ctx->occupancy[id];
   const int64_t need = (n_items + kStreamWarps - 1) / kStreamWarps;
@@ -584,8 +593,8 @@ static windq_status launch_stream_G(windq_ctx* ctx, StreamArgs& args, cudaStream
 // One matrix, n_plans plans, clip indices supplied.  Arguments have been checked by the caller.
 windq_status launch_apply_stream(windq_ctx* ctx, int G, const void* W, int64_t R, int64_t C, int64_t ldw, const float* s,
                                  const float* clip_grid, int K, const uint8_t* clip_idx, const void* scale_in,
-                                 const float* thr_grid, int thr_K, const uint8_t* thr_idx, const windq_plan_out* plans,
-                                 int n_plans, cudaStream_t st) {
+                                 const float* thr_grid, int thr_K, const uint8_t* thr_idx, const void* lowbit,
+                                 const windq_plan_out* plans, int n_plans, cudaStream_t st) {
   StreamArgs args;
   memset(&args, 0, sizeof(args));
   args.W = (const __half*)W;
@@ -595,6 +604,7 @@ windq_status launch_apply_stream(windq_ctx* ctx, int G, const void* W, int64_t R
   args.scale_in = (const __half*)scale_in;
   args.thr_grid = thr_grid;
   args.thr_idx = thr_idx;
+  args.lowbit = (const __half*)lowbit;
   args.ldw = ldw;
   args.R = (int)R;
   args.U = (int)(C / G);
@@ -634,7 +644,7 @@ static windq_status check_plan(windq_ctx* ctx, const char* who, int p, const win
 
 extern "C" windq_status windq_apply_plan_multi(windq_ctx* ctx, const void* W, int64_t R, int64_t C, int64_t ldw, int G,
                                                const float* s, const float* clip_grid, int K, const uint8_t* clip_idx,
-                                               const windq_plan_out* plans, int n_plans, void* stream) {
+                                               const void* lowbit, const windq_plan_out* plans, int n_plans, void* stream) {
   using namespace windq;
   const char* who = "windq_apply_plan_multi";
   if (!ctx) return fail(nullptr, WINDQ_ERR_NULL, "%s: ctx is NULL", who);
@@ -651,8 +661,9 @@ extern "C" windq_status windq_apply_plan_multi(windq_ctx* ctx, const void* W, in
                              plans[p].zeros_out != plans[o].zeros_out && (plans[p].Wq_out == nullptr || plans[p].Wq_out != plans[o].Wq_out),
                     WINDQ_ERR_ARG, "%s: plans %d and %d share an output array", who, o, p);
   }
+  WINDQ_REQUIRE(ctx, ((uintptr_t)lowbit & 1) == 0, WINDQ_ERR_ALIGN, "%s: lowbit is misaligned", who);
   DeviceGuard guard(ctx->device);
-  return launch_apply_stream(ctx, G, W, R, C, ldw, s, clip_grid, K, clip_idx, nullptr, nullptr, 0, nullptr, plans, n_plans,
+  return launch_apply_stream(ctx, G, W, R, C, ldw, s, clip_grid, K, clip_idx, nullptr, nullptr, 0, nullptr, lowbit, plans, n_plans,
                              (cudaStream_t)stream);
 }
 
@@ -673,6 +684,6 @@ extern "C" windq_status windq_apply_plan_searched(windq_ctx* ctx, const void* W,
   const windq_plan_out pl = {actions, code_offsets, codes_out, scales_out, zeros_out, Wq_out};
   if (windq_status st = check_plan(ctx, who, 0, pl, W)) return st;
   DeviceGuard guard(ctx->device);
-  return launch_apply_stream(ctx, G, W, R, C, ldw, s, clip_grid, K, clip_idx, nullptr, thr_grid, thr_K, thr_idx, &pl, 1,
+  return launch_apply_stream(ctx, G, W, R, C, ldw, s, clip_grid, K, clip_idx, nullptr, thr_grid, thr_K, thr_idx, nullptr, &pl, 1,
                              (cudaStream_t)stream);
 }

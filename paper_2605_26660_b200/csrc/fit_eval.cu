@@ -39,6 +39,7 @@ struct FitJobs {
   float* group_err[kFitMaxJobs];
   float* err[kFitMaxJobs];
   float* energy[kFitMaxJobs];
+  __half* lowbit[kFitMaxJobs];  // [3][U][R]: 1.58-bit scale, 1-bit scale, 1.58-bit threshold (rounded towards zero), or NULL
   long long ldw[kFitMaxJobs];
   int R[kFitMaxJobs];
   int U[kFitMaxJobs];
@@ -196,6 +197,16 @@ fit_eval_kernel(const __half* __restrict__ W_one, int R_one, int U_one, int64_t 
       if (live && q == 0 && group_err_out) {
         group_err_out[((int64_t)4 * U + u) * R + row] = low.err_t;
         group_err_out[((int64_t)5 * U + u) * R + row] = low.err_b;
+      }
+      if (BATCH) {
+        // the parameters of the two low-bit fits, for a plan application that wants to skip their sums
+        __half* lb = jobs.lowbit[jfeat];
+        if (lb && live && q == 0) {
+          const int64_t o = (int64_t)u * R + row, plane = (int64_t)U * R;
+          lb[o] = __float2half_rn(low.alpha_t);               // exact: the value of an fp16 number
+          lb[plane + o] = __float2half_rn(low.alpha_b);
+          lb[2 * plane + o] = __float2half_rz(low.delta);      // |w| > delta for an fp16 |w| is |w| > this
+        }
       }
     }
 
@@ -445,6 +456,8 @@ static windq_status fit_batch_any(windq_ctx* ctx, const char* who, const windq_f
     fj.group_err[j] = b.group_err_out;
     fj.err[j] = b.err_out;
     fj.energy[j] = b.energy_out;
+    fj.lowbit[j] = (__half*)b.lowbit_out;
+    WINDQ_REQUIRE(ctx, ((uintptr_t)b.lowbit_out & 1) == 0, WINDQ_ERR_ALIGN, "%s: job %d: lowbit_out is misaligned", who, j);
     fj.ldw[j] = b.ldw;
     fj.R[j] = (int)b.R;
     fj.U[j] = (int)(b.C / G);
@@ -535,6 +548,7 @@ windq_status windq_features_fit_batch(windq_ctx* ctx, const windq_featfit_job* j
     fit[j].energy_out = jobs[j].energy_out;
     fit[j].clip_idx_out = jobs[j].clip_idx_out;
     fit[j].group_err_out = jobs[j].group_err_out;
+    fit[j].lowbit_out = jobs[j].lowbit_out;
     feat[j] = jobs[j].feat_out;
     if (!feat[j]) return windq::fail(ctx, WINDQ_ERR_NULL, "%s: job %d: feat_out is NULL", who, j);
   }

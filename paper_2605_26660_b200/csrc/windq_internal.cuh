@@ -85,12 +85,12 @@ windq_status check_matrix(windq_ctx* ctx, const char* who, const void* W, int64_
 // The clip grid lives on the device and is used as given; only K can be checked on the host.
 windq_status check_K(windq_ctx* ctx, const char* who, int K);
 
-// The streaming plan kernel (apply_stream.cu): one matrix, n_plans plans, clip indices supplied; scale_in, thr_grid
-// and thr_idx may be NULL.  Arguments must have been checked.
+// The streaming plan kernel (apply_stream.cu): one matrix, n_plans plans, clip indices supplied; scale_in, thr_grid,
+// thr_idx and lowbit may be NULL.  Arguments must have been checked.
 windq_status launch_apply_stream(windq_ctx* ctx, int G, const void* W, int64_t R, int64_t C, int64_t ldw, const float* s,
                                  const float* clip_grid, int K, const uint8_t* clip_idx, const void* scale_in,
-                                 const float* thr_grid, int thr_K, const uint8_t* thr_idx, const windq_plan_out* plans,
-                                 int n_plans, cudaStream_t st);
+                                 const float* thr_grid, int thr_K, const uint8_t* thr_idx, const void* lowbit,
+                                 const windq_plan_out* plans, int n_plans, cudaStream_t st);
 
 // The state features of every unit of n_jobs matrices from per-unit histograms of |w| bit patterns (32768 bins each,
 // units of all jobs in a row) and per-unit sums of w, as the fused fit pass leaves them (unit_features.cu).

@@ -126,3 +126,43 @@ def test_multi_argument_checks(wq, ctx):
     out = wq.windq_apply_plan_multi(ctx, W, 128, s, gd, idx, [plan(), plan()])
     torch.cuda.synchronize()
     assert out[0]["wq"] is None and bool((out[0]["codes"][:2048] == 0).all())
+
+
+@pytest.mark.parametrize("G,shapes", [(128, [(300, 1024), (1100, 512)]), (64, [(133, 512), (40, 256)]), (32, [(200, 256)]),
+                                      (256, [(19, 2048)]), (512, [(67, 1024)])])
+def test_low_bit_parameters_from_the_fit_give_the_same_plans(wq, ctx, oracle, G, shapes):
+    """windq_fit_eval_batch can leave the scales (and the 1.58-bit threshold) of its two low-bit fits in a table that
+    windq_apply_plan_multi takes in place of forming the sums again: every output equals the call without the table,
+    and the table's scales are the oracle's."""
+    grid = ws.clip_grid(20)
+    gd = torch.from_numpy(grid).cuda()
+    Ws = [ws.weights(R, C, 860 + i, "student_t").cuda() for i, (R, C) in enumerate(shapes)]
+    for W in Ws:
+        W[::5, :G] = 0                              # some all-zero groups (empty support)
+    ss = [(torch.rand(C, generator=torch.Generator().manual_seed(i)) * 3).cuda() for i, (R, C) in enumerate(shapes)]
+    for s in ss:
+        s[G // 2:G] = 0                             # and groups whose support may carry no activation weight
+    fits = wq.windq_fit_eval_batch(ctx, Ws, G, ss, gd, want_lowbit=True)
+    rng = np.random.default_rng(G)
+    for W, s, fit in zip(Ws, ss, fits):
+        R, C = W.shape
+        U = C // G
+        plans_a, plans_b, acts_np = [], [], []
+        for p in range(3):
+            acts = rng.choice([5, 6, 5, 6, 4, 0, 2], U).astype(np.uint8)
+            acts_np.append(acts)
+            a_d = torch.from_numpy(acts).cuda()
+            eb = wq.windq_effective_bits(ctx, a_d, R, G)
+            n = int(eb["code_offsets"][-1].item())
+            for plans in (plans_a, plans_b):
+                plans.append(dict(actions=a_d, code_offsets=eb["code_offsets"], codes=torch.full((n,), 0xEE, dtype=torch.uint8, device="cuda")))
+        with_table = wq.windq_apply_plan_multi(ctx, W, G, s, gd, fit["clip_idx"], plans_a, lowbit=fit["lowbit"])
+        without = wq.windq_apply_plan_multi(ctx, W, G, s, gd, fit["clip_idx"], plans_b)
+        torch.cuda.synchronize()
+        for a, b in zip(with_table, without):
+            for k in ("codes", "scales", "zeros", "wq"):
+                assert torch.equal(a[k].view(torch.uint8), b[k].view(torch.uint8)), k
+        want = oracle.apply_plan(W.cpu().numpy(), G, s.cpu().numpy(), grid, np.full(U, 5, np.uint8), fit["clip_idx"].cpu().numpy())
+        assert np.array_equal(u16(fit["lowbit"][0]), want["scales"])
+        want = oracle.apply_plan(W.cpu().numpy(), G, s.cpu().numpy(), grid, np.full(U, 6, np.uint8), fit["clip_idx"].cpu().numpy())
+        assert np.array_equal(u16(fit["lowbit"][1]), want["scales"])

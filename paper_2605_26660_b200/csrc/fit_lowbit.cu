@@ -4,8 +4,8 @@
 // caller's threshold ratios one after the other, each fitted and scored exactly like the single threshold of
 // windq_fit_eval, and keeps the first of the least error.
 //
-// Bound by the FP32 pipes like the other fits: per threshold ratio about 10 binary32 operations per weight (the
-// support sums, then the error with the scale those sums give).  Same layout: LG = G / 32 lanes per group hold 32
+// Bound by the FP32 pipes like the other fits: per threshold ratio six packed binary32 operations and four
+// comparisons per pair of weights (the support sums, then the error with the scale those sums give).  Same layout: LG = G / 32 lanes per group hold 32
 // magnitudes and 32 statistics in registers, one warp per item of GPW rows of a unit, persistent grid, items
 // claimed from a counter; sums in PSUM8 order, so thresholds, scales and group errors are reproducible bit for bit.
 #include "fit_device.cuh"
@@ -74,22 +74,22 @@ fit_ternary_search_kernel(const __half* __restrict__ W, int R, int U, int64_t ld
 #pragma unroll 1
     for (int k = 0; k < Kt; ++k) {
       const float delta = __fmul_rn(thr_s[k], meanA);
-      // support sums, weighted by s
-      float Bt[4], Ct[4];
+      // support sums, weighted by s.  The support enters as a factor m = 1 or 0 per weight: s (|w| m) and s m are
+      // exact products of the terms the definition adds, so the sums round as they do there; leaves 2 h and
+      // 2 h + 1 run side by side in the two halves of the packed operations.
+      const float2 zero2 = make_float2(0.0f, 0.0f);
+      float2 bt[2] = {zero2, zero2}, ct[2] = {zero2, zero2};
 #pragma unroll
-      for (int l = 0; l < 4; ++l) {
-        float bt = 0.0f, ct = 0.0f;
+      for (int h = 0; h < 2; ++h)
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
-          const float aw = av.get(l, i), sj = sv.get(l, i);
-          const bool in = aw > delta;
-          bt = __fmaf_rn(sj, in ? aw : 0.0f, bt);
-          ct = __fadd_rn(ct, in ? sj : 0.0f);
+          const float2 aw = av.v[h][i], sj = sv.v[h][i];
+          const float2 m = make_float2(aw.x > delta ? 1.0f : 0.0f, aw.y > delta ? 1.0f : 0.0f);
+          bt[h] = fma2(sj, mul2(aw, m), bt[h]);
+          ct[h] = fma2(sj, m, ct[h]);
         }
-        Bt[l] = bt; Ct[l] = ct;
-      }
-      float sumBt = group_tree<G>(Bt[0], Bt[1], Bt[2], Bt[3]);
-      float sumCt = group_tree<G>(Ct[0], Ct[1], Ct[2], Ct[3]);
+      float sumBt = group_tree<G>(bt[0], bt[1]);
+      float sumCt = group_tree<G>(ct[0], ct[1]);
       // a weighted sum of zero: no activation weight on the support, or no support at all; the unweighted sums
       // decide which, and give the scale in the first case
       bool nonempty = some;
@@ -118,19 +118,19 @@ fit_ternary_search_kernel(const __half* __restrict__ W, int R, int U, int64_t ld
       const float alpha = nonempty ? __half2float(__float2half_rn(__fdiv_rn(sumBt, sumCt))) : 0.0f;
       // error: the difference between the reconstruction and the weight has the magnitude |alpha - |w|| on the
       // support and |w| off it; its sign does not matter to (s d) d, and rounding is symmetric in sign
-      float Et[4];
+      // (m alpha is alpha or 0 exactly, so |w| - m alpha rounds once, like the difference itself)
+      const float2 nalpha2 = make_float2(-alpha, -alpha);
+      float2 et[2] = {zero2, zero2};
 #pragma unroll
-      for (int l = 0; l < 4; ++l) {
-        float et = 0.0f;
+      for (int h = 0; h < 2; ++h)
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
-          const float aw = av.get(l, i), sj = sv.get(l, i);
-          const float d = __fsub_rn(aw > delta ? alpha : 0.0f, aw);
-          et = __fmaf_rn(__fmul_rn(sj, d), d, et);
+          const float2 aw = av.v[h][i];
+          const float2 m = make_float2(aw.x > delta ? 1.0f : 0.0f, aw.y > delta ? 1.0f : 0.0f);
+          const float2 d = fma2(m, nalpha2, aw);
+          et[h] = fma2(mul2(sv.v[h][i], d), d, et[h]);
         }
-        Et[l] = et;
-      }
-      const float e = group_tree<G>(Et[0], Et[1], Et[2], Et[3]);
+      const float e = group_tree<G>(et[0], et[1]);
       if (e < best_e) {
         best_e = e;
         best_k = k;

@@ -5,7 +5,7 @@
     python bench.py --impl reference --steps K --warmup W    # the CPU oracle, as it stands
 
 A step is one pass of the whole hot path over a LLaMA-7B-shaped model of synthetic weights and
-calibration activations (32 decoder blocks; see windq_synth.CONFIGS): per block 4 x act_stats;
+calibration activations (32 decoder blocks; see windq_synth.CONFIGS): per block act_stats of its inputs;
 per matrix and chunk width (64, 128) unit_features + fit_eval over every unit; then, at chunk
 width 128, effective_bits + apply_plan for three seeded random plans (1.58, 2.0, 3.0 bits).
 The metric is unit x bit-width candidate evaluations per second (6 per unit and chunk width).
@@ -357,9 +357,9 @@ def score_block(wq, ctx, spec, Wb, Xb, plans_b, buf, grid_d, timer=None, sink=No
     receives every result (the e2e leg copies them to the host)."""
     launches = 0
     mats = matrices_of(spec)
-    for i, X in Xb.items():
-        wq.windq_act_stats(ctx, X, buf.s[i])
-        launches += 2
+    ids = sorted(Xb)
+    wq.windq_act_stats_batch(ctx, [Xb[i] for i in ids], [buf.s[i] for i in ids])
+    launches += 1
     if BATCH_FITS:
         # chunk widths G and 2 G: the features of both come out of one pass at G (windq_unit_features_batch2)
         nested = (not FUSED_FEATURES and len(spec.chunk_widths) == 2 and spec.chunk_widths[1] == 2 * spec.chunk_widths[0]

@@ -93,6 +93,21 @@ int64_t windq_scratch_bytes_fit_eval(int64_t R, int64_t C, int G);
 windq_status windq_act_stats(windq_ctx* ctx, const void* X, int64_t T, int64_t C, int64_t ldx,
                              float* s_out, void* stream);
 
+/* windq_act_stats for several calibration inputs in one launch (the paper has no counterpart: a decoder block has
+ * a handful of distinct inputs of a few tens of megabytes, each too short a read to amortise a launch of its own).
+ * Every job is one windq_act_stats call -- X, T, C, ldx, s_out as there -- and gives the same bits.
+ *   jobs: HOST array of n_jobs descriptors (1 <= n_jobs <= WINDQ_MAX_ACT_JOBS), read during the call only.
+ * The channels of all jobs together may number at most 4 194 304.
+ * Scratch: windq_scratch_bytes_act_stats_batch (the sum of the jobs' windq_scratch_bytes_act_stats). */
+#define WINDQ_MAX_ACT_JOBS 16
+typedef struct {
+  const void* X;  /* fp16 [T][ldx] */
+  int64_t T, C, ldx;
+  float* s_out;   /* fp32 [C] */
+} windq_act_job;
+int64_t windq_scratch_bytes_act_stats_batch(const windq_act_job* jobs, int n_jobs);
+windq_status windq_act_stats_batch(windq_ctx* ctx, const windq_act_job* jobs, int n_jobs, void* stream);
+
 /* Variant of windq_act_stats that allocates nothing.  (The paper has no counterpart: this entry
  * point exists for the sake of callers, not of the method.)
  *

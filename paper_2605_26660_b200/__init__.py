@@ -55,6 +55,9 @@ def _load() -> ctypes.CDLL:
         getattr(lib, name).restype = i64
     lib.windq_act_stats.argtypes = [vp, vp, i64, i64, i64, vp, vp]
     lib.windq_act_stats_noalloc.argtypes = [vp, vp, i64, i64, i64, vp, vp]
+    lib.windq_act_stats_batch.argtypes = [vp, vp, i32, vp]
+    lib.windq_scratch_bytes_act_stats_batch.restype = i64
+    lib.windq_scratch_bytes_act_stats_batch.argtypes = [vp, i32]
     lib.windq_unit_features.argtypes = [vp, vp, i64, i64, i64, i32, vp, vp, vp]
     lib.windq_fit_eval.argtypes = [vp, vp, i64, i64, i64, i32, vp, vp, i32, vp, vp, vp, vp, vp]
     lib.windq_apply_plan_batch.argtypes = [vp, vp, i32, i32, vp, i32, vp]
@@ -199,6 +202,43 @@ def windq_act_stats(ctx: Context, X: torch.Tensor, s_out: torch.Tensor | None = 
     _need(s_out, torch.float32, "s_out", 1)
     ctx._check(_lib.windq_act_stats(ctx._h, _ptr(X), T, C, ldx, _ptr(s_out), _stream(stream)))
     return s_out
+
+
+MAX_ACT_JOBS = 16   # WINDQ_MAX_ACT_JOBS of the header
+
+
+class _ActJob(ctypes.Structure):
+    _fields_ = [("X", ctypes.c_void_p), ("T", ctypes.c_int64), ("C", ctypes.c_int64), ("ldx", ctypes.c_int64),
+                ("s_out", ctypes.c_void_p)]
+
+
+def windq_act_stats_batch(ctx: Context, Xs, s_outs=None, stream=None):
+    """windq_act_stats of up to 16 inputs in one launch.  ``s_outs`` may hold one preallocated fp32 [C] tensor
+    per input.  Returns the list of statistics."""
+    if not Xs:
+        raise ValueError("Xs must be non-empty")
+    if s_outs is not None and len(s_outs) != len(Xs):
+        raise ValueError("s_outs must have one entry per input")
+    jobs = (_ActJob * len(Xs))()
+    outs = []
+    for j, X in enumerate(Xs):
+        T, C, ldx = _matrix(X, "X")
+        s = s_outs[j] if s_outs is not None else torch.empty(C, dtype=torch.float32, device=X.device)
+        _need(s, torch.float32, "s_out", 1)
+        if s.numel() < C:
+            raise ValueError("s_out must have at least C entries")
+        jobs[j] = _ActJob(X.data_ptr(), T, C, ldx, s.data_ptr())
+        outs.append(s)
+    ctx._check(_lib.windq_act_stats_batch(ctx._h, ctypes.cast(jobs, ctypes.c_void_p), len(Xs), _stream(stream)))
+    return outs
+
+
+def windq_scratch_bytes_act_stats_batch(shapes) -> int:
+    """Scratch of a windq_act_stats_batch call over inputs of the given (T, C) shapes."""
+    jobs = (_ActJob * len(shapes))()
+    for j, (T, C) in enumerate(shapes):
+        jobs[j] = _ActJob(None, int(T), int(C), int(C), None)
+    return int(_lib.windq_scratch_bytes_act_stats_batch(ctypes.cast(jobs, ctypes.c_void_p), len(shapes)))
 
 
 NOALLOC_SCRATCH_BYTES = 4 * 1024 * 1024   # WINDQ_NOALLOC_SCRATCH_BYTES of the header

@@ -85,8 +85,19 @@ windq_status windq_create(windq_ctx** out, int device) {
   if (prop.major != 10)
     return windq::fail(nullptr, WINDQ_ERR_UNSUPPORTED, "windq_create: device %d is sm_%d%d, this library is built for sm_100a",
                        device, prop.major, prop.minor);
+  unsigned int* sync = nullptr;
+  {
+    windq::DeviceGuard guard(device);
+    if (cudaMalloc(&sync, windq::kSyncCounters * sizeof(unsigned int)) != cudaSuccess ||
+        cudaMemset(sync, 0, windq::kSyncCounters * sizeof(unsigned int)) != cudaSuccess) {
+      cudaGetLastError();
+      if (sync) cudaFree(sync);
+      return windq::fail(nullptr, WINDQ_ERR_CUDA, "windq_create: cannot allocate the arrival counters on device %d", device);
+    }
+  }
   windq_ctx* ctx = new windq_ctx;
   ctx->device = device;
+  ctx->sync = sync;
   ctx->sm_count = prop.multiProcessorCount;
   ctx->scratch = nullptr;
   ctx->scratch_bytes = 0;
@@ -101,10 +112,9 @@ void windq_destroy(windq_ctx* ctx) {
   if (!ctx) return;
   {
     windq::DeviceGuard guard(ctx->device);
-    if (ctx->scratch) {
-      cudaDeviceSynchronize();
-      cudaFree(ctx->scratch);
-    }
+    cudaDeviceSynchronize();
+    if (ctx->scratch) cudaFree(ctx->scratch);
+    cudaFree(ctx->sync);
   }
   delete ctx;
 }

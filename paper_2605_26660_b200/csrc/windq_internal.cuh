@@ -14,12 +14,15 @@ struct windq_ctx {
   int sm_count;
   void* scratch;
   int64_t scratch_bytes;
+  unsigned int* sync;  // kSyncCounters arrival counters, zero between launches
   unsigned long long prepared[2];  // kernels whose attributes have been set on this context's device (bit per KernelId)
   int occupancy[128];              // resident blocks per SM of those kernels (0 where not asked)
   char err[256];
 };
 
 namespace windq {
+
+constexpr int64_t kSyncCounters = 16384;
 
 windq_status fail(windq_ctx* ctx, windq_status st, const char* fmt, ...);
 // Makes the context's scratch at least `bytes` large (may cudaMalloc).

@@ -75,6 +75,39 @@ def test_act_stats_strided_rows(wq, ctx, oracle):
     assert close(got.cpu().numpy(), oracle.act_stats(X.numpy())).all()
 
 
+def test_act_stats_batch(wq, ctx, oracle):
+    """Several inputs of different shapes in one launch: the oracle's values, the bits of the separate calls,
+    nothing written past an output, and the same again on a second call (the arrival
+    counters are back at zero)."""
+    shapes = [(300, 11008), (77, 264), (1, 8), (512, 4096), (65, 1000), (1100, 28672)]
+    Xs = [ws.activations(T, C, 700 + j) for j, (T, C) in enumerate(shapes)]
+    tiny = torch.randint(1, 1024, (70, 64), generator=torch.Generator().manual_seed(5), dtype=torch.int16)
+    Xs.append((tiny | (tiny << 15)).view(torch.float16))      # subnormal fp16 values of both signs: nothing is flushed
+    shapes.append((70, 64))
+    Xd = [X.cuda() for X in Xs]
+    wide = torch.zeros((65, 1280), dtype=torch.float16, device="cuda")     # a strided view as one of the jobs
+    wide[:, :1000] = Xd[4]
+    Xd[4] = wide[:, :1000]
+    pairs = [guarded((C,), torch.float32) for _, C in shapes]
+    for rep in range(2):
+        for out, _ in pairs:
+            out.fill_(-1.0)
+        wq.windq_act_stats_batch(ctx, Xd, [out for out, _ in pairs])
+        torch.cuda.synchronize()
+        for (out, intact), X, Xg in zip(pairs, Xs, Xd):
+            assert intact()
+            assert close(out.cpu().numpy(), oracle.act_stats(X.numpy())).all()
+            assert torch.equal(out, wq.windq_act_stats(ctx, Xg))
+            assert close(wq.windq_act_stats_noalloc(ctx, Xg, torch.empty_like(out)).cpu().numpy(), oracle.act_stats(X.numpy())).all()
+    # the subnormal input on its own terms (its statistics are far below the absolute tolerance above)
+    assert np.allclose(pairs[-1][0].cpu().numpy(), oracle.act_stats(Xs[-1].numpy()), rtol=1e-5, atol=0.0)
+    assert wq.windq_scratch_bytes_act_stats_batch(shapes) == sum(wq.windq_scratch_bytes_act_stats(T, C) for T, C in shapes)
+    with pytest.raises(wq.WindqError):
+        wq.windq_act_stats_batch(ctx, [Xd[0]] * 17)
+    with pytest.raises(wq.WindqError):
+        wq.windq_act_stats_batch(ctx, [Xd[0], torch.zeros((4, 12), dtype=torch.float16, device="cuda")])
+
+
 # ------------------------------------------------------------------ unit_features
 @pytest.mark.parametrize("R,C,G", [(300, 512, 128), (64, 256, 32), (1000, 1024, 512), (97, 256, 64), (4096, 512, 256)])
 def test_unit_features(wq, ctx, oracle, R, C, G):

@@ -787,8 +787,10 @@ def main():
     evals_per_step = 6 * sum(units.values())
     job_evals = evals_per_step if strong else world * evals_per_step   # what all ranks together score in a step
     elems_rank, _ = workload_counts(spec, len(blocks))               # what this rank's fits read
+    wq.windq_fit_work(ctx, reset=True)
     ms, launches, fit_ms, clocks = run_device_leg(wq, ctx, spec, model, plans, plan_index, buf, grid_d, args.steps, args.warmup,
                                                   local_rank, sync)
+    evaluated, searched = wq.windq_fit_work(ctx, reset=True)      # clip candidates the fits evaluated in full / all of them
     ms = sharding.max_float(ms)
     value = job_evals * args.steps / (ms * 1e-3)
 
@@ -815,6 +817,13 @@ def main():
                     weight_gbs=2.0 * fit_elem / (fit_ms * 1e-3) / 1e9, hbm_frac=hbm_time / (fit_ms * 1e-3),
                     elem_cand_per_s=fit_elem * (4 * spec.K + 2) / (fit_ms * 1e-3),
                     peak_source="%d SMs x 128 lanes x %.0f MHz (%s)" % (sm_count, peaks["sm_max_mhz"], peaks["source"]))
+    # `frac` credits the search with all its candidates (the count the method defines).  The eight-bit search skips
+    # candidates that provably cannot win; what the kernel executed is the evaluated share of the 28 K operations,
+    # the ten once per weight, and the bound of the eight-bit candidates (seven operations on two of a lane's 32 weights)
+    share = evaluated / max(1, searched)
+    ops_executed = 28 * spec.K * share + 10 + 7 * spec.K / 16.0
+    roofline["executed"] = dict(candidates_evaluated_share=share, ops_per_element=ops_executed,
+                                frac=fit_elem * ops_executed / (fit_ms * 1e-3) / 1e12 / alu_peak)
 
     e2e = None
     if not args.no_e2e:

@@ -79,6 +79,15 @@ const char* windq_last_error(const windq_ctx* ctx);
  * the number of values for which they do not: 0 on every GPU this library supports. */
 windq_status windq_selfcheck(windq_ctx* ctx, int64_t* n_failures_out, void* stream);
 
+/* How much of the clip search the fits skipped (the paper has no counterpart; a measurement aid).  The eight-bit
+ * search of windq_fit_eval and its variants leaves out candidates that provably cannot win (the error of a group
+ * is at least the error term of any one of its weights; see windq_fit_eval), so the work of a fit depends on the
+ * data.  Every fit kernel of the context adds to two counters: the clip candidates of its searches, counted once
+ * per warp pass (a pass covers the 1024 weights a warp holds), and those of them it evaluated in full.
+ *   evaluated_out, searched_out: HOST pointers to one int64 each; reset != 0 puts both counters back to zero.
+ * Synchronises the device (a blocking copy). */
+windq_status windq_fit_work(windq_ctx* ctx, int64_t* evaluated_out, int64_t* searched_out, int reset);
+
 /* Grows the context's scratch buffer to at least `bytes` now (synchronises the device), so that
  * later calls do not allocate.  windq_scratch_bytes_* tell how much a call will need. */
 windq_status windq_reserve(windq_ctx* ctx, int64_t bytes);
@@ -166,7 +175,12 @@ windq_status windq_unit_features(windq_ctx* ctx, const void* W, int64_t R, int64
  *   clip_idx_out u8   [4][U][R]  best clip index for 8, 4, 3, 2 bit; nullable
  *   group_err_out fp32 [6][U][R] best error of every group; nullable
  * clip_grid: fp32 [K] (device).  Group-level results (clip indices, group errors) are
- * bit-reproducible: every operation is a fixed IEEE binary32 sequence. */
+ * bit-reproducible: every operation is a fixed IEEE binary32 sequence.
+ * s must be >= 0 (it is a mean of squares).  The eight-bit search relies on it: every term s_j d_j^2 of an error is
+ * then >= 0 and rounding is monotone, so the error of a candidate is at least the term of any single weight, and
+ * a candidate for which the term of a group's least or greatest weight already exceeds the least error found is
+ * skipped without changing any result (windq_fit_work tells how many were).  With negative s the results are
+ * unspecified, like those of non-finite input. */
 windq_status windq_fit_eval(windq_ctx* ctx, const void* W, int64_t R, int64_t C, int64_t ldw, int G,
                             const float* s, const float* clip_grid, int K, float* err_out,
                             float* energy_out, uint8_t* clip_idx_out, float* group_err_out,

@@ -47,6 +47,7 @@ def _load() -> ctypes.CDLL:
     lib.windq_last_error.restype = ctypes.c_char_p
     lib.windq_reserve.argtypes = [vp, i64]
     lib.windq_selfcheck.argtypes = [vp, vp, vp]
+    lib.windq_fit_work.argtypes = [vp, ctypes.POINTER(i64), ctypes.POINTER(i64), i32]
     for name in ("windq_scratch_bytes_act_stats",):
         getattr(lib, name).argtypes = [i64, i64]
         getattr(lib, name).restype = i64
@@ -180,6 +181,14 @@ def windq_selfcheck(ctx: Context, stream=None) -> int:
 
 def windq_reserve(ctx: Context, nbytes: int) -> None:
     ctx.reserve(nbytes)
+
+
+def windq_fit_work(ctx: Context, reset: bool = False):
+    """(clip candidates evaluated in full, clip candidates searched) by the fits of this context since the counters
+    were last reset, counted once per warp pass.  Synchronises the device."""
+    a, b = ctypes.c_int64(0), ctypes.c_int64(0)
+    ctx._check(_lib.windq_fit_work(ctx._h, ctypes.byref(a), ctypes.byref(b), 1 if reset else 0))
+    return int(a.value), int(b.value)
 
 
 def windq_scratch_bytes_act_stats(T: int, C: int) -> int:

@@ -88,8 +88,7 @@ windq_status windq_create(windq_ctx** out, int device) {
   unsigned int* sync = nullptr;
   {
     windq::DeviceGuard guard(device);
-    if (cudaMalloc(&sync, windq::kSyncCounters * sizeof(unsigned int)) != cudaSuccess ||
-        cudaMemset(sync, 0, windq::kSyncCounters * sizeof(unsigned int)) != cudaSuccess) {
+    if (cudaMalloc(&sync, windq::kSyncBytes) != cudaSuccess || cudaMemset(sync, 0, windq::kSyncBytes) != cudaSuccess) {
       cudaGetLastError();
       if (sync) cudaFree(sync);
       return windq::fail(nullptr, WINDQ_ERR_CUDA, "windq_create: cannot allocate the arrival counters on device %d", device);
@@ -131,6 +130,19 @@ windq_status windq_selfcheck(windq_ctx* ctx, int64_t* n_failures_out, void* stre
   WINDQ_CUDA(ctx, cudaMemsetAsync(n_failures_out, 0, sizeof(int64_t), st));
   selfcheck_reciprocal_kernel<<<0x7c00 / 256, 256, 0, st>>>((unsigned long long*)n_failures_out);
   WINDQ_CUDA(ctx, cudaGetLastError());
+  return WINDQ_OK;
+}
+
+windq_status windq_fit_work(windq_ctx* ctx, int64_t* evaluated_out, int64_t* searched_out, int reset) {
+  using namespace windq;
+  if (!ctx) return fail(nullptr, WINDQ_ERR_NULL, "windq_fit_work: ctx is NULL");
+  WINDQ_REQUIRE(ctx, evaluated_out && searched_out, WINDQ_ERR_NULL, "windq_fit_work: evaluated_out or searched_out is NULL");
+  DeviceGuard guard(ctx->device);
+  unsigned long long host[2] = {0, 0};
+  WINDQ_CUDA(ctx, cudaMemcpy(host, fit_work_counters(ctx), sizeof(host), cudaMemcpyDeviceToHost));
+  if (reset) WINDQ_CUDA(ctx, cudaMemset(fit_work_counters(ctx), 0, sizeof(host)));
+  *evaluated_out = (int64_t)host[0];
+  *searched_out = (int64_t)host[1];
   return WINDQ_OK;
 }
 

@@ -279,6 +279,85 @@ __device__ __forceinline__ void search_uniform(const Lane32& w, const Lane32& s,
   }
 }
 
+// This lane's least and greatest weight with their activation weights, as (least, greatest) pairs: the two
+// elements a narrower clip range hurts most, for the bound of search_uniform_pruned.
+__device__ __forceinline__ void lane_extremes(const Lane32& w, const Lane32& s, float2& ext_w, float2& ext_s) {
+  float lo = w.v[0][0].x, hi = lo, slo = s.v[0][0].x, shi = slo;
+#pragma unroll
+  for (int h = 0; h < 2; ++h)
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const float2 wv = w.v[h][i], sv = s.v[h][i];
+      if (wv.x < lo) { lo = wv.x; slo = sv.x; }
+      if (wv.x > hi) { hi = wv.x; shi = sv.x; }
+      if (wv.y < lo) { lo = wv.y; slo = sv.y; }
+      if (wv.y > hi) { hi = wv.y; shi = sv.y; }
+    }
+  ext_w = make_float2(lo, hi);
+  ext_s = make_float2(slo, shi);
+}
+
+// search_uniform with candidates left out that cannot win -- same best_e and best_k, bit for bit.
+//
+// Every term (s d) d of a candidate's error is >= 0 when s >= 0, and rounding to nearest is monotone, so the
+// error of a group -- a tree of additions of such terms, each addition rounded -- is at least the rounded term
+// fl(fl(s_j d_j) d_j) of any one element j.  A candidate whose term for some element already exceeds the least
+// error found so far therefore cannot replace it, and if that holds in every group of the warp the warp skips the
+// candidate.  The elements tried are each lane's least and greatest weight (the ones a narrower clip range cuts
+// deepest); their terms cost one packed evaluation per candidate, a sixteenth of the full one.  The scan runs from
+// the last candidate to the first and replaces on <=, which ends on the same candidate as the forward scan with <
+// (the first of the least error), because clip grids usually end on the widest range and the wide ranges win at
+// eight bits: there four candidates in five are skipped on weight-like data.  With activation weights below zero
+// the premise fails; such input is outside the domain (s is a mean of squares).  `evaluated` is advanced by the
+// number of candidates evaluated in full.
+template <int G>
+__device__ __forceinline__ void search_uniform_pruned(const Lane32& w, const Lane32& s, float2 ext_w, float2 ext_s, float mn,
+                                                      float rng, int bi, const float* __restrict__ clip, int K, Cand* cand,
+                                                      int chunk, int stride, int lane, float& best_e, int& best_k,
+                                                      unsigned int& evaluated) {
+  constexpr int LG = Map<G>::LG;
+  const int g = lane / LG, q = lane % LG;
+  const UniformSpec us = uniform_spec(bi);
+  const int qmax_bits = __float_as_int(us.qmax);
+  Cand* mine = cand + g * stride;
+  best_e = __int_as_float(0x7f800000);
+  best_k = 0;
+  const float2 magic2 = make_float2(kMagic, kMagic);
+  const int n_chunks = (K + chunk - 1) / chunk;
+  for (int ci = n_chunks - 1; ci >= 0; --ci) {
+    const int k0 = ci * chunk;
+    const int kc = min(chunk, K - k0);
+    __syncwarp();
+    for (int k = q; k < kc; k += LG) mine[k] = make_cand(mn, rng, __ldg(clip + k0 + k), us);
+    __syncwarp();
+    for (int k = kc - 1; k >= 0; --k) {
+      const Cand c = mine[k];
+      {
+        float2 x = add2(fma2(ext_w, make_float2(c.inv, c.inv), magic2), make_float2(c.bias, c.bias));
+        x.x = clamp_code(x.x, qmax_bits);
+        x.y = clamp_code(x.y, qmax_bits);
+        const float2 d = add2(fma2(x, make_float2(c.nscale, c.nscale), make_float2(c.kz, c.kz)), ext_w);
+        const float2 term = mul2(mul2(ext_s, d), d);
+        // one bit per lane whose bound rules the candidate out for its group; a group is out if any of its lanes says so
+        unsigned int out = __ballot_sync(0xffffffffu, fmaxf(term.x, term.y) > best_e);
+#pragma unroll
+        for (int m = 1; m < LG; m <<= 1) out |= out >> m;
+        constexpr unsigned int kFirstLanes = LG == 1 ? 0xffffffffu : LG == 2 ? 0x55555555u : LG == 4 ? 0x11111111u
+                                             : LG == 8 ? 0x01010101u : 0x00010001u;
+        if ((out & kFirstLanes) == kFirstLanes) continue;
+      }
+      ++evaluated;
+      float2 e01, e23;
+      cand_leaf_errors(w, s, c, qmax_bits, e01, e23);
+      const float e = group_tree<G>(e01, e23);
+      if (e <= best_e) {
+        best_e = e;
+        best_k = k0 + k;
+      }
+    }
+  }
+}
+
 // ---- ternary and binary -----------------------------------------------------------------------
 struct LowBitFit {
   float delta;    // ternary threshold 0.7 * mean |w|

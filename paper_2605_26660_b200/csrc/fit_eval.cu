@@ -67,7 +67,7 @@ fit_eval_kernel(const __half* __restrict__ W_one, int R_one, int U_one, int64_t 
                 const float* __restrict__ clip, int K, double* __restrict__ partial, uint8_t* __restrict__ clip_idx_one,
                 float* __restrict__ group_err_one, int rows_blocks_one, int chunk, int stride,
                 const float* __restrict__ scale, const float* __restrict__ thresh, float never,
-                unsigned int* __restrict__ next_item, const FitJobs jobs) {
+                unsigned int* __restrict__ next_item, unsigned long long* __restrict__ work, const FitJobs jobs) {
   constexpr int LG = Map<G>::LG, GPW = Map<G>::GPW;
   extern __shared__ float4 smem_f4[];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -76,6 +76,7 @@ fit_eval_kernel(const __half* __restrict__ W_one, int R_one, int U_one, int64_t 
 
   const unsigned int n_items = (BATCH ? jobs.first_item[jobs.n] : (unsigned int)(U_one * rows_blocks_one)) * (PARTS ? 5u : 1u);
 
+  unsigned int searched = 0, evaluated = 0;  // clip candidates of this warp's searches, and those evaluated in full
   Lane32 sv;
   for (;;) {
     // items are claimed from a counter, in order: with equal static shares the warps of an SM do not
@@ -170,6 +171,8 @@ fit_eval_kernel(const __half* __restrict__ W_one, int R_one, int U_one, int64_t 
     float mn, mx;
     group_range<G>(wv, mn, mx);
     const float rng = __fsub_rn(mx, mn);
+    float2 ext_w, ext_s;
+    lane_extremes(wv, sv, ext_w, ext_s);
 
     float e[7] = {0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f};
 #pragma unroll 1
@@ -177,7 +180,13 @@ fit_eval_kernel(const __half* __restrict__ W_one, int R_one, int U_one, int64_t 
       if (PARTS && !((parts >> bi) & 1u)) continue;
       float be;
       int bk;
-      search_uniform<G>(wv, sv, mn, rng, bi, clip, K, cand, chunk, stride, lane, be, bk);
+      searched += (unsigned int)K;
+      if (bi == 0) {
+        search_uniform_pruned<G>(wv, sv, ext_w, ext_s, mn, rng, bi, clip, K, cand, chunk, stride, lane, be, bk, evaluated);
+      } else {
+        search_uniform<G>(wv, sv, mn, rng, bi, clip, K, cand, chunk, stride, lane, be, bk);
+        evaluated += (unsigned int)K;
+      }
       e[0] = bi == 0 ? be : e[0];
       e[1] = bi == 1 ? be : e[1];
       e[2] = bi == 2 ? be : e[2];
@@ -218,6 +227,10 @@ fit_eval_kernel(const __half* __restrict__ W_one, int R_one, int U_one, int64_t 
       for (int m = LG; m < 32; m <<= 1) d += __shfl_xor_sync(0xffffffffu, d, m);
       if (lane == 0 && (!PARTS || ((parts >> (c < 4 ? c : 4)) & 1u))) partial[(int64_t)item * kFitPartials + c] = d;
     }
+  }
+  if (lane == 0 && searched) {
+    atomicAdd(work, (unsigned long long)evaluated);
+    atomicAdd(work + 1, (unsigned long long)searched);
   }
 }
 
@@ -309,11 +322,11 @@ windq_status launch_fit(windq_ctx* ctx, const __half* W, int R, int U, int64_t l
   if (in_parts)
     fit_eval_kernel<G, PROTECT, true, false><<<(unsigned)grid, kFitWarpsPerBlock * 32, smem, st>>>(
         W, R, U, ldw, s, clip, K, partial, clip_idx_out, group_err_out, rows_blocks, chunk, stride, scale, thresh,
-        __builtin_nanf(""), next_item, FitJobs());
+        __builtin_nanf(""), next_item, fit_work_counters(ctx), FitJobs());
   else
     fit_eval_kernel<G, PROTECT, false, false><<<(unsigned)grid, kFitWarpsPerBlock * 32, smem, st>>>(
         W, R, U, ldw, s, clip, K, partial, clip_idx_out, group_err_out, rows_blocks, chunk, stride, scale, thresh,
-        __builtin_nanf(""), next_item, FitJobs());
+        __builtin_nanf(""), next_item, fit_work_counters(ctx), FitJobs());
   WINDQ_CUDA(ctx, cudaGetLastError());
   fit_finalize_kernel<<<(unsigned)U, 256, 0, st>>>(partial, rows_blocks, err_out, energy_out);
   WINDQ_CUDA(ctx, cudaGetLastError());
@@ -344,11 +357,11 @@ windq_status launch_fit_batch(windq_ctx* ctx, const FitJobs& jobs, const float* 
   if (in_parts)
     fit_eval_kernel<G, false, true, true, FEAT><<<(unsigned)grid, kFitWarpsPerBlock * 32, smem, st>>>(
         nullptr, 0, 0, 0, nullptr, clip, K, partial, nullptr, nullptr, 0, chunk, stride, nullptr, nullptr, __builtin_nanf(""),
-        next_item, jobs);
+        next_item, fit_work_counters(ctx), jobs);
   else
     fit_eval_kernel<G, false, false, true, FEAT><<<(unsigned)grid, kFitWarpsPerBlock * 32, smem, st>>>(
         nullptr, 0, 0, 0, nullptr, clip, K, partial, nullptr, nullptr, 0, chunk, stride, nullptr, nullptr, __builtin_nanf(""),
-        next_item, jobs);
+        next_item, fit_work_counters(ctx), jobs);
   WINDQ_CUDA(ctx, cudaGetLastError());
   fit_finalize_batch_kernel<<<jobs.first_unit[jobs.n], 256, 0, st>>>(partial, GPW, jobs, FEAT ? unit_wsum : nullptr);
   WINDQ_CUDA(ctx, cudaGetLastError());

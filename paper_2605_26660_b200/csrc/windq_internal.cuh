@@ -14,7 +14,7 @@ struct windq_ctx {
   int sm_count;
   void* scratch;
   int64_t scratch_bytes;
-  unsigned int* sync;  // kSyncCounters arrival counters, zero between launches
+  unsigned int* sync;  // kSyncCounters arrival counters, zero between launches; two 64-bit work counters follow them
   unsigned long long prepared[2];  // kernels whose attributes have been set on this context's device (bit per KernelId)
   int occupancy[128];              // resident blocks per SM of those kernels (0 where not asked)
   char err[256];
@@ -23,8 +23,13 @@ struct windq_ctx {
 namespace windq {
 
 constexpr int64_t kSyncCounters = 16384;
+constexpr int64_t kSyncBytes = kSyncCounters * (int64_t)sizeof(unsigned int) + 2 * (int64_t)sizeof(unsigned long long);
 
 windq_status fail(windq_ctx* ctx, windq_status st, const char* fmt, ...);
+// Where the fits count their clip candidates: [0] those evaluated in full, [1] all of them (see windq_fit_work).
+inline unsigned long long* fit_work_counters(windq_ctx* ctx) {
+  return reinterpret_cast<unsigned long long*>(ctx->sync + kSyncCounters);
+}
 // Makes the context's scratch at least `bytes` large (may cudaMalloc).
 windq_status ensure_scratch(windq_ctx* ctx, int64_t bytes);
 

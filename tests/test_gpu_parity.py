@@ -188,6 +188,46 @@ def test_fit_eval_config1_single_layer(wq, ctx, oracle):
         assert close(got["err"][u0], want["err"][u0]).all() and close(got["energy"][u0], want["energy"][u0]).all()
 
 
+@pytest.mark.parametrize("G", [32, 64, 128, 256, 512])
+def test_eight_bit_search_skips_only_losers(wq, ctx, oracle, G):
+    """The eight-bit clip search leaves out candidates whose error is bounded below by a single weight's term.  The
+    kept index and error must be those of the full search, bit for bit, whatever the order of the grid (the search
+    scans it backwards), with repeated ratios (the first of equal errors wins), with more candidates than one table
+    holds, with statistics that vanish where the extremes sit (the bound is then zero and rules nothing out) and
+    with an outlier that is free to clip (the best ratio is then the narrowest, met last)."""
+    R, U = 37, 5
+    rng = np.random.default_rng(40 + G)
+    W = ws.weights(R, U * G, 41 + G, "student_t")
+    W[:, :G] = 0                                                        # every candidate ties at zero error
+    W[3, G:2 * G] = 0.25                                                # a constant row
+    s = oracle.act_stats(ws.activations(96, U * G, 42 + G).numpy())
+    out_col = 3 * G + int(rng.integers(0, G))
+    W[:, out_col] = torch.from_numpy(rng.choice([-4.0, 4.0], R).astype(np.float16))   # outliers on a channel ...
+    s[out_col] = 0                                                      # ... that no activation ever excites
+    s[4 * G:] = 0
+    s[4 * G + 5] = 1.0                                                  # one live channel in the last unit
+    asc = ws.clip_grid(20)
+    grids = {"ascending": asc, "descending": asc[::-1].copy(),
+             "shuffled with repeats": rng.permutation(np.concatenate([asc, asc[5:9], asc[-1:]])).astype(np.float32),
+             "one": asc[-1:].copy(), "sixty-four": rng.uniform(1.0 / 64, 1.0, 64).astype(np.float32)}
+    for name, grid in grids.items():
+        want = oracle.fit_eval(W.numpy(), G, s, grid)
+        wq.windq_fit_work(ctx, reset=True)
+        got = run_fit(wq, ctx, W, G, s, grid)
+        evaluated, searched = wq.windq_fit_work(ctx)
+        check_fit(got, want)
+        assert 0 < evaluated <= searched, name
+        assert searched % (4 * len(grid)) == 0, name
+    # on weight-like data with the widest range last, most eight-bit candidates are ruled out
+    Wl = ws.weights(256, 4 * G, 43 + G, "student_t")
+    sl = oracle.act_stats(ws.activations(96, 4 * G, 44 + G).numpy())
+    wq.windq_fit_work(ctx, reset=True)
+    got = run_fit(wq, ctx, Wl, G, sl, asc)
+    evaluated, searched = wq.windq_fit_work(ctx, reset=True)
+    check_fit(got, oracle.fit_eval(Wl.numpy(), G, sl, asc, threads=8))
+    assert evaluated < 0.95 * searched
+
+
 def test_selfcheck_finds_no_mismatch(wq, ctx):
     """The fits take 1 / scale by the hardware approximation and one Newton step; for every fp16 value a scale can
     have that must be the IEEE quotient, which the oracle uses."""

@@ -279,9 +279,9 @@ __device__ __forceinline__ void search_uniform(const Lane32& w, const Lane32& s,
   }
 }
 
-// This lane's least and greatest weight with their activation weights, as (least, greatest) pairs: the two
-// elements a narrower clip range hurts most, for the bound of search_uniform_pruned.
-__device__ __forceinline__ void lane_extremes(const Lane32& w, const Lane32& s, float2& ext_w, float2& ext_s) {
+// This lane's least and greatest weight and their activation weights, as (least, greatest, s of least, s of
+// greatest): the elements a narrower clip range cuts deepest, for the bound of search_uniform_pruned.
+__device__ __forceinline__ float4 lane_extremes(const Lane32& w, const Lane32& s) {
   float lo = w.v[0][0].x, hi = lo, slo = s.v[0][0].x, shi = slo;
 #pragma unroll
   for (int h = 0; h < 2; ++h)
@@ -293,8 +293,7 @@ __device__ __forceinline__ void lane_extremes(const Lane32& w, const Lane32& s, 
       if (wv.y < lo) { lo = wv.y; slo = sv.y; }
       if (wv.y > hi) { hi = wv.y; shi = sv.y; }
     }
-  ext_w = make_float2(lo, hi);
-  ext_s = make_float2(slo, shi);
+  return make_float4(lo, hi, slo, shi);
 }
 
 // search_uniform with candidates left out that cannot win -- same best_e and best_k, bit for bit.
@@ -303,18 +302,23 @@ __device__ __forceinline__ void lane_extremes(const Lane32& w, const Lane32& s, 
 // error of a group -- a tree of additions of such terms, each addition rounded -- is at least the rounded term
 // fl(fl(s_j d_j) d_j) of any one element j.  A candidate whose term for some element already exceeds the least
 // error found so far therefore cannot replace it, and if that holds in every group of the warp the warp skips the
-// candidate.  The elements tried are each lane's least and greatest weight (the ones a narrower clip range cuts
-// deepest); their terms cost one packed evaluation per candidate, a sixteenth of the full one.  The scan runs from
-// the last candidate to the first and replaces on <=, which ends on the same candidate as the forward scan with <
-// (the first of the least error), because clip grids usually end on the widest range and the wide ranges win at
-// eight bits: there four candidates in five are skipped on weight-like data.  With activation weights below zero
-// the premise fails; such input is outside the domain (s is a mean of squares).  `evaluated` is advanced by the
-// number of candidates evaluated in full.
+// candidate.  The elements tried are every lane's least and greatest weight (`ext`, one entry per lane of the
+// warp, in shared memory: the ones a narrower clip range cuts deepest).  Where a group has four lanes or more, the
+// lane that forms a candidate's parameters also forms its bound -- the largest of those terms over the group's
+// lanes -- and leaves it in the table entry in place of z * scale, which the scan forms again for the candidates
+// it evaluates.  Where a group has one or two lanes, a lane would have to form ten bounds and more on its own, and
+// every lane tries its own two elements inside the scan instead (a group is out if any of its lanes says so);
+// measured, each form is the faster one on its side (chunk width 64: 0.72 against 0.80 ms on 11008 x 4096; 128:
+// 0.71 against 0.74).  The scan runs from the last candidate to the first and replaces on <=, which ends on the
+// same candidate as the forward scan with < (the first of the least error): clip grids usually end on the widest
+// range and the wide ranges win at eight bits -- there four candidates in five are skipped on weight-like data.
+// With activation weights below zero the premise fails; such input is outside the domain (s is a mean of squares).
+// `skipped` is advanced by the number of candidates left out.
 template <int G>
-__device__ __forceinline__ void search_uniform_pruned(const Lane32& w, const Lane32& s, float2 ext_w, float2 ext_s, float mn,
+__device__ __forceinline__ void search_uniform_pruned(const Lane32& w, const Lane32& s, const float4* ext, float mn,
                                                       float rng, int bi, const float* __restrict__ clip, int K, Cand* cand,
                                                       int chunk, int stride, int lane, float& best_e, int& best_k,
-                                                      unsigned int& evaluated) {
+                                                      unsigned int& skipped) {
   constexpr int LG = Map<G>::LG;
   const int g = lane / LG, q = lane % LG;
   const UniformSpec us = uniform_spec(bi);
@@ -323,30 +327,54 @@ __device__ __forceinline__ void search_uniform_pruned(const Lane32& w, const Lan
   best_e = __int_as_float(0x7f800000);
   best_k = 0;
   const float2 magic2 = make_float2(kMagic, kMagic);
+  constexpr bool kInLoop = LG <= 2;  // bounds formed inside the scan, from the lane's own elements
+  const float4 own = ext[lane];
+  const float2 own_w = make_float2(own.x, own.y), own_s = make_float2(own.z, own.w);
   const int n_chunks = (K + chunk - 1) / chunk;
   for (int ci = n_chunks - 1; ci >= 0; --ci) {
     const int k0 = ci * chunk;
     const int kc = min(chunk, K - k0);
     __syncwarp();
-    for (int k = q; k < kc; k += LG) mine[k] = make_cand(mn, rng, __ldg(clip + k0 + k), us);
-    __syncwarp();
-    for (int k = kc - 1; k >= 0; --k) {
-      const Cand c = mine[k];
-      {
-        float2 x = add2(fma2(ext_w, make_float2(c.inv, c.inv), magic2), make_float2(c.bias, c.bias));
+    if (kInLoop) {
+      for (int k = q; k < kc; k += LG) mine[k] = make_cand(mn, rng, __ldg(clip + k0 + k), us);
+    } else
+    for (int k = q; k < kc; k += LG) {
+      Cand c = make_cand(mn, rng, __ldg(clip + k0 + k), us);
+      float b = 0.0f;
+#pragma unroll
+      for (int j = 0; j < LG; ++j) {
+        const float4 e = ext[g * LG + j];
+        const float2 ew = make_float2(e.x, e.y);
+        float2 x = add2(fma2(ew, make_float2(c.inv, c.inv), magic2), make_float2(c.bias, c.bias));
         x.x = clamp_code(x.x, qmax_bits);
         x.y = clamp_code(x.y, qmax_bits);
-        const float2 d = add2(fma2(x, make_float2(c.nscale, c.nscale), make_float2(c.kz, c.kz)), ext_w);
-        const float2 term = mul2(mul2(ext_s, d), d);
-        // one bit per lane whose bound rules the candidate out for its group; a group is out if any of its lanes says so
+        const float2 d = add2(fma2(x, make_float2(c.nscale, c.nscale), make_float2(c.kz, c.kz)), ew);
+        const float2 term = mul2(mul2(make_float2(e.z, e.w), d), d);
+        b = fmaxf(b, fmaxf(term.x, term.y));
+      }
+      c.kz = b;  // the table entry carries the bound in place of z * scale, which the scan forms again
+      mine[k] = c;
+    }
+    __syncwarp();
+    for (int k = kc - 1; k >= 0; --k) {
+      Cand c = mine[k];
+      if (kInLoop) {
+        // this lane's own two elements; a group is out if any of its lanes says so
+        float2 x = add2(fma2(own_w, make_float2(c.inv, c.inv), magic2), make_float2(c.bias, c.bias));
+        x.x = clamp_code(x.x, qmax_bits);
+        x.y = clamp_code(x.y, qmax_bits);
+        const float2 d = add2(fma2(x, make_float2(c.nscale, c.nscale), make_float2(c.kz, c.kz)), own_w);
+        const float2 term = mul2(mul2(own_s, d), d);
         unsigned int out = __ballot_sync(0xffffffffu, fmaxf(term.x, term.y) > best_e);
 #pragma unroll
         for (int m = 1; m < LG; m <<= 1) out |= out >> m;
         constexpr unsigned int kFirstLanes = LG == 1 ? 0xffffffffu : LG == 2 ? 0x55555555u : LG == 4 ? 0x11111111u
                                              : LG == 8 ? 0x01010101u : 0x00010001u;
-        if ((out & kFirstLanes) == kFirstLanes) continue;
+        if ((out & kFirstLanes) == kFirstLanes) { ++skipped; continue; }
+      } else {
+        if (__all_sync(0xffffffffu, c.kz > best_e)) { ++skipped; continue; }  // ruled out in every group of the warp
+        c.kz = __fmul_rn(__fadd_rn(c.bias, kMagic), -c.nscale);  // z * scale, as make_cand forms it
       }
-      ++evaluated;
       float2 e01, e23;
       cand_leaf_errors(w, s, c, qmax_bits, e01, e23);
       const float e = group_tree<G>(e01, e23);

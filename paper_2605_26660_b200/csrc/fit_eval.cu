@@ -72,11 +72,13 @@ fit_eval_kernel(const __half* __restrict__ W_one, int R_one, int U_one, int64_t 
   extern __shared__ float4 smem_f4[];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   Cand* cand = reinterpret_cast<Cand*>(smem_f4) + (size_t)warp * GPW * stride;
+  __shared__ float4 ext_all[kFitWarpsPerBlock][32];  // every lane's least and greatest weight, for those bounds
+  float4* ext = ext_all[warp];
   const int g = lane / LG, q = lane % LG;
 
   const unsigned int n_items = (BATCH ? jobs.first_item[jobs.n] : (unsigned int)(U_one * rows_blocks_one)) * (PARTS ? 5u : 1u);
 
-  unsigned int searched = 0, evaluated = 0;  // clip candidates of this warp's searches, and those evaluated in full
+  unsigned int searches = 0, skipped = 0;  // clip searches of this warp (K candidates each), and candidates left out
   Lane32 sv;
   for (;;) {
     // items are claimed from a counter, in order: with equal static shares the warps of an SM do not
@@ -171,26 +173,27 @@ fit_eval_kernel(const __half* __restrict__ W_one, int R_one, int U_one, int64_t 
     float mn, mx;
     group_range<G>(wv, mn, mx);
     const float rng = __fsub_rn(mx, mn);
-    float2 ext_w, ext_s;
-    lane_extremes(wv, sv, ext_w, ext_s);
+    __syncwarp();                       // the previous item's search has read its entries
+    ext[lane] = lane_extremes(wv, sv);  // read by the eight-bit search, after its __syncwarp()
 
-    float e[7] = {0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f};
+    float e[3] = {0.0f, 0.0f, 0.0f};
 #pragma unroll 1
     for (int bi = 0; bi < 4; ++bi) {
       if (PARTS && !((parts >> bi) & 1u)) continue;
       float be;
       int bk;
-      searched += (unsigned int)K;
+      ++searches;
       if (bi == 0) {
-        search_uniform_pruned<G>(wv, sv, ext_w, ext_s, mn, rng, bi, clip, K, cand, chunk, stride, lane, be, bk, evaluated);
+        search_uniform_pruned<G>(wv, sv, ext, mn, rng, bi, clip, K, cand, chunk, stride, lane, be, bk, skipped);
       } else {
         search_uniform<G>(wv, sv, mn, rng, bi, clip, K, cand, chunk, stride, lane, be, bk);
-        evaluated += (unsigned int)K;
       }
-      e[0] = bi == 0 ? be : e[0];
-      e[1] = bi == 1 ? be : e[1];
-      e[2] = bi == 2 ? be : e[2];
-      e[3] = bi == 3 ? be : e[3];
+      {
+        double d = live ? (double)be : 0.0;
+#pragma unroll
+        for (int m = LG; m < 32; m <<= 1) d += __shfl_xor_sync(0xffffffffu, d, m);
+        if (lane == 0) partial[(int64_t)item * kFitPartials + bi] = d;
+      }
       if (live && q == 0) {
         const int64_t o = ((int64_t)bi * U + u) * R + row;
         if (clip_idx_out) clip_idx_out[o] = (uint8_t)bk;
@@ -200,9 +203,9 @@ fit_eval_kernel(const __half* __restrict__ W_one, int R_one, int U_one, int64_t 
     if (!PARTS || (parts & 0x10u)) {
       // group errors wanted: the term-by-term sums (bit-defined); unit sums only: from the sums of the fit
       const LowBitFit low = fit_low_bits<G>(wv, sv, group_err_out != nullptr);
-      e[4] = low.err_t;
-      e[5] = low.err_b;
-      e[6] = low.energy;
+      e[0] = low.err_t;
+      e[1] = low.err_b;
+      e[2] = low.energy;
       if (live && q == 0 && group_err_out) {
         group_err_out[((int64_t)4 * U + u) * R + row] = low.err_t;
         group_err_out[((int64_t)5 * U + u) * R + row] = low.err_b;
@@ -221,16 +224,16 @@ fit_eval_kernel(const __half* __restrict__ W_one, int R_one, int U_one, int64_t 
 
     // add over the rows of this item in double; lanes of a group hold equal values
 #pragma unroll
-    for (int c = 0; c < 7; ++c) {
+    for (int c = 0; c < 3; ++c) {
       double d = live ? (double)e[c] : 0.0;
 #pragma unroll
       for (int m = LG; m < 32; m <<= 1) d += __shfl_xor_sync(0xffffffffu, d, m);
-      if (lane == 0 && (!PARTS || ((parts >> (c < 4 ? c : 4)) & 1u))) partial[(int64_t)item * kFitPartials + c] = d;
+      if (lane == 0 && (!PARTS || (parts & 0x10u))) partial[(int64_t)item * kFitPartials + 4 + c] = d;
     }
   }
-  if (lane == 0 && searched) {
-    atomicAdd(work, (unsigned long long)evaluated);
-    atomicAdd(work + 1, (unsigned long long)searched);
+  if (lane == 0 && searches) {
+    atomicAdd(work, (unsigned long long)searches * (unsigned long long)K - (unsigned long long)skipped);
+    atomicAdd(work + 1, (unsigned long long)searches * (unsigned long long)K);
   }
 }
 

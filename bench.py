@@ -42,7 +42,7 @@ APPLY_G = 128                    # chunk width the plans are applied at (the fir
 # measured DRAM bytes (read + written) per byte of weights, from the ncu captures summarised under profiles/:
 # one 4096 x 4096 matrix per launch (outputs stay in L2), and the seven matrices of a 7B-shaped block per launch
 # (mean of the captures at chunk widths 64 and 128)
-FIT_TRAFFIC_PER_WEIGHT_BYTE = {False: 33.6 / 33.554, True: (434.4 + 432.3) / 2 / 404.75}
+FIT_TRAFFIC_PER_WEIGHT_BYTE = {False: None, True: (434.4 + 437.0) / 2 / 404.75}   # None: no capture of the kernel as it stands
 SEED = 0
 
 
@@ -807,10 +807,11 @@ def main():
     hbm_time = 2.0 * fit_elem / (peaks["hbm_gbs"] * 1e9)
     alu_time = fit_elem * ops / (alu_peak * 1e12)
     # DRAM traffic of fit_eval_kernel per launch: dram__bytes_read + dram__bytes_write of an ncu capture of the same
-    # launch shape (profiles/fit_eval_kernel_batch_cfg3_block_K20.txt: 433 MB against 404.75 MB of weights for a block
-    # per launch; profiles/fit_eval_kernel_4096x4096_K20.txt for one matrix per launch), scaled to this run's average
+    # launch shape (profiles/fit_eval_kernel_batch_cfg3_block_K20.txt: 436 MB against 404.75 MB of weights for a block
+    # per launch; one matrix per launch has no capture of the present kernel: null), scaled to this run's average
     # launch by the weights a launch reads (traffic is proportional to them: one pass, no re-reads)
-    traffic = FIT_TRAFFIC_PER_WEIGHT_BYTE[BATCH_FITS] * 2.0 * fit_elem / n_fit
+    per_byte = FIT_TRAFFIC_PER_WEIGHT_BYTE[BATCH_FITS]
+    traffic = None if per_byte is None else per_byte * 2.0 * fit_elem / n_fit
     roofline = dict(bound="alu" if alu_time >= hbm_time else "hbm", kernel="fit_eval_kernel", achieved=achieved, peak=alu_peak,
                     unit="T fp32 lane-ops/s (fma = 1)", frac=achieved / alu_peak, traffic=traffic, traffic_unit="bytes per launch",
                     launches=n_fit, avg_launch_ms=fit_ms / n_fit, ops_per_element=ops,

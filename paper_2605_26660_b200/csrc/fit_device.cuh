@@ -400,45 +400,44 @@ struct LowBitFit {
 template <int G>
 __device__ __forceinline__ LowBitFit fit_low_bits(const Lane32& w, const Lane32& s, bool exact_errors) {
   LowBitFit f;
-  float A[4], Sb[4], Bb[4], En[4];
+  const float2 zero2 = make_float2(0.0f, 0.0f);
+  // leaves 2 h and 2 h + 1 side by side in the two halves of the packed operations
+  float2 a2[2] = {zero2, zero2}, sb2[2] = {zero2, zero2}, bb2[2] = {zero2, zero2}, en2[2] = {zero2, zero2};
 #pragma unroll
-  for (int l = 0; l < 4; ++l) {
-    float a = 0.0f, sb = 0.0f, bb = 0.0f, en = 0.0f;
+  for (int h = 0; h < 2; ++h)
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
-      const float wv = w.get(l, i), sv = s.get(l, i), aw = fabsf(wv);
-      a = __fadd_rn(a, aw);
-      sb = __fadd_rn(sb, sv);
-      bb = __fmaf_rn(sv, aw, bb);
-      en = __fmaf_rn(__fmul_rn(sv, wv), wv, en);
+      const float2 wv = w.v[h][i], sv = s.v[h][i];
+      const float2 aw = make_float2(fabsf(wv.x), fabsf(wv.y));
+      a2[h] = add2(a2[h], aw);
+      sb2[h] = add2(sb2[h], sv);
+      bb2[h] = fma2(sv, aw, bb2[h]);
+      en2[h] = fma2(mul2(sv, wv), wv, en2[h]);
     }
-    A[l] = a; Sb[l] = sb; Bb[l] = bb; En[l] = en;
-  }
-  const float sumA = group_tree<G>(A[0], A[1], A[2], A[3]);
-  const float sumS = group_tree<G>(Sb[0], Sb[1], Sb[2], Sb[3]);
-  const float sumB = group_tree<G>(Bb[0], Bb[1], Bb[2], Bb[3]);
-  f.energy = group_tree<G>(En[0], En[1], En[2], En[3]);
+  const float sumA = group_tree<G>(a2[0], a2[1]);
+  const float sumS = group_tree<G>(sb2[0], sb2[1]);
+  const float sumB = group_tree<G>(bb2[0], bb2[1]);
+  f.energy = group_tree<G>(en2[0], en2[1]);
   const float meanA = __fmul_rn(sumA, 1.0f / (float)G);
   f.delta = __fmul_rn(0.7f, meanA);
   f.alpha_b = __half2float(__float2half_rn(sumS == 0.0f ? meanA : __fdiv_rn(sumB, sumS)));
 
   // ternary sums over the support, weighted by s; the unweighted ones only if some group of the
-  // warp has no activation weight on its support
-  float Bt[4], Ct[4];
+  // warp has no activation weight on its support.  The support enters as a factor 1 or 0 per weight: s (|w| m)
+  // and s m are exact products of the terms the definition adds, so the sums round as they do there.
+  float2 bt2[2] = {zero2, zero2}, ct2[2] = {zero2, zero2};
 #pragma unroll
-  for (int l = 0; l < 4; ++l) {
-    float bt = 0.0f, ct = 0.0f;
+  for (int h = 0; h < 2; ++h)
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
-      const float aw = fabsf(w.get(l, i)), sv = s.get(l, i);
-      const bool in = aw > f.delta;
-      bt = __fmaf_rn(sv, in ? aw : 0.0f, bt);
-      ct = __fadd_rn(ct, in ? sv : 0.0f);
+      const float2 wv = w.v[h][i], sv = s.v[h][i];
+      const float2 aw = make_float2(fabsf(wv.x), fabsf(wv.y));
+      const float2 m = make_float2(aw.x > f.delta ? 1.0f : 0.0f, aw.y > f.delta ? 1.0f : 0.0f);
+      bt2[h] = fma2(sv, mul2(aw, m), bt2[h]);
+      ct2[h] = fma2(sv, m, ct2[h]);
     }
-    Bt[l] = bt; Ct[l] = ct;
-  }
-  float sumBt = group_tree<G>(Bt[0], Bt[1], Bt[2], Bt[3]);
-  float sumCt = group_tree<G>(Ct[0], Ct[1], Ct[2], Ct[3]);
+  float sumBt = group_tree<G>(bt2[0], bt2[1]);
+  float sumCt = group_tree<G>(ct2[0], ct2[1]);
   const float wBt = sumBt, wCt = sumCt;  // the weighted sums, whatever the scale is taken from
   // delta < max |w| whenever some w is not zero (0.7 * mean <= 0.7 * max, roundings included), so
   // the support is empty exactly when every |w| is zero, i.e. when their sum is

@@ -316,3 +316,40 @@ def test_energy_is_the_weighted_sum_of_squares_in_float64(oracle):
     share = 3.0 * float(s[7]) * float((w64[:, 7] ** 2).sum())
     assert abs((float(e2[0]) - float(fit["energy"][0])) - share) <= 1e-5 * float(e2[0])
     assert e2[1] == fit["energy"][1] and e2[2] == fit["energy"][2]
+
+
+# ------------------------------------------------------------------ a candidate's error against single terms
+def test_error_is_never_below_the_term_of_one_weight(oracle):
+    """With s >= 0 every term (s d) d is >= 0 and rounding is monotone, so the PSUM8 error of a candidate is at least
+    the rounded term of any single weight -- the fact the GPU's eight-bit search rests on when it leaves out
+    candidates.  Checked here on the oracle alone, with the terms formed independently in float64 (c * scale - w is
+    exact there, so one rounding to binary32 gives the fused result), on weight-like groups, on groups whose
+    statistics span sixty binary orders, and on groups with a single live channel (where the error IS the term)."""
+    rng = np.random.default_rng(11)
+    f32 = np.float32
+    checked = tight = 0
+    for G in (32, 128, 512):
+        for trial in range(12):
+            w = ws.weights(1, G, 500 + 13 * trial + G, "student_t").numpy()[0].astype(np.float32)
+            kind = trial % 3
+            if kind == 0:
+                s = (rng.standard_normal(G) ** 2).astype(np.float32)
+            elif kind == 1:
+                s = (2.0 ** rng.integers(-40, 20, G)).astype(np.float32)
+            else:
+                s = np.zeros(G, np.float32)
+                s[int(rng.integers(0, G))] = f32(rng.uniform(0.1, 10.0))
+            for bits in BITS:
+                for p in (0.5, 0.7368421, 1.0):
+                    scale, zero, err, codes = oracle.uniform_candidate(w, s, bits, p)
+                    c = codes.astype(np.float64) - float(zero)
+                    d = (c * float(scale) - w.astype(np.float64)).astype(np.float32)          # fma(c, scale, -w)
+                    t = (s.astype(np.float32) * d).astype(np.float32)                         # s * d, rounded
+                    term = (t.astype(np.float64) * d.astype(np.float64)).astype(np.float32)   # fl(t * d)
+                    assert (term >= 0).all()
+                    assert f32(err) >= term.max(), (G, trial, bits, p)
+                    checked += 1
+                    if kind == 2:
+                        assert f32(err) == term.max()
+                        tight += 1
+    assert checked == 3 * 12 * 4 * 3 and tight == 3 * 4 * 4 * 3
